@@ -1,0 +1,183 @@
+/*
+ * alx.h -- C ABI of the B200 (sm_100a) implicit-ALS half-epoch library.
+ *
+ * The method is implicit Alternating Least Squares as stated in "ALX: Large Scale Matrix
+ * Factorization on TPUs" (arXiv 2112.02194): model Eq. 1, objective Eq. 3, row update Eq. 4,
+ * order of operations Algorithm 1.  One GPU, both embedding tables and the sparse matrix
+ * resident in device memory.  Every step runs in this library's own CUDA kernels.
+ *
+ * Conventions
+ *   - Every call returns an alx_status; nothing throws across this boundary; on error the
+ *     out-parameters are left untouched and alx_last_error() describes the failure.
+ *   - The caller owns every pointer it passes.  Calls copy what they need; the context never
+ *     keeps a caller pointer.  "on_device" arguments say whether a pointer is a device pointer
+ *     (read or written on the context's stream) or a host pointer.
+ *   - W is the table of the matrix's rows (n_rows x d), H the table of its columns (n_cols x d),
+ *     both row-major, contiguous, in the storage type chosen at creation.
+ *   - Kernels are launched asynchronously on the context's stream.  Problems a kernel detects
+ *     (index out of range, non-positive pivot) set a device status word that the next
+ *     synchronising call (alx_synchronize, alx_loss, alx_get_*) turns into an error code.
+ *     Nothing traps or asserts on the device.
+ *   - Results are run-to-run deterministic: no floating-point atomics, all partial sums are
+ *     combined in a fixed order that depends only on the problem sizes.
+ */
+#ifndef ALX_H_
+#define ALX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct alx_ctx alx_ctx; /* opaque; owns all device state */
+
+typedef enum {
+    ALX_OK = 0,
+    ALX_ERR_INVALID_ARG = 1,
+    ALX_ERR_BAD_STATE = 2,   /* call order: e.g. half-epoch before the matrix or tables are set */
+    ALX_ERR_OOM = 3,
+    ALX_ERR_CUDA = 4,
+    ALX_ERR_BAD_CSR = 5,     /* rowptr not monotone / index out of range / row not strictly ascending */
+    ALX_ERR_NOT_SPD = 6,     /* a pivot was not positive (cannot happen for lambda > 0 in exact arithmetic) */
+    ALX_ERR_UNSUPPORTED = 7
+} alx_status;
+
+typedef enum { ALX_ROWS = 0, ALX_COLS = 1 } alx_side; /* which table is SOLVED; the other is held fixed */
+typedef enum { ALX_F32 = 0, ALX_BF16 = 1 } alx_dtype;
+
+/* number of degree classes and the default split threshold, see alx_get_buckets */
+#define ALX_N_CLASSES 12
+#define ALX_DEFAULT_SPLIT 8192
+
+typedef void *(*alx_alloc_fn)(size_t bytes, void *user); /* returns a device pointer, 256-byte aligned, or NULL */
+typedef void (*alx_free_fn)(void *ptr, void *user);
+
+typedef struct alx_options {
+    int64_t n_rows, n_cols;  /* 1 <= n < 2^31 each */
+    int32_t d;               /* embedding dimension: 16, 32, 64 or 128 */
+    float lambda;            /* L2 weight of Eq. 3; must be > 0 (guarantees a unique minimiser) */
+    float alpha0;            /* weight of the all-pairs term of Eq. 3 (the paper's alpha); >= 0 */
+    int32_t storage;         /* alx_dtype of both tables.  ALX_BF16 follows Sec. 4.4 of the paper:
+                                tables in bfloat16, statistics and solve in float32, result rounded
+                                to nearest even on the way back */
+    int32_t device;          /* CUDA device ordinal, -1 = the current device */
+    void *stream;            /* cudaStream_t all work is ordered on; NULL = the legacy default stream */
+    alx_alloc_fn alloc;      /* device allocator; NULL => cudaMalloc */
+    alx_free_fn free;        /* NULL => cudaFree */
+    void *alloc_user;
+    int64_t split;           /* rows longer than this are cut into chunks of this many entries that
+                                different thread blocks accumulate; 0 => ALX_DEFAULT_SPLIT; >= 16 */
+    int32_t kernels;         /* 0 = best available for (d, storage); 1 = force the plain FP32-ALU
+                                kernels (reference path inside the library; every d, every storage) */
+    int32_t reserved;
+} alx_options;
+
+typedef struct alx_stats {
+    int64_t nnz;
+    int64_t rows_in_class[2][ALX_N_CLASSES]; /* [side][class] */
+    int64_t n_chunks[2];                     /* chunk descriptors of the split class, per side */
+    int64_t not_spd;                         /* rows whose factorisation met a non-positive pivot, so far */
+    double ms_gramian, ms_rows, ms_half_epoch; /* device time of the phases of the LAST half-epoch */
+    int64_t kernel_launches;                 /* kernels this context has launched so far */
+    int64_t workspace_bytes;                 /* device memory the context holds */
+    int32_t kernel_path[2];                  /* [side]: 0 = FP32-ALU kernels, 1 = tensor-core kernels */
+} alx_stats;
+
+/* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.
+   (Problem statement, Sec. 3: S subset of U x I x R, W in R^{U x d}, H in R^{I x d}.) */
+alx_status alx_create(int64_t n_rows, int64_t n_cols, int32_t d, float lambda, float alpha0, alx_ctx **out);
+alx_status alx_create_ex(const alx_options *opt, alx_ctx **out);
+alx_status alx_destroy(alx_ctx *ctx);
+
+/*
+ * Give the observed entries S (Sec. 3) as CSR over the matrix's rows:
+ * rowptr[n_rows + 1] (int64, rowptr[0] = 0, rowptr[n_rows] = nnz), colidx[nnz] (int32, strictly
+ * ascending inside each row: S is a set of pairs), values[nnz] (float labels y, or NULL: y = 1).
+ * The call copies the arrays, validates them on the device (ALX_ERR_BAD_CSR, never a trap), builds
+ * the transpose (CSC, row ids ascending inside each column; "a similar pass over the item side",
+ * Alg. 1 line 11, needs it), and for both orientations the degree-class order of the rows and the
+ * chunk descriptors of the rows longer than `split`.  Integer work only; synchronises.
+ */
+alx_status alx_set_csr(alx_ctx *ctx, const int64_t *rowptr, const int32_t *colidx, const float *values,
+                       int64_t nnz, int on_device);
+
+/* Overwrite one table from n x d row-major data of type src_dtype (converted with round-to-nearest-even). */
+alx_status alx_set_embeddings(alx_ctx *ctx, alx_side side, const void *src, alx_dtype src_dtype, int on_device);
+
+/*
+ * One half-epoch (Alg. 1 lines 2-10 for solved_side = ALX_ROWS; line 11 for ALX_COLS):
+ *   G <- X^T X over ALL rows of the fixed table X            (Alg. 1 line 2; Gramian remark under Eq. 4)
+ *   for every row u of the solved side:
+ *       b <- sum_{(u,i,y) in S} y x_i ;  A <- alpha0 G + lambda I + sum_{(u,i,y) in S} x_i (x) x_i
+ *       row u <- A^-1 b                                      (Eq. 4), rounded to the storage type
+ *   rows without observations become exactly 0.
+ * Asynchronous on the context's stream.
+ */
+alx_status alx_half_epoch(alx_ctx *ctx, alx_side solved_side);
+
+/* alx_half_epoch(ALX_ROWS) then alx_half_epoch(ALX_COLS): the column pass sees the new W (Alg. 1). */
+alx_status alx_epoch(alx_ctx *ctx);
+
+/*
+ * As alx_half_epoch, and additionally returns, for the k listed rows of the solved side, the
+ * float32 solution BEFORE it is rounded to the storage type (x_out: k x d floats, host memory).
+ * Used to check the residual |A x - b| / |b| of the solver itself.  Synchronises.
+ */
+alx_status alx_half_epoch_capture(alx_ctx *ctx, alx_side solved_side, const int64_t *row_ids, int64_t k,
+                                  float *x_out);
+
+/*
+ * The objective of Eq. 3 at the current tables:
+ *   components[0] = sum_S (y - <w_u, h_i>)^2
+ *   components[1] = alpha0 * sum_u sum_i <w_u, h_i>^2   (computed as <W^T W, H^T H>_F)
+ *   components[2] = lambda * (|W|_F^2 + |H|_F^2)
+ * total = their sum.  Products in float32, every accumulation across entries in float64 in a fixed
+ * order.  components may be NULL.  Synchronises.
+ */
+alx_status alx_loss(alx_ctx *ctx, double *total, double *components);
+
+/* Copy rows [row_begin, row_begin + row_count) of one table to dst (row_count x d, dst_dtype). Synchronises. */
+alx_status alx_get_embeddings(alx_ctx *ctx, alx_side side, void *dst, alx_dtype dst_dtype, int64_t row_begin,
+                              int64_t row_count, int on_device);
+
+/* ---- diagnostics used by tests and the benchmark ---- */
+
+/* The Gramian the last alx_half_epoch(solved = side) or alx_loss computed for the table of `fixed_side`
+   (d x d doubles, host).  ALX_ERR_BAD_STATE if none has been computed yet. */
+alx_status alx_get_gramian(alx_ctx *ctx, alx_side fixed_side, double *dst);
+/* Compute only the Gramian of one table now (the first step of a half-epoch) and return it. */
+alx_status alx_gramian(alx_ctx *ctx, alx_side table, double *dst);
+
+/* The transpose built by alx_set_csr: colptr[n_cols + 1], rowidx[nnz], values_t[nnz] (may be NULL). Host memory. */
+alx_status alx_get_transpose(alx_ctx *ctx, int64_t *colptr, int32_t *rowidx, float *values_t);
+
+/*
+ * The degree-class structure of one orientation (side = which table's rows are ordered).
+ *   class(deg) = 0 if deg = 0; ALX_N_CLASSES-1 if deg > split; otherwise the smallest c >= 1 with
+ *   deg <= 16 * 2^(c-1), capped at ALX_N_CLASSES-2.
+ *   order[n]              : row ids sorted by (class, id)
+ *   class_offsets[13]     : start of each class inside `order`
+ *   chunk_desc[4*n_chunks]: for the rows of the last class in ascending id, consecutive pieces of
+ *                           `split` entries (the last one shorter): row, begin, end, slot (int64 each)
+ * Pass NULL for arrays that are not wanted; *n_chunks (may be NULL) receives the descriptor count. Host memory.
+ */
+alx_status alx_get_buckets(alx_ctx *ctx, alx_side side, int32_t *order, int64_t *class_offsets,
+                           int64_t *chunk_desc, int64_t *n_chunks);
+
+alx_status alx_get_stats(alx_ctx *ctx, alx_stats *out);
+
+/* Wait for the context's stream and report any device-detected problem since the last check. */
+alx_status alx_synchronize(alx_ctx *ctx);
+
+/* Text of the last error on this context ("" if none).  Valid until the next call on the context. */
+const char *alx_last_error(const alx_ctx *ctx);
+
+/* Library version string, e.g. "alx-b200 0.1 (sm_100a)". */
+const char *alx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALX_H_ */

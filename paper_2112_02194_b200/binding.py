@@ -1,0 +1,266 @@
+"""Thin Python binding of the C ABI in ``include/alx.h``: argument marshalling only.
+
+Every step of the method runs inside ``libalx_b200.so``.  PyTorch is used here for device memory
+(the context's allocator callbacks hand out ``torch.empty`` buffers) and for the CUDA stream.
+Importing this module needs the built library; there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import (CFUNCTYPE, POINTER, Structure, byref, c_char_p, c_double, c_float, c_int, c_int32, c_int64,
+                    c_size_t, c_void_p)
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libalx_b200.so")
+
+ALX_OK = 0
+ALX_ROWS, ALX_COLS = 0, 1
+ALX_F32, ALX_BF16 = 0, 1
+ALX_N_CLASSES = 12
+ALX_DEFAULT_SPLIT = 8192
+STATUS_NAMES = ["ALX_OK", "ALX_ERR_INVALID_ARG", "ALX_ERR_BAD_STATE", "ALX_ERR_OOM", "ALX_ERR_CUDA",
+                "ALX_ERR_BAD_CSR", "ALX_ERR_NOT_SPD", "ALX_ERR_UNSUPPORTED"]
+
+ALLOC_FN = CFUNCTYPE(c_void_p, c_size_t, c_void_p)
+FREE_FN = CFUNCTYPE(None, c_void_p, c_void_p)
+
+
+class alx_options(Structure):
+    _fields_ = [("n_rows", c_int64), ("n_cols", c_int64), ("d", c_int32), ("lambda_", c_float),
+                ("alpha0", c_float), ("storage", c_int32), ("device", c_int32), ("stream", c_void_p),
+                ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_user", c_void_p), ("split", c_int64),
+                ("kernels", c_int32), ("reserved", c_int32)]
+
+
+class alx_stats(Structure):
+    _fields_ = [("nnz", c_int64), ("rows_in_class", (c_int64 * ALX_N_CLASSES) * 2), ("n_chunks", c_int64 * 2),
+                ("not_spd", c_int64), ("ms_gramian", c_double), ("ms_rows", c_double),
+                ("ms_half_epoch", c_double), ("kernel_launches", c_int64), ("workspace_bytes", c_int64),
+                ("kernel_path", c_int32 * 2)]
+
+
+EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_half_epoch",
+           "alx_epoch", "alx_half_epoch_capture", "alx_loss", "alx_get_embeddings", "alx_get_gramian",
+           "alx_gramian", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
+           "alx_last_error", "alx_version"]
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libalx_b200.so (built in-tree by ``build.py``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: run `python -m paper_2112_02194_b200.build` first "
+                          "(there is no CPU or library fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P = c_void_p
+    lib.alx_create.argtypes = [c_int64, c_int64, c_int32, c_float, c_float, POINTER(P)]
+    lib.alx_create_ex.argtypes = [POINTER(alx_options), POINTER(P)]
+    lib.alx_destroy.argtypes = [P]
+    lib.alx_set_csr.argtypes = [P, P, P, P, c_int64, c_int]
+    lib.alx_set_embeddings.argtypes = [P, c_int, P, c_int, c_int]
+    lib.alx_half_epoch.argtypes = [P, c_int]
+    lib.alx_epoch.argtypes = [P]
+    lib.alx_half_epoch_capture.argtypes = [P, c_int, P, c_int64, P]
+    lib.alx_loss.argtypes = [P, POINTER(c_double), POINTER(c_double)]
+    lib.alx_get_embeddings.argtypes = [P, c_int, P, c_int, c_int64, c_int64, c_int]
+    lib.alx_get_gramian.argtypes = [P, c_int, P]
+    lib.alx_gramian.argtypes = [P, c_int, P]
+    lib.alx_get_transpose.argtypes = [P, P, P, P]
+    lib.alx_get_buckets.argtypes = [P, c_int, P, P, P, POINTER(c_int64)]
+    lib.alx_get_stats.argtypes = [P, POINTER(alx_stats)]
+    lib.alx_synchronize.argtypes = [P]
+    lib.alx_last_error.argtypes = [P]
+    lib.alx_last_error.restype = c_char_p
+    lib.alx_version.restype = c_char_p
+    for name in EXPORTS:
+        if name not in ("alx_last_error", "alx_version"):
+            getattr(lib, name).restype = c_int
+    _lib = lib
+    return lib
+
+
+class AlxError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {message}")
+        self.status = status
+
+
+def _np_ptr(a):
+    return None if a is None else a.ctypes.data_as(c_void_p)
+
+
+class Alx:
+    """One context.  Methods carry the C names without the ``alx_`` prefix and only marshal arguments."""
+
+    def __init__(self, n_rows, n_cols, d, lam, alpha0, storage="f32", split=0, kernels=0, device=None,
+                 use_torch_allocator=True):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("alx needs a CUDA device (B200, sm_100a); there is no CPU path")
+        self.lib = load_library()
+        self.torch = torch
+        self.n_rows, self.n_cols, self.d = int(n_rows), int(n_cols), int(d)
+        self.storage = storage
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        self._buffers = {}
+        opt = alx_options()
+        opt.n_rows, opt.n_cols, opt.d = self.n_rows, self.n_cols, self.d
+        opt.lambda_, opt.alpha0 = lam, alpha0
+        opt.storage = ALX_BF16 if storage == "bf16" else ALX_F32
+        opt.device = self.device
+        opt.stream = torch.cuda.current_stream(self.device).cuda_stream
+        opt.split = split
+        opt.kernels = kernels
+        if use_torch_allocator:
+            dev = torch.device("cuda", self.device)
+
+            def _alloc(nbytes, _user):
+                try:
+                    t = torch.empty(int(nbytes), dtype=torch.uint8, device=dev)
+                except Exception:
+                    return None
+                self._buffers[t.data_ptr()] = t
+                return t.data_ptr()
+
+            def _free(ptr, _user):
+                self._buffers.pop(ptr, None)
+
+            self._alloc_cb, self._free_cb = ALLOC_FN(_alloc), FREE_FN(_free)
+            opt.alloc, opt.free = self._alloc_cb, self._free_cb
+        self._opt = opt
+        self.ctx = c_void_p()
+        st = self.lib.alx_create_ex(byref(opt), byref(self.ctx))
+        if st != ALX_OK:
+            raise AlxError(st, "alx_create_ex failed")
+
+    # -- helpers
+    def _check(self, st):
+        if st != ALX_OK:
+            raise AlxError(st, self.lib.alx_last_error(self.ctx).decode())
+
+    def _n(self, side):
+        return self.n_rows if side == ALX_ROWS else self.n_cols
+
+    def destroy(self):
+        if getattr(self, "ctx", None) is not None and self.ctx:
+            self.lib.alx_destroy(self.ctx)
+            self.ctx = None
+            self._buffers.clear()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    # -- the ABI
+    def set_csr(self, rowptr, colidx, values=None):
+        """numpy arrays (host) or torch CUDA tensors (device): int64 rowptr, int32 colidx, float32 values."""
+        torch = self.torch
+        if isinstance(rowptr, torch.Tensor):
+            assert rowptr.dtype == torch.int64 and colidx.dtype == torch.int32 and rowptr.is_cuda and colidx.is_cuda
+            assert rowptr.is_contiguous() and colidx.is_contiguous()
+            v = None
+            if values is not None:
+                assert values.dtype == torch.float32 and values.is_cuda and values.is_contiguous()
+                v = values.data_ptr()
+            self._check(self.lib.alx_set_csr(self.ctx, rowptr.data_ptr(), colidx.data_ptr(), v,
+                                             int(colidx.numel()), 1))
+        else:
+            rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+            colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+            v = None if values is None else np.ascontiguousarray(values, dtype=np.float32)
+            self._check(self.lib.alx_set_csr(self.ctx, _np_ptr(rowptr), _np_ptr(colidx), _np_ptr(v),
+                                             int(colidx.size), 0))
+
+    def set_embeddings(self, side, src, dtype=None):
+        """src: numpy float32 / uint16 (bf16 bit patterns) array, or a torch CUDA tensor (float32 / bfloat16)."""
+        torch = self.torch
+        if isinstance(src, torch.Tensor):
+            assert src.is_cuda and src.is_contiguous() and src.numel() == self._n(side) * self.d
+            dt = ALX_BF16 if src.dtype == torch.bfloat16 else ALX_F32
+            assert src.dtype in (torch.bfloat16, torch.float32)
+            self._check(self.lib.alx_set_embeddings(self.ctx, side, src.data_ptr(), dt, 1))
+        else:
+            src = np.ascontiguousarray(src)
+            assert src.size == self._n(side) * self.d
+            if src.dtype == np.uint16:
+                dt = ALX_BF16
+            else:
+                src = np.ascontiguousarray(src, dtype=np.float32)
+                dt = ALX_F32
+            self._check(self.lib.alx_set_embeddings(self.ctx, side, _np_ptr(src), dt, 0))
+
+    def half_epoch(self, side):
+        self._check(self.lib.alx_half_epoch(self.ctx, side))
+
+    def epoch(self):
+        self._check(self.lib.alx_epoch(self.ctx))
+
+    def half_epoch_capture(self, side, row_ids):
+        ids = np.ascontiguousarray(row_ids, dtype=np.int64)
+        out = np.empty((ids.size, self.d), dtype=np.float32)
+        self._check(self.lib.alx_half_epoch_capture(self.ctx, side, _np_ptr(ids), int(ids.size), _np_ptr(out)))
+        return out
+
+    def loss(self):
+        total = c_double()
+        comp = (c_double * 3)()
+        self._check(self.lib.alx_loss(self.ctx, byref(total), comp))
+        return total.value, (comp[0], comp[1], comp[2])
+
+    def get_embeddings(self, side, dtype="f32", row_begin=0, row_count=None, out=None):
+        """Host copy as numpy (float32, or uint16 bf16 bits); or into a torch CUDA tensor given as ``out``."""
+        if row_count is None:
+            row_count = self._n(side) - row_begin
+        if out is not None:
+            dt = ALX_BF16 if out.dtype == self.torch.bfloat16 else ALX_F32
+            assert out.is_cuda and out.is_contiguous() and out.numel() == row_count * self.d
+            self._check(self.lib.alx_get_embeddings(self.ctx, side, out.data_ptr(), dt, row_begin, row_count, 1))
+            return out
+        arr = np.empty((row_count, self.d), dtype=np.uint16 if dtype == "bf16" else np.float32)
+        self._check(self.lib.alx_get_embeddings(self.ctx, side, _np_ptr(arr), ALX_BF16 if dtype == "bf16" else ALX_F32,
+                                                row_begin, row_count, 0))
+        return arr
+
+    def gramian(self, table_side):
+        g = np.empty((self.d, self.d), dtype=np.float64)
+        self._check(self.lib.alx_gramian(self.ctx, table_side, _np_ptr(g)))
+        return g
+
+    def get_gramian(self, table_side):
+        g = np.empty((self.d, self.d), dtype=np.float64)
+        self._check(self.lib.alx_get_gramian(self.ctx, table_side, _np_ptr(g)))
+        return g
+
+    def get_transpose(self, nnz, with_values=False):
+        colptr = np.empty(self.n_cols + 1, dtype=np.int64)
+        rowidx = np.empty(nnz, dtype=np.int32)
+        vt = np.empty(nnz, dtype=np.float32) if with_values else None
+        self._check(self.lib.alx_get_transpose(self.ctx, _np_ptr(colptr), _np_ptr(rowidx), _np_ptr(vt)))
+        return colptr, rowidx, vt
+
+    def get_buckets(self, side):
+        n = self._n(side)
+        order = np.empty(n, dtype=np.int32)
+        offs = np.empty(ALX_N_CLASSES + 1, dtype=np.int64)
+        nch = c_int64()
+        self._check(self.lib.alx_get_buckets(self.ctx, side, None, None, None, byref(nch)))
+        desc = np.empty((nch.value, 4), dtype=np.int64)
+        self._check(self.lib.alx_get_buckets(self.ctx, side, _np_ptr(order), _np_ptr(offs), _np_ptr(desc), byref(nch)))
+        return order, offs, desc
+
+    def get_stats(self):
+        s = alx_stats()
+        self._check(self.lib.alx_get_stats(self.ctx, byref(s)))
+        return s
+
+    def synchronize(self):
+        self._check(self.lib.alx_synchronize(self.ctx))

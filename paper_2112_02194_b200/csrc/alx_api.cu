@@ -1,0 +1,603 @@
+// C ABI of the library (declared in include/alx.h): context, argument checks, device memory,
+// and the order in which the kernels of one half-epoch are launched.  No arithmetic of the method
+// happens on the host.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include "../../include/alx.h"
+#include "alx_common.cuh"
+
+using namespace alx;
+
+struct alx_ctx {
+    alx_options opt{};
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int bf16 = 0;
+    size_t elem = 4;
+    int64_t n[2] = {0, 0};   // n[ALX_ROWS] = n_rows, n[ALX_COLS] = n_cols
+    int64_t nnz = -1;
+    int64_t split = ALX_DEFAULT_SPLIT;
+    bool has_values = false;
+    bool have_table[2] = {false, false};
+    bool have_gram[2] = {false, false};
+
+    // per orientation: [ALX_ROWS] = CSR (rows of the matrix), [ALX_COLS] = CSC
+    int64_t *ptr[2] = {nullptr, nullptr};
+    int32_t *idx[2] = {nullptr, nullptr};
+    float *val[2] = {nullptr, nullptr};
+    int32_t *order[2] = {nullptr, nullptr};
+    int64_t *class_offs_dev[2] = {nullptr, nullptr};
+    int64_t class_offs[2][ALX_N_CLASSES + 1] = {};
+    int64_t *chunk_desc[2] = {nullptr, nullptr};
+    int64_t *split_first[2] = {nullptr, nullptr};
+    int64_t n_chunks[2] = {0, 0};
+    int64_t n_split_rows[2] = {0, 0};
+
+    void *table[2] = {nullptr, nullptr};
+    double *G64[2] = {nullptr, nullptr};   // Gramian of table [side]
+    float *Bmat = nullptr;
+    float *gram_partials = nullptr;
+    float *split_partials = nullptr;
+    double *loss_partials_buf = nullptr;
+    double *loss_result = nullptr;
+    DevStatus *status = nullptr;
+
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    alx_stats stats{};
+    int64_t launches = 0;
+    int64_t bytes_held = 0;
+    std::vector<std::pair<void *, size_t>> owned;
+    std::string err;
+};
+
+namespace {
+
+alx_status fail(alx_ctx *c, alx_status code, const char *fmt, ...)
+{
+    if (c) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        c->err = buf;
+    }
+    return code;
+}
+
+#define ALX_CUDA(c, expr)                                                                          \
+    do {                                                                                           \
+        cudaError_t e_ = (expr);                                                                   \
+        if (e_ != cudaSuccess)                                                                     \
+            return fail((c), e_ == cudaErrorMemoryAllocation ? ALX_ERR_OOM : ALX_ERR_CUDA,         \
+                        "%s failed: %s", #expr, cudaGetErrorString(e_));                           \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+void *dev_alloc(alx_ctx *c, size_t bytes)
+{
+    if (bytes == 0) bytes = 256;
+    void *p = nullptr;
+    if (c->opt.alloc) {
+        p = c->opt.alloc(bytes, c->opt.alloc_user);
+    } else if (cudaMalloc(&p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        p = nullptr;
+    }
+    if (p) {
+        c->owned.emplace_back(p, bytes);
+        c->bytes_held += (int64_t)bytes;
+    }
+    return p;
+}
+
+void dev_free(alx_ctx *c, void *p)
+{
+    if (!p) return;
+    for (size_t k = 0; k < c->owned.size(); ++k)
+        if (c->owned[k].first == p) {
+            c->bytes_held -= (int64_t)c->owned[k].second;
+            c->owned.erase(c->owned.begin() + k);
+            break;
+        }
+    if (c->opt.free) c->opt.free(p, c->opt.alloc_user); else cudaFree(p);
+}
+
+template <typename T> bool alloc_into(alx_ctx *c, T *&dst, size_t count)
+{
+    dst = static_cast<T *>(dev_alloc(c, count * sizeof(T)));
+    return dst != nullptr;
+}
+
+#define ALX_ALLOC(c, dst, count)                                                                   \
+    do {                                                                                           \
+        if (!alloc_into((c), (dst), (size_t)(count)))                                              \
+            return fail((c), ALX_ERR_OOM, "device allocation of %zu bytes failed",                 \
+                        (size_t)(count) * sizeof(*(dst)));                                         \
+    } while (0)
+
+// read and clear the device status word (after a stream synchronise)
+alx_status check_device_status(alx_ctx *c)
+{
+    DevStatus h;
+    ALX_CUDA(c, cudaMemcpyAsync(&h, c->status, sizeof h, cudaMemcpyDeviceToHost, c->stream));
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    c->stats.not_spd += (int64_t)h.not_spd;
+    if (h.flags == 0) return ALX_OK;
+    ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));
+    if (h.flags & kFlagBadRowptr) return fail(c, ALX_ERR_BAD_CSR, "rowptr is not a monotone offset array (near row %lld)", h.first_bad);
+    if (h.flags & kFlagBadCol) return fail(c, ALX_ERR_BAD_CSR, "column index out of range at entry %lld", h.first_bad);
+    if (h.flags & kFlagUnsorted) return fail(c, ALX_ERR_BAD_CSR, "column indices not strictly ascending inside a row at entry %lld", h.first_bad);
+    if (h.flags & kFlagNotSpd) return fail(c, ALX_ERR_NOT_SPD, "%llu rows met a non-positive pivot (first: row %lld); they were set to zero", h.not_spd, h.first_bad);
+    if (h.flags & kFlagTimeout) return fail(c, ALX_ERR_CUDA, "a bounded wait inside a kernel ran out (item %lld)", h.first_bad);
+    return fail(c, ALX_ERR_CUDA, "device status flags 0x%x", h.flags);
+}
+
+SideView side_view(const alx_ctx *c, int side)
+{
+    SideView v;
+    v.ptr = c->ptr[side];
+    v.idx = c->idx[side];
+    v.val = c->val[side];
+    v.order = c->order[side];
+    v.chunk_desc = c->chunk_desc[side];
+    v.split_first = c->split_first[side];
+    v.n = c->n[side];
+    return v;
+}
+
+// degree classes, order and chunk descriptors of one orientation
+alx_status build_buckets(alx_ctx *c, int side, int64_t *scratch_a, int64_t *scratch_b, int64_t *scan_scratch,
+                         int64_t scan_elems)
+{
+    const int64_t n = c->n[side];
+    ALX_CUDA(c, launch_bucket(c->ptr[side], n, c->split, scratch_a, scratch_b, scan_scratch, scan_elems,
+                              c->order[side], c->class_offs_dev[side], c->stream, &c->launches));
+    ALX_CUDA(c, cudaMemcpyAsync(c->class_offs[side], c->class_offs_dev[side], sizeof(int64_t) * (ALX_N_CLASSES + 1),
+                                cudaMemcpyDeviceToHost, c->stream));
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    const int64_t *offs = c->class_offs[side];
+    const int64_t n_split = offs[ALX_N_CLASSES] - offs[ALX_N_CLASSES - 1];
+    c->n_split_rows[side] = n_split;
+    c->n_chunks[side] = 0;
+    if (n_split > 0) {
+        int64_t *counts = nullptr;
+        ALX_ALLOC(c, counts, n_split);
+        ALX_ALLOC(c, c->split_first[side], n_split + 1);
+        const int32_t *split_rows = c->order[side] + offs[ALX_N_CLASSES - 1];
+        ALX_CUDA(c, launch_chunk_counts(c->ptr[side], split_rows, n_split, c->split, counts, c->stream, &c->launches));
+        ALX_CUDA(c, scan_exclusive(counts, true, c->split_first[side], n_split, scan_scratch, scan_elems, c->stream,
+                                   &c->launches));
+        int64_t total = 0;
+        ALX_CUDA(c, cudaMemcpyAsync(&total, c->split_first[side] + n_split, sizeof total, cudaMemcpyDeviceToHost, c->stream));
+        ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        c->n_chunks[side] = total;
+        ALX_ALLOC(c, c->chunk_desc[side], 4 * total);
+        ALX_CUDA(c, launch_chunk_fill(c->ptr[side], split_rows, n_split, c->split, c->split_first[side],
+                                      c->chunk_desc[side], c->stream, &c->launches));
+        ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        dev_free(c, counts);
+    }
+    for (int k = 0; k < ALX_N_CLASSES; ++k) c->stats.rows_in_class[side][k] = offs[k + 1] - offs[k];
+    c->stats.n_chunks[side] = c->n_chunks[side];
+    return ALX_OK;
+}
+
+void release_matrix(alx_ctx *c)
+{
+    for (int s = 0; s < 2; ++s) {
+        dev_free(c, c->ptr[s]); c->ptr[s] = nullptr;
+        dev_free(c, c->idx[s]); c->idx[s] = nullptr;
+        dev_free(c, c->val[s]); c->val[s] = nullptr;
+        dev_free(c, c->order[s]); c->order[s] = nullptr;
+        dev_free(c, c->chunk_desc[s]); c->chunk_desc[s] = nullptr;
+        dev_free(c, c->split_first[s]); c->split_first[s] = nullptr;
+    }
+    dev_free(c, c->split_partials); c->split_partials = nullptr;
+    dev_free(c, c->loss_partials_buf); c->loss_partials_buf = nullptr;
+    c->nnz = -1;
+}
+
+alx_status gramian_of(alx_ctx *c, int table_side)
+{
+    ALX_CUDA(c, launch_gramian(c->table[table_side], c->bf16, c->n[table_side], c->opt.d, c->gram_partials,
+                               c->G64[table_side], c->Bmat, c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
+    c->have_gram[table_side] = true;
+    return ALX_OK;
+}
+
+alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float *cap_out)
+{
+    if (c->nnz < 0) return fail(c, ALX_ERR_BAD_STATE, "alx_half_epoch before alx_set_csr");
+    const int fixed = 1 - side;
+    if (!c->have_table[fixed]) return fail(c, ALX_ERR_BAD_STATE, "the fixed table has not been set");
+    ALX_CUDA(c, cudaEventRecord(c->ev[0], c->stream));
+    alx_status st = gramian_of(c, fixed);
+    if (st != ALX_OK) return st;
+    ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
+    RowOut out{c->table[side], cap_slot, cap_out};
+    ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
+                                   c->table[fixed], c->bf16, c->opt.d, c->Bmat, c->split_partials, out, c->status,
+                                   c->stream, &c->launches));
+    c->stats.kernel_path[side] = 0;
+    ALX_CUDA(c, cudaEventRecord(c->ev[2], c->stream));
+    c->have_table[side] = true;
+    c->have_gram[side] = false;
+    return ALX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *alx_version(void) { return "alx-b200 0.1 (sm_100a)"; }
+
+const char *alx_last_error(const alx_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+alx_status alx_create(int64_t n_rows, int64_t n_cols, int32_t d, float lambda, float alpha0, alx_ctx **out)
+{
+    alx_options o;
+    memset(&o, 0, sizeof o);
+    o.n_rows = n_rows; o.n_cols = n_cols; o.d = d; o.lambda = lambda; o.alpha0 = alpha0;
+    o.storage = ALX_F32; o.device = -1;
+    return alx_create_ex(&o, out);
+}
+
+alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
+{
+    if (!opt || !out) return ALX_ERR_INVALID_ARG;
+    if (opt->n_rows < 1 || opt->n_cols < 1 || opt->n_rows >= (1ll << 31) || opt->n_cols >= (1ll << 31))
+        return ALX_ERR_INVALID_ARG;
+    if (opt->d != 16 && opt->d != 32 && opt->d != 64 && opt->d != 128) return ALX_ERR_UNSUPPORTED;
+    if (!(opt->lambda > 0.f)) return ALX_ERR_UNSUPPORTED;   // lambda = 0: minimiser not unique
+    if (!(opt->alpha0 >= 0.f)) return ALX_ERR_INVALID_ARG;
+    if (opt->storage != ALX_F32 && opt->storage != ALX_BF16) return ALX_ERR_INVALID_ARG;
+    if ((opt->alloc == nullptr) != (opt->free == nullptr)) return ALX_ERR_INVALID_ARG;
+    if (opt->split != 0 && opt->split < 16) return ALX_ERR_INVALID_ARG;
+    int dev = opt->device;
+    if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return ALX_ERR_CUDA;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || dev >= count) return ALX_ERR_CUDA;
+
+    alx_ctx *c = new (std::nothrow) alx_ctx();
+    if (!c) return ALX_ERR_OOM;
+    c->opt = *opt;
+    c->device = dev;
+    c->stream = static_cast<cudaStream_t>(opt->stream);
+    c->bf16 = opt->storage == ALX_BF16;
+    c->elem = c->bf16 ? 2 : 4;
+    c->n[ALX_ROWS] = opt->n_rows;
+    c->n[ALX_COLS] = opt->n_cols;
+    c->split = opt->split ? opt->split : ALX_DEFAULT_SPLIT;
+    DeviceGuard guard(dev);
+    auto body = [&]() -> alx_status {
+        const int d = opt->d;
+        for (int s = 0; s < 2; ++s) {
+            void *t = dev_alloc(c, (size_t)c->n[s] * d * c->elem);
+            if (!t) return fail(c, ALX_ERR_OOM, "device allocation of a %lld x %d table failed", (long long)c->n[s], d);
+            c->table[s] = t;
+            ALX_ALLOC(c, c->G64[s], d * d);
+            ALX_ALLOC(c, c->class_offs_dev[s], ALX_N_CLASSES + 1);
+        }
+        ALX_ALLOC(c, c->Bmat, d * d);
+        const int64_t nmax = c->n[0] > c->n[1] ? c->n[0] : c->n[1];
+        ALX_ALLOC(c, c->gram_partials, gramian_partials(nmax) * d * d);
+        ALX_ALLOC(c, c->loss_result, 4);
+        ALX_ALLOC(c, c->status, 1);
+        ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));
+        for (auto &e : c->ev) ALX_CUDA(c, cudaEventCreate(&e));
+        ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        return ALX_OK;
+    };
+    alx_status st = body();
+    if (st != ALX_OK) {
+        alx_destroy(c);
+        return st;
+    }
+    *out = c;
+    return ALX_OK;
+}
+
+alx_status alx_destroy(alx_ctx *c)
+{
+    if (!c) return ALX_OK;
+    DeviceGuard guard(c->device);
+    cudaStreamSynchronize(c->stream);
+    for (auto &e : c->ev) if (e) cudaEventDestroy(e);
+    std::vector<std::pair<void *, size_t>> owned = c->owned;
+    for (auto &p : owned) dev_free(c, p.first);
+    delete c;
+    return ALX_OK;
+}
+
+alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx, const float *values, int64_t nnz,
+                       int on_device)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!rowptr || nnz < 0 || (nnz > 0 && !colidx)) return fail(c, ALX_ERR_INVALID_ARG, "null array or negative nnz");
+    DeviceGuard guard(c->device);
+    release_matrix(c);
+    const int64_t n_rows = c->n[ALX_ROWS], n_cols = c->n[ALX_COLS];
+    const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    const size_t nz = (size_t)(nnz > 0 ? nnz : 1);
+    c->has_values = values != nullptr;
+    ALX_ALLOC(c, c->ptr[0], n_rows + 1);
+    ALX_ALLOC(c, c->idx[0], nz);
+    ALX_CUDA(c, cudaMemcpyAsync(c->ptr[0], rowptr, sizeof(int64_t) * (n_rows + 1), kind, c->stream));
+    if (nnz > 0) ALX_CUDA(c, cudaMemcpyAsync(c->idx[0], colidx, sizeof(int32_t) * nnz, kind, c->stream));
+    if (values) {
+        ALX_ALLOC(c, c->val[0], nz);
+        if (nnz > 0) ALX_CUDA(c, cudaMemcpyAsync(c->val[0], values, sizeof(float) * nnz, kind, c->stream));
+    }
+    // validate before anything indexes with these arrays
+    ALX_CUDA(c, launch_validate(c->ptr[0], c->idx[0], n_rows, n_cols, nnz, c->status, c->stream, &c->launches));
+    alx_status st = check_device_status(c);
+    if (st != ALX_OK) { release_matrix(c); return st; }
+    c->nnz = nnz;
+
+    // scratch shared by the scans and the bucket passes
+    const int64_t nmax = n_rows > n_cols ? n_rows : n_cols;
+    const int64_t nb = bucket_blocks(nmax);
+    const int64_t scan_elems = scan_scratch_elems(nb * kNClasses > nmax ? nb * kNClasses : nmax) + 16;
+    int64_t *scan_scratch = nullptr, *blk_counts = nullptr, *blk_offs = nullptr;
+    int32_t *counts = nullptr;
+    ALX_ALLOC(c, scan_scratch, scan_elems);
+    ALX_ALLOC(c, blk_counts, nb * kNClasses);
+    ALX_ALLOC(c, blk_offs, nb * kNClasses + 1);
+    ALX_ALLOC(c, counts, n_cols);
+
+    // transpose: count, prefix sum, degree classes of the columns, fill, sort each column, labels
+    ALX_ALLOC(c, c->ptr[1], n_cols + 1);
+    ALX_ALLOC(c, c->idx[1], nz);
+    ALX_CUDA(c, cudaMemsetAsync(counts, 0, sizeof(int32_t) * n_cols, c->stream));
+    ALX_CUDA(c, launch_count_cols(c->idx[0], nnz, counts, c->stream, &c->launches));
+    ALX_CUDA(c, scan_exclusive(counts, false, c->ptr[1], n_cols, scan_scratch, scan_elems, c->stream, &c->launches));
+    for (int s = 0; s < 2; ++s) ALX_ALLOC(c, c->order[s], c->n[s]);
+    st = build_buckets(c, ALX_COLS, blk_counts, blk_offs, scan_scratch, scan_elems);
+    if (st != ALX_OK) return st;
+    ALX_CUDA(c, cudaMemsetAsync(counts, 0, sizeof(int32_t) * n_cols, c->stream));
+    ALX_CUDA(c, launch_fill_transpose(c->ptr[0], c->idx[0], n_rows, nnz, c->ptr[1], counts, c->idx[1], c->stream,
+                                      &c->launches));
+    ALX_CUDA(c, launch_sort_segments(c->ptr[1], c->idx[1], c->order[1], c->class_offs[1], c->stream, &c->launches));
+    if (values) {
+        ALX_ALLOC(c, c->val[1], nz);
+        ALX_CUDA(c, launch_values_transpose(c->ptr[0], c->idx[0], c->val[0], c->ptr[1], c->idx[1], n_cols, nnz,
+                                            c->val[1], c->stream, &c->launches));
+    }
+    st = build_buckets(c, ALX_ROWS, blk_counts, blk_offs, scan_scratch, scan_elems);
+    if (st != ALX_OK) return st;
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    dev_free(c, counts);
+    dev_free(c, blk_offs);
+    dev_free(c, blk_counts);
+    dev_free(c, scan_scratch);
+
+    const int d = c->opt.d;
+    const int64_t max_chunks = c->n_chunks[0] > c->n_chunks[1] ? c->n_chunks[0] : c->n_chunks[1];
+    if (max_chunks > 0) ALX_ALLOC(c, c->split_partials, max_chunks * (int64_t)(d * d + d));
+    ALX_ALLOC(c, c->loss_partials_buf, loss_partials(nnz));
+    c->stats.nnz = nnz;
+    return ALX_OK;
+}
+
+alx_status alx_set_embeddings(alx_ctx *c, alx_side side, const void *src, alx_dtype src_dtype, int on_device)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!src || (side != ALX_ROWS && side != ALX_COLS) || (src_dtype != ALX_F32 && src_dtype != ALX_BF16))
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_set_embeddings");
+    DeviceGuard guard(c->device);
+    const int64_t count = c->n[side] * c->opt.d;
+    const size_t src_bytes = (size_t)count * (src_dtype == ALX_BF16 ? 2 : 4);
+    const void *dev_src = src;
+    void *staging = nullptr;
+    if (!on_device) {
+        if ((src_dtype == ALX_BF16) == (c->bf16 != 0)) {
+            ALX_CUDA(c, cudaMemcpyAsync(c->table[side], src, src_bytes, cudaMemcpyHostToDevice, c->stream));
+            ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+            c->have_table[side] = true;
+            c->have_gram[side] = false;
+            return ALX_OK;
+        }
+        staging = dev_alloc(c, src_bytes);
+        if (!staging) return fail(c, ALX_ERR_OOM, "staging allocation failed");
+        ALX_CUDA(c, cudaMemcpyAsync(staging, src, src_bytes, cudaMemcpyHostToDevice, c->stream));
+        dev_src = staging;
+    }
+    ALX_CUDA(c, launch_convert(dev_src, src_dtype == ALX_BF16, c->table[side], c->bf16, count, c->stream, &c->launches));
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (staging) dev_free(c, staging);
+    c->have_table[side] = true;
+    c->have_gram[side] = false;
+    return ALX_OK;
+}
+
+alx_status alx_get_embeddings(alx_ctx *c, alx_side side, void *dst, alx_dtype dst_dtype, int64_t row_begin,
+                              int64_t row_count, int on_device)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!dst || (side != ALX_ROWS && side != ALX_COLS) || (dst_dtype != ALX_F32 && dst_dtype != ALX_BF16) ||
+        row_begin < 0 || row_count < 0 || row_begin + row_count > c->n[side])
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_get_embeddings");
+    if (!c->have_table[side]) return fail(c, ALX_ERR_BAD_STATE, "table has not been set or solved yet");
+    DeviceGuard guard(c->device);
+    const int d = c->opt.d;
+    const int64_t count = row_count * d;
+    const char *src = static_cast<const char *>(c->table[side]) + (size_t)row_begin * d * c->elem;
+    const size_t dst_bytes = (size_t)count * (dst_dtype == ALX_BF16 ? 2 : 4);
+    const bool same = (dst_dtype == ALX_BF16) == (c->bf16 != 0);
+    if (on_device) {
+        ALX_CUDA(c, launch_convert(src, c->bf16, dst, dst_dtype == ALX_BF16, count, c->stream, &c->launches));
+    } else if (same) {
+        ALX_CUDA(c, cudaMemcpyAsync(dst, src, dst_bytes, cudaMemcpyDeviceToHost, c->stream));
+    } else {
+        void *staging = dev_alloc(c, dst_bytes);
+        if (!staging) return fail(c, ALX_ERR_OOM, "staging allocation failed");
+        ALX_CUDA(c, launch_convert(src, c->bf16, staging, dst_dtype == ALX_BF16, count, c->stream, &c->launches));
+        ALX_CUDA(c, cudaMemcpyAsync(dst, staging, dst_bytes, cudaMemcpyDeviceToHost, c->stream));
+        ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        dev_free(c, staging);
+    }
+    return check_device_status(c);
+}
+
+alx_status alx_half_epoch(alx_ctx *c, alx_side side)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (side != ALX_ROWS && side != ALX_COLS) return fail(c, ALX_ERR_INVALID_ARG, "bad side");
+    DeviceGuard guard(c->device);
+    return half_epoch_impl(c, side, nullptr, nullptr);
+}
+
+alx_status alx_epoch(alx_ctx *c)
+{
+    alx_status st = alx_half_epoch(c, ALX_ROWS);
+    if (st != ALX_OK) return st;
+    return alx_half_epoch(c, ALX_COLS);
+}
+
+alx_status alx_half_epoch_capture(alx_ctx *c, alx_side side, const int64_t *row_ids, int64_t k, float *x_out)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if ((side != ALX_ROWS && side != ALX_COLS) || k < 0 || (k > 0 && (!row_ids || !x_out)))
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_half_epoch_capture");
+    for (int64_t j = 0; j < k; ++j)
+        if (row_ids[j] < 0 || row_ids[j] >= c->n[side]) return fail(c, ALX_ERR_INVALID_ARG, "row id out of range");
+    DeviceGuard guard(c->device);
+    const int64_t n = c->n[side];
+    const int d = c->opt.d;
+    int32_t *slot = nullptr;
+    float *cap = nullptr;
+    ALX_ALLOC(c, slot, n);
+    ALX_ALLOC(c, cap, (k > 0 ? k : 1) * d);
+    std::vector<int32_t> h(n, -1);
+    for (int64_t j = 0; j < k; ++j) h[row_ids[j]] = (int32_t)j;   // a repeated id keeps its last slot
+    ALX_CUDA(c, cudaMemcpyAsync(slot, h.data(), sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream));
+    alx_status st = half_epoch_impl(c, side, slot, cap);
+    if (st == ALX_OK) {
+        std::vector<float> tmp((size_t)(k > 0 ? k : 1) * d);
+        ALX_CUDA(c, cudaMemcpyAsync(tmp.data(), cap, sizeof(float) * k * d, cudaMemcpyDeviceToHost, c->stream));
+        ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        for (int64_t j = 0; j < k; ++j)
+            memcpy(x_out + j * d, tmp.data() + (size_t)h[row_ids[j]] * d, sizeof(float) * d);
+        st = check_device_status(c);
+    } else {
+        cudaStreamSynchronize(c->stream);
+    }
+    dev_free(c, slot);
+    dev_free(c, cap);
+    return st;
+}
+
+alx_status alx_gramian(alx_ctx *c, alx_side table, double *dst)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!dst || (table != ALX_ROWS && table != ALX_COLS)) return fail(c, ALX_ERR_INVALID_ARG, "bad argument");
+    if (!c->have_table[table]) return fail(c, ALX_ERR_BAD_STATE, "table has not been set");
+    DeviceGuard guard(c->device);
+    alx_status st = gramian_of(c, table);
+    if (st != ALX_OK) return st;
+    return alx_get_gramian(c, table, dst);
+}
+
+alx_status alx_get_gramian(alx_ctx *c, alx_side side, double *dst)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!dst || (side != ALX_ROWS && side != ALX_COLS)) return fail(c, ALX_ERR_INVALID_ARG, "bad argument");
+    if (!c->have_gram[side]) return fail(c, ALX_ERR_BAD_STATE, "no Gramian of that table is current");
+    DeviceGuard guard(c->device);
+    const int d = c->opt.d;
+    ALX_CUDA(c, cudaMemcpyAsync(dst, c->G64[side], sizeof(double) * d * d, cudaMemcpyDeviceToHost, c->stream));
+    return check_device_status(c);
+}
+
+alx_status alx_loss(alx_ctx *c, double *total, double *components)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!total) return fail(c, ALX_ERR_INVALID_ARG, "null output");
+    if (c->nnz < 0) return fail(c, ALX_ERR_BAD_STATE, "alx_loss before alx_set_csr");
+    if (!c->have_table[0] || !c->have_table[1]) return fail(c, ALX_ERR_BAD_STATE, "both tables must be set");
+    DeviceGuard guard(c->device);
+    for (int s = 0; s < 2; ++s)
+        if (!c->have_gram[s]) {
+            alx_status st = gramian_of(c, s);
+            if (st != ALX_OK) return st;
+        }
+    ALX_CUDA(c, launch_loss_obs(c->ptr[0], c->idx[0], c->val[0], c->n[0], c->nnz, c->table[0], c->table[1], c->bf16,
+                                c->opt.d, c->loss_partials_buf, c->loss_result, c->stream, &c->launches));
+    ALX_CUDA(c, launch_loss_finish(c->loss_partials_buf, c->nnz > 0 ? loss_partials(c->nnz) : 0, c->G64[0], c->G64[1],
+                                   c->opt.d, (double)c->opt.alpha0, (double)c->opt.lambda, c->loss_result, c->stream,
+                                   &c->launches));
+    double h[3];
+    ALX_CUDA(c, cudaMemcpyAsync(h, c->loss_result, sizeof h, cudaMemcpyDeviceToHost, c->stream));
+    alx_status st = check_device_status(c);
+    if (st != ALX_OK) return st;
+    *total = h[0] + h[1] + h[2];
+    if (components) { components[0] = h[0]; components[1] = h[1]; components[2] = h[2]; }
+    return ALX_OK;
+}
+
+alx_status alx_get_transpose(alx_ctx *c, int64_t *colptr, int32_t *rowidx, float *values_t)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (c->nnz < 0) return fail(c, ALX_ERR_BAD_STATE, "alx_get_transpose before alx_set_csr");
+    DeviceGuard guard(c->device);
+    if (colptr) ALX_CUDA(c, cudaMemcpyAsync(colptr, c->ptr[1], sizeof(int64_t) * (c->n[1] + 1), cudaMemcpyDeviceToHost, c->stream));
+    if (rowidx && c->nnz > 0) ALX_CUDA(c, cudaMemcpyAsync(rowidx, c->idx[1], sizeof(int32_t) * c->nnz, cudaMemcpyDeviceToHost, c->stream));
+    if (values_t) {
+        if (!c->has_values) return fail(c, ALX_ERR_BAD_STATE, "the matrix was set without labels");
+        if (c->nnz > 0) ALX_CUDA(c, cudaMemcpyAsync(values_t, c->val[1], sizeof(float) * c->nnz, cudaMemcpyDeviceToHost, c->stream));
+    }
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ALX_OK;
+}
+
+alx_status alx_get_buckets(alx_ctx *c, alx_side side, int32_t *order, int64_t *class_offsets, int64_t *chunk_desc,
+                           int64_t *n_chunks)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (side != ALX_ROWS && side != ALX_COLS) return fail(c, ALX_ERR_INVALID_ARG, "bad side");
+    if (c->nnz < 0) return fail(c, ALX_ERR_BAD_STATE, "alx_get_buckets before alx_set_csr");
+    DeviceGuard guard(c->device);
+    if (order) ALX_CUDA(c, cudaMemcpyAsync(order, c->order[side], sizeof(int32_t) * c->n[side], cudaMemcpyDeviceToHost, c->stream));
+    if (class_offsets) memcpy(class_offsets, c->class_offs[side], sizeof(int64_t) * (ALX_N_CLASSES + 1));
+    if (n_chunks) *n_chunks = c->n_chunks[side];
+    if (chunk_desc && c->n_chunks[side] > 0)
+        ALX_CUDA(c, cudaMemcpyAsync(chunk_desc, c->chunk_desc[side], sizeof(int64_t) * 4 * c->n_chunks[side], cudaMemcpyDeviceToHost, c->stream));
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ALX_OK;
+}
+
+alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
+{
+    if (!c || !out) return ALX_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]) == cudaSuccess) c->stats.ms_gramian = ms; else cudaGetLastError();
+    if (cudaEventElapsedTime(&ms, c->ev[1], c->ev[2]) == cudaSuccess) c->stats.ms_rows = ms; else cudaGetLastError();
+    if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[2]) == cudaSuccess) c->stats.ms_half_epoch = ms; else cudaGetLastError();
+    c->stats.kernel_launches = c->launches;
+    c->stats.workspace_bytes = c->bytes_held;
+    *out = c->stats;
+    return ALX_OK;
+}
+
+alx_status alx_synchronize(alx_ctx *c)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    return check_device_status(c);
+}
+
+}  // extern "C"

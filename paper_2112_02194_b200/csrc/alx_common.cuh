@@ -1,0 +1,134 @@
+// Shared declarations of the CUDA side of the library: device status word, storage-type helpers,
+// launch descriptors.  Host entry points of each .cu file are declared at the bottom.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace alx {
+
+constexpr int kNClasses = 12;
+
+// bits of DevStatus::flags
+enum : unsigned {
+    kFlagBadRowptr = 1u,
+    kFlagBadCol = 2u,
+    kFlagUnsorted = 4u,
+    kFlagNotSpd = 8u,
+    kFlagTimeout = 16u,   // a bounded wait inside a kernel ran out
+    kFlagInternal = 32u,
+};
+
+struct DevStatus {
+    unsigned flags;
+    unsigned pad;
+    unsigned long long not_spd;   // rows whose factorisation met a non-positive pivot
+    long long first_bad;          // an offending position (entry or row) for error messages
+};
+
+__device__ __forceinline__ void raise_flag(DevStatus *st, unsigned f, long long where)
+{
+    unsigned old = atomicOr(&st->flags, f);
+    if (!(old & f)) st->first_bad = where;
+}
+
+// ---- storage types -------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void store_elem(float *p, float v) { *p = v; }
+__device__ __forceinline__ void store_elem(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+// 16-byte chunk of a table row -> floats (4 for fp32, 8 for bf16)
+template <typename T> struct Chunk16;
+template <> struct Chunk16<float> {
+    static constexpr int kElems = 4;
+    __device__ static __forceinline__ void load(const float *p, float *out)
+    {
+        float4 v = __ldg(reinterpret_cast<const float4 *>(p));
+        out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+    }
+};
+template <> struct Chunk16<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    __device__ static __forceinline__ void load(const __nv_bfloat16 *p, float *out)
+    {
+        uint4 v = __ldg(reinterpret_cast<const uint4 *>(p));
+        const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            out[2 * k] = __uint_as_float(w[k] << 16);
+            out[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        }
+    }
+};
+
+// ---- what a half-epoch hands to the row kernels -------------------------------------------
+struct SideView {
+    const int64_t *ptr;    // [n + 1] offsets of the solved side's rows
+    const int32_t *idx;    // [nnz] ids into the fixed table, ascending inside a row
+    const float *val;      // [nnz] labels or nullptr (all 1)
+    const int32_t *order;  // [n] rows by (class, id)
+    const int64_t *chunk_desc;   // [4 * n_chunks]
+    const int64_t *split_first;  // [n_split_rows + 1]
+    int64_t n;
+};
+
+struct RowOut {
+    void *table;             // solved table, storage type, row-major [n x d]
+    const int32_t *cap_slot; // nullptr, or per-row capture slot (-1 = none)
+    float *cap_out;          // [slots x d] fp32 solutions before rounding
+};
+
+// ---- host entry points (one per .cu) ----------------------------------------------------------
+struct ScanScratch;
+
+// alx_setup.cu
+cudaError_t scan_exclusive(const void *in, bool in_is_i64, int64_t *out, int64_t n, int64_t *scratch,
+                           int64_t scratch_elems, cudaStream_t s, int64_t *launches);
+int64_t scan_scratch_elems(int64_t n);
+cudaError_t launch_validate(const int64_t *rowptr, const int32_t *colidx, int64_t n_rows, int64_t n_cols,
+                            int64_t nnz, DevStatus *st, cudaStream_t s, int64_t *launches);
+cudaError_t launch_degrees(const int64_t *ptr, int64_t n, int32_t *deg, cudaStream_t s, int64_t *launches);
+cudaError_t launch_count_cols(const int32_t *colidx, int64_t nnz, int32_t *counts, cudaStream_t s, int64_t *launches);
+cudaError_t launch_fill_transpose(const int64_t *rowptr, const int32_t *colidx, int64_t n_rows, int64_t nnz,
+                                  const int64_t *colptr, int32_t *cursor, int32_t *rowidx, cudaStream_t s,
+                                  int64_t *launches);
+cudaError_t launch_sort_segments(const int64_t *colptr, int32_t *rowidx, const int32_t *order,
+                                 const int64_t *class_offs_host, cudaStream_t s, int64_t *launches);
+cudaError_t launch_values_transpose(const int64_t *rowptr, const int32_t *colidx, const float *values,
+                                    const int64_t *colptr, const int32_t *rowidx, int64_t n_cols, int64_t nnz,
+                                    float *values_t, cudaStream_t s, int64_t *launches);
+// order by (class, id): block_counts scratch is [kNClasses * n_blocks] int64 (+ scan scratch)
+int64_t bucket_blocks(int64_t n);
+cudaError_t launch_bucket(const int64_t *ptr, int64_t n, int64_t split, int64_t *block_counts,
+                          int64_t *block_offsets, int64_t *scan_scratch, int64_t scan_scratch_elems,
+                          int32_t *order, int64_t *class_offs_dev, cudaStream_t s, int64_t *launches);
+cudaError_t launch_chunk_counts(const int64_t *ptr, const int32_t *split_rows, int64_t n_split, int64_t split,
+                                int64_t *counts, cudaStream_t s, int64_t *launches);
+cudaError_t launch_chunk_fill(const int64_t *ptr, const int32_t *split_rows, int64_t n_split, int64_t split,
+                              const int64_t *first, int64_t *desc, cudaStream_t s, int64_t *launches);
+cudaError_t launch_convert(const void *src, int src_bf16, void *dst, int dst_bf16, int64_t count, cudaStream_t s,
+                           int64_t *launches);
+
+// alx_gramian.cu
+constexpr int kGramRowsPerPartial = 4096;
+int64_t gramian_partials(int64_t n);
+cudaError_t launch_gramian(const void *X, int bf16, int64_t n, int d, float *partials, double *G64, float *Bmat,
+                           float alpha0, float lambda, cudaStream_t s, int64_t *launches);
+
+// alx_rows.cu
+cudaError_t launch_rows_simple(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
+                               int64_t n_split_rows, const void *X, int bf16, int d, const float *Bmat,
+                               float *split_partials, RowOut out, DevStatus *st, cudaStream_t s,
+                               int64_t *launches);
+
+// alx_loss.cu
+int64_t loss_partials(int64_t nnz);
+cudaError_t launch_loss_obs(const int64_t *rowptr, const int32_t *colidx, const float *values, int64_t n_rows,
+                            int64_t nnz, const void *W, const void *H, int bf16, int d, double *partials,
+                            double *result, cudaStream_t s, int64_t *launches);
+cudaError_t launch_loss_finish(const double *partials, int64_t n_partials, const double *GW, const double *GH, int d,
+                               double alpha0, double lambda, double *result, cudaStream_t s, int64_t *launches);
+
+}  // namespace alx

@@ -1,0 +1,110 @@
+// Gramian of the fixed table, G = X^T X over all of its rows (Alg. 1 line 2; the remark under Eq. 4
+// that sum_i h_i (x) h_i does not depend on the row being solved), and the base matrix
+// alpha0 G + lambda I that every row's normal matrix starts from (Alg. 1 line 5).
+//
+// The table is cut into pieces of kGramRowsPerPartial rows (a function of the table size only); each
+// piece is summed in fp32 by one thread block, and the pieces are added in ascending order in fp64,
+// so the result does not depend on how blocks are scheduled.
+#include "alx_common.cuh"
+
+namespace alx {
+
+namespace {
+
+constexpr int kStageRows = 32;
+
+// FP32-ALU version: works for every d in {16, 32, 64, 128} and both storage types
+template <int D, typename T>
+__global__ void __launch_bounds__(256) k_gramian_simple(const T *__restrict__ X, int64_t n,
+                                                        float *__restrict__ partials)
+{
+    constexpr int TT = D / 16;
+    constexpr int LDS = D + 4;
+    constexpr int CH = D / Chunk16<T>::kElems;   // 16-byte chunks per row
+    __shared__ __align__(16) float hs[kStageRows * LDS];
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int64_t r0 = (int64_t)blockIdx.x * kGramRowsPerPartial;
+    const int64_t r1 = (r0 + kGramRowsPerPartial < n) ? r0 + kGramRowsPerPartial : n;
+    float acc[TT][TT];
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < TT; ++b) acc[a][b] = 0.f;
+
+    for (int64_t base = r0; base < r1; base += kStageRows) {
+        const int rc = (int)((r1 - base < kStageRows) ? r1 - base : kStageRows);
+        for (int pr = tid; pr < rc * CH; pr += 256) {
+            const int r = pr / CH, ch = pr % CH;
+            float v[Chunk16<T>::kElems];
+            Chunk16<T>::load(X + (base + r) * D + ch * Chunk16<T>::kElems, v);
+#pragma unroll
+            for (int k = 0; k < Chunk16<T>::kElems; ++k) hs[r * LDS + ch * Chunk16<T>::kElems + k] = v[k];
+        }
+        __syncthreads();
+        for (int r = 0; r < rc; ++r) {
+            float ai[TT], bl[TT];
+#pragma unroll
+            for (int a = 0; a < TT; ++a) ai[a] = hs[r * LDS + ty + 16 * a];
+#pragma unroll
+            for (int b = 0; b < TT; ++b) bl[b] = hs[r * LDS + tx + 16 * b];
+#pragma unroll
+            for (int a = 0; a < TT; ++a)
+#pragma unroll
+                for (int b = 0; b < TT; ++b) acc[a][b] = fmaf(ai[a], bl[b], acc[a][b]);
+        }
+        __syncthreads();
+    }
+    float *out = partials + (int64_t)blockIdx.x * D * D;
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < TT; ++b) out[(ty + 16 * a) * D + tx + 16 * b] = acc[a][b];
+}
+
+// pieces added in ascending order in fp64; also writes alpha0 G + lambda I in fp32
+__global__ void k_gramian_reduce(const float *__restrict__ partials, int64_t n_partials, int d,
+                                 double *__restrict__ G64, float *__restrict__ Bmat, float alpha0, float lambda)
+{
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= d * d) return;
+    double s = 0.0;
+    for (int64_t p = 0; p < n_partials; ++p) s += (double)partials[p * d * d + e];
+    G64[e] = s;
+    const int i = e / d, l = e % d;
+    Bmat[e] = (float)((double)alpha0 * s + (i == l ? (double)lambda : 0.0));
+}
+
+template <int D>
+cudaError_t gramian_simple_d(const void *X, int bf16, int64_t n, float *partials, cudaStream_t s)
+{
+    const unsigned grid = (unsigned)gramian_partials(n);
+    if (bf16)
+        k_gramian_simple<D, __nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)X, n, partials);
+    else
+        k_gramian_simple<D, float><<<grid, 256, 0, s>>>((const float *)X, n, partials);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int64_t gramian_partials(int64_t n) { return (n + kGramRowsPerPartial - 1) / kGramRowsPerPartial; }
+
+cudaError_t launch_gramian(const void *X, int bf16, int64_t n, int d, float *partials, double *G64, float *Bmat,
+                           float alpha0, float lambda, cudaStream_t s, int64_t *launches)
+{
+    cudaError_t e;
+    switch (d) {
+    case 16: e = gramian_simple_d<16>(X, bf16, n, partials, s); break;
+    case 32: e = gramian_simple_d<32>(X, bf16, n, partials, s); break;
+    case 64: e = gramian_simple_d<64>(X, bf16, n, partials, s); break;
+    case 128: e = gramian_simple_d<128>(X, bf16, n, partials, s); break;
+    default: return cudaErrorInvalidValue;
+    }
+    ++*launches;
+    if (e != cudaSuccess) return e;
+    k_gramian_reduce<<<(d * d + 255) / 256, 256, 0, s>>>(partials, gramian_partials(n), d, G64, Bmat, alpha0, lambda);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace alx

@@ -1,0 +1,255 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from oracle import ials
+from tests import problems
+
+pytestmark = pytest.mark.gpu
+
+ROWS, COLS = 0, 1
+
+
+def make_ctx(p, kernels=0):
+    from paper_2112_02194_b200 import Alx
+    a = Alx(p.n_rows, p.n_cols, p.d, p.lam, p.alpha, storage=p.storage, split=p.split, kernels=kernels)
+    a.set_csr(p.rowptr, p.colidx, p.values)
+    a.set_embeddings(ROWS, p.W0)
+    a.set_embeddings(COLS, p.H0)
+    return a
+
+
+def rel_fro(x, ref):
+    return np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-300)
+
+
+def row_rel(x, ref):
+    num = np.linalg.norm(x - ref, axis=1)
+    den = np.linalg.norm(ref, axis=1)
+    ok = den > 0
+    return num[ok] / den[ok]
+
+
+SUITE = problems.small_suite()
+IDS = ["tiny", "zipf_d64_f32", "local_d128_bf16", "split_d128_bf16", "split_d32_f32_labels", "alpha0_d16_bf16",
+       "default_split_d64_bf16"]
+
+
+@pytest.fixture(scope="module", params=list(range(len(SUITE))), ids=IDS)
+def prob(request):
+    return SUITE[request.param]()
+
+
+def test_transpose_and_buckets_bit_exact(prob):
+    p = prob
+    a = make_ctx(p)
+    split = p.split or ials.SPLIT
+    colptr, rowidx, vt = a.get_transpose(p.nnz, with_values=p.values is not None)
+    o_colptr, o_rowidx, o_vt = ials.transpose(p.n_rows, p.n_cols, p.rowptr, p.colidx, p.values)
+    np.testing.assert_array_equal(colptr, o_colptr)
+    np.testing.assert_array_equal(rowidx, o_rowidx)
+    if p.values is not None:
+        np.testing.assert_array_equal(vt, o_vt)
+    for side, ptr in ((ROWS, p.rowptr), (COLS, o_colptr)):
+        order, offs, desc = a.get_buckets(side)
+        o_order, o_offs = ials.bucket_rows(ptr, split=split)
+        o_desc, _ = ials.chunks(ptr, split=split)
+        np.testing.assert_array_equal(order, o_order)
+        np.testing.assert_array_equal(offs, o_offs)
+        np.testing.assert_array_equal(desc, o_desc)
+    a.destroy()
+
+
+def test_gramian_matches_oracle(prob):
+    p = prob
+    a = make_ctx(p)
+    for side, tab in ((ROWS, p.W0), (COLS, p.H0)):
+        G = a.gramian(side)
+        ref = ials.gramian(p.f64(tab))
+        assert np.abs(G - ref).max() <= 1e-6 * np.abs(ref).max()
+        np.testing.assert_array_equal(G, G.T)
+    a.destroy()
+
+
+def test_epoch_embeddings_residual_and_loss(prob):
+    p = prob
+    a = make_ctx(p)
+    W0, H0 = p.f64(p.W0), p.f64(p.H0)
+    colptr, rowidx, vt = ials.transpose(p.n_rows, p.n_cols, p.rowptr, p.colidx, p.values)
+    vals64 = None if p.values is None else p.values.astype(np.float64)
+    vt64 = None if vt is None else vt.astype(np.float64)
+
+    # loss at the initial tables: isolates the loss kernels
+    tot, comp = a.loss()
+    o_tot, o_comp = ials.loss(p.rowptr, p.colidx, vals64, W0, H0, p.alpha, p.lam)
+    np.testing.assert_allclose(comp, o_comp, rtol=1e-6, atol=1e-12 * o_tot)
+
+    # --- rows half-step, with the fp32 solutions before rounding captured for every row
+    ids = np.arange(p.n_rows, dtype=np.int64)
+    x32 = a.half_epoch_capture(ROWS, ids)
+    W_gpu = p.f64(a.get_embeddings(ROWS, dtype=p.storage))
+    G = ials.gramian(H0)
+    W_ref, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, G=G, return_raw=True)
+    assert rel_fro(W_gpu, W_ref) <= p.emb_tol
+    assert np.quantile(row_rel(W_gpu, W_ref), 0.999) <= 10 * p.emb_tol
+    deg = np.diff(p.rowptr)
+    assert np.all(W_gpu[deg == 0] == 0.0)
+    # residual gate |A x - b| / |b| <= 1e-4 on the solver's own fp32 solution, A and b rebuilt in fp64
+    worst = 0.0
+    check = np.unique(np.concatenate([np.argsort(deg)[-40:], np.arange(0, p.n_rows, max(1, p.n_rows // 150))]))
+    for u in check:
+        if deg[u] == 0:
+            assert np.all(x32[u] == 0)
+            continue
+        A, b = ials.row_system(p.rowptr, p.colidx, vals64, H0, G, p.alpha, p.lam, int(u))
+        worst = max(worst, np.linalg.norm(A @ x32[u].astype(np.float64) - b) / np.linalg.norm(b))
+    assert worst <= 1e-4, worst
+    assert rel_fro(x32.astype(np.float64), W_raw) <= 1e-3
+
+    # --- columns half-step on the GPU's own new W (trajectories may differ by storage rounding)
+    a.half_epoch(COLS)
+    H_gpu = p.f64(a.get_embeddings(COLS, dtype=p.storage))
+    H_ref_same = ials.half_step(colptr, rowidx, vt64, W_gpu, p.alpha, p.lam, p.storage)
+    assert rel_fro(H_gpu, H_ref_same) <= p.emb_tol
+    # and end to end against the oracle's own trajectory
+    H_ref = ials.half_step(colptr, rowidx, vt64, W_ref, p.alpha, p.lam, p.storage)
+    assert rel_fro(H_gpu, H_ref) <= p.emb_tol
+    cdeg = np.diff(colptr)
+    assert np.all(H_gpu[cdeg == 0] == 0.0)
+
+    # loss: kernel on the GPU's tables vs oracle on the same tables; and end to end
+    tot, comp = a.loss()
+    o_tot, o_comp = ials.loss(p.rowptr, p.colidx, vals64, W_gpu, H_gpu, p.alpha, p.lam)
+    assert abs(tot - o_tot) <= 1e-6 * o_tot
+    e_tot, _ = ials.loss(p.rowptr, p.colidx, vals64, W_ref, H_ref, p.alpha, p.lam)
+    assert abs(tot - e_tot) <= 1e-4 * e_tot
+    st = a.get_stats()
+    assert st.not_spd == 0 and st.nnz == p.nnz
+    a.destroy()
+
+
+def test_run_to_run_bitwise_determinism(prob):
+    p = prob
+    outs = []
+    for _ in range(2):
+        a = make_ctx(p)
+        a.epoch()
+        outs.append((a.get_embeddings(ROWS, dtype=p.storage).copy(), a.get_embeddings(COLS, dtype=p.storage).copy(),
+                     a.loss()[0]))
+        a.destroy()
+    np.testing.assert_array_equal(outs[0][0], outs[1][0])
+    np.testing.assert_array_equal(outs[0][1], outs[1][1])
+    assert outs[0][2] == outs[1][2]
+
+
+def test_three_epochs_loss_tracks_oracle_and_decreases():
+    p = SUITE[1]()            # d = 64, fp32: the shape of the "3 epochs with loss tracked" configuration
+    a = make_ctx(p)
+    W, H = p.f64(p.W0), p.f64(p.H0)
+    colptr, rowidx, vt = ials.transpose(p.n_rows, p.n_cols, p.rowptr, p.colidx, None)
+    prev = a.loss()[0]
+    for ep in range(3):
+        a.epoch()
+        W = ials.half_step(p.rowptr, p.colidx, None, H, p.alpha, p.lam, p.storage)
+        H = ials.half_step(colptr, rowidx, None, W, p.alpha, p.lam, p.storage)
+        tot = a.loss()[0]
+        ref = ials.loss(p.rowptr, p.colidx, None, W, H, p.alpha, p.lam)[0]
+        assert abs(tot - ref) <= 1e-4 * ref
+        assert tot <= prev * (1 + 1e-6)
+        prev = tot
+    a.destroy()
+
+
+def test_device_pointers_and_ranged_reads():
+    import torch
+    p = SUITE[2]()
+    from paper_2112_02194_b200 import Alx
+    a = Alx(p.n_rows, p.n_cols, p.d, p.lam, p.alpha, storage=p.storage)
+    dev = torch.device("cuda")
+    a.set_csr(torch.from_numpy(p.rowptr).to(dev), torch.from_numpy(p.colidx).to(dev))
+    H_t = torch.from_numpy(p.H0.view(np.int16)).to(dev).view(torch.bfloat16)
+    a.set_embeddings(COLS, H_t)
+    a.set_embeddings(ROWS, p.f64(p.W0).astype(np.float32))     # fp32 source into a bf16 table: converted
+    np.testing.assert_array_equal(a.get_embeddings(ROWS, dtype="bf16"), p.W0)
+    a.half_epoch(ROWS)
+    full = a.get_embeddings(ROWS, dtype="bf16")
+    part = a.get_embeddings(ROWS, dtype="bf16", row_begin=100, row_count=37)
+    np.testing.assert_array_equal(part, full[100:137])
+    out = torch.empty((37, p.d), dtype=torch.float32, device=dev)
+    a.get_embeddings(ROWS, row_begin=100, row_count=37, out=out)
+    np.testing.assert_array_equal(out.cpu().numpy(), p.f64(part).astype(np.float32))
+    b = make_ctx(p)
+    b.half_epoch(ROWS)
+    np.testing.assert_array_equal(b.get_embeddings(ROWS, dtype="bf16"), full)
+    a.destroy(); b.destroy()
+
+
+def test_error_paths_return_status_codes():
+    from paper_2112_02194_b200 import Alx, AlxError
+    with pytest.raises(AlxError) as e:
+        Alx(10, 10, 16, 0.0, 0.1)                       # lambda = 0: minimiser not unique
+    assert e.value.status == 7
+    with pytest.raises(AlxError) as e:
+        Alx(10, 10, 24, 0.1, 0.1)                       # unsupported d
+    assert e.value.status == 7
+    with pytest.raises(AlxError) as e:
+        Alx(0, 10, 16, 0.1, 0.1)
+    assert e.value.status == 1
+    a = Alx(4, 5, 16, 0.1, 0.1)
+    with pytest.raises(AlxError) as e:
+        a.half_epoch(ROWS)                              # before the matrix is set
+    assert e.value.status == 2
+    rowptr = np.array([0, 2, 2, 3, 5], dtype=np.int64)
+    good = np.array([0, 3, 1, 2, 4], dtype=np.int32)
+    for bad_cols, code in ((np.array([3, 0, 1, 2, 4], dtype=np.int32), 5),      # not ascending
+                           (np.array([0, 0, 1, 2, 4], dtype=np.int32), 5),      # duplicate
+                           (np.array([0, 5, 1, 2, 4], dtype=np.int32), 5),      # out of range
+                           (np.array([0, -1, 1, 2, 4], dtype=np.int32), 5)):
+        with pytest.raises(AlxError) as e:
+            a.set_csr(rowptr, bad_cols)
+        assert e.value.status == code
+    with pytest.raises(AlxError) as e:
+        a.set_csr(np.array([0, 3, 2, 3, 5], dtype=np.int64), good)             # rowptr not monotone
+    assert e.value.status == 5
+    a.set_csr(rowptr, good)                                                    # the context is still usable
+    with pytest.raises(AlxError) as e:
+        a.half_epoch(ROWS)                                                     # fixed table not set
+    assert e.value.status == 2
+    a.set_embeddings(COLS, np.ones((5, 16), dtype=np.float32))
+    a.half_epoch(ROWS)
+    w = a.get_embeddings(ROWS)
+    assert np.all(w[1] == 0) and np.all(np.isfinite(w))
+    with pytest.raises(AlxError):
+        a.get_embeddings(ROWS, row_begin=3, row_count=5)
+    a.destroy()
+
+
+def test_empty_matrix_gives_zero_tables():
+    from paper_2112_02194_b200 import Alx
+    a = Alx(7, 9, 32, 0.1, 0.01)
+    a.set_csr(np.zeros(8, dtype=np.int64), np.zeros(0, dtype=np.int32))
+    a.set_embeddings(ROWS, np.ones((7, 32), dtype=np.float32))
+    a.set_embeddings(COLS, np.ones((9, 32), dtype=np.float32))
+    a.epoch()
+    assert np.all(a.get_embeddings(ROWS) == 0) and np.all(a.get_embeddings(COLS) == 0)
+    assert a.loss()[0] == 0.0
+    a.destroy()
+
+
+def test_device_generators_match_numpy():
+    import torch
+    from synth import device, graphs
+    n = 20000
+    deg = graphs.zipf_degrees(n, 500000, 1.1, 6000, 5)
+    for spec in (graphs.GraphSpec(n, n, 9, law=graphs.LAW_LOCAL, delta=200),
+                 graphs.GraphSpec(n, n, 9, qtable=graphs.zipf_quantile_table(n, 1.1, 0.01)),
+                 graphs.GraphSpec(n, n - 777, 10)):
+        rowptr, colidx = graphs.build_csr(spec, deg)
+        rp_t, ci_t = device.device_csr(spec, deg)
+        np.testing.assert_array_equal(rp_t.cpu().numpy(), rowptr)
+        np.testing.assert_array_equal(ci_t.cpu().numpy(), colidx)
+    for storage in ("f32", "bf16"):
+        ref = graphs.init_embeddings(3000, 128, 7, 2, storage)
+        t = device.device_embeddings(3000, 128, 7, 2, storage)
+        got = t.view(torch.int16).cpu().numpy().view(np.uint16) if storage == "bf16" else t.cpu().numpy()
+        np.testing.assert_array_equal(got, ref)
