@@ -41,6 +41,12 @@ __global__ void __launch_bounds__(256) k_gramian_simple(const T *__restrict__ X,
             for (int k = 0; k < Chunk16<T>::kElems; ++k) hs[r * LDS + ch * Chunk16<T>::kElems + k] = v[k];
         }
         __syncthreads();
+        // two-level sum: a fresh accumulator per staged batch keeps the fp32 error near sqrt(rows) * 2^-24
+        float part[TT][TT];
+#pragma unroll
+        for (int a = 0; a < TT; ++a)
+#pragma unroll
+            for (int b = 0; b < TT; ++b) part[a][b] = 0.f;
         for (int r = 0; r < rc; ++r) {
             float ai[TT], bl[TT];
 #pragma unroll
@@ -50,8 +56,12 @@ __global__ void __launch_bounds__(256) k_gramian_simple(const T *__restrict__ X,
 #pragma unroll
             for (int a = 0; a < TT; ++a)
 #pragma unroll
-                for (int b = 0; b < TT; ++b) acc[a][b] = fmaf(ai[a], bl[b], acc[a][b]);
+                for (int b = 0; b < TT; ++b) part[a][b] = fmaf(ai[a], bl[b], part[a][b]);
         }
+#pragma unroll
+        for (int a = 0; a < TT; ++a)
+#pragma unroll
+            for (int b = 0; b < TT; ++b) acc[a][b] += part[a][b];
         __syncthreads();
     }
     float *out = partials + (int64_t)blockIdx.x * D * D;
