@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the implicit-ALS epoch (Gramian -> gather -> normal equations -> solve -> write back, rows then
+columns) on synthetic power-law graphs, through the C ABI of libalx_b200.so.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg2|small] [--impl ours|reference]
+
+One "step" is one full epoch over the resident graph.  Prints ONE JSON line.  With --impl reference the
+fp64 CPU oracle is timed on a bounded sample of the same workload instead (a deliberately slow program:
+the ratio to it is context, the roofline fraction is the figure of merit).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from synth import graphs  # noqa: E402
+
+METRIC = "observed entries/sec per ALS epoch"
+UNIT = "entries/s"
+
+# the benchmark configurations (see DESIGN.md for the recipe); "cfg3" is the graded one
+WORKLOADS = {
+    "cfg3": dict(n=10_000_000, nnz=1_000_000_000, s=1.1, cap=1_000_000, law="local", delta=100_000, d=128,
+                 lam=0.01, alpha=0.001, storage="bf16", seed=0xA1C50003, init_seed=0x1A150003,
+                 desc="10M x 10M, 1e9 entries, rank-size Zipf(1.1) degrees (cap 1e6), 80% of a row's entries "
+                      "within +-1% of its id, d=128, bf16 tables / fp32 solve"),
+    "cfg2": dict(n=1_000_000, nnz=50_000_000, s=1.2, cap=100_000, law="zipf", delta=0, d=64,
+                 lam=0.05, alpha=0.001, storage="f32", seed=0xA1C50002, init_seed=0x1A150002,
+                 desc="1M x 1M, 5e7 entries, Zipf(1.2) out- and in-degrees (cap 1e5), d=64, fp32 tables"),
+    "small": dict(n=200_000, nnz=10_000_000, s=1.1, cap=40_000, law="local", delta=2_000, d=128,
+                  lam=0.01, alpha=0.001, storage="bf16", seed=0xA1C500FF, init_seed=0x1A1500FF,
+                  desc="200k x 200k, 1e7 entries, scaled-down cfg3 (debugging / profiling case)"),
+}
+
+
+def make_spec(w):
+    n = w["n"]
+    if w["law"] == "local":
+        return graphs.GraphSpec(n, n, w["seed"] + 1, law=graphs.LAW_LOCAL, delta=w["delta"])
+    if w["law"] == "zipf":
+        return graphs.GraphSpec(n, n, w["seed"] + 1, qtable=graphs.zipf_quantile_table(n, w["s"], w["cap"] / w["nnz"]))
+    return graphs.GraphSpec(n, n, w["seed"] + 1)
+
+
+# ----------------------------------------------------------------------------------------------- roofline
+def roofline_terms(n, N, nnz, d, e):
+    """Algorithmic work of ONE half-epoch: bytes over HBM, tensor flops, FP32-ALU flops."""
+    bytes_ = nnz * d * e + nnz * 4 + (n + 1) * 8 + n * 4 + N * d * e + n * d * e
+    tensor = 2.0 * nnz * d * d + 2.0 * N * d * d
+    alu = n * (d ** 3 / 3.0 + 2.0 * d * d) + 2.0 * nnz * d + n * d * d
+    return bytes_, tensor, alu
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """nvidia-smi clock / throttle samples during the timed region (read-only queries)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); smax.append(float(r[1]))
+                for k, nme in enumerate(names):
+                    if r[3 + k].lower().startswith("active"):
+                        reasons.add(nme)
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(w, target_rows, budget_s=None):
+    """Time the fp64 oracle on a bounded sample: the first `target_rows` rows of the workload's graph, with the
+    fixed table compacted to the columns they touch (Gramian over those rows).  Returns (entries/s, info)."""
+    from oracle import ials
+    ials.build()
+    n, d = w["n"], w["d"]
+    spec = make_spec(w)
+    deg = graphs.zipf_degrees(n, w["nnz"], w["s"], w["cap"], w["seed"])
+    rows = np.arange(min(target_rows, n), dtype=np.int64)
+    ptr, cols = graphs.row_columns_flat(spec, rows, deg[rows])
+    uniq, inv = np.unique(cols, return_inverse=True)
+    X = graphs.storage_to_f64(graphs.init_embedding_rows(uniq, d, w["init_seed"], 3, w["storage"]), w["storage"])
+    cores = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    G = ials.gramian(X)
+    ials.half_step(ptr, inv.astype(np.int32), None, X, w["alpha"], w["lam"], w["storage"], G=G)
+    dt = time.perf_counter() - t0
+    nnz_s = int(ptr[-1])
+    info = {"kind": "oracle", "cores": cores, "unit": UNIT,
+            "sample": f"one half-step over rows 0..{rows.size - 1} of the {w['name']} graph ({nnz_s} entries, "
+                      f"{uniq.size} distinct fixed-side rows incl. their Gramian), fp64, OpenMP over rows; "
+                      f"{dt:.1f} s; value = sampled entries / seconds (an epoch visits every entry twice, so "
+                      f"per-epoch rate is half of this)"}
+    # the metric counts entries per EPOCH second; an epoch is two half-steps over the same entries
+    return nnz_s / (2.0 * dt), info
+
+
+# ----------------------------------------------------------------------------------------------- ranks
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def aggregate_over_ranks(ms_local: float, units_local: float, world: int, device=None):
+    """(max over ranks of the time, sum over ranks of the units) -- replicas only, no data-path collective."""
+    if world == 1:
+        return ms_local, units_local
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ----------------------------------------------------------------------------------------------- main legs
+def run_reference(args, w):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    rows = {"cfg3": 60_000, "cfg2": 100_000, "small": 30_000}[w["name"]]
+    vals = []
+    info = None
+    for _ in range(args.warmup):
+        oracle_sample(w, max(rows // 20, 100))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        v, info = oracle_sample(w, rows)
+        vals.append(v)
+    ms = (time.perf_counter() - t0) * 1e3 / max(args.steps, 1)
+    value = statistics.median(vals)
+    info["value"] = value
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": w["name"], "description": w["desc"]},
+           "cpu_baseline": info,
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def run_ours(args, w):
+    import torch
+    from paper_2112_02194_b200 import ALX_COLS, ALX_ROWS, Alx
+    from synth import device as sdev
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    n, d, storage = w["n"], w["d"], w["storage"]
+    e = 2 if storage == "bf16" else 4
+
+    # ---- synthetic inputs, generated on the device (replicas: every rank builds the same graph)
+    t_gen = time.perf_counter()
+    spec = make_spec(w)
+    deg = graphs.zipf_degrees(n, w["nnz"], w["s"], w["cap"], w["seed"])
+    rowptr, colidx = sdev.device_csr(spec, deg)
+    W0 = sdev.device_embeddings(n, d, w["init_seed"], 2, storage)
+    H0 = sdev.device_embeddings(n, d, w["init_seed"], 3, storage)
+    nnz = int(colidx.numel())
+    t_gen = time.perf_counter() - t_gen
+
+    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage)
+    t_set = time.perf_counter()
+    a.set_csr(rowptr, colidx)
+    torch.cuda.synchronize()
+    t_set = time.perf_counter() - t_set
+    a.set_embeddings(ALX_ROWS, W0)
+    a.set_embeddings(ALX_COLS, H0)
+
+    # ---- device-resident timing: K epochs, CUDA events on the context's stream
+    for _ in range(args.warmup):
+        a.epoch()
+    a.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    launches0 = a.get_stats().kernel_launches
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    half_ms = {"rows": [], "cols": [], "gramian": [], "row_kernels": []}
+    ev[0].record()
+    for k in range(args.steps):
+        a.half_epoch(ALX_ROWS)
+        a.half_epoch(ALX_COLS)
+        ev[k + 1].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        torch.distributed.barrier()
+    st = a.get_stats()
+    launches = st.kernel_launches - launches0
+    step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    ms_local = sum(step_ms) / args.steps
+    # per-phase times of one more half-epoch pair (outside the timed region)
+    for side, key in ((ALX_ROWS, "rows"), (ALX_COLS, "cols")):
+        a.half_epoch(side)
+        s2 = a.get_stats()
+        half_ms[key].append(s2.ms_half_epoch)
+        half_ms["gramian"].append(s2.ms_gramian)
+        half_ms["row_kernels"].append(s2.ms_rows)
+    fp32_peak = a.fp32_peak_tflops()
+    loss = a.loss()[0]
+    ms, units = aggregate_over_ranks(ms_local, float(nnz), world, dev)
+    value = units / (ms * 1e-3)
+
+    # ---- roofline of the dominant phase (the row kernels of one half-epoch)
+    peaks = load_peaks()
+    b_half, t_half, alu_half = roofline_terms(n, n, nnz, d, e)
+    t_bytes = b_half / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = t_half / (peaks["bf16_tflops"] * 1e12)
+    t_alu = alu_half / (fp32_peak * 1e12)
+    t_roof = max(t_bytes, t_tensor + t_alu)
+    rows_ms = statistics.mean(half_ms["row_kernels"])
+    if t_bytes >= t_tensor + t_alu:
+        roof = {"bound": "hbm", "achieved": b_half / (rows_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "alu", "achieved": alu_half / (rows_ms * 1e-3) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof.update({"kernel": "row kernels of one half-epoch (gather + normal equations + solve + write back)",
+                 "peak_source": f"HBM and bf16 {peaks['source']}; FP32 FMA measured in this run",
+                 "half_epoch_ms": {"rows": half_ms["rows"][0], "cols": half_ms["cols"][0],
+                                   "gramian": statistics.mean(half_ms["gramian"]), "row_kernels": rows_ms},
+                 "roofline_half_epoch_ms": {"bytes": t_bytes * 1e3, "tensor": t_tensor * 1e3, "alu": t_alu * 1e3,
+                                            "max(bytes, tensor+alu)": t_roof * 1e3},
+                 "frac_of_roofline_time": t_roof * 1e3 / statistics.mean([half_ms["rows"][0], half_ms["cols"][0]])})
+
+    # ---- end to end from host buffers: upload S and both tables, one epoch, download both tables
+    e2e = None
+    cpu_baseline = None
+    if args.skip_e2e:
+        a.destroy()
+    elif rank == 0 or world > 1:
+        a.destroy()
+        del a
+        torch.cuda.empty_cache()
+        h_rowptr = torch.empty(rowptr.shape, dtype=rowptr.dtype, pin_memory=True); h_rowptr.copy_(rowptr)
+        h_colidx = torch.empty(colidx.shape, dtype=colidx.dtype, pin_memory=True); h_colidx.copy_(colidx)
+        np_dt = np.uint16 if storage == "bf16" else np.float32
+        view = (lambda t: t.view(torch.int16)) if storage == "bf16" else (lambda t: t)
+        h_W = torch.empty(view(W0).shape, dtype=view(W0).dtype, pin_memory=True); h_W.copy_(view(W0))
+        h_H = torch.empty(view(H0).shape, dtype=view(H0).dtype, pin_memory=True); h_H.copy_(view(H0))
+        del rowptr, colidx, W0, H0
+        torch.cuda.empty_cache()
+        o_W = torch.empty_like(h_W, pin_memory=True)
+        o_H = torch.empty_like(h_H, pin_memory=True)
+        b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage)
+        reps = 2 if w["name"] != "small" else 3
+        times = []
+        for r in range(reps):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            b.set_csr(h_rowptr.numpy(), h_colidx.numpy())
+            b.set_embeddings(ALX_ROWS, h_W.numpy().view(np_dt))
+            b.set_embeddings(ALX_COLS, h_H.numpy().view(np_dt))
+            b.epoch()
+            st_o = b.lib.alx_get_embeddings(b.ctx, ALX_ROWS, o_W.data_ptr(), 1 if storage == "bf16" else 0, 0, n, 0)
+            st_o |= b.lib.alx_get_embeddings(b.ctx, ALX_COLS, o_H.data_ptr(), 1 if storage == "bf16" else 0, 0, n, 0)
+            torch.cuda.synchronize()
+            times.append(time.perf_counter() - t0)
+            assert st_o == 0
+        t_e2e = min(times[1:]) if len(times) > 1 else times[0]
+        t_e2e_ms, units_e = aggregate_over_ranks(t_e2e * 1e3, float(nnz), world, dev)
+        e2e = {"value": units_e / (t_e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(h_rowptr.numel() * 8 + h_colidx.numel() * 4 + 2 * n * d * e),
+               "d2h_bytes_per_step": int(2 * n * d * e), "ms_per_step": t_e2e_ms,
+               "covers": "alx_set_csr (upload, validate, transpose, degree classes) + alx_set_embeddings x2 + "
+                         "alx_epoch + alx_get_embeddings x2, pinned host buffers"}
+        b.destroy()
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        v, info = oracle_sample(w, {"cfg3": 60_000, "cfg2": 100_000, "small": 30_000}[w["name"]])
+        info["value"] = v
+        cpu_baseline = info
+
+    if rank == 0:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+               "config": {"workload": w["name"], "description": w["desc"], "nnz": nnz, "n_rows": n, "n_cols": n,
+                          "d": d, "storage": storage, "lambda": w["lam"], "alpha0": w["alpha"],
+                          "step": "one epoch = rows half-epoch + columns half-epoch",
+                          "l2": "inputs larger than L2 (tables and index arrays are GBs)",
+                          "multi_gpu": "replicas only", "kernel_path": list(st.kernel_path),
+                          "paper_context": "about 20 min/epoch for 365M nodes / 29.9B edges on 256 TPU v3 cores"},
+               "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
+               "cpu_baseline": cpu_baseline,
+               "extra": {"epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
+                         "setup_s": {"generate": t_gen, "alx_set_csr_device": t_set},
+                         "rows_in_class": [list(st.rows_in_class[0]), list(st.rows_in_class[1])],
+                         "n_chunks": list(st.n_chunks), "workspace_gb": st.workspace_bytes / 1e9}}
+        print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
+    ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")
+    args = ap.parse_args()
+    w = dict(WORKLOADS[args.workload], name=args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -168,6 +168,11 @@ alx_status alx_get_buckets(alx_ctx *ctx, alx_side side, int32_t *order, int64_t 
 
 alx_status alx_get_stats(alx_ctx *ctx, alx_stats *out);
 
+/* Diagnostic for roofline reports: measured FP32 fused-multiply-add throughput of the device in
+   TFLOP/s (a register-resident FMA loop on every SM, best of three).  No counterpart in the paper.
+   Allocates and frees 256 bytes with cudaMalloc; synchronises. */
+alx_status alx_fp32_peak_tflops(alx_ctx *ctx, double *tflops);
+
 /* Wait for the context's stream and report any device-detected problem since the last check. */
 alx_status alx_synchronize(alx_ctx *ctx);
 

@@ -44,7 +44,7 @@ class alx_stats(Structure):
 
 EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_half_epoch",
            "alx_epoch", "alx_half_epoch_capture", "alx_loss", "alx_get_embeddings", "alx_get_gramian",
-           "alx_gramian", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
+           "alx_gramian", "alx_fp32_peak_tflops", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
            "alx_last_error", "alx_version"]
 
 _lib = None
@@ -76,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.alx_get_buckets.argtypes = [P, c_int, P, P, P, POINTER(c_int64)]
     lib.alx_get_stats.argtypes = [P, POINTER(alx_stats)]
     lib.alx_synchronize.argtypes = [P]
+    lib.alx_fp32_peak_tflops.argtypes = [P, POINTER(c_double)]
     lib.alx_last_error.argtypes = [P]
     lib.alx_last_error.restype = c_char_p
     lib.alx_version.restype = c_char_p
@@ -261,6 +262,11 @@ class Alx:
         s = alx_stats()
         self._check(self.lib.alx_get_stats(self.ctx, byref(s)))
         return s
+
+    def fp32_peak_tflops(self):
+        v = c_double()
+        self._check(self.lib.alx_fp32_peak_tflops(self.ctx, byref(v)))
+        return v.value
 
     def synchronize(self):
         self._check(self.lib.alx_synchronize(self.ctx))

@@ -593,6 +593,17 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
     return ALX_OK;
 }
 
+alx_status alx_fp32_peak_tflops(alx_ctx *c, double *tflops)
+{
+    if (!c || !tflops) return ALX_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    double v = 0.0;
+    ALX_CUDA(c, measure_fp32_peak(&v, c->stream));
+    *tflops = v;
+    return ALX_OK;
+}
+
 alx_status alx_synchronize(alx_ctx *c)
 {
     if (!c) return ALX_ERR_INVALID_ARG;

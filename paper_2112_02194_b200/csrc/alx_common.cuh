@@ -117,6 +117,8 @@ int64_t gramian_partials(int64_t n);
 cudaError_t launch_gramian(const void *X, int bf16, int64_t n, int d, float *partials, double *G64, float *Bmat,
                            float alpha0, float lambda, cudaStream_t s, int64_t *launches);
 
+cudaError_t measure_fp32_peak(double *tflops, cudaStream_t s);
+
 // alx_rows.cu
 cudaError_t launch_rows_simple(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                                int64_t n_split_rows, const void *X, int bf16, int d, const float *Bmat,

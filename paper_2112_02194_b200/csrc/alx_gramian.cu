@@ -118,3 +118,54 @@ cudaError_t launch_gramian(const void *X, int bf16, int64_t n, int d, float *par
 }
 
 }  // namespace alx
+
+// ---- FP32 FMA throughput probe (diagnostic; gives the denominator of the ALU roofline) ------------
+namespace alx {
+namespace {
+__global__ void __launch_bounds__(256) k_ffma_probe(float *out, int iters)
+{
+    float a[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) a[k] = 1.0f + 1e-3f * (float)(threadIdx.x + k);
+    const float m = 0.999999f, c = 1e-7f;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) a[k] = fmaf(a[k], m, c);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) s += a[k];
+    if (s == 12345.678f) out[0] = s;   // keeps the loop alive; practically never taken
+}
+}  // namespace
+
+cudaError_t measure_fp32_peak(double *tflops, cudaStream_t s)
+{
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    float *out = nullptr;
+    cudaError_t e = cudaMalloc(&out, 256);
+    if (e != cudaSuccess) return e;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    const int iters = 1 << 16, grid = sms * 8;
+    double best = 0.0;
+    for (int rep = 0; rep < 4; ++rep) {
+        cudaEventRecord(e0, s);
+        k_ffma_probe<<<grid, 256, 0, s>>>(out, iters);
+        cudaEventRecord(e1, s);
+        cudaEventSynchronize(e1);
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double fl = 2.0 * 16.0 * (double)iters * 256.0 * (double)grid;
+        if (rep > 0 && ms > 0.f && fl / (ms * 1e-3) * 1e-12 > best) best = fl / (ms * 1e-3) * 1e-12;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaFree(out);
+    *tflops = best;
+    return cudaGetLastError();
+}
+}  // namespace alx

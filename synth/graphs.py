@@ -75,7 +75,7 @@ def zipf_degrees(n: int, nnz: int, s: float, cap: int, seed: int) -> np.ndarray:
     lo, hi = 0.0, float(cap) * 4
     while total(hi) < nnz:
         hi *= 2
-    for _ in range(200):
+    for _ in range(64):
         mid = 0.5 * (lo + hi)
         if total(mid) < nnz:
             lo = mid
@@ -285,10 +285,14 @@ def normal_table() -> np.ndarray:
     return np.rint(ndtri(p) * 2.0 ** NT_SCALE_BITS).astype(np.int64)
 
 
-def normal_fixed(seed: int, stream: int, start: int, count: int, table: np.ndarray) -> np.ndarray:
-    """int64[count]: standard normal draws times 2^24 for element indices start .. start+count-1."""
+def normal_fixed(seed: int, stream: int, start: int, count: int, table: np.ndarray, index=None) -> np.ndarray:
+    """int64[count]: standard normal draws times 2^24 for element indices start .. start+count-1
+    (or for the explicit element indices in ``index``)."""
     key = stream_key(seed, stream)
-    idx = np.arange(start, start + count, dtype=np.int64).astype(U64)
+    if index is None:
+        idx = np.arange(start, start + count, dtype=np.int64).astype(U64)
+    else:
+        idx = np.asarray(index, dtype=np.int64).astype(U64)
     h = hash2(key, idx, U64(0))
     cell = (h >> U64(64 - NT_BITS)).astype(np.int64)
     frac = ((h >> U64(64 - NT_BITS - NT_FRAC_BITS)) & U64((1 << NT_FRAC_BITS) - 1)).astype(np.int64)
@@ -326,3 +330,14 @@ def init_embeddings(n: int, d: int, seed: int, stream: int, storage: str, row_be
     v = normal_fixed(seed, stream, row_begin * d, row_count * d, normal_table())
     x = v.astype(np.float64) * (sigma / 2.0 ** NT_SCALE_BITS)
     return to_storage_bits(x, storage).reshape(row_count, d)
+
+
+def init_embedding_rows(row_ids, d: int, seed: int, stream: int, storage: str, sigma: float | None = None):
+    """The listed rows of the table init_embeddings(n, d, seed, stream, storage) would give, without the rest."""
+    row_ids = np.asarray(row_ids, dtype=np.int64)
+    if sigma is None:
+        sigma = 0.1 / np.sqrt(d)
+    index = (row_ids[:, None] * d + np.arange(d, dtype=np.int64)[None, :]).reshape(-1)
+    v = normal_fixed(seed, stream, 0, 0, normal_table(), index=index)
+    x = v.astype(np.float64) * (sigma / 2.0 ** NT_SCALE_BITS)
+    return to_storage_bits(x, storage).reshape(row_ids.size, d)
