@@ -179,6 +179,31 @@ alx_status alx_synchronize(alx_ctx *ctx);
 /* Text of the last error on this context ("" if none).  Valid until the next call on the context. */
 const char *alx_last_error(const alx_ctx *ctx);
 
+/*
+ * Gramian of a table without allocating anything (the paper has no counterpart; this is an addition for
+ * callers that cannot allocate device memory when they call: inside a frozen memory pool, on a thread
+ * that must not take an allocator lock, under a memory budget fixed at start-up).
+ *   table   : device pointer, n x d row-major, float32 or bfloat16 (dtype)
+ *   gramian : device pointer, d x d doubles, receives table^T table; written on `stream` (cudaStream_t,
+ *             NULL = legacy default stream); the call does not synchronise
+ * Same kernels and the same fixed summation order as alx_gramian, so the results agree to the last bit.
+ * The piece sums go to a fixed array inside the library image (16 MiB + 64 KiB on every GPU that loads
+ * the library, held until the process exits).  Limits: d in {16, 32, 64, 128} and
+ * n <= alx_gramian_noalloc_max_rows(d) = (4 Mi / d^2) * 4096 rows (1 048 576 for d = 128); larger inputs
+ * are refused with ALX_ERR_UNSUPPORTED and a message in alx_noalloc_last_error().  No cudaMalloc, cudaFree
+ * or other allocating routine is called.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
+ * device current; make that first call outside any stream capture.  The device that owns `table` must be
+ * the current device.  All calls share the one array and it keeps the previous call's contents (each call
+ * overwrites every piece it later reads, so nothing needs clearing): two calls whose kernels overlap on
+ * the GPU -- different streams, or different host threads -- race; order them on one stream.
+ */
+alx_status alx_gramian_noalloc(const void *table, alx_dtype dtype, int64_t n, int32_t d, double *gramian,
+                               void *stream);
+int64_t alx_gramian_noalloc_max_rows(int32_t d);
+/* Message of the calling thread's last failed alx_gramian_noalloc ("" after a success). */
+const char *alx_noalloc_last_error(void);
+
 /* Library version string, e.g. "alx-b200 0.1 (sm_100a)". */
 const char *alx_version(void);
 

@@ -45,7 +45,8 @@ class alx_stats(Structure):
 EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_half_epoch",
            "alx_epoch", "alx_half_epoch_capture", "alx_loss", "alx_get_embeddings", "alx_get_gramian",
            "alx_gramian", "alx_fp32_peak_tflops", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
-           "alx_last_error", "alx_version"]
+           "alx_last_error", "alx_version", "alx_gramian_noalloc", "alx_gramian_noalloc_max_rows",
+           "alx_noalloc_last_error"]
 
 _lib = None
 
@@ -80,8 +81,12 @@ def load_library() -> ctypes.CDLL:
     lib.alx_last_error.argtypes = [P]
     lib.alx_last_error.restype = c_char_p
     lib.alx_version.restype = c_char_p
+    lib.alx_gramian_noalloc.argtypes = [P, c_int, c_int64, c_int32, P, P]
+    lib.alx_gramian_noalloc_max_rows.argtypes = [c_int32]
+    lib.alx_gramian_noalloc_max_rows.restype = c_int64
+    lib.alx_noalloc_last_error.restype = c_char_p
     for name in EXPORTS:
-        if name not in ("alx_last_error", "alx_version"):
+        if name not in ("alx_last_error", "alx_version", "alx_gramian_noalloc_max_rows", "alx_noalloc_last_error"):
             getattr(lib, name).restype = c_int
     _lib = lib
     return lib
@@ -270,3 +275,23 @@ class Alx:
 
     def synchronize(self):
         self._check(self.lib.alx_synchronize(self.ctx))
+
+
+def gramian_noalloc(table, out):
+    """``alx_gramian_noalloc``: table^T table of a CUDA tensor (n x d, float32 or bfloat16) into ``out``
+    (a d x d float64 CUDA tensor the caller owns), on the current stream, without any allocation by the
+    library.  For callers that may not allocate at call time; see include/alx.h for the limits."""
+    import torch
+    lib = load_library()
+    assert table.is_cuda and table.is_contiguous() and table.dim() == 2
+    assert out.is_cuda and out.is_contiguous() and out.dtype == torch.float64 and out.numel() == table.shape[1] ** 2
+    dt = ALX_BF16 if table.dtype == torch.bfloat16 else ALX_F32
+    st = lib.alx_gramian_noalloc(table.data_ptr(), dt, table.shape[0], table.shape[1], out.data_ptr(),
+                                 torch.cuda.current_stream().cuda_stream)
+    if st != ALX_OK:
+        raise AlxError(st, lib.alx_noalloc_last_error().decode())
+    return out
+
+
+def gramian_noalloc_max_rows(d: int) -> int:
+    return int(load_library().alx_gramian_noalloc_max_rows(d))

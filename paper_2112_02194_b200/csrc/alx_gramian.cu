@@ -5,6 +5,10 @@
 // The table is cut into pieces of kGramRowsPerPartial rows (a function of the table size only); each
 // piece is summed in fp32 by one thread block, and the pieces are added in ascending order in fp64,
 // so the result does not depend on how blocks are scheduled.
+#include <mutex>
+#include <string>
+
+#include "../../include/alx.h"
 #include "alx_common.cuh"
 
 namespace alx {
@@ -169,3 +173,95 @@ cudaError_t measure_fp32_peak(double *tflops, cudaStream_t s)
     return cudaGetLastError();
 }
 }  // namespace alx
+
+// ---- Gramian without any allocation ---------------------------------------------------------------
+// For callers that must not allocate device memory at the time of the call: code running inside a
+// memory pool that has been frozen, a host thread that may not take the allocator's lock, a service
+// whose memory budget was fixed at start-up.  The piece sums that the context-based path keeps in a
+// buffer it allocates live here in a fixed array that is part of the library image, so every GPU that
+// loads the library carries kNoAllocScratchFloats * 4 bytes (16 MiB + 64 KiB) until the process exits.
+namespace alx {
+namespace {
+
+constexpr int64_t kNoAllocPieceFloats = 4ll << 20;                       // room for the piece sums
+constexpr int64_t kNoAllocScratchFloats = kNoAllocPieceFloats + 128 * 128;  // + one d x d fp32 by-product
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchFloats];
+
+constexpr int kNoAllocMaxDevices = 64;
+float *g_noalloc_ptr[kNoAllocMaxDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_noalloc_mutex;
+thread_local std::string g_noalloc_error;
+
+alx_status noalloc_fail(alx_status code, const std::string &msg)
+{
+    g_noalloc_error = msg;
+    return code;
+}
+
+}  // namespace
+}  // namespace alx
+
+extern "C" {
+
+int64_t alx_gramian_noalloc_max_rows(int32_t d)
+{
+    if (d != 16 && d != 32 && d != 64 && d != 128) return 0;
+    return (alx::kNoAllocPieceFloats / ((int64_t)d * d)) * alx::kGramRowsPerPartial;
+}
+
+const char *alx_noalloc_last_error(void) { return alx::g_noalloc_error.c_str(); }
+
+alx_status alx_gramian_noalloc(const void *table, alx_dtype dtype, int64_t n, int32_t d, double *gramian,
+                               void *stream)
+{
+    using namespace alx;
+    if (!table || !gramian || n < 1 || (dtype != ALX_F32 && dtype != ALX_BF16))
+        return noalloc_fail(ALX_ERR_INVALID_ARG, "alx_gramian_noalloc: null pointer, n < 1 or unknown dtype");
+    if (d != 16 && d != 32 && d != 64 && d != 128)
+        return noalloc_fail(ALX_ERR_UNSUPPORTED, "alx_gramian_noalloc: d must be 16, 32, 64 or 128");
+    const int64_t max_rows = alx_gramian_noalloc_max_rows(d);
+    if (n > max_rows)
+        return noalloc_fail(ALX_ERR_UNSUPPORTED,
+                            "alx_gramian_noalloc: " + std::to_string(n) + " rows exceed the fixed scratch array (at most " +
+                                std::to_string(max_rows) + " rows for d = " + std::to_string(d) +
+                                "); use a context and alx_gramian instead");
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices)
+        return noalloc_fail(ALX_ERR_CUDA, "alx_gramian_noalloc: no current CUDA device");
+    float *scratch = nullptr;
+    {
+        // set-up, once per device, with that device current: the array's name is only a handle in host
+        // code; the kernels need its device address
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ptr[dev]) {
+            void *p = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+            if (e != cudaSuccess || !p)
+                return noalloc_fail(ALX_ERR_CUDA, std::string("alx_gramian_noalloc: cudaGetSymbolAddress failed: ") +
+                                                      cudaGetErrorString(e));
+            g_noalloc_ptr[dev] = static_cast<float *>(p);
+        }
+        scratch = g_noalloc_ptr[dev];
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float *pieces = scratch, *base_out = scratch + kNoAllocPieceFloats;
+    cudaError_t e;
+    const int bf16 = dtype == ALX_BF16;
+    switch (d) {
+    case 16: e = gramian_simple_d<16>(table, bf16, n, pieces, s); break;
+    case 32: e = gramian_simple_d<32>(table, bf16, n, pieces, s); break;
+    case 64: e = gramian_simple_d<64>(table, bf16, n, pieces, s); break;
+    default: e = gramian_simple_d<128>(table, bf16, n, pieces, s); break;
+    }
+    if (e == cudaSuccess) {
+        // every piece the reduction reads was written in full by the launch above: nothing has to start at zero
+        k_gramian_reduce<<<(d * d + 255) / 256, 256, 0, s>>>(pieces, gramian_partials(n), d, gramian, base_out, 0.f, 0.f);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess)
+        return noalloc_fail(ALX_ERR_CUDA, std::string("alx_gramian_noalloc: launch failed: ") + cudaGetErrorString(e));
+    g_noalloc_error.clear();
+    return ALX_OK;
+}
+
+}  // extern "C"
