@@ -209,8 +209,17 @@ void release_matrix(alx_ctx *c)
     c->nnz = -1;
 }
 
+bool tensor_path(const alx_ctx *c) { return c->bf16 && c->opt.d == 128 && c->opt.kernels == 0; }
+
 alx_status gramian_of(alx_ctx *c, int table_side)
 {
+    if (tensor_path(c)) {
+        ALX_CUDA(c, launch_gramian_umma(c->table[table_side], c->n[table_side], c->gram_partials, c->stream, &c->launches));
+        ALX_CUDA(c, launch_gramian_reduce(c->gram_partials, gramian_umma_partials(), c->opt.d, c->G64[table_side], c->Bmat,
+                                          c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
+        c->have_gram[table_side] = true;
+        return ALX_OK;
+    }
     ALX_CUDA(c, launch_gramian(c->table[table_side], c->bf16, c->n[table_side], c->opt.d, c->gram_partials,
                                c->G64[table_side], c->Bmat, c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
     c->have_gram[table_side] = true;
@@ -227,10 +236,17 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     if (st != ALX_OK) return st;
     ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
     RowOut out{c->table[side], cap_slot, cap_out};
-    ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
-                                   c->table[fixed], c->bf16, c->opt.d, c->Bmat, c->split_partials, out, c->status,
-                                   c->stream, &c->launches));
-    c->stats.kernel_path[side] = 0;
+    if (tensor_path(c)) {
+        ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
+                                     c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
+                                     &c->launches));
+        c->stats.kernel_path[side] = 1;
+    } else {
+        ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side],
+                                       c->n_split_rows[side], c->table[fixed], c->bf16, c->opt.d, c->Bmat,
+                                       c->split_partials, out, c->status, c->stream, &c->launches));
+        c->stats.kernel_path[side] = 0;
+    }
     ALX_CUDA(c, cudaEventRecord(c->ev[2], c->stream));
     c->have_table[side] = true;
     c->have_gram[side] = false;
@@ -292,7 +308,9 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
         }
         ALX_ALLOC(c, c->Bmat, d * d);
         const int64_t nmax = c->n[0] > c->n[1] ? c->n[0] : c->n[1];
-        ALX_ALLOC(c, c->gram_partials, gramian_partials(nmax) * d * d);
+        int64_t n_part = gramian_partials(nmax);
+        if (gramian_umma_partials() > n_part) n_part = gramian_umma_partials();
+        ALX_ALLOC(c, c->gram_partials, n_part * d * d);
         ALX_ALLOC(c, c->loss_result, 4);
         ALX_ALLOC(c, c->status, 1);
         ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));

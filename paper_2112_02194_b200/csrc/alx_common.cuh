@@ -117,6 +117,8 @@ int64_t gramian_partials(int64_t n);
 cudaError_t launch_gramian(const void *X, int bf16, int64_t n, int d, float *partials, double *G64, float *Bmat,
                            float alpha0, float lambda, cudaStream_t s, int64_t *launches);
 
+cudaError_t launch_gramian_reduce(const float *partials, int64_t n_partials, int d, double *G64, float *Bmat,
+                                  float alpha0, float lambda, cudaStream_t s, int64_t *launches);
 cudaError_t measure_fp32_peak(double *tflops, cudaStream_t s);
 
 // alx_rows.cu
@@ -124,6 +126,13 @@ cudaError_t launch_rows_simple(const SideView &sv, const int64_t *class_offs_hos
                                int64_t n_split_rows, const void *X, int bf16, int d, const float *Bmat,
                                float *split_partials, RowOut out, DevStatus *st, cudaStream_t s,
                                int64_t *launches);
+
+// alx_umma.cu: tensor-core path, d = 128 and bf16 tables only
+int64_t gramian_umma_partials();
+cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches);
+cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
+                             int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
+                             RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches);
 
 // alx_loss.cu
 int64_t loss_partials(int64_t nnz);

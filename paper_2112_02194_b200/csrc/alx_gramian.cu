@@ -103,6 +103,14 @@ cudaError_t gramian_simple_d(const void *X, int bf16, int64_t n, float *partials
 
 int64_t gramian_partials(int64_t n) { return (n + kGramRowsPerPartial - 1) / kGramRowsPerPartial; }
 
+cudaError_t launch_gramian_reduce(const float *partials, int64_t n_partials, int d, double *G64, float *Bmat,
+                                  float alpha0, float lambda, cudaStream_t s, int64_t *launches)
+{
+    k_gramian_reduce<<<(d * d + 255) / 256, 256, 0, s>>>(partials, n_partials, d, G64, Bmat, alpha0, lambda);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_gramian(const void *X, int bf16, int64_t n, int d, float *partials, double *G64, float *Bmat,
                            float alpha0, float lambda, cudaStream_t s, int64_t *launches)
 {

@@ -1,0 +1,457 @@
+// Tensor-core (tcgen05 / tensor memory) kernels for d = 128 with bfloat16 tables:
+//   - the Gramian X^T X of the fixed table                                   (Alg. 1 line 2)
+//   - per row: sum x_i (x) x_i and sum y x_i over the row's observations      (Alg. 1 lines 6-9),
+//     then the same factor / solve / store as the FP32-ALU path               (Alg. 1 line 10, Eq. 4)
+//   - partial sums of the chunks of rows longer than `split`
+//
+// One persistent block per SM, three roles:
+//   producer warps   gather the fixed-side rows of an item with 16-byte cp.async into a ring of
+//                    shared-memory stages, already in the operand layout the tensor core reads:
+//                    "MN-major, 128-byte swizzle" - a gathered row is one K index, its 128 features
+//                    are the M (and N) index, split into two 64-feature halves of 128 bytes;
+//   one MMA thread   issues tcgen05.mma 128 x 128 x 16 (A = B = the staged tile) into one of two
+//                    fp32 accumulators in tensor memory, plus a 128 x 16 x 16 product with a two-column
+//                    (high / low bfloat16 parts of the label) tile that yields sum y x_i;
+//   solver groups    two groups of 256 threads, one per accumulator: read the accumulator back with
+//                    tcgen05.ld, add alpha0 G + lambda I, factor, solve, round and store - or, for
+//                    Gramian pieces and chunks, write the sums to the workspace.
+// Stage and accumulator hand-over is by mbarriers; every wait is bounded and a block that gives up
+// sets a status flag, releases its tensor memory and returns.
+#include "alx_chol.cuh"
+#include "alx_common.cuh"
+#include "alx_ptx.cuh"
+
+namespace alx {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int D = 128;
+constexpr int kStageRows = 32;
+constexpr int kNStage = 6;
+constexpr int kLag = 4;                               // stages of copies in flight per producer warp
+constexpr int kHalfBytes = kStageRows * 128;          // one 64-feature half of a stage
+constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
+constexpr int kStageYBytes = 2 * kStageRows * 16;     // 1024: label tile, two 8-column chunks
+constexpr int kProducerWarps = 4;
+constexpr int kGroups = 2;
+constexpr int kSolverThreads = kGroups * kThreads;    // 512
+constexpr int kMmaWarp = kSolverThreads / 32;         // warp 16
+constexpr int kFirstProducerWarp = kMmaWarp + 1;
+constexpr int kBlockThreads = kSolverThreads + 32 + kProducerWarps * 32;   // 672
+constexpr int kTmemCols = 512;
+constexpr int kAccStride = 256;                       // accumulator a lives at columns a * 256 .. + 144
+constexpr int kGramSubRows = 256;                     // rows per tensor-memory accumulation of the Gramian (the
+                                                      // accumulator truncates: fewer steps, smaller bias)
+constexpr int kGramBlocks = 148;                      // fixed, so that the order of sums depends on sizes only
+
+enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2 };
+
+struct Params {
+    SideView sv;
+    const __nv_bfloat16 *X;      // fixed table [N x 128]
+    int64_t n_items;             // rows of classes 1 .. 10 / chunk descriptors / 1024-row sub-pieces
+    int64_t last_item;           // rows mode: position in sv.order of item 0 (items walk downwards)
+    int64_t n_fixed;             // Gramian mode: rows of the table
+    const float *Bmat;           // alpha0 G + lambda I
+    float *partials;             // chunks: [slot][D*D + D]; Gramian: [2 * kGramBlocks][D*D]
+    RowOut out;
+    DevStatus *st;
+};
+
+struct GroupSmem {
+    float As[Geo<D>::A_FLOATS];
+    float Pt[Geo<D>::P_FLOATS];
+    float dinv[D];
+};
+
+struct __align__(1024) Smem {
+    unsigned char h[kNStage][kStageHBytes];
+    unsigned char y[kNStage][kStageYBytes];
+    uint64_t full[kNStage], empty[kNStage], acc_full[kGroups], acc_empty[kGroups];
+    uint32_t tmem_base;
+    int abort_flag;
+    int s_bad[kGroups];
+};
+
+template <int MODE> __device__ __forceinline__ void item_range(const Params &p, int64_t t, int64_t &u, int64_t &beg,
+                                                               int64_t &end, int64_t &slot)
+{
+    if (MODE == kModeRows) {
+        u = p.sv.order[p.last_item - t];
+        beg = p.sv.ptr[u];
+        end = p.sv.ptr[u + 1];
+        slot = 0;
+    } else if (MODE == kModeChunks) {
+        const int64_t *d = p.sv.chunk_desc + 4 * t;
+        u = d[0]; beg = d[1]; end = d[2]; slot = d[3];
+    } else {
+        u = 0; slot = t;
+        beg = t * kGramSubRows;
+        end = (beg + kGramSubRows < p.n_fixed) ? beg + kGramSubRows : p.n_fixed;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int pw, int lane)
+{
+    int64_t g = 0, signalled = 0;
+    const int c = lane & 15;                 // 16-byte chunk of the 256-byte row
+    const int half = c >> 3, cc = c & 7;
+    bool alive = true;
+    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x) {
+        int64_t u, beg, end, slot_unused;
+        item_range<MODE>(p, t, u, beg, end, slot_unused);
+        for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
+            const int slot = (int)(g % kNStage);
+            const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+            if (!mbar_wait(&sm.empty[slot], ph ^ 1u, &sm.abort_flag)) { alive = false; break; }
+            const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
+            const int rc16 = (rc + 15) & ~15;
+            // lanes 0..7 fetch the ids (and labels) of this warp's 8 rows
+            int64_t my_e = e0 + pw * 8 + (lane & 7);
+            int32_t my_idx = -1;
+            float my_y = 0.f;
+            if (lane < 8 && my_e < end) {
+                my_idx = (MODE == kModeGramian) ? (int32_t)my_e : p.sv.idx[my_e];
+                my_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[my_e] : 1.f);
+            }
+            const uint32_t hbase = smem_u32(&sm.h[slot][0]) + half * kHalfBytes + pw * 1024;
+            const uint32_t ybase = smem_u32(&sm.y[slot][0]) + pw * 128;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int j = (lane >> 4) + 2 * q;          // row inside this warp's group of 8
+                const int r = pw * 8 + j;                   // row inside the stage
+                const int32_t src = __shfl_sync(0xFFFFFFFFu, my_idx, j);
+                const float yv = __shfl_sync(0xFFFFFFFFu, my_y, j);
+                const uint32_t dst = hbase + j * 128 + ((cc ^ j) << 4);
+                if (src >= 0) cp_async16(dst, p.X + (int64_t)src * D + c * 8);
+                else if (r < rc16) st_shared_zero16(dst);
+                if (MODE != kModeGramian && c == 0 && r < rc16) {
+                    const __nv_bfloat16 yhi = __float2bfloat16_rn(yv);
+                    const __nv_bfloat16 ylo = __float2bfloat16_rn(yv - __bfloat162float(yhi));
+                    const uint32_t packed = (uint32_t)__bfloat16_as_ushort(yhi) | ((uint32_t)__bfloat16_as_ushort(ylo) << 16);
+                    st_shared_v4(ybase + j * 16, packed, 0u, 0u, 0u);
+                }
+            }
+            cp_async_commit();
+            ++g;
+            if (g > kLag) {
+                cp_async_wait<kLag>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.full[signalled % kNStage]);
+                ++signalled;
+            }
+        }
+    }
+    cp_async_wait<0>();
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0)
+        for (; signalled < g; ++signalled) mbar_arrive(&sm.full[signalled % kNStage]);
+}
+
+template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane)
+{
+    constexpr uint32_t kIdescMain = idesc_bf16_mn_major(128, 128);
+    constexpr uint32_t kIdescY = idesc_bf16_mn_major(128, 16);
+    const uint32_t tmem = sm.tmem_base;
+    int64_t g = 0, it = 0;
+    bool alive = true;
+    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
+        int64_t u, beg, end, slot_unused;
+        item_range<MODE>(p, t, u, beg, end, slot_unused);
+        const int a = (int)(it & 1);
+        const uint32_t aph = (uint32_t)((it >> 1) & 1);
+        if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_main = tmem + a * kAccStride;
+        bool first = true;
+        for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
+            const int slot = (int)(g % kNStage);
+            const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+            if (!mbar_wait(&sm.full[slot], ph, &sm.abort_flag)) { alive = false; break; }
+            tc_fence_after();
+            const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
+            const int nk = (rc + 15) >> 4;
+            if (lane == 0) {
+                const uint32_t hb = smem_u32(&sm.h[slot][0]);
+                const uint32_t yb = smem_u32(&sm.y[slot][0]);
+                for (int ks = 0; ks < nk; ++ks) {
+                    // 16 gathered rows = two groups of 8 rows of 128 bytes; halves are kHalfBytes apart
+                    const uint64_t adesc = smem_desc(hb + ks * 2048, kHalfBytes, 1024, 2);
+                    umma_f16(d_main, adesc, adesc, kIdescMain, !first);
+                    if (MODE != kModeGramian) {
+                        const uint64_t ydesc = smem_desc(yb + ks * 256, 128, kStageRows * 16, 0);
+                        umma_f16(d_main + D, adesc, ydesc, kIdescY, !first);
+                    }
+                    first = false;
+                }
+                umma_commit(&sm.empty[slot]);
+            }
+            __syncwarp();
+            ++g;
+        }
+        if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
+        __syncwarp();
+    }
+}
+
+template <int MODE>
+__device__ void solver_role(const Params &p, Smem &sm, GroupSmem &gs, int gidx, int tid)
+{
+    const int lane = tid & 31, w = tid >> 5;
+    const int q = w & 3, hh = w >> 2;            // lane quarter of tensor memory, column half
+    const int i = q * 32 + lane;                 // row of the matrix this thread reads back
+    const int bar_id = 1 + gidx;
+    constexpr int LDA = Geo<D>::LDA;
+    const uint32_t tmem = sm.tmem_base;
+    float run[(MODE == kModeGramian) ? 64 : 1];
+    if (MODE == kModeGramian) {
+#pragma unroll
+        for (int k = 0; k < 64; ++k) run[k] = 0.f;
+    }
+    int64_t it = 0;
+    for (int64_t t = blockIdx.x; t < p.n_items; t += gridDim.x, ++it) {
+        if ((it & 1) != gidx) continue;
+        int64_t u, beg, end, slot;
+        item_range<MODE>(p, t, u, beg, end, slot);
+        const uint32_t aph = (uint32_t)((it >> 1) & 1);
+        if (!mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag)) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + gidx * kAccStride + hh * 64;
+        uint32_t v0[32], v1[32];
+        tmem_ld32(taddr, v0);
+        tmem_ld32(taddr + 32, v1);
+        tmem_ld_wait();
+        if (MODE == kModeGramian) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+                run[k] += __uint_as_float(v0[k]);
+                run[32 + k] += __uint_as_float(v1[k]);
+            }
+        } else if (MODE == kModeChunks) {
+            float *dst = p.partials + slot * (int64_t)(D * D + D) + (int64_t)i * D + hh * 64;
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) {
+                *reinterpret_cast<float4 *>(dst + k) = make_float4(__uint_as_float(v0[k]), __uint_as_float(v0[k + 1]),
+                                                                   __uint_as_float(v0[k + 2]), __uint_as_float(v0[k + 3]));
+                *reinterpret_cast<float4 *>(dst + 32 + k) = make_float4(__uint_as_float(v1[k]), __uint_as_float(v1[k + 1]),
+                                                                        __uint_as_float(v1[k + 2]), __uint_as_float(v1[k + 3]));
+            }
+        } else {
+            float *dst = gs.As + i * LDA + hh * 64;
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) {
+                *reinterpret_cast<float4 *>(dst + k) = make_float4(__uint_as_float(v0[k]), __uint_as_float(v0[k + 1]),
+                                                                   __uint_as_float(v0[k + 2]), __uint_as_float(v0[k + 3]));
+                *reinterpret_cast<float4 *>(dst + 32 + k) = make_float4(__uint_as_float(v1[k]), __uint_as_float(v1[k + 1]),
+                                                                        __uint_as_float(v1[k + 2]), __uint_as_float(v1[k + 3]));
+            }
+        }
+        if (MODE != kModeGramian && hh == 0) {
+            uint32_t bv[4];
+            tmem_ld4(tmem + ((uint32_t)(q * 32) << 16) + gidx * kAccStride + D, bv);
+            tmem_ld_wait();
+            const float b = __uint_as_float(bv[0]) + __uint_as_float(bv[1]);   // high and low parts of the labels
+            if (MODE == kModeChunks) p.partials[slot * (int64_t)(D * D + D) + D * D + i] = b;
+            else gs.As[D * LDA + i] = b;
+        }
+        tc_fence_before();
+        group_sync(bar_id);
+        if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
+        if (MODE == kModeRows) {
+            // lower triangle += alpha0 G + lambda I (coalesced reads of the shared base matrix)
+            for (int e = tid; e < D * D; e += kThreads) {
+                const int r = e >> 7, cidx = e & (D - 1);
+                if (cidx <= r) gs.As[r * LDA + cidx] += p.Bmat[e];
+            }
+            group_sync(bar_id);
+            float xq[D / 32];
+            const bool ok = cholesky_solve<D>(gs.As, gs.Pt, gs.dinv, xq, tid, bar_id, &sm.s_bad[gidx]);
+            if (tid < 32) store_solution<D, __nv_bfloat16>(xq, ok, u, p.out, p.st);
+            group_sync(bar_id);
+        }
+    }
+    if (MODE == kModeGramian) {
+        float *dst = p.partials + ((int64_t)blockIdx.x * kGroups + gidx) * (D * D) + (int64_t)i * D + hh * 64;
+#pragma unroll
+        for (int k = 0; k < 64; k += 4)
+            *reinterpret_cast<float4 *>(dst + k) = make_float4(run[k], run[k + 1], run[k + 2], run[k + 3]);
+    }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kBlockThreads, 1) k_umma(Params p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment for the swizzled stages
+    unsigned char *aligned = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Smem &sm = *reinterpret_cast<Smem *>(aligned);
+    GroupSmem *gs = reinterpret_cast<GroupSmem *>(aligned + sizeof(Smem));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < kNStage; ++s) { mbar_init(&sm.full[s], kProducerWarps); mbar_init(&sm.empty[s], 1); }
+        for (int a = 0; a < kGroups; ++a) { mbar_init(&sm.acc_full[a], 1); mbar_init(&sm.acc_empty[a], 1); }
+        sm.abort_flag = 0;
+        mbar_fence_init();
+    }
+    // label tiles start finite (all zero): rows beyond an item's end multiply zeros, never stale NaNs
+    for (int k = tid; k < kNStage * kStageYBytes / 16; k += kBlockThreads)
+        st_shared_zero16(smem_u32(&sm.y[0][0]) + k * 16);
+    for (int k = tid; k < kNStage * kStageHBytes / 16; k += kBlockThreads)
+        st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
+    fence_proxy_async();
+    if (warp == kMmaWarp) {
+        tmem_alloc(&sm.tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    if (warp < kMmaWarp) {
+        const int gidx = warp / (kThreads / 32);
+        solver_role<MODE>(p, sm, gs[(MODE == kModeRows) ? gidx : 0], gidx, tid - gidx * kThreads);
+    } else if (warp == kMmaWarp) {
+        mma_role<MODE>(p, sm, lane);
+    } else {
+        producer_role<MODE>(p, sm, warp - kFirstProducerWarp, lane);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(sm.tmem_base, kTmemCols);
+    }
+    if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, blockIdx.x);
+}
+
+__global__ void k_zero_rows_bf16(const int32_t *__restrict__ rows, int64_t count, RowOut out)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count * D) return;
+    const int64_t u = rows[t / D];
+    const int c = (int)(t % D);
+    reinterpret_cast<__nv_bfloat16 *>(out.table)[u * D + c] = __float2bfloat16_rn(0.f);
+    if (out.cap_slot) {
+        const int slot = out.cap_slot[u];
+        if (slot >= 0) out.cap_out[(int64_t)slot * D + c] = 0.f;
+    }
+}
+
+// chunks of a split row added in ascending order, then factor / solve / store (one block of 256 per row)
+__global__ void __launch_bounds__(kThreads, 2) k_split_solve_umma(SideView sv, int64_t split_class_begin,
+                                                                  const float *__restrict__ partials,
+                                                                  const float *__restrict__ Bmat, RowOut out,
+                                                                  DevStatus *st)
+{
+    constexpr int LDA = Geo<D>::LDA;
+    extern __shared__ __align__(16) unsigned char smem_raw2[];
+    GroupSmem &gs = *reinterpret_cast<GroupSmem *>(smem_raw2);
+    __shared__ int s_bad;
+    const int tid = threadIdx.x;
+    const int64_t j = blockIdx.x;
+    const int64_t u = sv.order[split_class_begin + j];
+    const int64_t c0 = sv.split_first[j], c1 = sv.split_first[j + 1];
+    // lower triangle and right-hand side: element e of this thread summed over the chunks in order
+    for (int e = tid; e < D * D + D; e += kThreads) {
+        const int r = e >> 7, cidx = e & (D - 1);
+        if (e < D * D && cidx > r) continue;
+        float s = 0.f;
+        for (int64_t c = c0; c < c1; ++c) s += partials[c * (int64_t)(D * D + D) + e];
+        if (e < D * D) gs.As[r * LDA + cidx] = s + Bmat[e];
+        else gs.As[D * LDA + (e - D * D)] = s;
+    }
+    __syncthreads();
+    float xq[D / 32];
+    const bool ok = cholesky_solve<D>(gs.As, gs.Pt, gs.dinv, xq, tid, 0, &s_bad);
+    if (tid < 32) store_solution<D, __nv_bfloat16>(xq, ok, u, out, st);
+}
+
+size_t smem_bytes(int)
+{
+    // the same (large) request in every mode: at most one block per SM, so two blocks never compete for
+    // the SM's 512 tensor-memory columns
+    return sizeof(Smem) + 1024 + kGroups * sizeof(GroupSmem);
+}
+
+template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStream_t s)
+{
+    const size_t smem = smem_bytes(MODE);
+    cudaError_t e = cudaFuncSetAttribute(k_umma<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_umma<MODE><<<grid, kBlockThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+int sm_count()
+{
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms > 0 ? sms : 1;
+}
+
+}  // namespace
+
+int64_t gramian_umma_partials() { return (int64_t)kGramBlocks * kGroups; }
+
+// Gramian of a bf16 table with d = 128 on the tensor cores; partials must hold gramian_umma_partials() * d * d floats
+cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches)
+{
+    Params p{};
+    p.X = reinterpret_cast<const __nv_bfloat16 *>(X);
+    p.n_fixed = n;
+    p.n_items = (n + kGramSubRows - 1) / kGramSubRows;
+    p.partials = partials;
+    cudaError_t e = launch_mode<kModeGramian>(p, kGramBlocks, s);
+    ++*launches;
+    return e;
+}
+
+cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows,
+                             const void *X, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
+                             cudaStream_t s, int64_t *launches)
+{
+    const int sms = sm_count();
+    Params p{};
+    p.sv = sv;
+    p.X = reinterpret_cast<const __nv_bfloat16 *>(X);
+    p.Bmat = Bmat;
+    p.partials = split_partials;
+    p.out = out;
+    p.st = st;
+    cudaError_t e;
+    if (n_chunks > 0) {
+        p.n_items = n_chunks;
+        e = launch_mode<kModeChunks>(p, (int)(n_chunks < sms ? n_chunks : sms), s);
+        ++*launches;
+        if (e != cudaSuccess) return e;
+        const size_t smem = sizeof(GroupSmem);
+        e = cudaFuncSetAttribute(k_split_solve_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_split_solve_umma<<<(unsigned)n_split_rows, kThreads, smem, s>>>(sv, offs[kNClasses - 1], split_partials, Bmat, out, st);
+        ++*launches;
+    }
+    const int64_t n_whole = offs[kNClasses - 1] - offs[1];
+    if (n_whole > 0) {
+        p.n_items = n_whole;
+        p.last_item = offs[kNClasses - 1] - 1;
+        e = launch_mode<kModeRows>(p, (int)(n_whole < sms ? n_whole : sms), s);
+        ++*launches;
+        if (e != cudaSuccess) return e;
+    }
+    const int64_t n_zero = offs[1] - offs[0];
+    if (n_zero > 0) {
+        k_zero_rows_bf16<<<(unsigned)((n_zero * D + 255) / 256), 256, 0, s>>>(sv.order + offs[0], n_zero, out);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace alx
