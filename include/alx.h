@@ -186,7 +186,8 @@ const char *alx_last_error(const alx_ctx *ctx);
  *   table   : device pointer, n x d row-major, float32 or bfloat16 (dtype)
  *   gramian : device pointer, d x d doubles, receives table^T table; written on `stream` (cudaStream_t,
  *             NULL = legacy default stream); the call does not synchronise
- * Same kernels and the same fixed summation order as alx_gramian, so the results agree to the last bit.
+ * Same kernels and the same fixed summation order as alx_gramian on a context created with kernels = 1
+ * (the FP32-ALU kernels), so those results agree to the last bit.
  * The piece sums go to a fixed array inside the library image (16 MiB + 64 KiB on every GPU that loads
  * the library, held until the process exits).  Limits: d in {16, 32, 64, 128} and
  * n <= alx_gramian_noalloc_max_rows(d) = (4 Mi / d^2) * 4096 rows (1 048 576 for d = 128); larger inputs

@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 
 def reference_gramian(table_bits, storage, n, d):
     from paper_2112_02194_b200 import ALX_ROWS, Alx
-    a = Alx(n, 4, d, 0.1, 0.01, storage=storage)
+    # kernels=1: the FP32-ALU kernels, whose Gramian kernel the allocation-free entry point shares
+    a = Alx(n, 4, d, 0.1, 0.01, storage=storage, kernels=1)
     a.set_embeddings(ALX_ROWS, table_bits)
     G = a.gramian(ALX_ROWS)
     a.destroy()
