@@ -12,9 +12,11 @@
 //   one MMA thread   issues tcgen05.mma 128 x 128 x 16 (A = B = the staged tile) into one of two
 //                    fp32 accumulators in tensor memory, plus a 128 x 16 x 16 product with a two-column
 //                    (high / low bfloat16 parts of the label) tile that yields sum y x_i;
-//   solver groups    two groups of 256 threads, one per accumulator: read the accumulator back with
-//                    tcgen05.ld, add alpha0 G + lambda I, factor, solve, round and store - or, for
-//                    Gramian pieces and chunks, write the sums to the workspace.
+//   solver groups    rows: three groups of 128 threads, one per accumulator, thread i owning row i of
+//                    the normal matrix.  The matrix never leaves tensor memory: the group adds
+//                    alpha0 G + lambda I on first touch, factors it in place with a blocked right-looking
+//                    Cholesky (tcgen05.ld / tcgen05.st of 16-column row segments), solves and stores the
+//                    row.  Gramian pieces and chunks: two groups of 256 threads copy the sums out.
 // Stage and accumulator hand-over is by mbarriers; every wait is bounded and a block that gives up
 // sets a status flag, releases its tensor memory and returns.
 #include "alx_chol.cuh"
@@ -35,18 +37,24 @@ constexpr int kHalfBytes = kStageRows * 128;          // one 64-feature half of 
 constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
 constexpr int kStageYBytes = 2 * kStageRows * 16;     // 1024: label tile, two 8-column chunks
 constexpr int kProducerWarps = 4;
-constexpr int kGroups = 2;
-constexpr int kSolverThreads = kGroups * kThreads;    // 512
-constexpr int kMmaWarp = kSolverThreads / 32;         // warp 16
-constexpr int kFirstProducerWarp = kMmaWarp + 1;
-constexpr int kBlockThreads = kSolverThreads + 32 + kProducerWarps * 32;   // 672
 constexpr int kTmemCols = 512;
-constexpr int kAccStride = 256;                       // accumulator a lives at columns a * 256 .. + 144
+constexpr int kMaxGroups = 3;
 constexpr int kGramSubRows = 256;                     // rows per tensor-memory accumulation of the Gramian (the
                                                       // accumulator truncates: fewer steps, smaller bias)
 constexpr int kGramBlocks = 148;                      // fixed, so that the order of sums depends on sizes only
 
 enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2 };
+
+// thread layout per mode: solver groups (one accumulator each), then one MMA warp, then the producer warps
+template <int MODE> struct Cfg {
+    static constexpr int kGroups = (MODE == kModeRows) ? 3 : 2;
+    static constexpr int kGroupThreads = (MODE == kModeRows) ? 128 : 256;
+    static constexpr int kAccStride = (MODE == kModeRows) ? 160 : 256;   // accumulator a: columns a * stride .. + 144
+    static constexpr int kSolverThreads = kGroups * kGroupThreads;
+    static constexpr int kMmaWarp = kSolverThreads / 32;
+    static constexpr int kFirstProducerWarp = kMmaWarp + 1;
+    static constexpr int kBlockThreads = kSolverThreads + 32 + kProducerWarps * 32;
+};
 
 struct Params {
     SideView sv;
@@ -60,19 +68,28 @@ struct Params {
     DevStatus *st;
 };
 
-struct GroupSmem {
+struct GroupSmem {   // split-row solve: one matrix in shared memory
     float As[Geo<D>::A_FLOATS];
     float Pt[Geo<D>::P_FLOATS];
     float dinv[D];
 };
 
+constexpr int kLdB = D + 4;
+struct __align__(16) RowGroupSmem {   // scratch of one tensor-memory solver group (float4 access: 16-byte aligned)
+    float Ps[D][16];        // panel of the current block step, row i = what thread i computed
+    float Lkk[16][16];      // diagonal block of the current step
+    float dinv[16];
+    float z[16];            // the block's part of L^-1 b
+    float red[2][4][16];    // per-warp partial sums of the back substitution (double buffered)
+    int bad;
+};
+
 struct __align__(1024) Smem {
     unsigned char h[kNStage][kStageHBytes];
     unsigned char y[kNStage][kStageYBytes];
-    uint64_t full[kNStage], empty[kNStage], acc_full[kGroups], acc_empty[kGroups];
+    uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
     uint32_t tmem_base;
     int abort_flag;
-    int s_bad[kGroups];
 };
 
 template <int MODE> __device__ __forceinline__ void item_range(const Params &p, int64_t t, int64_t &u, int64_t &beg,
@@ -163,11 +180,11 @@ template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane
     for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
         int64_t u, beg, end, slot_unused;
         item_range<MODE>(p, t, u, beg, end, slot_unused);
-        const int a = (int)(it & 1);
-        const uint32_t aph = (uint32_t)((it >> 1) & 1);
+        const int a = (int)(it % Cfg<MODE>::kGroups);
+        const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
         if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag)) break;
         tc_fence_after();
-        const uint32_t d_main = tmem + a * kAccStride;
+        const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
         bool first = true;
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
@@ -200,13 +217,13 @@ template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane
 }
 
 template <int MODE>
-__device__ void solver_role(const Params &p, Smem &sm, GroupSmem &gs, int gidx, int tid)
+__device__ void copyout_role(const Params &p, Smem &sm, int gidx, int tid)
 {
+    constexpr int kAccStride = Cfg<MODE>::kAccStride;
     const int lane = tid & 31, w = tid >> 5;
     const int q = w & 3, hh = w >> 2;            // lane quarter of tensor memory, column half
     const int i = q * 32 + lane;                 // row of the matrix this thread reads back
     const int bar_id = 1 + gidx;
-    constexpr int LDA = Geo<D>::LDA;
     const uint32_t tmem = sm.tmem_base;
     float run[(MODE == kModeGramian) ? 64 : 1];
     if (MODE == kModeGramian) {
@@ -241,71 +258,299 @@ __device__ void solver_role(const Params &p, Smem &sm, GroupSmem &gs, int gidx, 
                 *reinterpret_cast<float4 *>(dst + 32 + k) = make_float4(__uint_as_float(v1[k]), __uint_as_float(v1[k + 1]),
                                                                         __uint_as_float(v1[k + 2]), __uint_as_float(v1[k + 3]));
             }
-        } else {
-            float *dst = gs.As + i * LDA + hh * 64;
-#pragma unroll
-            for (int k = 0; k < 32; k += 4) {
-                *reinterpret_cast<float4 *>(dst + k) = make_float4(__uint_as_float(v0[k]), __uint_as_float(v0[k + 1]),
-                                                                   __uint_as_float(v0[k + 2]), __uint_as_float(v0[k + 3]));
-                *reinterpret_cast<float4 *>(dst + 32 + k) = make_float4(__uint_as_float(v1[k]), __uint_as_float(v1[k + 1]),
-                                                                        __uint_as_float(v1[k + 2]), __uint_as_float(v1[k + 3]));
-            }
         }
         if (MODE != kModeGramian && hh == 0) {
             uint32_t bv[4];
             tmem_ld4(tmem + ((uint32_t)(q * 32) << 16) + gidx * kAccStride + D, bv);
             tmem_ld_wait();
             const float b = __uint_as_float(bv[0]) + __uint_as_float(bv[1]);   // high and low parts of the labels
-            if (MODE == kModeChunks) p.partials[slot * (int64_t)(D * D + D) + D * D + i] = b;
-            else gs.As[D * LDA + i] = b;
+            p.partials[slot * (int64_t)(D * D + D) + D * D + i] = b;
         }
         tc_fence_before();
         group_sync(bar_id);
         if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
-        if (MODE == kModeRows) {
-            // lower triangle += alpha0 G + lambda I (coalesced reads of the shared base matrix)
-            for (int e = tid; e < D * D; e += kThreads) {
-                const int r = e >> 7, cidx = e & (D - 1);
-                if (cidx <= r) gs.As[r * LDA + cidx] += p.Bmat[e];
-            }
-            group_sync(bar_id);
-            float xq[D / 32];
-            const bool ok = cholesky_solve<D>(gs.As, gs.Pt, gs.dinv, xq, tid, bar_id, &sm.s_bad[gidx]);
-            if (tid < 32) store_solution<D, __nv_bfloat16>(xq, ok, u, p.out, p.st);
-            group_sync(bar_id);
-        }
     }
     if (MODE == kModeGramian) {
-        float *dst = p.partials + ((int64_t)blockIdx.x * kGroups + gidx) * (D * D) + (int64_t)i * D + hh * 64;
+        float *dst = p.partials + ((int64_t)blockIdx.x * Cfg<MODE>::kGroups + gidx) * (D * D) + (int64_t)i * D + hh * 64;
 #pragma unroll
         for (int k = 0; k < 64; k += 4)
             *reinterpret_cast<float4 *>(dst + k) = make_float4(run[k], run[k + 1], run[k + 2], run[k + 3]);
     }
 }
 
-template <int MODE>
-__global__ void __launch_bounds__(kBlockThreads, 1) k_umma(Params p)
+
+// ---------------------------------------------------------------------------------------------------------
+// Rows mode: factor and solve in place in tensor memory.  128 threads, thread i = row i = tensor-memory lane i.
+// Blocked right-looking Cholesky, 16 columns per step:
+//   (1) every live row reads its 16 panel values; the 16 threads that own the diagonal block factor it with
+//       shuffles (their warp-mates take part in the shuffles only) and carry b along as a 17th column;
+//   (2) rows below the block do their own forward substitution against the block (from shared memory),
+//       publish their panel row, and fold the block's part of L^-1 b into their b; meanwhile each diagonal
+//       thread computes its column of the block's inverse, which it keeps in registers for step (4);
+//   (3) trailing update of the thread's own row, 16 columns at a time, against the published panel rows;
+//       the next block's diagonal threads only have one such column block, so their factorisation
+//       overlaps the other threads' update;
+//   (4) back substitution block by block from the end: per-block partial sums over the rows below are
+//       reduced in a fixed order (warp butterfly, then four warps in order), the diagonal threads apply
+//       their inverse columns.
+// alpha0 G + lambda I is added from shared memory when an element is first read (block step 0).
+__device__ __forceinline__ void warp_reduce16(float (&v)[16], int lane)
 {
+    // after the call, lane 2c (and 2c+1) holds the sum over the 32 lanes of v[c], in v[0]
+    float t8[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const bool up = (lane & 16) != 0;
+        const float send = up ? v[c] : v[c + 8];
+        const float keep = up ? v[c + 8] : v[c];
+        t8[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 16);
+    }
+    float t4[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const bool up = (lane & 8) != 0;
+        const float send = up ? t8[c] : t8[c + 4];
+        const float keep = up ? t8[c + 4] : t8[c];
+        t4[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 8);
+    }
+    float t2[2];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        const bool up = (lane & 4) != 0;
+        const float send = up ? t4[c] : t4[c + 2];
+        const float keep = up ? t4[c + 2] : t4[c];
+        t2[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 4);
+    }
+    {
+        const bool up = (lane & 2) != 0;
+        const float send = up ? t2[0] : t2[1];
+        const float keep = up ? t2[1] : t2[0];
+        v[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 2);
+    }
+    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
+}
+
+__device__ __forceinline__ void group128_sync(int bar_id)
+{
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+}
+
+__device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, const float *__restrict__ Bs, int gidx,
+                                 int tid)
+{
+    constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
+    const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory
+    const int i = tid;                           // my row
+    const int bar_id = 1 + gidx;
+    const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
+    const float *Brow = Bs + i * kLdB;
+    int64_t it = 0;
+    for (int64_t t = blockIdx.x; t < p.n_items; t += gridDim.x, ++it) {
+        if ((int)(it % kGroups) != gidx) continue;
+        int64_t u, beg, end, slot;
+        item_range<kModeRows>(p, t, u, beg, end, slot);
+        const uint32_t aph = (uint32_t)((it / kGroups) & 1);
+        if (!mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag)) break;
+        tc_fence_after();
+        if (tid == 0) gs.bad = 0;
+        float b;
+        {
+            uint32_t bv[4];
+            tmem_ld4(trow + D, bv);
+            tmem_ld_wait();
+            b = __uint_as_float(bv[0]) + __uint_as_float(bv[1]);   // high and low parts of the labels
+        }
+        float yinv[16];          // my column of the inverse of my diagonal block (set at my block step)
+#pragma unroll
+        for (int c = 0; c < 16; ++c) yinv[c] = 0.f;
+
+        for (int k = 0; k < D / 16; ++k) {
+            const int k0 = 16 * k;
+            float a[16];
+            const bool warp_live = (w * 32 + 31 >= k0);            // some row of my warp is at or below the block
+            if (warp_live) {
+                tmem_ld16(trow + k0, a);
+                if (k == 0) {
+#pragma unroll
+                    for (int c = 0; c < 16; c += 4) {
+                        const float4 bb = *reinterpret_cast<const float4 *>(Brow + c);
+                        a[c] += bb.x; a[c + 1] += bb.y; a[c + 2] += bb.z; a[c + 3] += bb.w;
+                    }
+                }
+            }
+            // (1) diagonal block
+            if (w == (k0 >> 5)) {
+                const int hb = k0 & 16;
+                const int l = lane - hb;
+                const bool is_diag = (l >= 0 && l < 16);
+                float my_inv = 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float pj = __shfl_sync(0xFFFFFFFFu, a[j], hb + j);
+                    const bool ok = pj > 0.f;
+                    float inv = ok ? rsqrtf(pj) : 0.f;
+                    inv = inv * fmaf(-0.5f * pj * inv, inv, 1.5f);
+                    if (!ok && lane == 0) gs.bad = 1;
+                    const float zj = __shfl_sync(0xFFFFFFFFu, b, hb + j) * inv;
+                    if (is_diag) {
+                        if (l == j) { a[j] = pj * inv; my_inv = inv; b = zj; }
+                        else { a[j] *= inv; if (l > j) b = fmaf(-a[j], zj, b); }
+                    }
+#pragma unroll
+                    for (int c = j + 1; c < 16; ++c) {
+                        const float lc = __shfl_sync(0xFFFFFFFFu, a[j], hb + c);
+                        if (is_diag) a[c] = fmaf(-a[j], lc, a[c]);
+                    }
+                }
+                if (is_diag) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) gs.Lkk[l][c] = (c <= l) ? a[c] : 0.f;
+                    gs.dinv[l] = my_inv;
+                    gs.z[l] = b;
+                }
+            }
+            group128_sync(bar_id);
+            // (2) rows below the block: forward substitution; diagonal threads: their column of the inverse
+            if (i >= k0 + 16) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    float s = a[c];
+#pragma unroll
+                    for (int pp = 0; pp < c; ++pp) s = fmaf(-a[pp], gs.Lkk[c][pp], s);
+                    a[c] = s * gs.dinv[c];
+                }
+                float acc = 0.f;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) acc = fmaf(a[c], gs.z[c], acc);
+                b -= acc;
+#pragma unroll
+                for (int c = 0; c < 16; c += 4)
+                    *reinterpret_cast<float4 *>(&gs.Ps[i][c]) = make_float4(a[c], a[c + 1], a[c + 2], a[c + 3]);
+            } else if (i >= k0) {
+                const int l = i - k0;
+                float tacc[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) tacc[c] = 0.f;
+#pragma unroll
+                for (int cp = 0; cp < 16; ++cp) {
+                    // y[cp] of the solve L y = e_l
+                    float ycp = (cp < l) ? 0.f : ((cp == l) ? gs.dinv[cp] : -tacc[cp] * gs.dinv[cp]);
+                    yinv[cp] = ycp;
+#pragma unroll
+                    for (int c = cp + 1; c < 16; ++c) tacc[c] = fmaf(gs.Lkk[c][cp], ycp, tacc[c]);
+                }
+            }
+            if (warp_live) {
+                tmem_st16(trow + k0, a);      // L (rows above the block rewrite what they read)
+                tmem_st_wait();
+            }
+            group128_sync(bar_id);
+            // (3) trailing update of my own row
+            for (int cb = k0 + 16; cb < (w + 1) * 32; cb += 16) {
+                float tt[16];
+                tmem_ld16(trow + cb, tt);
+                if (k == 0) {
+#pragma unroll
+                    for (int c = 0; c < 16; c += 4) {
+                        const float4 bb = *reinterpret_cast<const float4 *>(Brow + cb + c);
+                        tt[c] += bb.x; tt[c + 1] += bb.y; tt[c + 2] += bb.z; tt[c + 3] += bb.w;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const float4 p0 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][0]);
+                    const float4 p1 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][4]);
+                    const float4 p2 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][8]);
+                    const float4 p3 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][12]);
+                    float s = tt[c];
+                    s = fmaf(-a[0], p0.x, s); s = fmaf(-a[1], p0.y, s); s = fmaf(-a[2], p0.z, s); s = fmaf(-a[3], p0.w, s);
+                    s = fmaf(-a[4], p1.x, s); s = fmaf(-a[5], p1.y, s); s = fmaf(-a[6], p1.z, s); s = fmaf(-a[7], p1.w, s);
+                    s = fmaf(-a[8], p2.x, s); s = fmaf(-a[9], p2.y, s); s = fmaf(-a[10], p2.z, s); s = fmaf(-a[11], p2.w, s);
+                    s = fmaf(-a[12], p3.x, s); s = fmaf(-a[13], p3.y, s); s = fmaf(-a[14], p3.z, s); s = fmaf(-a[15], p3.w, s);
+                    tt[c] = s;
+                }
+                tmem_st16(trow + cb, tt);
+            }
+            tmem_st_wait();
+        }
+        // (4) back substitution L^T x = z; b now holds z_i
+        float x = 0.f;
+        for (int k = D / 16 - 1; k >= 0; --k) {
+            const int k0 = 16 * k;
+            float wv[16];
+            if (w * 32 + 31 >= k0 + 16) {
+                tmem_ld16(trow + k0, wv);
+                const float xm = (i >= k0 + 16) ? x : 0.f;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) wv[c] = (i >= k0 + 16) ? wv[c] * xm : 0.f;
+                warp_reduce16(wv, lane);
+            } else {
+                wv[0] = 0.f;
+            }
+            if ((lane & 1) == 0) gs.red[k & 1][w][lane >> 1] = wv[0];
+            group128_sync(bar_id);
+            if (w == (k0 >> 5)) {
+                const int hb = k0 & 16;
+                const int l = lane - hb;
+                const bool is_diag = (l >= 0 && l < 16);
+                float rhs = 0.f;
+                if (is_diag) rhs = b - (((gs.red[k & 1][0][l] + gs.red[k & 1][1][l]) + gs.red[k & 1][2][l]) + gs.red[k & 1][3][l]);
+                float acc = 0.f;
+#pragma unroll
+                for (int cp = 0; cp < 16; ++cp) {
+                    const float r = __shfl_sync(0xFFFFFFFFu, rhs, hb + cp);
+                    acc = fmaf(yinv[cp], r, acc);     // yinv[cp] = Linv[cp][l], zero for cp < l
+                }
+                if (is_diag) x = acc;
+            }
+        }
+        // tensor memory is free again for the next item of this accumulator
+        tc_fence_before();
+        group128_sync(bar_id);
+        if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
+        const bool ok = gs.bad == 0;
+        const float xo = ok ? x : 0.f;
+        reinterpret_cast<__nv_bfloat16 *>(p.out.table)[u * D + i] = __float2bfloat16_rn(xo);
+        if (p.out.cap_slot) {
+            const int cs = p.out.cap_slot[u];
+            if (cs >= 0) p.out.cap_out[(int64_t)cs * D + i] = xo;
+        }
+        if (!ok && tid == 0) {
+            atomicAdd(&p.st->not_spd, 1ull);
+            raise_flag(p.st, kFlagNotSpd, u);
+        }
+        group128_sync(bar_id);      // gs.bad is reset at the top of the next item
+    }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
+{
+    using C = Cfg<MODE>;
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled stages
     unsigned char *aligned = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Smem &sm = *reinterpret_cast<Smem *>(aligned);
-    GroupSmem *gs = reinterpret_cast<GroupSmem *>(aligned + sizeof(Smem));
+    float *Bs = reinterpret_cast<float *>(aligned + sizeof(Smem));
+    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(Smem) + sizeof(float) * D * kLdB);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
         for (int s = 0; s < kNStage; ++s) { mbar_init(&sm.full[s], kProducerWarps); mbar_init(&sm.empty[s], 1); }
-        for (int a = 0; a < kGroups; ++a) { mbar_init(&sm.acc_full[a], 1); mbar_init(&sm.acc_empty[a], 1); }
+        for (int a = 0; a < kMaxGroups; ++a) { mbar_init(&sm.acc_full[a], 1); mbar_init(&sm.acc_empty[a], 1); }
         sm.abort_flag = 0;
         mbar_fence_init();
     }
     // label tiles start finite (all zero): rows beyond an item's end multiply zeros, never stale NaNs
-    for (int k = tid; k < kNStage * kStageYBytes / 16; k += kBlockThreads)
+    for (int k = tid; k < kNStage * kStageYBytes / 16; k += C::kBlockThreads)
         st_shared_zero16(smem_u32(&sm.y[0][0]) + k * 16);
-    for (int k = tid; k < kNStage * kStageHBytes / 16; k += kBlockThreads)
+    for (int k = tid; k < kNStage * kStageHBytes / 16; k += C::kBlockThreads)
         st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
+    if (MODE == kModeRows) {
+        for (int e = tid; e < D * D; e += C::kBlockThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
+    }
     fence_proxy_async();
-    if (warp == kMmaWarp) {
+    if (warp == C::kMmaWarp) {
         tmem_alloc(&sm.tmem_base, kTmemCols);
         tmem_relinquish();
     }
@@ -313,18 +558,19 @@ __global__ void __launch_bounds__(kBlockThreads, 1) k_umma(Params p)
     __syncthreads();
     tc_fence_after();
 
-    if (warp < kMmaWarp) {
-        const int gidx = warp / (kThreads / 32);
-        solver_role<MODE>(p, sm, gs[(MODE == kModeRows) ? gidx : 0], gidx, tid - gidx * kThreads);
-    } else if (warp == kMmaWarp) {
+    if (warp < C::kMmaWarp) {
+        const int gidx = warp / (C::kGroupThreads / 32);
+        if (MODE == kModeRows) solver_rows_tmem(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
+        else copyout_role<MODE>(p, sm, gidx, tid - gidx * C::kGroupThreads);
+    } else if (warp == C::kMmaWarp) {
         mma_role<MODE>(p, sm, lane);
     } else {
-        producer_role<MODE>(p, sm, warp - kFirstProducerWarp, lane);
+        producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == kMmaWarp) {
+    if (warp == C::kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(sm.tmem_base, kTmemCols);
     }
@@ -373,19 +619,19 @@ __global__ void __launch_bounds__(kThreads, 2) k_split_solve_umma(SideView sv, i
     if (tid < 32) store_solution<D, __nv_bfloat16>(xq, ok, u, out, st);
 }
 
-size_t smem_bytes(int)
+size_t smem_bytes()
 {
     // the same (large) request in every mode: at most one block per SM, so two blocks never compete for
     // the SM's 512 tensor-memory columns
-    return sizeof(Smem) + 1024 + kGroups * sizeof(GroupSmem);
+    return sizeof(Smem) + 1024 + sizeof(float) * D * kLdB + kMaxGroups * sizeof(RowGroupSmem) + 48 * 1024;
 }
 
 template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStream_t s)
 {
-    const size_t smem = smem_bytes(MODE);
+    const size_t smem = smem_bytes();
     cudaError_t e = cudaFuncSetAttribute(k_umma<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_umma<MODE><<<grid, kBlockThreads, smem, s>>>(p);
+    k_umma<MODE><<<grid, Cfg<MODE>::kBlockThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -399,7 +645,7 @@ int sm_count()
 
 }  // namespace
 
-int64_t gramian_umma_partials() { return (int64_t)kGramBlocks * kGroups; }
+int64_t gramian_umma_partials() { return (int64_t)kGramBlocks * Cfg<kModeGramian>::kGroups; }
 
 // Gramian of a bf16 table with d = 128 on the tensor cores; partials must hold gramian_umma_partials() * d * d floats
 cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches)
