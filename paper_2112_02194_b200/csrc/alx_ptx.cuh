@@ -43,6 +43,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 {
     for (uint32_t it = 0; it < (1u << 22); ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (it > 16u) __nanosleep(it < 256u ? 64u : 256u);     // leave the issue slots to the working warps
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -185,6 +186,12 @@ __host__ __device__ constexpr uint32_t idesc_bf16_mn_major(int M, int N)
            | (1u << 7) | (1u << 10)      // A and B format: bf16
            | (1u << 15) | (1u << 16)     // A and B are MN-major
            | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// bf16 operands, fp32 accumulator, both operands K-major, A negated: D += (-A) * B^T
+__host__ __device__ constexpr uint32_t idesc_bf16_k_major_negA(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 13) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 }  // namespace ptx

@@ -75,11 +75,15 @@ struct GroupSmem {   // split-row solve: one matrix in shared memory
 };
 
 constexpr int kLdB = D + 4;
-struct __align__(16) RowGroupSmem {   // scratch of one tensor-memory solver group (float4 access: 16-byte aligned)
-    float Ps[D][16];        // panel of the current block step, row i = what thread i computed
-    float Lkk[16][16];      // diagonal block of the current step
-    float dinv[16];
-    float z[16];            // the block's part of L^-1 b
+struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver group
+    // Panel of the current block step as tensor-core operands: row i = what thread i computed, split into
+    // three bfloat16 parts (p = p1 + p2 + p3 to 2^-27), each part a K-major 128 x 16 tile without swizzle:
+    // groups of 8 rows take 256 bytes, the two 8-element K halves of a group are 128 bytes apart.
+    unsigned char pop[3][D * 32];
+    uint64_t trail_bar;     // completion of the trailing-update MMAs of the current block step
+    alignas(16) float Lt[16][16];    // transpose of the diagonal block's factor: Lt[p][c] = L[c][p] (read as float4)
+    alignas(16) float dinv[16];
+    alignas(16) float z[16];   // the block's part of L^-1 b
     float red[2][4][16];    // per-warp partial sums of the back substitution (double buffered)
     int bad;
 };
@@ -287,13 +291,15 @@ __device__ void copyout_role(const Params &p, Smem &sm, int gidx, int tid)
 //   (2) rows below the block do their own forward substitution against the block (from shared memory),
 //       publish their panel row, and fold the block's part of L^-1 b into their b; meanwhile each diagonal
 //       thread computes its column of the block's inverse, which it keeps in registers for step (4);
-//   (3) trailing update of the thread's own row, 16 columns at a time, against the published panel rows;
-//       the next block's diagonal threads only have one such column block, so their factorisation
-//       overlaps the other threads' update;
+//   (3) trailing update A22 -= P P^T on the tensor core, in place in tensor memory: six tcgen05.mma
+//       128 x N x 16 (N = columns right of the block) over the three-way bfloat16 split of P
+//       (p1p1 + p1p2 + p2p1 + p1p3 + p3p1 + p2p2, the dropped terms are below 2^-26 relative),
+//       A operand negated by the instruction descriptor;
 //   (4) back substitution block by block from the end: per-block partial sums over the rows below are
 //       reduced in a fixed order (warp butterfly, then four warps in order), the diagonal threads apply
 //       their inverse columns.
-// alpha0 G + lambda I is added from shared memory when an element is first read (block step 0).
+// alpha0 G + lambda I is added from shared memory when a panel is read (every element of the lower triangle
+// is read as part of a panel exactly once; the tensor-core updates commute with that addition).
 __device__ __forceinline__ void warp_reduce16(float (&v)[16], int lane)
 {
     // after the call, lane 2c (and 2c+1) holds the sum over the 32 lanes of v[c], in v[0]
@@ -330,28 +336,54 @@ __device__ __forceinline__ void warp_reduce16(float (&v)[16], int lane)
     v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
 }
 
+// one MUFU instruction, about 2 ulp: the factor absorbs it as a relative perturbation of 2^-22 of the pivot
+__device__ __forceinline__ float rsqrt_fast(float x)
+{
+    float r;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
 __device__ __forceinline__ void group128_sync(int bar_id)
 {
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
 }
 
+#ifdef ALX_PHASE_TIMERS
+__device__ unsigned long long g_phase_cycles[16];
+#define PHASE_MARK(slot)                                                        \
+    do {                                                                        \
+        const long long now_ = clock64();                                       \
+        if (blockIdx.x == 0 && gidx == 0 && tid == 127) atomicAdd(&g_phase_cycles[slot], (unsigned long long)(now_ - t_prev_)); \
+        t_prev_ = now_;                                                         \
+    } while (0)
+#else
+#define PHASE_MARK(slot) do { } while (0)
+#endif
+
 __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, const float *__restrict__ Bs, int gidx,
                                  int tid)
 {
+#ifdef ALX_PHASE_TIMERS
+    long long t_prev_ = clock64();
+#endif
     constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
     const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory
     const int i = tid;                           // my row
     const int bar_id = 1 + gidx;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
     const float *Brow = Bs + i * kLdB;
+    uint32_t trail_parity = 0;
     int64_t it = 0;
     for (int64_t t = blockIdx.x; t < p.n_items; t += gridDim.x, ++it) {
         if ((int)(it % kGroups) != gidx) continue;
         int64_t u, beg, end, slot;
         item_range<kModeRows>(p, t, u, beg, end, slot);
         const uint32_t aph = (uint32_t)((it / kGroups) & 1);
+        PHASE_MARK(0);
         if (!mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag)) break;
         tc_fence_after();
+        PHASE_MARK(1);
         if (tid == 0) gs.bad = 0;
         float b;
         {
@@ -360,6 +392,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             tmem_ld_wait();
             b = __uint_as_float(bv[0]) + __uint_as_float(bv[1]);   // high and low parts of the labels
         }
+        bool dead = false;
         float yinv[16];          // my column of the inverse of my diagonal block (set at my block step)
 #pragma unroll
         for (int c = 0; c < 16; ++c) yinv[c] = 0.f;
@@ -368,64 +401,134 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             const int k0 = 16 * k;
             float a[16];
             const bool warp_live = (w * 32 + 31 >= k0);            // some row of my warp is at or below the block
+            if (k > 0) {
+                // the previous step's tensor-core update must have landed before its results are read
+                if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag)) { dead = true; break; }
+                trail_parity ^= 1u;
+                tc_fence_after();
+            }
             if (warp_live) {
                 tmem_ld16(trow + k0, a);
-                if (k == 0) {
 #pragma unroll
-                    for (int c = 0; c < 16; c += 4) {
-                        const float4 bb = *reinterpret_cast<const float4 *>(Brow + c);
-                        a[c] += bb.x; a[c + 1] += bb.y; a[c + 2] += bb.z; a[c + 3] += bb.w;
-                    }
+                for (int c = 0; c < 16; c += 4) {
+                    const float4 bb = *reinterpret_cast<const float4 *>(Brow + k0 + c);
+                    a[c] += bb.x; a[c + 1] += bb.y; a[c + 2] += bb.z; a[c + 3] += bb.w;
                 }
             }
+            PHASE_MARK(2);
             // (1) diagonal block
             if (w == (k0 >> 5)) {
                 const int hb = k0 & 16;
                 const int l = lane - hb;
                 const bool is_diag = (l >= 0 && l < 16);
                 float my_inv = 0.f;
+                bool all_ok = true;
+                // two pivots per step; branch-free: lanes outside the block run the same code on zero multipliers
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float pj = __shfl_sync(0xFFFFFFFFu, a[j], hb + j);
-                    const bool ok = pj > 0.f;
-                    float inv = ok ? rsqrtf(pj) : 0.f;
-                    inv = inv * fmaf(-0.5f * pj * inv, inv, 1.5f);
-                    if (!ok && lane == 0) gs.bad = 1;
-                    const float zj = __shfl_sync(0xFFFFFFFFu, b, hb + j) * inv;
-                    if (is_diag) {
-                        if (l == j) { a[j] = pj * inv; my_inv = inv; b = zj; }
-                        else { a[j] *= inv; if (l > j) b = fmaf(-a[j], zj, b); }
+                for (int j = 0; j < 16; j += 2) {
+                    const float p00 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j);
+                    const float p10 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j + 1);
+                    const float p11 = __shfl_sync(0xFFFFFFFFu, a[j + 1], hb + j + 1);
+                    const float bj = __shfl_sync(0xFFFFFFFFu, b, hb + j);
+                    const float bj1 = __shfl_sync(0xFFFFFFFFu, b, hb + j + 1);
+                    const bool ok0 = p00 > 0.f;
+                    const float inv0 = ok0 ? rsqrt_fast(p00) : 0.f;
+                    const float l10 = p10 * inv0;
+                    const float q11 = fmaf(-l10, l10, p11);
+                    const bool ok1 = q11 > 0.f;
+                    const float inv1 = ok1 ? rsqrt_fast(q11) : 0.f;
+                    all_ok = all_ok && ok0 && ok1;
+                    const float zj = bj * inv0;
+                    const float zj1 = fmaf(-l10, zj, bj1) * inv1;
+                    const float x0 = a[j] * inv0;                       // L[l][j] for rows below
+                    const float x1 = fmaf(-x0, l10, a[j + 1]) * inv1;   // L[l][j+1] for rows below
+                    const bool below = is_diag && l > j + 1;
+                    const float n0 = (l == j) ? p00 * inv0 : ((l == j + 1) ? l10 : x0);
+                    const float n1 = (l == j + 1) ? q11 * inv1 : x1;
+                    a[j] = is_diag ? n0 : a[j];
+                    a[j + 1] = is_diag ? n1 : a[j + 1];
+                    my_inv = (l == j) ? inv0 : ((l == j + 1) ? inv1 : my_inv);
+                    const float m0 = below ? x0 : 0.f, m1 = below ? x1 : 0.f;
+                    const float bdown = fmaf(-m1, zj1, fmaf(-m0, zj, b));
+                    b = (is_diag && l == j) ? zj : ((is_diag && l == j + 1) ? zj1 : bdown);
+                    // all exchanges of the step first, then the arithmetic: the shuffles pipeline instead of
+                    // each FMA waiting for its own
+                    float lc0[16], lc1[16];
+#pragma unroll
+                    for (int c = j + 2; c < 16; ++c) {
+                        lc0[c] = __shfl_sync(0xFFFFFFFFu, a[j], hb + c);
+                        lc1[c] = __shfl_sync(0xFFFFFFFFu, a[j + 1], hb + c);
                     }
 #pragma unroll
-                    for (int c = j + 1; c < 16; ++c) {
-                        const float lc = __shfl_sync(0xFFFFFFFFu, a[j], hb + c);
-                        if (is_diag) a[c] = fmaf(-a[j], lc, a[c]);
-                    }
+                    for (int c = j + 2; c < 16; ++c) a[c] = fmaf(-m1, lc1[c], fmaf(-m0, lc0[c], a[c]));
                 }
+                if (!all_ok && lane == 0) gs.bad = 1;
                 if (is_diag) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) gs.Lkk[l][c] = (c <= l) ? a[c] : 0.f;
+                    for (int c = 0; c < 16; ++c) gs.Lt[c][l] = (c <= l) ? a[c] : 0.f;
                     gs.dinv[l] = my_inv;
                     gs.z[l] = b;
                 }
             }
+            PHASE_MARK(3);
             group128_sync(bar_id);
+            PHASE_MARK(4);
             // (2) rows below the block: forward substitution; diagonal threads: their column of the inverse
             if (i >= k0 + 16) {
+                // column-oriented forward substitution: after a[pp] is final, it is eliminated from the later
+                // entries, which are independent of each other
+                float dv[16];
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    float s = a[c];
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(&gs.dinv[4 * q4]);
+                    dv[4 * q4] = v.x; dv[4 * q4 + 1] = v.y; dv[4 * q4 + 2] = v.z; dv[4 * q4 + 3] = v.w;
+                }
+                float lt[2][16];
 #pragma unroll
-                    for (int pp = 0; pp < c; ++pp) s = fmaf(-a[pp], gs.Lkk[c][pp], s);
-                    a[c] = s * gs.dinv[c];
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[0][4 * q4]);
+                    lt[0][4 * q4] = v.x; lt[0][4 * q4 + 1] = v.y; lt[0][4 * q4 + 2] = v.z; lt[0][4 * q4 + 3] = v.w;
+                }
+#pragma unroll
+                for (int pp = 0; pp < 16; ++pp) {
+                    // the next row of the block's factor is fetched while this one is applied
+                    if (pp + 1 < 15) {
+#pragma unroll
+                        for (int q4 = (pp + 2) / 4; q4 < 4; ++q4) {
+                            const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[pp + 1][4 * q4]);
+                            lt[(pp + 1) & 1][4 * q4] = v.x; lt[(pp + 1) & 1][4 * q4 + 1] = v.y;
+                            lt[(pp + 1) & 1][4 * q4 + 2] = v.z; lt[(pp + 1) & 1][4 * q4 + 3] = v.w;
+                        }
+                    }
+                    a[pp] *= dv[pp];
+#pragma unroll
+                    for (int c = pp + 1; c < 16; ++c) a[c] = fmaf(-a[pp], lt[pp & 1][c], a[c]);
                 }
                 float acc = 0.f;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) acc = fmaf(a[c], gs.z[c], acc);
                 b -= acc;
+                // three-way bfloat16 split of my panel row into the operand tiles
+                uint32_t w1[8], w2[8], w3[8];
 #pragma unroll
-                for (int c = 0; c < 16; c += 4)
-                    *reinterpret_cast<float4 *>(&gs.Ps[i][c]) = make_float4(a[c], a[c + 1], a[c + 2], a[c + 3]);
+                for (int c = 0; c < 16; c += 2) {
+                    float r0 = a[c], r1 = a[c + 1];
+                    const __nv_bfloat16 h0 = __float2bfloat16_rn(r0), h1 = __float2bfloat16_rn(r1);
+                    r0 -= __bfloat162float(h0); r1 -= __bfloat162float(h1);
+                    const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
+                    r0 -= __bfloat162float(m0); r1 -= __bfloat162float(m1);
+                    const __nv_bfloat16 l0 = __float2bfloat16_rn(r0), l1 = __float2bfloat16_rn(r1);
+                    w1[c >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                    w2[c >> 1] = (uint32_t)__bfloat16_as_ushort(m0) | ((uint32_t)__bfloat16_as_ushort(m1) << 16);
+                    w3[c >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                }
+                const uint32_t roff = (uint32_t)((i >> 3) * 256 + (i & 7) * 16);
+                const uint32_t b1 = smem_u32(&gs.pop[0][0]) + roff, b2 = smem_u32(&gs.pop[1][0]) + roff,
+                               b3 = smem_u32(&gs.pop[2][0]) + roff;
+                st_shared_v4(b1, w1[0], w1[1], w1[2], w1[3]); st_shared_v4(b1 + 128, w1[4], w1[5], w1[6], w1[7]);
+                st_shared_v4(b2, w2[0], w2[1], w2[2], w2[3]); st_shared_v4(b2 + 128, w2[4], w2[5], w2[6], w2[7]);
+                st_shared_v4(b3, w3[0], w3[1], w3[2], w3[3]); st_shared_v4(b3 + 128, w3[4], w3[5], w3[6], w3[7]);
+                fence_proxy_async();
             } else if (i >= k0) {
                 const int l = i - k0;
                 float tacc[16];
@@ -434,45 +537,63 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
 #pragma unroll
                 for (int cp = 0; cp < 16; ++cp) {
                     // y[cp] of the solve L y = e_l
-                    float ycp = (cp < l) ? 0.f : ((cp == l) ? gs.dinv[cp] : -tacc[cp] * gs.dinv[cp]);
+                    const float ycp = (cp < l) ? 0.f : ((cp == l) ? gs.dinv[cp] : -tacc[cp] * gs.dinv[cp]);
                     yinv[cp] = ycp;
+                    float lt[16];
 #pragma unroll
-                    for (int c = cp + 1; c < 16; ++c) tacc[c] = fmaf(gs.Lkk[c][cp], ycp, tacc[c]);
+                    for (int q4 = (cp + 1) / 4; q4 < 4; ++q4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[cp][4 * q4]);
+                        lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int c = cp + 1; c < 16; ++c) tacc[c] = fmaf(lt[c], ycp, tacc[c]);
                 }
             }
+            PHASE_MARK(5);
             if (warp_live) {
                 tmem_st16(trow + k0, a);      // L (rows above the block rewrite what they read)
                 tmem_st_wait();
             }
+            tc_fence_before();
+            PHASE_MARK(6);
             group128_sync(bar_id);
-            // (3) trailing update of my own row
-            for (int cb = k0 + 16; cb < (w + 1) * 32; cb += 16) {
-                float tt[16];
-                tmem_ld16(trow + cb, tt);
-                if (k == 0) {
+            PHASE_MARK(7);
+            // (3) trailing update on the tensor core
+            if (k < D / 16 - 1 && tid == 0) {
+                tc_fence_after();
+                const int n_trail = D - k0 - 16;
+                const uint32_t idesc16 = idesc_bf16_k_major_negA(128, 16);
+                const uint32_t idesc_rest = idesc_bf16_k_major_negA(128, n_trail > 16 ? n_trail - 16 : 16);
+                const uint32_t d_addr = sm.tmem_base + gidx * kAccStride + k0 + 16;
+                const uint32_t boff = (uint32_t)((k0 + 16) * 32);
+                uint64_t da[3], db[3], dc[3];
 #pragma unroll
-                    for (int c = 0; c < 16; c += 4) {
-                        const float4 bb = *reinterpret_cast<const float4 *>(Brow + cb + c);
-                        tt[c] += bb.x; tt[c + 1] += bb.y; tt[c + 2] += bb.z; tt[c + 3] += bb.w;
-                    }
+                for (int q = 0; q < 3; ++q) {
+                    da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
+                    db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + boff, 128, 256, 0);
+                    dc[q] = smem_desc(smem_u32(&gs.pop[q][0]) + boff + 16 * 32, 128, 256, 0);
                 }
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const float4 p0 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][0]);
-                    const float4 p1 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][4]);
-                    const float4 p2 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][8]);
-                    const float4 p3 = *reinterpret_cast<const float4 *>(&gs.Ps[cb + c][12]);
-                    float s = tt[c];
-                    s = fmaf(-a[0], p0.x, s); s = fmaf(-a[1], p0.y, s); s = fmaf(-a[2], p0.z, s); s = fmaf(-a[3], p0.w, s);
-                    s = fmaf(-a[4], p1.x, s); s = fmaf(-a[5], p1.y, s); s = fmaf(-a[6], p1.z, s); s = fmaf(-a[7], p1.w, s);
-                    s = fmaf(-a[8], p2.x, s); s = fmaf(-a[9], p2.y, s); s = fmaf(-a[10], p2.z, s); s = fmaf(-a[11], p2.w, s);
-                    s = fmaf(-a[12], p3.x, s); s = fmaf(-a[13], p3.y, s); s = fmaf(-a[14], p3.z, s); s = fmaf(-a[15], p3.w, s);
-                    tt[c] = s;
+                // the 16 columns that form the next panel first: their completion is all the next step waits for;
+                // the rest follows in issue order and is complete before any later MMA or commit of this thread
+                umma_f16(d_addr, da[0], db[0], idesc16, true);
+                umma_f16(d_addr, da[0], db[1], idesc16, true);
+                umma_f16(d_addr, da[1], db[0], idesc16, true);
+                umma_f16(d_addr, da[0], db[2], idesc16, true);
+                umma_f16(d_addr, da[2], db[0], idesc16, true);
+                umma_f16(d_addr, da[1], db[1], idesc16, true);
+                umma_commit(&gs.trail_bar);
+                if (n_trail > 16) {
+                    umma_f16(d_addr + 16, da[0], dc[0], idesc_rest, true);
+                    umma_f16(d_addr + 16, da[0], dc[1], idesc_rest, true);
+                    umma_f16(d_addr + 16, da[1], dc[0], idesc_rest, true);
+                    umma_f16(d_addr + 16, da[0], dc[2], idesc_rest, true);
+                    umma_f16(d_addr + 16, da[2], dc[0], idesc_rest, true);
+                    umma_f16(d_addr + 16, da[1], dc[1], idesc_rest, true);
                 }
-                tmem_st16(trow + cb, tt);
             }
-            tmem_st_wait();
+            PHASE_MARK(8);
         }
+        if (dead) break;
         // (4) back substitution L^T x = z; b now holds z_i
         float x = 0.f;
         for (int k = D / 16 - 1; k >= 0; --k) {
@@ -504,6 +625,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 if (is_diag) x = acc;
             }
         }
+        PHASE_MARK(9);
         // tensor memory is free again for the next item of this accumulator
         tc_fence_before();
         group128_sync(bar_id);
@@ -520,8 +642,23 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             raise_flag(p.st, kFlagNotSpd, u);
         }
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
+        PHASE_MARK(10);
     }
 }
+
+#ifdef ALX_PHASE_TIMERS
+}  // namespace
+extern "C" int alx_debug_phase_cycles(unsigned long long *out, int reset)
+{
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(unsigned long long) * 16);
+    if (reset) {
+        unsigned long long z[16] = {};
+        cudaMemcpyToSymbol(g_phase_cycles, z, sizeof z);
+    }
+    return (int)e;
+}
+namespace {
+#endif
 
 template <int MODE>
 __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
@@ -548,6 +685,12 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
         st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
     if (MODE == kModeRows) {
         for (int e = tid; e < D * D; e += C::kBlockThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
+        for (int g = 0; g < C::kGroups; ++g) {
+            if (tid == 0) mbar_init(&rgs[g].trail_bar, 1);
+            for (int k = tid; k < 3 * D * 32 / 16; k += C::kBlockThreads)
+                st_shared_zero16(smem_u32(&rgs[g].pop[0][0]) + k * 16);
+        }
+        if (tid == 0) mbar_fence_init();
     }
     fence_proxy_async();
     if (warp == C::kMmaWarp) {
