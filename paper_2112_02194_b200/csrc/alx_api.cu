@@ -140,7 +140,7 @@ alx_status check_device_status(alx_ctx *c)
     if (h.flags & kFlagBadCol) return fail(c, ALX_ERR_BAD_CSR, "column index out of range at entry %lld", h.first_bad);
     if (h.flags & kFlagUnsorted) return fail(c, ALX_ERR_BAD_CSR, "column indices not strictly ascending inside a row at entry %lld", h.first_bad);
     if (h.flags & kFlagNotSpd) return fail(c, ALX_ERR_NOT_SPD, "%llu rows met a non-positive pivot (first: row %lld); they were set to zero", h.not_spd, h.first_bad);
-    if (h.flags & kFlagTimeout) return fail(c, ALX_ERR_CUDA, "a bounded wait inside a kernel ran out (item %lld)", h.first_bad);
+    if (h.flags & kFlagTimeout) return fail(c, ALX_ERR_CUDA, "a bounded wait inside a kernel ran out (wait site %lld, block %lld)", h.first_bad / 1000000, h.first_bad % 1000000);
     return fail(c, ALX_ERR_CUDA, "device status flags 0x%x", h.flags);
 }
 

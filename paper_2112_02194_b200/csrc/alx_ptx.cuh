@@ -23,13 +23,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+// non-blocking test of a phase's completion
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t"
         "}\n"
         : "=r"(ok)
@@ -37,17 +38,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Wait with an iteration limit.  Returns false if the limit ran out or another role of the block has
-// already given up (*abort_flag != 0); the caller then leaves its loop and the block winds down.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+// Wait with a hard limit (about a second: 2^21 polls with up to 0.5 us of sleep in between).  Returns false if
+// the limit ran out or another role of the block has already given up (*abort_flag != 0); the caller then
+// leaves its loop and the block winds down.  *abort_flag records which wait gave up (site code).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1)
 {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 16u) __nanosleep(it < 256u ? 64u : 256u);     // leave the issue slots to the working warps
+    for (uint32_t it = 0; it < (1u << 21); ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if (it > 16u) __nanosleep(it < 256u ? 32u : 500u);     // leave the issue slots to the working warps
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
-    *abort_flag = 1;
+    if (*abort_flag == 0) *abort_flag = site;
     return false;
+}
+
+// One lane polls, the warp follows: keeps the polling traffic of a waiting warp to a single thread.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, site) ? 1 : 0;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    return ok != 0;
 }
 
 // ---- cp.async (16 bytes, L2 only) and proxy fence ----------------------------------------------------

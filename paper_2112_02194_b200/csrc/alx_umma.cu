@@ -22,12 +22,26 @@
 #include "alx_chol.cuh"
 #include "alx_common.cuh"
 #include "alx_ptx.cuh"
+#include <cstring>
 
 namespace alx {
 
 namespace {
 
 using namespace ptx;
+
+#ifdef ALX_TRACE
+__device__ volatile unsigned int *g_trace = nullptr;     // mapped host memory: [block][32] progress words
+#define TRACE(slot, val)                                                                      \
+    do {                                                                                      \
+        if (g_trace && blockIdx.x < 160 && (threadIdx.x & 31) == 0) {                           \
+            g_trace[blockIdx.x * 32 + (slot)] = (unsigned)(val);                              \
+        }                                                                                     \
+    } while (0)
+#else
+#define TRACE(slot, val) do { } while (0)
+#endif
+
 
 constexpr int D = 128;
 constexpr int kStageRows = 32;
@@ -38,7 +52,8 @@ constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
 constexpr int kStageYBytes = 2 * kStageRows * 16;     // 1024: label tile, two 8-column chunks
 constexpr int kProducerWarps = 4;
 constexpr int kTmemCols = 512;
-constexpr int kMaxGroups = 3;
+constexpr int kMaxGroups = 4;
+constexpr int kBRing = 8;                             // rows mode: ring of per-item right-hand sides
 constexpr int kGramSubRows = 256;                     // rows per tensor-memory accumulation of the Gramian (the
                                                       // accumulator truncates: fewer steps, smaller bias)
 constexpr int kGramBlocks = 148;                      // fixed, so that the order of sums depends on sizes only
@@ -46,10 +61,13 @@ constexpr int kGramBlocks = 148;                      // fixed, so that the orde
 enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2 };
 
 // thread layout per mode: solver groups (one accumulator each), then one MMA warp, then the producer warps
+#ifndef ALX_DEBUG_ACTIVE_GROUPS
+#define ALX_DEBUG_ACTIVE_GROUPS 4
+#endif
 template <int MODE> struct Cfg {
-    static constexpr int kGroups = (MODE == kModeRows) ? 3 : 2;
+    static constexpr int kGroups = (MODE == kModeRows) ? ALX_DEBUG_ACTIVE_GROUPS : 2;
     static constexpr int kGroupThreads = (MODE == kModeRows) ? 128 : 256;
-    static constexpr int kAccStride = (MODE == kModeRows) ? 160 : 256;   // accumulator a: columns a * stride .. + 144
+    static constexpr int kAccStride = (MODE == kModeRows) ? 128 : 256;   // accumulator a: columns a * stride ..
     static constexpr int kSolverThreads = kGroups * kGroupThreads;
     static constexpr int kMmaWarp = kSolverThreads / 32;
     static constexpr int kFirstProducerWarp = kMmaWarp + 1;
@@ -77,15 +95,17 @@ struct GroupSmem {   // split-row solve: one matrix in shared memory
 constexpr int kLdB = D + 4;
 struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver group
     // Panel of the current block step as tensor-core operands: row i = what thread i computed, split into
-    // three bfloat16 parts (p = p1 + p2 + p3 to 2^-27), each part a K-major 128 x 16 tile without swizzle:
+    // three bfloat16 parts (p = p1 + p2 + p3 to 2^-24), each part a K-major 128 x 16 tile without swizzle:
     // groups of 8 rows take 256 bytes, the two 8-element K halves of a group are 128 bytes apart.
     unsigned char pop[3][D * 32];
     uint64_t trail_bar;     // completion of the trailing-update MMAs of the current block step
     alignas(16) float Lt[16][16];    // transpose of the diagonal block's factor: Lt[p][c] = L[c][p] (read as float4)
+    alignas(16) float xch[64];       // the two new columns of a diagonal-block step, double buffered
     alignas(16) float dinv[16];
     alignas(16) float z[16];   // the block's part of L^-1 b
     float red[2][4][16];    // per-warp partial sums of the back substitution (double buffered)
     int bad;
+    int stop;               // set by the polling thread when a wait gave up; read by the group after its barrier
 };
 
 struct __align__(1024) Smem {
@@ -94,6 +114,12 @@ struct __align__(1024) Smem {
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
     uint32_t tmem_base;
     int abort_flag;
+    // rows mode: the producer warps also sum y x_i of the rows they staged (four partial sums per item)
+    float ylab[kNStage][kStageRows];          // labels of the staged rows
+    int stage_meta[kNStage];                     // K steps of the stage (1 or 2) | 4 if it ends its item; -1: no more work
+    int rows_staged[kProducerWarps][kNStage];    // per producer warp: how many of its 8 rows of the stage are defined
+    int last_of_item[kProducerWarps][kNStage];   // per producer warp: 1 + ring index of the item whose last stage this is, else 0
+    alignas(16) float bpart[kBRing][kProducerWarps][D];
 };
 
 template <int MODE> __device__ __forceinline__ void item_range(const Params &p, int64_t t, int64_t &u, int64_t &beg,
@@ -115,19 +141,58 @@ template <int MODE> __device__ __forceinline__ void item_range(const Params &p, 
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// rows mode: sum y x over this warp's 8 rows of a landed stage (lane = features 4*lane .. 4*lane+3)
+__device__ __forceinline__ void stage_rhs(Smem &sm, int slot, int pw, int lane, float (&bacc)[4])
+{
+    const int f = 4 * lane;
+    const int half = f >> 6, cc = (f & 63) >> 3, inner = (f & 7) * 2;
+    const unsigned char *base = &sm.h[slot][0] + half * kHalfBytes + pw * 1024;
+    const int nrows = sm.rows_staged[pw][slot];      // rows of this warp that hold data or zeros
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if (j < nrows) {
+            const uint2 v = *reinterpret_cast<const uint2 *>(base + j * 128 + ((cc ^ j) << 4) + inner);
+            const float y = sm.ylab[slot][pw * 8 + j];
+            bacc[0] = fmaf(y, __uint_as_float(v.x << 16), bacc[0]);
+            bacc[1] = fmaf(y, __uint_as_float(v.x & 0xFFFF0000u), bacc[1]);
+            bacc[2] = fmaf(y, __uint_as_float(v.y << 16), bacc[2]);
+            bacc[3] = fmaf(y, __uint_as_float(v.y & 0xFFFF0000u), bacc[3]);
+        }
+    }
+}
+
+template <int MODE> __device__ __forceinline__ void producer_signal(Smem &sm, int64_t signalled, int pw, int lane,
+                                                                   float (&bacc)[4])
+{
+    const int slot = (int)(signalled % kNStage);
+    if (MODE == kModeRows) {
+        __syncwarp();      // every lane's copies of this stage have landed (each lane waited for its own)
+        stage_rhs(sm, slot, pw, lane, bacc);
+        const int last = sm.last_of_item[pw][slot];
+        if (last) {
+            *reinterpret_cast<float4 *>(&sm.bpart[last - 1][pw][4 * lane]) = make_float4(bacc[0], bacc[1], bacc[2], bacc[3]);
+            bacc[0] = bacc[1] = bacc[2] = bacc[3] = 0.f;
+        }
+    }
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.full[slot]);
+}
+
 template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int pw, int lane)
 {
-    int64_t g = 0, signalled = 0;
+    int64_t g = 0, signalled = 0, it = 0;
     const int c = lane & 15;                 // 16-byte chunk of the 256-byte row
     const int half = c >> 3, cc = c & 7;
+    float bacc[4] = {0.f, 0.f, 0.f, 0.f};
     bool alive = true;
-    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x) {
+    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
         int64_t u, beg, end, slot_unused;
         item_range<MODE>(p, t, u, beg, end, slot_unused);
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
-            if (!mbar_wait(&sm.empty[slot], ph ^ 1u, &sm.abort_flag)) { alive = false; break; }
+            if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int rc16 = (rc + 15) & ~15;
             // lanes 0..7 fetch the ids (and labels) of this warp's 8 rows
@@ -137,6 +202,14 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
             if (lane < 8 && my_e < end) {
                 my_idx = (MODE == kModeGramian) ? (int32_t)my_e : p.sv.idx[my_e];
                 my_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[my_e] : 1.f);
+            }
+            if (MODE == kModeRows) {
+                if (lane < 8) sm.ylab[slot][pw * 8 + lane] = my_y;
+                if (lane == 0) {
+                    sm.last_of_item[pw][slot] = (e0 + kStageRows >= end) ? 1 + (int)(it % kBRing) : 0;
+                    const int mine = rc16 - pw * 8;
+                    sm.rows_staged[pw][slot] = mine < 0 ? 0 : (mine > 8 ? 8 : mine);
+                }
             }
             const uint32_t hbase = smem_u32(&sm.h[slot][0]) + half * kHalfBytes + pw * 1024;
             const uint32_t ybase = smem_u32(&sm.y[slot][0]) + pw * 128;
@@ -149,7 +222,7 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
                 const uint32_t dst = hbase + j * 128 + ((cc ^ j) << 4);
                 if (src >= 0) cp_async16(dst, p.X + (int64_t)src * D + c * 8);
                 else if (r < rc16) st_shared_zero16(dst);
-                if (MODE != kModeGramian && c == 0 && r < rc16) {
+                if (MODE == kModeChunks && c == 0 && r < rc16) {
                     const __nv_bfloat16 yhi = __float2bfloat16_rn(yv);
                     const __nv_bfloat16 ylo = __float2bfloat16_rn(yv - __bfloat162float(yhi));
                     const uint32_t packed = (uint32_t)__bfloat16_as_ushort(yhi) | ((uint32_t)__bfloat16_as_ushort(ylo) << 16);
@@ -160,18 +233,13 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
             ++g;
             if (g > kLag) {
                 cp_async_wait<kLag>();
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.full[signalled % kNStage]);
+                producer_signal<MODE>(sm, signalled, pw, lane, bacc);
                 ++signalled;
             }
         }
     }
     cp_async_wait<0>();
-    fence_proxy_async();
-    __syncwarp();
-    if (lane == 0)
-        for (; signalled < g; ++signalled) mbar_arrive(&sm.full[signalled % kNStage]);
+    for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
 }
 
 template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane)
@@ -186,14 +254,14 @@ template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane
         item_range<MODE>(p, t, u, beg, end, slot_unused);
         const int a = (int)(it % Cfg<MODE>::kGroups);
         const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
-        if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag)) break;
+        if (!mbar_wait_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
         tc_fence_after();
         const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
         bool first = true;
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
-            if (!mbar_wait(&sm.full[slot], ph, &sm.abort_flag)) { alive = false; break; }
+            if (!mbar_wait_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) { alive = false; break; }
             tc_fence_after();
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int nk = (rc + 15) >> 4;
@@ -204,7 +272,7 @@ template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane
                     // 16 gathered rows = two groups of 8 rows of 128 bytes; halves are kHalfBytes apart
                     const uint64_t adesc = smem_desc(hb + ks * 2048, kHalfBytes, 1024, 2);
                     umma_f16(d_main, adesc, adesc, kIdescMain, !first);
-                    if (MODE != kModeGramian) {
+                    if (MODE == kModeChunks) {
                         const uint64_t ydesc = smem_desc(yb + ks * 256, 128, kStageRows * 16, 0);
                         umma_f16(d_main + D, adesc, ydesc, kIdescY, !first);
                     }
@@ -240,7 +308,7 @@ __device__ void copyout_role(const Params &p, Smem &sm, int gidx, int tid)
         int64_t u, beg, end, slot;
         item_range<MODE>(p, t, u, beg, end, slot);
         const uint32_t aph = (uint32_t)((it >> 1) & 1);
-        if (!mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag)) break;
+        if (!mbar_wait_warp(&sm.acc_full[gidx], aph, &sm.abort_flag, 50 + MODE)) break;
         tc_fence_after();
         const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + gidx * kAccStride + hh * 64;
         uint32_t v0[32], v1[32];
@@ -368,8 +436,14 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
     long long t_prev_ = clock64();
 #endif
     constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
-    const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory
-    const int i = tid;                           // my row
+    const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory (= the SM sub-partition)
+    const int i = tid;                           // my row of the matrix (= feature index = tensor-memory lane)
+    // Group g eliminates in the cyclic order rot, rot+1, ..., 127, 0, ..., rot-1 (a symmetric permutation of the
+    // matrix): the rows that stay active longest then sit in a different lane quarter, hence on a different
+    // sub-partition's scheduler, for every group.
+    const int rot = (32 * gidx) & (D - 1);
+    const int pos = (i - rot) & (D - 1);         // my place in the elimination order
+    const int wpos = pos & ~31;                  // first place of my warp
     const int bar_id = 1 + gidx;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
     const float *Brow = Bs + i * kLdB;
@@ -380,18 +454,20 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         int64_t u, beg, end, slot;
         item_range<kModeRows>(p, t, u, beg, end, slot);
         const uint32_t aph = (uint32_t)((it / kGroups) & 1);
+        if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000);
         PHASE_MARK(0);
-        if (!mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag)) break;
+        // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
+        if (tid == 0) {
+            gs.stop = mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
+            gs.bad = 0;
+        }
+        group128_sync(bar_id);
+        if (gs.stop) break;
         tc_fence_after();
         PHASE_MARK(1);
-        if (tid == 0) gs.bad = 0;
-        float b;
-        {
-            uint32_t bv[4];
-            tmem_ld4(trow + D, bv);
-            tmem_ld_wait();
-            b = __uint_as_float(bv[0]) + __uint_as_float(bv[1]);   // high and low parts of the labels
-        }
+        // right-hand side: the four producer warps' partial sums, in order
+        const float *bp = &sm.bpart[it % kBRing][0][i];
+        float b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
         bool dead = false;
         float yinv[16];          // my column of the inverse of my diagonal block (set at my block step)
 #pragma unroll
@@ -399,25 +475,27 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
 
         for (int k = 0; k < D / 16; ++k) {
             const int k0 = 16 * k;
+            const int ck = (k0 + rot) & (D - 1);                   // tensor-memory columns of this block
             float a[16];
-            const bool warp_live = (w * 32 + 31 >= k0);            // some row of my warp is at or below the block
+            const bool warp_live = (wpos + 31 >= k0);              // some row of my warp is at or after the block
             if (k > 0) {
-                // the previous step's tensor-core update must have landed before its results are read
-                if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag)) { dead = true; break; }
-                trail_parity ^= 1u;
+                // the previous step's tensor-core update of these columns has landed: the issuing thread waited
+                // for it before the group's barrier at the end of that step
+                if (gs.stop) { dead = true; break; }
                 tc_fence_after();
             }
             if (warp_live) {
-                tmem_ld16(trow + k0, a);
+                tmem_ld16(trow + ck, a);
 #pragma unroll
                 for (int c = 0; c < 16; c += 4) {
-                    const float4 bb = *reinterpret_cast<const float4 *>(Brow + k0 + c);
+                    const float4 bb = *reinterpret_cast<const float4 *>(Brow + ck + c);
                     a[c] += bb.x; a[c + 1] += bb.y; a[c + 2] += bb.z; a[c + 3] += bb.w;
                 }
             }
+            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 1);
             PHASE_MARK(2);
             // (1) diagonal block
-            if (w == (k0 >> 5)) {
+            if (wpos == (k0 & ~31)) {
                 const int hb = k0 & 16;
                 const int l = lane - hb;
                 const bool is_diag = (l >= 0 && l < 16);
@@ -451,16 +529,20 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     const float m0 = below ? x0 : 0.f, m1 = below ? x1 : 0.f;
                     const float bdown = fmaf(-m1, zj1, fmaf(-m0, zj, b));
                     b = (is_diag && l == j) ? zj : ((is_diag && l == j + 1) ? zj1 : bdown);
-                    // all exchanges of the step first, then the arithmetic: the shuffles pipeline instead of
-                    // each FMA waiting for its own
-                    float lc0[16], lc1[16];
+                    // the two new columns go through shared memory (shuffles are the slower path for 2 x 14 values)
+                    float *xb = &gs.xch[(j & 2) * 16];
+                    if (is_diag) { xb[l] = x0; xb[16 + l] = x1; }
+                    __syncwarp();
+                    float c0[16], c1[16];
 #pragma unroll
-                    for (int c = j + 2; c < 16; ++c) {
-                        lc0[c] = __shfl_sync(0xFFFFFFFFu, a[j], hb + c);
-                        lc1[c] = __shfl_sync(0xFFFFFFFFu, a[j + 1], hb + c);
+                    for (int q4 = (j + 2) / 4; q4 < 4; ++q4) {
+                        const float4 u4 = *reinterpret_cast<const float4 *>(&xb[4 * q4]);
+                        const float4 v4 = *reinterpret_cast<const float4 *>(&xb[16 + 4 * q4]);
+                        c0[4 * q4] = u4.x; c0[4 * q4 + 1] = u4.y; c0[4 * q4 + 2] = u4.z; c0[4 * q4 + 3] = u4.w;
+                        c1[4 * q4] = v4.x; c1[4 * q4 + 1] = v4.y; c1[4 * q4 + 2] = v4.z; c1[4 * q4 + 3] = v4.w;
                     }
 #pragma unroll
-                    for (int c = j + 2; c < 16; ++c) a[c] = fmaf(-m1, lc1[c], fmaf(-m0, lc0[c], a[c]));
+                    for (int c = j + 2; c < 16; ++c) a[c] = fmaf(-m1, c1[c], fmaf(-m0, c0[c], a[c]));
                 }
                 if (!all_ok && lane == 0) gs.bad = 1;
                 if (is_diag) {
@@ -470,57 +552,51 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     gs.z[l] = b;
                 }
             }
+            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 2);
             PHASE_MARK(3);
             group128_sync(bar_id);
+            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 3);
             PHASE_MARK(4);
-            // (2) rows below the block: forward substitution; diagonal threads: their column of the inverse
-            if (i >= k0 + 16) {
-                // column-oriented forward substitution: after a[pp] is final, it is eliminated from the later
-                // entries, which are independent of each other
+            // (2) rows after the block: forward substitution; diagonal threads: their column of the inverse
+            if (pos >= k0 + 16) {
                 float dv[16];
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     const float4 v = *reinterpret_cast<const float4 *>(&gs.dinv[4 * q4]);
                     dv[4 * q4] = v.x; dv[4 * q4 + 1] = v.y; dv[4 * q4 + 2] = v.z; dv[4 * q4 + 3] = v.w;
                 }
-                float lt[2][16];
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[0][4 * q4]);
-                    lt[0][4 * q4] = v.x; lt[0][4 * q4 + 1] = v.y; lt[0][4 * q4 + 2] = v.z; lt[0][4 * q4 + 3] = v.w;
-                }
+                // column-oriented: once a[pp] is final it is eliminated from the later entries, which are
+                // independent of each other
 #pragma unroll
                 for (int pp = 0; pp < 16; ++pp) {
-                    // the next row of the block's factor is fetched while this one is applied
-                    if (pp + 1 < 15) {
+                    float lt[16];
 #pragma unroll
-                        for (int q4 = (pp + 2) / 4; q4 < 4; ++q4) {
-                            const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[pp + 1][4 * q4]);
-                            lt[(pp + 1) & 1][4 * q4] = v.x; lt[(pp + 1) & 1][4 * q4 + 1] = v.y;
-                            lt[(pp + 1) & 1][4 * q4 + 2] = v.z; lt[(pp + 1) & 1][4 * q4 + 3] = v.w;
-                        }
+                    for (int q4 = (pp + 1) / 4; q4 < 4; ++q4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[pp][4 * q4]);
+                        lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
                     }
                     a[pp] *= dv[pp];
 #pragma unroll
-                    for (int c = pp + 1; c < 16; ++c) a[c] = fmaf(-a[pp], lt[pp & 1][c], a[c]);
+                    for (int c = pp + 1; c < 16; ++c) a[c] = fmaf(-a[pp], lt[c], a[c]);
                 }
                 float acc = 0.f;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) acc = fmaf(a[c], gs.z[c], acc);
                 b -= acc;
-                // three-way bfloat16 split of my panel row into the operand tiles
+                PHASE_MARK(11);
                 uint32_t w1[8], w2[8], w3[8];
 #pragma unroll
                 for (int c = 0; c < 16; c += 2) {
-                    float r0 = a[c], r1 = a[c + 1];
-                    const __nv_bfloat16 h0 = __float2bfloat16_rn(r0), h1 = __float2bfloat16_rn(r1);
-                    r0 -= __bfloat162float(h0); r1 -= __bfloat162float(h1);
-                    const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
-                    r0 -= __bfloat162float(m0); r1 -= __bfloat162float(m1);
-                    const __nv_bfloat16 l0 = __float2bfloat16_rn(r0), l1 = __float2bfloat16_rn(r1);
-                    w1[c >> 1] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                    w2[c >> 1] = (uint32_t)__bfloat16_as_ushort(m0) | ((uint32_t)__bfloat16_as_ushort(m1) << 16);
-                    w3[c >> 1] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                    // part 1 rounds to nearest (one packed conversion); parts 2 and 3 keep the leading 8 bits of
+                    // what is left, so p1 + p2 + p3 = p up to 2^-24
+                    const __nv_bfloat162 hpair = __floats2bfloat162_rn(a[c], a[c + 1]);
+                    const uint32_t hw = *reinterpret_cast<const uint32_t *>(&hpair);
+                    const float r0 = a[c] - __uint_as_float(hw << 16), r1 = a[c + 1] - __uint_as_float(hw & 0xFFFF0000u);
+                    const uint32_t m0 = __float_as_uint(r0) & 0xFFFF0000u, m1 = __float_as_uint(r1) & 0xFFFF0000u;
+                    const float s0 = r0 - __uint_as_float(m0), s1 = r1 - __uint_as_float(m1);
+                    w1[c >> 1] = hw;
+                    w2[c >> 1] = (m0 >> 16) | m1;
+                    w3[c >> 1] = (__float_as_uint(s0) >> 16) | (__float_as_uint(s1) & 0xFFFF0000u);
                 }
                 const uint32_t roff = (uint32_t)((i >> 3) * 256 + (i & 7) * 16);
                 const uint32_t b1 = smem_u32(&gs.pop[0][0]) + roff, b2 = smem_u32(&gs.pop[1][0]) + roff,
@@ -528,9 +604,11 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 st_shared_v4(b1, w1[0], w1[1], w1[2], w1[3]); st_shared_v4(b1 + 128, w1[4], w1[5], w1[6], w1[7]);
                 st_shared_v4(b2, w2[0], w2[1], w2[2], w2[3]); st_shared_v4(b2 + 128, w2[4], w2[5], w2[6], w2[7]);
                 st_shared_v4(b3, w3[0], w3[1], w3[2], w3[3]); st_shared_v4(b3 + 128, w3[4], w3[5], w3[6], w3[7]);
+                PHASE_MARK(12);
                 fence_proxy_async();
-            } else if (i >= k0) {
-                const int l = i - k0;
+                PHASE_MARK(13);
+            } else if (pos >= k0) {
+                const int l = pos - k0;
                 float tacc[16];
 #pragma unroll
                 for (int c = 0; c < 16; ++c) tacc[c] = 0.f;
@@ -551,45 +629,53 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             }
             PHASE_MARK(5);
             if (warp_live) {
-                tmem_st16(trow + k0, a);      // L (rows above the block rewrite what they read)
+                tmem_st16(trow + ck, a);      // L (rows before the block rewrite what they read)
                 tmem_st_wait();
             }
             tc_fence_before();
+            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 4);
             PHASE_MARK(6);
             group128_sync(bar_id);
+            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 5);
             PHASE_MARK(7);
             // (3) trailing update on the tensor core
             if (k < D / 16 - 1 && tid == 0) {
                 tc_fence_after();
-                const int n_trail = D - k0 - 16;
-                const uint32_t idesc16 = idesc_bf16_k_major_negA(128, 16);
-                const uint32_t idesc_rest = idesc_bf16_k_major_negA(128, n_trail > 16 ? n_trail - 16 : 16);
-                const uint32_t d_addr = sm.tmem_base + gidx * kAccStride + k0 + 16;
-                const uint32_t boff = (uint32_t)((k0 + 16) * 32);
-                uint64_t da[3], db[3], dc[3];
+                const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
+                uint64_t da[3];
 #pragma unroll
-                for (int q = 0; q < 3; ++q) {
-                    da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
-                    db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + boff, 128, 256, 0);
-                    dc[q] = smem_desc(smem_u32(&gs.pop[q][0]) + boff + 16 * 32, 128, 256, 0);
-                }
-                // the 16 columns that form the next panel first: their completion is all the next step waits for;
-                // the rest follows in issue order and is complete before any later MMA or commit of this thread
-                umma_f16(d_addr, da[0], db[0], idesc16, true);
-                umma_f16(d_addr, da[0], db[1], idesc16, true);
-                umma_f16(d_addr, da[1], db[0], idesc16, true);
-                umma_f16(d_addr, da[0], db[2], idesc16, true);
-                umma_f16(d_addr, da[2], db[0], idesc16, true);
-                umma_f16(d_addr, da[1], db[1], idesc16, true);
+                for (int q = 0; q < 3; ++q) da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
+                // columns [c_lo, c_lo + n) of the matrix (= panel rows c_lo ..) -= P P^T restricted to them
+                auto update = [&](int c_lo, int n) {
+                    const uint32_t idesc = idesc_bf16_k_major_negA(128, n);
+                    uint64_t db[3];
+#pragma unroll
+                    for (int q = 0; q < 3; ++q) db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + (uint32_t)(c_lo * 32), 128, 256, 0);
+                    umma_f16(d_base + c_lo, da[0], db[0], idesc, true);
+                    umma_f16(d_base + c_lo, da[0], db[1], idesc, true);
+                    umma_f16(d_base + c_lo, da[1], db[0], idesc, true);
+                    umma_f16(d_base + c_lo, da[0], db[2], idesc, true);
+                    umma_f16(d_base + c_lo, da[2], db[0], idesc, true);
+                    umma_f16(d_base + c_lo, da[1], db[1], idesc, true);
+                };
+                // the 16 columns of the next panel first: their completion is all the next step waits for; the rest
+                // follows in issue order and is complete before any later MMA or commit of this thread
+                update((k0 + 16 + rot) & (D - 1), 16);
                 umma_commit(&gs.trail_bar);
-                if (n_trail > 16) {
-                    umma_f16(d_addr + 16, da[0], dc[0], idesc_rest, true);
-                    umma_f16(d_addr + 16, da[0], dc[1], idesc_rest, true);
-                    umma_f16(d_addr + 16, da[1], dc[0], idesc_rest, true);
-                    umma_f16(d_addr + 16, da[0], dc[2], idesc_rest, true);
-                    umma_f16(d_addr + 16, da[2], dc[0], idesc_rest, true);
-                    umma_f16(d_addr + 16, da[1], dc[1], idesc_rest, true);
+                const int n_rest = D - k0 - 32;
+                if (n_rest > 0) {
+                    const int cs = (k0 + 32 + rot) & (D - 1);
+                    const int n1 = (n_rest < D - cs) ? n_rest : D - cs;     // up to the wrap-around
+                    update(cs, n1);
+                    if (n_rest > n1) update(0, n_rest - n1);
                 }
+                TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 6);
+                if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag, 70)) gs.stop = 1;
+                TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 7);
+            }
+            if (k < D / 16 - 1) {
+                trail_parity ^= 1u;
+                group128_sync(bar_id);
             }
             PHASE_MARK(8);
         }
@@ -598,19 +684,20 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         float x = 0.f;
         for (int k = D / 16 - 1; k >= 0; --k) {
             const int k0 = 16 * k;
+            const int ck = (k0 + rot) & (D - 1);
             float wv[16];
-            if (w * 32 + 31 >= k0 + 16) {
-                tmem_ld16(trow + k0, wv);
-                const float xm = (i >= k0 + 16) ? x : 0.f;
+            if (wpos + 31 >= k0 + 16) {
+                tmem_ld16(trow + ck, wv);
+                const float xm = (pos >= k0 + 16) ? x : 0.f;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) wv[c] = (i >= k0 + 16) ? wv[c] * xm : 0.f;
+                for (int c = 0; c < 16; ++c) wv[c] = (pos >= k0 + 16) ? wv[c] * xm : 0.f;
                 warp_reduce16(wv, lane);
             } else {
                 wv[0] = 0.f;
             }
             if ((lane & 1) == 0) gs.red[k & 1][w][lane >> 1] = wv[0];
             group128_sync(bar_id);
-            if (w == (k0 >> 5)) {
+            if (wpos == (k0 & ~31)) {
                 const int hb = k0 & 16;
                 const int l = lane - hb;
                 const bool is_diag = (l >= 0 && l < 16);
@@ -625,10 +712,13 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 if (is_diag) x = acc;
             }
         }
+        if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + 900);
         PHASE_MARK(9);
         // tensor memory is free again for the next item of this accumulator
         tc_fence_before();
+        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 1);
         group128_sync(bar_id);
+        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 2);
         if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
         const bool ok = gs.bad == 0;
         const float xo = ok ? x : 0.f;
@@ -641,10 +731,21 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             atomicAdd(&p.st->not_spd, 1ull);
             raise_flag(p.st, kFlagNotSpd, u);
         }
+        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 3);
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
+        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 4);
         PHASE_MARK(10);
     }
 }
+
+#ifdef ALX_TRACE
+}  // namespace
+extern "C" int alx_debug_set_trace(void *dev_ptr)
+{
+    return (int)cudaMemcpyToSymbol(g_trace, &dev_ptr, sizeof dev_ptr);
+}
+namespace {
+#endif
 
 #ifdef ALX_PHASE_TIMERS
 }  // namespace
@@ -665,8 +766,9 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
 {
     using C = Cfg<MODE>;
     extern __shared__ unsigned char smem_raw[];
-    // 1024-byte alignment for the swizzled stages
-    unsigned char *aligned = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte alignment for the swizzled stages; plain offset arithmetic on the shared array, so that the
+    // compiler keeps every access below in the shared address space (no generic loads)
+    unsigned char *aligned = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     Smem &sm = *reinterpret_cast<Smem *>(aligned);
     float *Bs = reinterpret_cast<float *>(aligned + sizeof(Smem));
     RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(Smem) + sizeof(float) * D * kLdB);
@@ -705,19 +807,25 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
         const int gidx = warp / (C::kGroupThreads / 32);
         if (MODE == kModeRows) solver_rows_tmem(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
         else copyout_role<MODE>(p, sm, gidx, tid - gidx * C::kGroupThreads);
+        if ((warp & 3) == 0) TRACE(16 + gidx, 1 + 10 * MODE);
     } else if (warp == C::kMmaWarp) {
         mma_role<MODE>(p, sm, lane);
+        TRACE(7, 1 + 10 * MODE);
     } else {
         producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
+        TRACE(20 + warp - C::kFirstProducerWarp, 1 + 10 * MODE);
     }
 
     tc_fence_before();
     __syncthreads();
+    if (tid == 0) TRACE(24, 1 + 10 * MODE);
+    if (warp == C::kMmaWarp) TRACE(25, 1 + 10 * MODE);
     if (warp == C::kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(sm.tmem_base, kTmemCols);
+        TRACE(25, 2 + 10 * MODE);
     }
-    if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, blockIdx.x);
+    if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, (long long)sm.abort_flag * 1000000 + blockIdx.x);
 }
 
 __global__ void k_zero_rows_bf16(const int32_t *__restrict__ rows, int64_t count, RowOut out)
@@ -766,7 +874,7 @@ size_t smem_bytes()
 {
     // the same (large) request in every mode: at most one block per SM, so two blocks never compete for
     // the SM's 512 tensor-memory columns
-    return sizeof(Smem) + 1024 + sizeof(float) * D * kLdB + kMaxGroups * sizeof(RowGroupSmem) + 48 * 1024;
+    return sizeof(Smem) + 1024 + sizeof(float) * D * kLdB + kMaxGroups * sizeof(RowGroupSmem);   // about 200 KB
 }
 
 template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStream_t s)
