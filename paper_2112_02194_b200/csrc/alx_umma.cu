@@ -30,17 +30,6 @@ namespace {
 
 using namespace ptx;
 
-#ifdef ALX_TRACE
-__device__ volatile unsigned int *g_trace = nullptr;     // mapped host memory: [block][32] progress words
-#define TRACE(slot, val)                                                                      \
-    do {                                                                                      \
-        if (g_trace && blockIdx.x < 160 && (threadIdx.x & 31) == 0) {                           \
-            g_trace[blockIdx.x * 32 + (slot)] = (unsigned)(val);                              \
-        }                                                                                     \
-    } while (0)
-#else
-#define TRACE(slot, val) do { } while (0)
-#endif
 
 
 constexpr int D = 128;
@@ -53,7 +42,7 @@ constexpr int kStageYBytes = 2 * kStageRows * 16;     // 1024: label tile, two 8
 constexpr int kProducerWarps = 4;
 constexpr int kTmemCols = 512;
 constexpr int kMaxGroups = 4;
-constexpr int kBRing = 8;                             // rows mode: ring of per-item right-hand sides
+constexpr int kBRing = 16;                            // rows mode: ring of per-item right-hand sides
 constexpr int kGramSubRows = 256;                     // rows per tensor-memory accumulation of the Gramian (the
                                                       // accumulator truncates: fewer steps, smaller bias)
 constexpr int kGramBlocks = 148;                      // fixed, so that the order of sums depends on sizes only
@@ -98,7 +87,8 @@ struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver gr
     // three bfloat16 parts (p = p1 + p2 + p3 to 2^-24), each part a K-major 128 x 16 tile without swizzle:
     // groups of 8 rows take 256 bytes, the two 8-element K halves of a group are 128 bytes apart.
     unsigned char pop[3][D * 32];
-    uint64_t trail_bar;     // completion of the trailing-update MMAs of the current block step
+    uint64_t trail_bar;     // completion of the next-panel part of the trailing update of the current block step
+    uint64_t rest_bar;      // completion of the remaining part (the operand tiles may be rewritten after it)
     alignas(16) float Lt[16][16];    // transpose of the diagonal block's factor: Lt[p][c] = L[c][p] (read as float4)
     alignas(16) float xch[64];       // the two new columns of a diagonal-block step, double buffered
     alignas(16) float dinv[16];
@@ -454,7 +444,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         int64_t u, beg, end, slot;
         item_range<kModeRows>(p, t, u, beg, end, slot);
         const uint32_t aph = (uint32_t)((it / kGroups) & 1);
-        if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000);
         PHASE_MARK(0);
         // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
         if (tid == 0) {
@@ -492,7 +481,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     a[c] += bb.x; a[c + 1] += bb.y; a[c + 2] += bb.z; a[c + 3] += bb.w;
                 }
             }
-            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 1);
             PHASE_MARK(2);
             // (1) diagonal block
             if (wpos == (k0 & ~31)) {
@@ -552,10 +540,10 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     gs.z[l] = b;
                 }
             }
-            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 2);
             PHASE_MARK(3);
+            // the previous step's whole tensor-core update has read its operand tiles before they are rewritten
+            if (k > 0 && tid == 0 && !mbar_wait(&gs.rest_bar, trail_parity ^ 1u, &sm.abort_flag, 80)) gs.stop = 1;
             group128_sync(bar_id);
-            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 3);
             PHASE_MARK(4);
             // (2) rows after the block: forward substitution; diagonal threads: their column of the inverse
             if (pos >= k0 + 16) {
@@ -633,10 +621,8 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 tmem_st_wait();
             }
             tc_fence_before();
-            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 4);
             PHASE_MARK(6);
             group128_sync(bar_id);
-            if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 5);
             PHASE_MARK(7);
             // (3) trailing update on the tensor core
             if (k < D / 16 - 1 && tid == 0) {
@@ -669,9 +655,8 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     update(cs, n1);
                     if (n_rest > n1) update(0, n_rest - n1);
                 }
-                TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 6);
+                umma_commit(&gs.rest_bar);
                 if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag, 70)) gs.stop = 1;
-                TRACE(8 + gidx, (unsigned)it * 1000 + k * 10 + 7);
             }
             if (k < D / 16 - 1) {
                 trail_parity ^= 1u;
@@ -712,13 +697,10 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 if (is_diag) x = acc;
             }
         }
-        if (w == 0) TRACE(8 + gidx, (unsigned)it * 1000 + 900);
         PHASE_MARK(9);
         // tensor memory is free again for the next item of this accumulator
         tc_fence_before();
-        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 1);
         group128_sync(bar_id);
-        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 2);
         if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
         const bool ok = gs.bad == 0;
         const float xo = ok ? x : 0.f;
@@ -731,21 +713,11 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             atomicAdd(&p.st->not_spd, 1ull);
             raise_flag(p.st, kFlagNotSpd, u);
         }
-        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 3);
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
-        TRACE(26 + (w & 3), 1000 * (unsigned)gidx + 4);
         PHASE_MARK(10);
     }
 }
 
-#ifdef ALX_TRACE
-}  // namespace
-extern "C" int alx_debug_set_trace(void *dev_ptr)
-{
-    return (int)cudaMemcpyToSymbol(g_trace, &dev_ptr, sizeof dev_ptr);
-}
-namespace {
-#endif
 
 #ifdef ALX_PHASE_TIMERS
 }  // namespace
@@ -788,7 +760,7 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
     if (MODE == kModeRows) {
         for (int e = tid; e < D * D; e += C::kBlockThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
         for (int g = 0; g < C::kGroups; ++g) {
-            if (tid == 0) mbar_init(&rgs[g].trail_bar, 1);
+            if (tid == 0) { mbar_init(&rgs[g].trail_bar, 1); mbar_init(&rgs[g].rest_bar, 1); }
             for (int k = tid; k < 3 * D * 32 / 16; k += C::kBlockThreads)
                 st_shared_zero16(smem_u32(&rgs[g].pop[0][0]) + k * 16);
         }
@@ -807,23 +779,17 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
         const int gidx = warp / (C::kGroupThreads / 32);
         if (MODE == kModeRows) solver_rows_tmem(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
         else copyout_role<MODE>(p, sm, gidx, tid - gidx * C::kGroupThreads);
-        if ((warp & 3) == 0) TRACE(16 + gidx, 1 + 10 * MODE);
     } else if (warp == C::kMmaWarp) {
         mma_role<MODE>(p, sm, lane);
-        TRACE(7, 1 + 10 * MODE);
     } else {
         producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
-        TRACE(20 + warp - C::kFirstProducerWarp, 1 + 10 * MODE);
     }
 
     tc_fence_before();
     __syncthreads();
-    if (tid == 0) TRACE(24, 1 + 10 * MODE);
-    if (warp == C::kMmaWarp) TRACE(25, 1 + 10 * MODE);
     if (warp == C::kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(sm.tmem_base, kTmemCols);
-        TRACE(25, 2 + 10 * MODE);
     }
     if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, (long long)sm.abort_flag * 1000000 + blockIdx.x);
 }
