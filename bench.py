@@ -39,6 +39,9 @@ WORKLOADS = {
     "cfg2": dict(n=1_000_000, nnz=50_000_000, s=1.2, cap=100_000, law="zipf", delta=0, d=64,
                  lam=0.05, alpha=0.001, storage="f32", seed=0xA1C50002, init_seed=0x1A150002,
                  desc="1M x 1M, 5e7 entries, Zipf(1.2) out- and in-degrees (cap 1e5), d=64, fp32 tables"),
+    "medium": dict(n=2_000_000, nnz=200_000_000, s=1.1, cap=200_000, law="local", delta=20_000, d=128,
+                   lam=0.01, alpha=0.001, storage="bf16", seed=0xA1C500FE, init_seed=0x1A1500FE,
+                   desc="2M x 2M, 2e8 entries, scaled-down cfg3 whose tables exceed L2 (profiling case)"),
     "small": dict(n=200_000, nnz=10_000_000, s=1.1, cap=40_000, law="local", delta=2_000, d=128,
                   lam=0.01, alpha=0.001, storage="bf16", seed=0xA1C500FF, init_seed=0x1A1500FF,
                   desc="200k x 200k, 1e7 entries, scaled-down cfg3 (debugging / profiling case)"),
@@ -129,7 +132,8 @@ def oracle_sample(w, target_rows, budget_s=None):
     rows = np.arange(min(target_rows, n), dtype=np.int64)
     ptr, cols = graphs.row_columns_flat(spec, rows, deg[rows])
     uniq, inv = np.unique(cols, return_inverse=True)
-    X = graphs.storage_to_f64(graphs.init_embedding_rows(uniq, d, w["init_seed"], 3, w["storage"]), w["storage"])
+    from synth import host as synth_host
+    X = graphs.storage_to_f64(synth_host.embedding_rows(d, w["init_seed"], 3, w["storage"], rows=uniq), w["storage"])
     cores = os.cpu_count() or 1
     t0 = time.perf_counter()
     G = ials.gramian(X)
@@ -171,7 +175,7 @@ def run_reference(args, w):
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    rows = {"cfg3": 60_000, "cfg2": 100_000, "small": 30_000}[w["name"]]
+    rows = {"cfg3": 60_000, "cfg2": 100_000, "small": 30_000, "medium": 30_000}[w["name"]]
     vals = []
     info = None
     for _ in range(args.warmup):
@@ -327,7 +331,7 @@ def run_ours(args, w):
                          "alx_epoch + alx_get_embeddings x2, pinned host buffers"}
         b.destroy()
     if rank == 0 and world == 1 and not args.skip_cpu:
-        v, info = oracle_sample(w, {"cfg3": 60_000, "cfg2": 100_000, "small": 30_000}[w["name"]])
+        v, info = oracle_sample(w, {"cfg3": 60_000, "cfg2": 100_000, "small": 30_000, "medium": 30_000}[w["name"]])
         info["value"] = v
         cpu_baseline = info
 

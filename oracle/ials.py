@@ -72,6 +72,15 @@ def gramian(X):
     return G
 
 
+def gramian_stream(block_fn, N, d, block_rows=250_000):
+    """Gramian of a table too large to hold in fp64: ``block_fn(row_begin, row_count)`` returns that block of
+    rows as fp64 (already rounded to the storage type); blocks are added in order."""
+    G = np.zeros((d, d), dtype=np.float64)
+    for r0 in range(0, N, block_rows):
+        G += gramian(block_fn(r0, min(block_rows, N - r0)))
+    return G
+
+
 def half_step(rowptr, colidx, values, X_fixed, alpha, lam, storage="f64", row_ids=None, G=None,
               return_raw=False, counters=None):
     """Eq. 4 for every row (or the rows in ``row_ids``) of the solved side.

@@ -20,9 +20,10 @@
  *   - alxo_transpose      : CSR -> CSC, row ids ascending inside each column
  *   - alxo_degree_class / alxo_bucket_rows / alxo_chunks
  *
- * Loops are in the paper's order.  The only parallelism is "omp parallel for" over the
- * rows of the side being solved, which Alg. 2's parfor over rows licenses: a row reads
- * only the fixed table, G and its own observations.
+ * Loops are in the paper's order.  The only parallelism is over rows: "omp parallel for" over the
+ * rows of the side being solved, which Alg. 2's parfor over rows licenses (a row reads only the
+ * fixed table, G and its own observations), and contiguous blocks of fixed-side rows in the Gramian
+ * (Alg. 2 lines 5-6: per-part Gramians added up), combined in block order.
  *
  * Pins (tests run without a GPU): brute-force stacked least squares via QR on tiny inputs,
  * closed forms (d = 1, single observation with and without the all-pairs term, orthogonal
@@ -64,14 +65,28 @@ void alxo_round_array(double *x, int64_t n, int storage)
 }
 
 /* ---- Gramian: G = sum over ALL rows of the fixed side of h (x) h ---- */
+/* The sum over rows is split into one contiguous block of rows per thread (the only parallelism: over rows),
+   each block summed in row order, the blocks added in block order. */
 void alxo_gramian(const double *X, int64_t N, int d, double *G)
 {
     memset(G, 0, sizeof(double) * (size_t)d * d);
-    for (int64_t i = 0; i < N; ++i) {
-        const double *h = X + i * d;
-        for (int a = 0; a < d; ++a)
-            for (int b = 0; b < d; ++b)
-                G[a * d + b] += h[a] * h[b];
+#pragma omp parallel
+    {
+        double *P = (double *)calloc((size_t)d * d, sizeof(double));
+#pragma omp for schedule(static) ordered
+        for (int64_t blk = 0; blk < 64; ++blk) {
+            const int64_t i0 = N * blk / 64, i1 = N * (blk + 1) / 64;
+            memset(P, 0, sizeof(double) * (size_t)d * d);
+            for (int64_t i = i0; i < i1; ++i) {
+                const double *h = X + i * d;
+                for (int a = 0; a < d; ++a)
+                    for (int b = 0; b < d; ++b)
+                        P[a * d + b] += h[a] * h[b];
+            }
+#pragma omp ordered
+            for (int k = 0; k < d * d; ++k) G[k] += P[k];
+        }
+        free(P);
     }
 }
 
