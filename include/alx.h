@@ -83,6 +83,7 @@ typedef struct alx_stats {
     int64_t kernel_launches;                 /* kernels this context has launched so far */
     int64_t workspace_bytes;                 /* device memory the context holds */
     int32_t kernel_path[2];                  /* [side]: 0 = FP32-ALU kernels, 1 = tensor-core kernels */
+    double ms_main_kernel;                   /* tensor path: device time of the whole-rows kernel of the LAST half-epoch, else 0 */
 } alx_stats;
 
 /* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.

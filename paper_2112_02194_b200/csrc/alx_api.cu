@@ -48,7 +48,8 @@ struct alx_ctx {
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
 
-    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool main_timed = false;
     alx_stats stats{};
     int64_t launches = 0;
     int64_t bytes_held = 0;
@@ -239,8 +240,9 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     if (tensor_path(c)) {
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
-                                     &c->launches));
+                                     &c->launches, c->ev[3], c->ev[4]));
         c->stats.kernel_path[side] = 1;
+        c->main_timed = true;
     } else {
         ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side],
                                        c->n_split_rows[side], c->table[fixed], c->bf16, c->opt.d, c->Bmat,
@@ -605,6 +607,10 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
     if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]) == cudaSuccess) c->stats.ms_gramian = ms; else cudaGetLastError();
     if (cudaEventElapsedTime(&ms, c->ev[1], c->ev[2]) == cudaSuccess) c->stats.ms_rows = ms; else cudaGetLastError();
     if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[2]) == cudaSuccess) c->stats.ms_half_epoch = ms; else cudaGetLastError();
+    c->stats.ms_main_kernel = 0.0;
+    if (c->main_timed) {
+        if (cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]) == cudaSuccess) c->stats.ms_main_kernel = ms; else cudaGetLastError();
+    }
     c->stats.kernel_launches = c->launches;
     c->stats.workspace_bytes = c->bytes_held;
     *out = c->stats;

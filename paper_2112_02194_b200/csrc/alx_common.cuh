@@ -132,7 +132,8 @@ int64_t gramian_umma_partials();
 cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches);
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                              int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
-                             RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches);
+                             RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,
+                             cudaEvent_t main_end);
 
 // alx_loss.cu
 int64_t loss_partials(int64_t nnz);

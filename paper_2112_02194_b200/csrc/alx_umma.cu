@@ -879,7 +879,7 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
 
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows,
                              const void *X, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
-                             cudaStream_t s, int64_t *launches)
+                             cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end)
 {
     const int sms = sm_count();
     Params p{};
@@ -905,7 +905,9 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
     if (n_whole > 0) {
         p.n_items = n_whole;
         p.last_item = offs[kNClasses - 1] - 1;
+        if (main_begin) cudaEventRecord(main_begin, s);
         e = launch_mode<kModeRows>(p, (int)(n_whole < sms ? n_whole : sms), s);
+        if (main_end) cudaEventRecord(main_end, s);
         ++*launches;
         if (e != cudaSuccess) return e;
     }
