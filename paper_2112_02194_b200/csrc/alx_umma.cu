@@ -458,9 +458,10 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         const float *bp = &sm.bpart[it % kBRing][0][i];
         float b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
         bool dead = false;
-        float yinv[16];          // my column of the inverse of my diagonal block (set at my block step)
+        float lrow[16];          // my row of my diagonal block's factor (kept for the block inverse at the end)
+        float my_dinv = 0.f;     // 1 / L[i][i]
 #pragma unroll
-        for (int c = 0; c < 16; ++c) yinv[c] = 0.f;
+        for (int c = 0; c < 16; ++c) lrow[c] = 0.f;
 
         for (int k = 0; k < D / 16; ++k) {
             const int k0 = 16 * k;
@@ -535,14 +536,19 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 if (!all_ok && lane == 0) gs.bad = 1;
                 if (is_diag) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) gs.Lt[c][l] = (c <= l) ? a[c] : 0.f;
+                    for (int c = 0; c < 16; ++c) {
+                        const float v = (c <= l) ? a[c] : 0.f;
+                        gs.Lt[c][l] = v;
+                        lrow[c] = v;
+                    }
                     gs.dinv[l] = my_inv;
                     gs.z[l] = b;
+                    my_dinv = my_inv;
                 }
             }
             PHASE_MARK(3);
             // the previous step's whole tensor-core update has read its operand tiles before they are rewritten
-            if (k > 0 && tid == 0 && !mbar_wait(&gs.rest_bar, trail_parity ^ 1u, &sm.abort_flag, 80)) gs.stop = 1;
+            if (k > 0 && lane == 0 && wpos == ((k0 + 64) & 96) && !mbar_wait(&gs.rest_bar, trail_parity ^ 1u, &sm.abort_flag, 80)) gs.stop = 1;
             group128_sync(bar_id);
             PHASE_MARK(4);
             // (2) rows after the block: forward substitution; diagonal threads: their column of the inverse
@@ -595,25 +601,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 PHASE_MARK(12);
                 fence_proxy_async();
                 PHASE_MARK(13);
-            } else if (pos >= k0) {
-                const int l = pos - k0;
-                float tacc[16];
-#pragma unroll
-                for (int c = 0; c < 16; ++c) tacc[c] = 0.f;
-#pragma unroll
-                for (int cp = 0; cp < 16; ++cp) {
-                    // y[cp] of the solve L y = e_l
-                    const float ycp = (cp < l) ? 0.f : ((cp == l) ? gs.dinv[cp] : -tacc[cp] * gs.dinv[cp]);
-                    yinv[cp] = ycp;
-                    float lt[16];
-#pragma unroll
-                    for (int q4 = (cp + 1) / 4; q4 < 4; ++q4) {
-                        const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[cp][4 * q4]);
-                        lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
-                    }
-#pragma unroll
-                    for (int c = cp + 1; c < 16; ++c) tacc[c] = fmaf(lt[c], ycp, tacc[c]);
-                }
             }
             PHASE_MARK(5);
             if (warp_live) {
@@ -624,47 +611,82 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             PHASE_MARK(6);
             group128_sync(bar_id);
             PHASE_MARK(7);
-            // (3) trailing update on the tensor core
-            if (k < D / 16 - 1 && tid == 0) {
+            // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
+            // blocks of 32 rows further on in the elimination order, which never holds the next diagonal block.  It
+            // issues the 16 columns of the next panel, waits for them, releases the group through the barrier and
+            // only then issues the remaining columns (a tcgen05.mma takes the issuing thread about 50 cycles).
+            const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
+            uint64_t da[3];
+            const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
+            // columns [c_lo, c_lo + n) of the matrix (= panel rows c_lo ..) -= P P^T restricted to them
+            auto update = [&](int c_lo, int n) {
+                const uint32_t idesc = idesc_bf16_k_major_negA(128, n);
+                uint64_t db[3];
+#pragma unroll
+                for (int q = 0; q < 3; ++q) db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + (uint32_t)(c_lo * 32), 128, 256, 0);
+                umma_f16(d_base + c_lo, da[0], db[0], idesc, true);
+                umma_f16(d_base + c_lo, da[0], db[1], idesc, true);
+                umma_f16(d_base + c_lo, da[1], db[0], idesc, true);
+                umma_f16(d_base + c_lo, da[0], db[2], idesc, true);
+                umma_f16(d_base + c_lo, da[2], db[0], idesc, true);
+                umma_f16(d_base + c_lo, da[1], db[1], idesc, true);
+            };
+            if (k < D / 16 - 1 && issuer) {
                 tc_fence_after();
-                const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
-                uint64_t da[3];
 #pragma unroll
                 for (int q = 0; q < 3; ++q) da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
-                // columns [c_lo, c_lo + n) of the matrix (= panel rows c_lo ..) -= P P^T restricted to them
-                auto update = [&](int c_lo, int n) {
-                    const uint32_t idesc = idesc_bf16_k_major_negA(128, n);
-                    uint64_t db[3];
-#pragma unroll
-                    for (int q = 0; q < 3; ++q) db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + (uint32_t)(c_lo * 32), 128, 256, 0);
-                    umma_f16(d_base + c_lo, da[0], db[0], idesc, true);
-                    umma_f16(d_base + c_lo, da[0], db[1], idesc, true);
-                    umma_f16(d_base + c_lo, da[1], db[0], idesc, true);
-                    umma_f16(d_base + c_lo, da[0], db[2], idesc, true);
-                    umma_f16(d_base + c_lo, da[2], db[0], idesc, true);
-                    umma_f16(d_base + c_lo, da[1], db[1], idesc, true);
-                };
-                // the 16 columns of the next panel first: their completion is all the next step waits for; the rest
-                // follows in issue order and is complete before any later MMA or commit of this thread
                 update((k0 + 16 + rot) & (D - 1), 16);
                 umma_commit(&gs.trail_bar);
-                const int n_rest = D - k0 - 32;
-                if (n_rest > 0) {
-                    const int cs = (k0 + 32 + rot) & (D - 1);
-                    const int n1 = (n_rest < D - cs) ? n_rest : D - cs;     // up to the wrap-around
-                    update(cs, n1);
-                    if (n_rest > n1) update(0, n_rest - n1);
-                }
-                umma_commit(&gs.rest_bar);
                 if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag, 70)) gs.stop = 1;
             }
             if (k < D / 16 - 1) {
                 trail_parity ^= 1u;
                 group128_sync(bar_id);
+                if (issuer) {
+                    const int n_rest = D - k0 - 32;
+                    if (n_rest > 0) {
+                        const int cs = (k0 + 32 + rot) & (D - 1);
+                        const int n1 = (n_rest < D - cs) ? n_rest : D - cs;     // up to the wrap-around
+                        update(cs, n1);
+                        if (n_rest > n1) update(0, n_rest - n1);
+                    }
+                    umma_commit(&gs.rest_bar);
+                }
             }
             PHASE_MARK(8);
         }
         if (dead) break;
+        // my column of the inverse of my diagonal block.  The eight blocks go through shared memory, in the operand
+        // tiles: every trailing update has completed (the last one was waited for before the last block step).
+        float yinv[16];
+        {
+            float *Lall = reinterpret_cast<float *>(&gs.pop[0][0]);      // [8 blocks][16][16], transposed
+            float *dall = Lall + 8 * 256;                                 // [128] reciprocals of the diagonal
+            float *Lb = Lall + (pos >> 4) * 256;
+            const int l = pos & 15;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) Lb[c * 16 + l] = lrow[c];
+            dall[pos] = my_dinv;
+            __syncwarp();
+            const float *dvb = dall + (pos & ~15);
+            float tacc[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) tacc[c] = 0.f;
+#pragma unroll
+            for (int cp = 0; cp < 16; ++cp) {
+                // y[cp] of the solve L y = e_l
+                const float ycp = (cp < l) ? 0.f : ((cp == l) ? dvb[cp] : -tacc[cp] * dvb[cp]);
+                yinv[cp] = ycp;
+                float lt[16];
+#pragma unroll
+                for (int q4 = (cp + 1) / 4; q4 < 4; ++q4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(&Lb[cp * 16 + 4 * q4]);
+                    lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
+                }
+#pragma unroll
+                for (int c = cp + 1; c < 16; ++c) tacc[c] = fmaf(lt[c], ycp, tacc[c]);
+            }
+        }
         // (4) back substitution L^T x = z; b now holds z_i
         float x = 0.f;
         for (int k = D / 16 - 1; k >= 0; --k) {
