@@ -182,6 +182,17 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+            // No free slot yet: the copies in flight have time to land, so hand over every stage issued so far
+            // before blocking (otherwise up to kLag landed stages would stay unannounced until the next issue).
+            {
+                int free_now = 1;
+                if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
+                free_now = __shfl_sync(0xFFFFFFFFu, free_now, 0);
+                if (!free_now && signalled < g) {
+                    cp_async_wait<0>();
+                    for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
+                }
+            }
             if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int rc16 = (rc + 15) & ~15;
@@ -221,7 +232,7 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
             }
             cp_async_commit();
             ++g;
-            if (g > kLag) {
+            if (g - signalled > kLag) {     // the oldest unannounced stage is kLag issues back: its copies have landed
                 cp_async_wait<kLag>();
                 producer_signal<MODE>(sm, signalled, pw, lane, bacc);
                 ++signalled;
