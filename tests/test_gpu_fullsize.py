@@ -1,26 +1,34 @@
-"""Parity at the benchmark's full size (10M x 10M, 1e9 entries, d = 128, bf16), on sampled rows.
+"""Parity at the benchmark configurations' full sizes, on sampled rows.
 
 The graph and the tables exist only on the device (same generator bits as the host recipe).  For a sample of
-rows -- random ones plus the longest, which are split into chunks -- the oracle recomputes the rows half-step
-from regenerated inputs: the rows' own column lists, the initial embeddings of just the columns they touch, and
-the Gramian of the whole fixed table streamed through the host in blocks.  The same launch configuration as
-``bench.py`` (same context options, whole half-epoch)."""
+rows -- random ones, the longest (which are split into chunks) and rows at the degree-class boundaries -- the
+oracle recomputes the rows half-step from regenerated inputs: the rows' own column lists, the initial embeddings
+of just the columns they touch, and the Gramian of the whole fixed table streamed through the host in blocks.
+The same launch configuration as ``bench.py`` (same context options, whole half-epoch).
+
+Configuration 3 (the one the headline metric is quoted on) and configuration 2 run by default.  Configurations 4
+and 5 (50M and 150M rows: minutes of host-side streaming for the oracle's Gramian, 40 and 130 GB on the device)
+run when ``ALX_TEST_FULLSIZE`` names them, e.g. ``ALX_TEST_FULLSIZE=cfg4,cfg5``."""
+import os
+
 import numpy as np
 import pytest
 
 pytestmark = pytest.mark.gpu
 
+_OPT_IN = {x.strip() for x in os.environ.get("ALX_TEST_FULLSIZE", "").split(",") if x.strip()}
 
-def test_cfg3_rows_half_epoch_sampled_rows_match_oracle():
+
+def _sampled_rows_half_epoch(name, n_random, min_memory, n_heavy=6):
     import torch
-    if torch.cuda.get_device_properties(0).total_memory < 60e9:
+    if torch.cuda.get_device_properties(0).total_memory < min_memory:
         pytest.skip("needs a large-memory GPU")
     import bench
     from oracle import ials
     from paper_2112_02194_b200 import ALX_COLS, ALX_ROWS, Alx
     from synth import device as sdev, graphs, host as shost
 
-    w = dict(bench.WORKLOADS["cfg3"], name="cfg3")
+    w = dict(bench.WORKLOADS[name], name=name)
     n, d, storage = w["n"], w["d"], w["storage"]
     spec = bench.make_spec(w)
     deg = graphs.zipf_degrees(n, w["nnz"], w["s"], w["cap"], w["seed"])
@@ -30,18 +38,25 @@ def test_cfg3_rows_half_epoch_sampled_rows_match_oracle():
     a.set_csr(rowptr, colidx)
     del colidx
     a.set_embeddings(ALX_COLS, H0)
+    del H0
+    torch.cuda.empty_cache()
 
-    # sample: 1500 random rows, the 6 longest rows (split into chunks), a few rows around the class boundaries
+    # sample: random rows, the longest rows (split into chunks), a few rows around the class boundaries
     rng = np.random.Generator(np.random.PCG64(12345))
-    heavy = np.argsort(deg)[-6:]
-    near = np.concatenate([np.nonzero(deg == k)[0][:3] for k in (1, 16, 17, 127, 128, 129, 8192, 8193) if np.any(deg == k)])
-    ids = np.unique(np.concatenate([rng.integers(0, n, 1500), heavy, near])).astype(np.int64)
+    heavy = np.argsort(deg)[-n_heavy:]
+    near = [np.nonzero(deg == k)[0][:3] for k in (1, 16, 17, 127, 128, 129, 8192, 8193) if np.any(deg == k)]
+    ids = np.unique(np.concatenate([rng.integers(0, n, n_random), heavy] + near)).astype(np.int64)
     x32 = a.half_epoch_capture(ALX_ROWS, ids)
     W_gpu = graphs.storage_to_f64(np.concatenate([a.get_embeddings(ALX_ROWS, dtype=storage, row_begin=int(u), row_count=1)
                                                   for u in ids]), storage)
     G_gpu = a.get_gramian(ALX_COLS)
     st = a.get_stats()
-    assert st.not_spd == 0 and st.kernel_path[0] == 1 and st.n_chunks[0] > 0
+    assert st.not_spd == 0
+    if storage == "bf16" and d == 128:
+        assert st.kernel_path[0] == 1          # the tensor-core kernels ran
+    if deg.max() > 8192:
+        assert st.n_chunks[0] > 0              # and the split-row path with them
+    a.destroy()
 
     # oracle side, from regenerated inputs only
     ptr, cols = graphs.row_columns_flat(spec, ids, deg[ids])
@@ -50,11 +65,12 @@ def test_cfg3_rows_half_epoch_sampled_rows_match_oracle():
     G = ials.gramian_stream(
         lambda r0, cnt: graphs.storage_to_f64(shost.embedding_rows(d, w["init_seed"], 3, storage, row_begin=r0, row_count=cnt), storage),
         n, d, block_rows=500_000)
-    assert np.abs(G_gpu - G).max() <= 2e-6 * np.abs(G).max()
+    # tensor-core Gramian: the fp32 accumulator truncates (bias below 2e-6 relative); FP32-ALU Gramian: 1e-6
+    assert np.abs(G_gpu - G).max() <= (2e-6 if storage == "bf16" else 1e-6) * np.abs(G).max()
     W_ref, W_raw = ials.half_step(ptr, inv.astype(np.int32), None, X, w["alpha"], w["lam"], storage, G=G, return_raw=True)
 
     rel = np.linalg.norm(W_gpu - W_ref) / np.linalg.norm(W_ref)
-    assert rel <= 2e-2, rel
+    assert rel <= (2e-2 if storage == "bf16" else 1e-3), rel
     raw_rel = np.linalg.norm(x32.astype(np.float64) - W_raw) / np.linalg.norm(W_raw)
     assert raw_rel <= 1e-3, raw_rel
     # residual of the solver's own fp32 solution, A and b rebuilt in fp64
@@ -63,4 +79,21 @@ def test_cfg3_rows_half_epoch_sampled_rows_match_oracle():
         A, b = ials.row_system(ptr, inv.astype(np.int32), None, X, G, w["alpha"], w["lam"], k)
         worst = max(worst, np.linalg.norm(A @ x32[k].astype(np.float64) - b) / np.linalg.norm(b))
     assert worst <= 1e-4, worst
-    a.destroy()
+
+
+def test_cfg3_rows_half_epoch_sampled_rows_match_oracle():
+    _sampled_rows_half_epoch("cfg3", 1500, 60e9)
+
+
+def test_cfg2_rows_half_epoch_sampled_rows_match_oracle():
+    _sampled_rows_half_epoch("cfg2", 1500, 8e9)
+
+
+@pytest.mark.skipif("cfg4" not in _OPT_IN, reason="opt-in: ALX_TEST_FULLSIZE=cfg4")
+def test_cfg4_rows_half_epoch_sampled_rows_match_oracle():
+    _sampled_rows_half_epoch("cfg4", 600, 100e9, n_heavy=3)
+
+
+@pytest.mark.skipif("cfg5" not in _OPT_IN, reason="opt-in: ALX_TEST_FULLSIZE=cfg5")
+def test_cfg5_rows_half_epoch_sampled_rows_match_oracle():
+    _sampled_rows_half_epoch("cfg5", 400, 170e9, n_heavy=3)
