@@ -46,7 +46,7 @@ WORKLOADS = {
     "cfg5": dict(n=150_000_000, nnz=5_000_000_000, s=1.1, cap=1_000_000, law="zipf", delta=0, d=128,
                  lam=0.01, alpha=0.0005, storage="bf16", seed=0xA1C50005, init_seed=0x1A150005,
                  desc="150M x 150M, 5e9 entries, Zipf(1.1) degrees (cap 1e6), d=128, bf16 tables (77 GB) plus CSR and "
-                      "its transpose (42 GB) resident"),
+                      "its transpose (42 GB) resident, 24 GB of chunk sums for the rows longer than 8192 entries"),
     "medium": dict(n=2_000_000, nnz=200_000_000, s=1.1, cap=200_000, law="local", delta=20_000, d=128,
                    lam=0.01, alpha=0.001, storage="bf16", seed=0xA1C500FE, init_seed=0x1A1500FE,
                    desc="2M x 2M, 2e8 entries, scaled-down cfg3 whose tables exceed L2 (profiling case)"),
@@ -54,6 +54,16 @@ WORKLOADS = {
                   lam=0.01, alpha=0.001, storage="bf16", seed=0xA1C500FF, init_seed=0x1A1500FF,
                   desc="200k x 200k, 1e7 entries, scaled-down cfg3 (debugging / profiling case)"),
 }
+
+
+def set_initial_table(a, side, w, stream, slice_rows=8_000_000):
+    """Initial embeddings of one side, generated on the device in slices (a second full copy of a 38 GB table does
+    not fit beside the largest configuration)."""
+    from synth import device as sdev
+    n = w["n"]
+    for r0 in range(0, n, slice_rows):
+        cnt = min(slice_rows, n - r0)
+        a.set_embedding_rows(side, r0, sdev.device_embeddings(cnt, w["d"], w["init_seed"], stream, w["storage"], row_begin=r0))
 
 
 def make_spec(w):
@@ -224,18 +234,30 @@ def run_ours(args, w):
     spec = make_spec(w)
     deg = graphs.zipf_degrees(n, w["nnz"], w["s"], w["cap"], w["seed"])
     rowptr, colidx = sdev.device_csr(spec, deg)
-    W0 = sdev.device_embeddings(n, d, w["init_seed"], 2, storage)
-    H0 = sdev.device_embeddings(n, d, w["init_seed"], 3, storage)
+    # the largest configurations leave no room for second copies of the tables and the graph: their tables are
+    # generated in slices straight into the context and the end-to-end leg (host copies of everything) is left out
+    lean = 2.0 * n * d * e > 32e9
+    if lean:
+        args.skip_e2e = True
+    else:
+        W0 = sdev.device_embeddings(n, d, w["init_seed"], 2, storage)
+        H0 = sdev.device_embeddings(n, d, w["init_seed"], 3, storage)
     nnz = int(colidx.numel())
     t_gen = time.perf_counter() - t_gen
 
-    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage)
+    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0))
     t_set = time.perf_counter()
     a.set_csr(rowptr, colidx)
     torch.cuda.synchronize()
     t_set = time.perf_counter() - t_set
-    a.set_embeddings(ALX_ROWS, W0)
-    a.set_embeddings(ALX_COLS, H0)
+    if lean:
+        del colidx
+        torch.cuda.empty_cache()
+        set_initial_table(a, ALX_ROWS, w, 2)
+        set_initial_table(a, ALX_COLS, w, 3)
+    else:
+        a.set_embeddings(ALX_ROWS, W0)
+        a.set_embeddings(ALX_COLS, H0)
 
     # ---- device-resident timing: K epochs, CUDA events on the context's stream
     for _ in range(args.warmup):
@@ -248,7 +270,7 @@ def run_ours(args, w):
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    half_ms = {"rows": [], "cols": [], "gramian": [], "row_kernels": [], "main_kernel": []}
+    half_ms = {"rows": [], "cols": [], "gramian": [], "row_kernels": [], "main_kernel": [], "dual_rows": []}
     ev[0].record()
     for k in range(args.steps):
         a.half_epoch(ALX_ROWS)
@@ -270,6 +292,7 @@ def run_ours(args, w):
         half_ms["gramian"].append(s2.ms_gramian)
         half_ms["row_kernels"].append(s2.ms_rows)
         half_ms["main_kernel"].append(s2.ms_main_kernel)
+        half_ms["dual_rows"].append(s2.dual_rows)
     fp32_peak = a.fp32_peak_tflops()
     loss = a.loss()[0]
     ms, units = aggregate_over_ranks(ms_local, float(nnz), world, dev)
@@ -286,10 +309,14 @@ def run_ours(args, w):
     main_ms = statistics.mean(half_ms["main_kernel"]) or rows_ms
     n_whole = [sum(st.rows_in_class[sd][1:11]) for sd in (0, 1)]
     n_split = [st.rows_in_class[sd][11] for sd in (0, 1)]
-    # dominant kernel: the whole-rows kernel (every row of at most `split` entries: gather, outer products,
-    # factor, solve, store).  Its algorithmic work per launch, averaged over the two sides:
-    ent_whole = nnz - statistics.mean([st.n_chunks[sd] for sd in (0, 1)]) * 8192 * 0.97   # entries outside split rows (approx.)
-    rows_whole = statistics.mean(n_whole)
+    # dominant kernel: the whole-rows kernel (every row of more than 16 and at most `split` entries, plus the shorter
+    # ones when the dual form stepped aside: gather, outer products, factor, solve, store).  Its algorithmic work per
+    # launch, averaged over the two sides:
+    split = w.get("split", 0) or 8192
+    ent_whole = nnz - statistics.mean([st.n_chunks[sd] for sd in (0, 1)]) * split * 0.97   # entries outside split rows (approx.)
+    dual_rows = statistics.mean(half_ms["dual_rows"])
+    rows_whole = statistics.mean(n_whole) - dual_rows
+    ent_whole -= 4.0 * dual_rows          # rows of 1 .. 16 entries, about 4 on average under the rank-size law (approx.)
     alu_main = rows_whole * (d ** 3 / 3.0 + 3.0 * d * d) + 2.0 * ent_whole * d
     bytes_main = ent_whole * (d * e + 4) + rows_whole * (d * e + 12)
     if t_bytes >= t_tensor + t_alu:
@@ -303,6 +330,8 @@ def run_ours(args, w):
     roof["traffic"] = 4.81e9 / 2.0e6 * rows_whole if w["name"] == "cfg3" else None
     roof.update({"kernel": "k_umma<0>: whole rows (gather, tcgen05 outer products, Cholesky in tensor memory, solve, store)",
                  "main_kernel_ms": main_ms, "rows_per_launch": rows_whole,
+                 "rows_in_dual_form": {"rows": half_ms["dual_rows"][0], "cols": half_ms["dual_rows"][1],
+                                       "note": "rows with at most 16 entries, solved by k_dual outside the dominant kernel"},
                  "peak_source": f"HBM and bf16 {peaks['source']} (sustained bf16); FP32 FMA measured in this run",
                  "half_epoch_ms": {"rows": half_ms["rows"][0], "cols": half_ms["cols"][0],
                                    "gramian": statistics.mean(half_ms["gramian"]), "row_kernels": rows_ms},
@@ -330,7 +359,7 @@ def run_ours(args, w):
         torch.cuda.empty_cache()
         o_W = torch.empty_like(h_W, pin_memory=True)
         o_H = torch.empty_like(h_H, pin_memory=True)
-        b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage)
+        b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0))
         reps = 2 if w["name"] != "small" else 3
         times = []
         for r in range(reps):

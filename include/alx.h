@@ -69,8 +69,11 @@ typedef struct alx_options {
     void *alloc_user;
     int64_t split;           /* rows longer than this are cut into chunks of this many entries that
                                 different thread blocks accumulate; 0 => ALX_DEFAULT_SPLIT; >= 16 */
-    int32_t kernels;         /* 0 = best available for (d, storage); 1 = force the plain FP32-ALU
-                                kernels (reference path inside the library; every d, every storage) */
+    int32_t kernels;         /* 0 = best available for (d, storage): for d = 128 with bf16 tables the tensor-core
+                                kernels, rows with at most 16 observations solved in the dual (push-through) form
+                                of Eq. 4 while alpha0 G + lambda I is well conditioned; 1 = force the plain FP32-ALU
+                                kernels (reference path inside the library; every d, every storage); 2 = as 0 but
+                                every row in the primal form */
     int32_t reserved;
 } alx_options;
 
@@ -84,6 +87,8 @@ typedef struct alx_stats {
     int64_t workspace_bytes;                 /* device memory the context holds */
     int32_t kernel_path[2];                  /* [side]: 0 = FP32-ALU kernels, 1 = tensor-core kernels */
     double ms_main_kernel;                   /* tensor path: device time of the whole-rows kernel of the LAST half-epoch, else 0 */
+    int64_t dual_rows;                       /* rows the LAST half-epoch solved in the dual form of Eq. 4 (0: none, or the
+                                                form stepped aside because alpha0 G + lambda I was ill conditioned) */
 } alx_stats;
 
 /* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.
@@ -106,6 +111,13 @@ alx_status alx_set_csr(alx_ctx *ctx, const int64_t *rowptr, const int32_t *colid
 
 /* Overwrite one table from n x d row-major data of type src_dtype (converted with round-to-nearest-even). */
 alx_status alx_set_embeddings(alx_ctx *ctx, alx_side side, const void *src, alx_dtype src_dtype, int on_device);
+
+/* The same for rows row_begin .. row_begin + row_count - 1 only (src holds row_count x d values).  For tables that
+   are filled in slices because a second full copy would not fit beside them; the table counts as set from the
+   first call on, rows no call has written hold unspecified values.  Synchronises.  (Initialisation of W and H:
+   Alg. 1 takes them as given.) */
+alx_status alx_set_embedding_rows(alx_ctx *ctx, alx_side side, int64_t row_begin, int64_t row_count, const void *src,
+                                  alx_dtype src_dtype, int on_device);
 
 /*
  * One half-epoch (Alg. 1 lines 2-10 for solved_side = ALX_ROWS; line 11 for ALX_COLS):

@@ -39,10 +39,11 @@ class alx_stats(Structure):
     _fields_ = [("nnz", c_int64), ("rows_in_class", (c_int64 * ALX_N_CLASSES) * 2), ("n_chunks", c_int64 * 2),
                 ("not_spd", c_int64), ("ms_gramian", c_double), ("ms_rows", c_double),
                 ("ms_half_epoch", c_double), ("kernel_launches", c_int64), ("workspace_bytes", c_int64),
-                ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double)]
+                ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double), ("dual_rows", c_int64)]
 
 
-EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_half_epoch",
+EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_set_embedding_rows",
+           "alx_half_epoch",
            "alx_epoch", "alx_half_epoch_capture", "alx_loss", "alx_get_embeddings", "alx_get_gramian",
            "alx_gramian", "alx_fp32_peak_tflops", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
            "alx_last_error", "alx_version", "alx_gramian_noalloc", "alx_gramian_noalloc_max_rows",
@@ -66,6 +67,7 @@ def load_library() -> ctypes.CDLL:
     lib.alx_destroy.argtypes = [P]
     lib.alx_set_csr.argtypes = [P, P, P, P, c_int64, c_int]
     lib.alx_set_embeddings.argtypes = [P, c_int, P, c_int, c_int]
+    lib.alx_set_embedding_rows.argtypes = [P, c_int, c_int64, c_int64, P, c_int, c_int]
     lib.alx_half_epoch.argtypes = [P, c_int]
     lib.alx_epoch.argtypes = [P]
     lib.alx_half_epoch_capture.argtypes = [P, c_int, P, c_int64, P]
@@ -203,6 +205,25 @@ class Alx:
                 src = np.ascontiguousarray(src, dtype=np.float32)
                 dt = ALX_F32
             self._check(self.lib.alx_set_embeddings(self.ctx, side, _np_ptr(src), dt, 0))
+
+    def set_embedding_rows(self, side, row_begin, src):
+        """Rows row_begin .. of one table from a torch CUDA tensor (float32 / bfloat16) or a numpy array
+        (float32 / uint16 bf16 bit patterns) holding whole rows."""
+        torch = self.torch
+        if isinstance(src, torch.Tensor):
+            assert src.is_cuda and src.is_contiguous() and src.numel() % self.d == 0
+            assert src.dtype in (torch.bfloat16, torch.float32)
+            dt = ALX_BF16 if src.dtype == torch.bfloat16 else ALX_F32
+            self._check(self.lib.alx_set_embedding_rows(self.ctx, side, row_begin, src.numel() // self.d, src.data_ptr(), dt, 1))
+        else:
+            src = np.ascontiguousarray(src)
+            assert src.size % self.d == 0
+            if src.dtype == np.uint16:
+                dt = ALX_BF16
+            else:
+                src = np.ascontiguousarray(src, dtype=np.float32)
+                dt = ALX_F32
+            self._check(self.lib.alx_set_embedding_rows(self.ctx, side, row_begin, src.size // self.d, _np_ptr(src), dt, 0))
 
     def half_epoch(self, side):
         self._check(self.lib.alx_half_epoch(self.ctx, side))

@@ -44,6 +44,8 @@ struct alx_ctx {
     float *Bmat = nullptr;
     float *gram_partials = nullptr;
     float *split_partials = nullptr;
+    void *dual_ws = nullptr;      // tensor path: B^-1 operand tiles and the flag of the dual form
+    int64_t dual_candidates = 0;  // rows of class 1 of the last half-epoch (solved in the dual form if the flag is set)
     double *loss_partials_buf = nullptr;
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
@@ -210,7 +212,8 @@ void release_matrix(alx_ctx *c)
     c->nnz = -1;
 }
 
-bool tensor_path(const alx_ctx *c) { return c->bf16 && c->opt.d == 128 && c->opt.kernels == 0; }
+bool tensor_path(const alx_ctx *c) { return c->bf16 && c->opt.d == 128 && c->opt.kernels != 1; }
+bool dual_form(const alx_ctx *c) { return tensor_path(c) && c->opt.kernels == 0; }
 
 alx_status gramian_of(alx_ctx *c, int table_side)
 {
@@ -218,6 +221,7 @@ alx_status gramian_of(alx_ctx *c, int table_side)
         ALX_CUDA(c, launch_gramian_umma(c->table[table_side], c->n[table_side], c->gram_partials, c->stream, &c->launches));
         ALX_CUDA(c, launch_gramian_reduce(c->gram_partials, gramian_umma_partials(), c->opt.d, c->G64[table_side], c->Bmat,
                                           c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
+        if (dual_form(c)) ALX_CUDA(c, launch_dual_prepare(c->Bmat, c->dual_ws, c->stream, &c->launches));
         c->have_gram[table_side] = true;
         return ALX_OK;
     }
@@ -240,14 +244,16 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     if (tensor_path(c)) {
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
-                                     &c->launches, c->ev[3], c->ev[4]));
+                                     &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
+        c->dual_candidates = dual_form(c) ? c->class_offs[side][2] - c->class_offs[side][1] : 0;
     } else {
         ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side],
                                        c->n_split_rows[side], c->table[fixed], c->bf16, c->opt.d, c->Bmat,
                                        c->split_partials, out, c->status, c->stream, &c->launches));
         c->stats.kernel_path[side] = 0;
+        c->dual_candidates = 0;
     }
     ALX_CUDA(c, cudaEventRecord(c->ev[2], c->stream));
     c->have_table[side] = true;
@@ -309,6 +315,10 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
             ALX_ALLOC(c, c->class_offs_dev[s], ALX_N_CLASSES + 1);
         }
         ALX_ALLOC(c, c->Bmat, d * d);
+        if (dual_form(c)) {
+            c->dual_ws = dev_alloc(c, dual_workspace_bytes());
+            if (!c->dual_ws) return fail(c, ALX_ERR_OOM, "device allocation of the dual-form workspace failed");
+        }
         const int64_t nmax = c->n[0] > c->n[1] ? c->n[0] : c->n[1];
         int64_t n_part = gramian_partials(nmax);
         if (gramian_umma_partials() > n_part) n_part = gramian_umma_partials();
@@ -435,6 +445,39 @@ alx_status alx_set_embeddings(alx_ctx *c, alx_side side, const void *src, alx_dt
         dev_src = staging;
     }
     ALX_CUDA(c, launch_convert(dev_src, src_dtype == ALX_BF16, c->table[side], c->bf16, count, c->stream, &c->launches));
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (staging) dev_free(c, staging);
+    c->have_table[side] = true;
+    c->have_gram[side] = false;
+    return ALX_OK;
+}
+
+alx_status alx_set_embedding_rows(alx_ctx *c, alx_side side, int64_t row_begin, int64_t row_count, const void *src,
+                                  alx_dtype src_dtype, int on_device)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!src || (side != ALX_ROWS && side != ALX_COLS) || (src_dtype != ALX_F32 && src_dtype != ALX_BF16) ||
+        row_begin < 0 || row_count < 0 || row_begin + row_count > c->n[side])
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_set_embedding_rows");
+    if (row_count == 0) return ALX_OK;
+    DeviceGuard guard(c->device);
+    const int64_t count = row_count * c->opt.d;
+    const size_t src_bytes = (size_t)count * (src_dtype == ALX_BF16 ? 2 : 4);
+    char *dst = static_cast<char *>(c->table[side]) + (size_t)row_begin * c->opt.d * c->elem;
+    const void *dev_src = src;
+    void *staging = nullptr;
+    const bool same = (src_dtype == ALX_BF16) == (c->bf16 != 0);
+    if (same) {
+        ALX_CUDA(c, cudaMemcpyAsync(dst, src, src_bytes, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
+    } else {
+        if (!on_device) {
+            staging = dev_alloc(c, src_bytes);
+            if (!staging) return fail(c, ALX_ERR_OOM, "staging allocation failed");
+            ALX_CUDA(c, cudaMemcpyAsync(staging, src, src_bytes, cudaMemcpyHostToDevice, c->stream));
+            dev_src = staging;
+        }
+        ALX_CUDA(c, launch_convert(dev_src, src_dtype == ALX_BF16, dst, c->bf16, count, c->stream, &c->launches));
+    }
     ALX_CUDA(c, cudaStreamSynchronize(c->stream));
     if (staging) dev_free(c, staging);
     c->have_table[side] = true;
@@ -610,6 +653,12 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
     c->stats.ms_main_kernel = 0.0;
     if (c->main_timed) {
         if (cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]) == cudaSuccess) c->stats.ms_main_kernel = ms; else cudaGetLastError();
+    }
+    c->stats.dual_rows = 0;
+    if (c->dual_candidates > 0 && c->dual_ws) {
+        int flag = 0;
+        ALX_CUDA(c, cudaMemcpy(&flag, dual_flag_ptr(c->dual_ws), sizeof flag, cudaMemcpyDeviceToHost));
+        c->stats.dual_rows = flag ? c->dual_candidates : 0;
     }
     c->stats.kernel_launches = c->launches;
     c->stats.workspace_bytes = c->bytes_held;

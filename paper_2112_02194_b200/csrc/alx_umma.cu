@@ -70,6 +70,8 @@ struct Params {
     int64_t last_item;           // rows mode: position in sv.order of item 0 (items walk downwards)
     int64_t n_fixed;             // Gramian mode: rows of the table
     const float *Bmat;           // alpha0 G + lambda I
+    const int *dual_flag;        // rows mode: set when the rows of class 1 are solved in the dual form elsewhere
+    int64_t n_items_primal;      // rows mode: items without the rows of class 1 (the last ones of the walk)
     float *partials;             // chunks: [slot][D*D + D]; Gramian: [2 * kGramBlocks][D*D]
     RowOut out;
     DevStatus *st;
@@ -770,6 +772,10 @@ template <int MODE>
 __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
 {
     using C = Cfg<MODE>;
+    if (MODE == kModeRows && p.dual_flag && *p.dual_flag) {
+        p.n_items = p.n_items_primal;
+        if ((int64_t)blockIdx.x >= p.n_items) return;      // block-uniform, before any barrier or allocation
+    }
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled stages; plain offset arithmetic on the shared array, so that the
     // compiler keeps every access below in the shared address space (no generic loads)
@@ -912,7 +918,8 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
 
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows,
                              const void *X, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
-                             cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end)
+                             cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
+                             const void *dual_ws)
 {
     const int sms = sm_count();
     Params p{};
@@ -935,6 +942,13 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         ++*launches;
     }
     const int64_t n_whole = offs[kNClasses - 1] - offs[1];
+    if (dual_ws && offs[2] > offs[1]) {
+        // rows with 1 .. 16 observations: dual form, if the flag (set on the device) allows it
+        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], X, dual_ws, out, st, s, launches);
+        if (e != cudaSuccess) return e;
+        p.dual_flag = dual_flag_ptr(dual_ws);
+        p.n_items_primal = offs[kNClasses - 1] - offs[2];
+    }
     if (n_whole > 0) {
         p.n_items = n_whole;
         p.last_item = offs[kNClasses - 1] - 1;

@@ -61,8 +61,9 @@ def device_csr(spec: graphs.GraphSpec, deg: np.ndarray):
     return rowptr, colidx
 
 
-def device_embeddings(n: int, d: int, seed: int, stream: int, storage: str, sigma: float | None = None):
-    """n x d CUDA tensor (float32 or bfloat16) with the same bits as graphs.init_embeddings."""
+def device_embeddings(n: int, d: int, seed: int, stream: int, storage: str, sigma: float | None = None, row_begin: int = 0):
+    """n x d CUDA tensor (float32 or bfloat16) with the same bits as rows row_begin .. row_begin + n - 1 of
+    graphs.init_embeddings."""
     import torch
     if sigma is None:
         sigma = 0.1 / np.sqrt(d)
@@ -71,7 +72,7 @@ def device_embeddings(n: int, d: int, seed: int, stream: int, storage: str, sigm
     out = torch.empty((n, d), dtype=torch.bfloat16 if storage == "bf16" else torch.float32, device=dev)
     key = int(graphs.stream_key(seed, stream))
     scale = float(sigma / 2.0 ** graphs.NT_SCALE_BITS)
-    err = lib().synth_normal(ctypes.c_ulonglong(key), ctypes.c_void_p(table.data_ptr()), ctypes.c_longlong(0),
+    err = lib().synth_normal(ctypes.c_ulonglong(key), ctypes.c_void_p(table.data_ptr()), ctypes.c_longlong(row_begin * d),
                              ctypes.c_longlong(n * d), ctypes.c_double(scale), ctypes.c_int(storage == "bf16"),
                              ctypes.c_void_p(out.data_ptr()),
                              ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))

@@ -33,18 +33,16 @@ def _sampled_rows_half_epoch(name, n_random, min_memory, n_heavy=6):
     spec = bench.make_spec(w)
     deg = graphs.zipf_degrees(n, w["nnz"], w["s"], w["cap"], w["seed"])
     rowptr, colidx = sdev.device_csr(spec, deg)
-    H0 = sdev.device_embeddings(n, d, w["init_seed"], 3, storage)
-    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage)
+    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0))
     a.set_csr(rowptr, colidx)
     del colidx
-    a.set_embeddings(ALX_COLS, H0)
-    del H0
     torch.cuda.empty_cache()
+    bench.set_initial_table(a, ALX_COLS, w, 3)      # in slices: no second copy of a 38 GB table
 
     # sample: random rows, the longest rows (split into chunks), a few rows around the class boundaries
     rng = np.random.Generator(np.random.PCG64(12345))
     heavy = np.argsort(deg)[-n_heavy:]
-    near = [np.nonzero(deg == k)[0][:3] for k in (1, 16, 17, 127, 128, 129, 8192, 8193) if np.any(deg == k)]
+    near = [np.nonzero(deg == k)[0][:3] for k in (1, 16, 17, 127, 128, 129, 8192, 8193, 65536, 65537) if np.any(deg == k)]
     ids = np.unique(np.concatenate([rng.integers(0, n, n_random), heavy] + near)).astype(np.int64)
     x32 = a.half_epoch_capture(ALX_ROWS, ids)
     W_gpu = graphs.storage_to_f64(np.concatenate([a.get_embeddings(ALX_ROWS, dtype=storage, row_begin=int(u), row_count=1)
@@ -54,7 +52,7 @@ def _sampled_rows_half_epoch(name, n_random, min_memory, n_heavy=6):
     assert st.not_spd == 0
     if storage == "bf16" and d == 128:
         assert st.kernel_path[0] == 1          # the tensor-core kernels ran
-    if deg.max() > 8192:
+    if deg.max() > (w.get("split", 0) or 8192):
         assert st.n_chunks[0] > 0              # and the split-row path with them
     a.destroy()
 

@@ -255,3 +255,67 @@ def test_device_generators_match_numpy():
         t = device.device_embeddings(3000, 128, 7, 2, storage)
         got = t.view(torch.int16).cpu().numpy().view(np.uint16) if storage == "bf16" else t.cpu().numpy()
         np.testing.assert_array_equal(got, ref)
+
+
+def _problem(name):
+    for make in problems.small_suite():
+        p = make()
+        if p.name == name:
+            return p
+    raise KeyError(name)
+
+
+def _class1_rows(p):
+    deg = np.diff(p.rowptr)
+    return np.nonzero((deg >= 1) & (deg <= 16))[0].astype(np.int64)
+
+
+def test_dual_form_for_short_rows_matches_oracle_and_primal_form():
+    """Rows with at most 16 observations are solved through the push-through identity (a k x k system); the
+    result must satisfy the same residual gate as the primal form and agree with it."""
+    p = _problem("local_d128_bf16")
+    ids = _class1_rows(p)
+    assert ids.size > 100
+    H0 = p.f64(p.H0)
+    G = ials.gramian(H0)
+    sols = {}
+    for kernels in (0, 2):
+        a = make_ctx(p, kernels=kernels)
+        sols[kernels] = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+        st = a.get_stats()
+        assert st.dual_rows == (ids.size if kernels == 0 else 0)
+        assert st.not_spd == 0
+        a.destroy()
+    _, W_raw = ials.half_step(p.rowptr, p.colidx, None, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G, return_raw=True)
+    for kernels in (0, 2):
+        assert rel_fro(sols[kernels], W_raw) <= 1e-4
+    worst = 0.0
+    for n, u in enumerate(ids):
+        A, b = ials.row_system(p.rowptr, p.colidx, None, H0, G, p.alpha, p.lam, int(u))
+        worst = max(worst, np.linalg.norm(A @ sols[0][n] - b) / np.linalg.norm(b))
+    assert worst <= 1e-4, worst
+
+
+def test_dual_form_steps_aside_when_base_matrix_is_ill_conditioned():
+    """alpha0 G + lambda I with a condition number of about 4e4: the dual form would lose four digits, so the
+    library must take the primal form for every row (and still meet the residual gate)."""
+    from synth import graphs
+    p = _problem("local_d128_bf16")
+    rng = np.random.Generator(np.random.PCG64(77))
+    H0 = 0.05 + 0.002 * rng.standard_normal((p.n_cols, p.d))
+    p.H0 = graphs.to_storage_bits(H0, p.storage)
+    p.alpha, p.lam = 0.5, 0.01
+    ids = _class1_rows(p)
+    a = make_ctx(p)
+    x32 = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+    st = a.get_stats()
+    assert st.dual_rows == 0 and st.kernel_path[0] == 1 and st.not_spd == 0
+    a.destroy()
+    H0r = p.f64(p.H0)
+    G = ials.gramian(H0r)
+    assert np.linalg.cond(p.alpha * G + p.lam * np.eye(p.d)) > 1e4
+    worst = 0.0
+    for n in range(0, ids.size, 7):
+        A, b = ials.row_system(p.rowptr, p.colidx, None, H0r, G, p.alpha, p.lam, int(ids[n]))
+        worst = max(worst, np.linalg.norm(A @ x32[n] - b) / np.linalg.norm(b))
+    assert worst <= 1e-4, worst
