@@ -181,9 +181,30 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
     for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
         int64_t u, beg, end, slot_unused;
         item_range<MODE>(p, t, u, beg, end, slot_unused);
+        // ids (and labels) of this warp's 8 rows of a stage are fetched one stage ahead by lanes 0..7
+        int32_t nxt_idx = -1;
+        float nxt_y = 0.f;
+        {
+            const int64_t e = beg + pw * 8 + (lane & 7);
+            if (lane < 8 && e < end) {
+                nxt_idx = (MODE == kModeGramian) ? (int32_t)e : p.sv.idx[e];
+                nxt_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[e] : 1.f);
+            }
+        }
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+            const int32_t my_idx = nxt_idx;
+            const float my_y = nxt_y;
+            {
+                const int64_t e = e0 + kStageRows + pw * 8 + (lane & 7);
+                nxt_idx = -1;
+                nxt_y = 0.f;
+                if (lane < 8 && e < end) {
+                    nxt_idx = (MODE == kModeGramian) ? (int32_t)e : p.sv.idx[e];
+                    nxt_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[e] : 1.f);
+                }
+            }
             // No free slot yet: the copies in flight have time to land, so hand over every stage issued so far
             // before blocking (otherwise up to kLag landed stages would stay unannounced until the next issue).
             {
@@ -198,14 +219,6 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
             if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int rc16 = (rc + 15) & ~15;
-            // lanes 0..7 fetch the ids (and labels) of this warp's 8 rows
-            int64_t my_e = e0 + pw * 8 + (lane & 7);
-            int32_t my_idx = -1;
-            float my_y = 0.f;
-            if (lane < 8 && my_e < end) {
-                my_idx = (MODE == kModeGramian) ? (int32_t)my_e : p.sv.idx[my_e];
-                my_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[my_e] : 1.f);
-            }
             if (MODE == kModeRows) {
                 if (lane < 8) sm.ylab[slot][pw * 8 + lane] = my_y;
                 if (lane == 0) {
