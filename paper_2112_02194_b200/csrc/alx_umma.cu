@@ -34,8 +34,12 @@ using namespace ptx;
 
 constexpr int D = 128;
 constexpr int kStageRows = 32;
-constexpr int kNStage = 6;
-constexpr int kLag = 4;                               // stages of copies in flight per producer warp
+// ring of stages: rows mode shares shared memory with the solver groups' scratch and alpha0 G + lambda I, the two
+// streaming modes (chunks, Gramian) use that space for a deeper ring, which is what keeps HBM busy
+template <int MODE> struct Ring {
+    static constexpr int kNStage = (MODE == 0) ? 6 : 18;
+    static constexpr int kLag = (MODE == 0) ? 4 : 14;     // stages of copies in flight per producer warp
+};
 constexpr int kHalfBytes = kStageRows * 128;          // one 64-feature half of a stage
 constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
 constexpr int kStageYBytes = 2 * kStageRows * 16;     // 1024: label tile, two 8-column chunks
@@ -60,7 +64,12 @@ template <int MODE> struct Cfg {
     static constexpr int kSolverThreads = kGroups * kGroupThreads;
     static constexpr int kMmaWarp = kSolverThreads / 32;
     static constexpr int kFirstProducerWarp = kMmaWarp + 1;
-    static constexpr int kBlockThreads = kSolverThreads + 32 + kProducerWarps * 32;
+    // rows mode: the four producer warps share every stage (8 rows each; their partial right-hand sides are summed in
+    // a fixed order); streaming modes: eight producer warps, each fills whole stages of its own (a stage costs a
+    // warp about 2000 cycles of waits, fences and address arithmetic whatever its share of the rows)
+    static constexpr int kProducers = (MODE == kModeRows) ? kProducerWarps : 8;
+    static constexpr int kFullArrivals = (MODE == kModeRows) ? kProducerWarps : 1;
+    static constexpr int kBlockThreads = kSolverThreads + 32 + kProducers * 32;
 };
 
 struct Params {
@@ -100,7 +109,8 @@ struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver gr
     int stop;               // set by the polling thread when a wait gave up; read by the group after its barrier
 };
 
-struct __align__(1024) Smem {
+template <int MODE> struct __align__(1024) SmemT {
+    static constexpr int kNStage = Ring<MODE>::kNStage;
     unsigned char h[kNStage][kStageHBytes];
     unsigned char y[kNStage][kStageYBytes];
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
@@ -134,6 +144,8 @@ template <int MODE> __device__ __forceinline__ void item_range(const Params &p, 
 
 // ---------------------------------------------------------------------------------------------------------
 // rows mode: sum y x over this warp's 8 rows of a landed stage (lane = features 4*lane .. 4*lane+3)
+using Smem = SmemT<0>;       // rows mode
+
 __device__ __forceinline__ void stage_rhs(Smem &sm, int slot, int pw, int lane, float (&bacc)[4])
 {
     const int f = 4 * lane;
@@ -153,11 +165,12 @@ __device__ __forceinline__ void stage_rhs(Smem &sm, int slot, int pw, int lane, 
     }
 }
 
-template <int MODE> __device__ __forceinline__ void producer_signal(Smem &sm, int64_t signalled, int pw, int lane,
+template <int MODE> __device__ __forceinline__ void producer_signal(SmemT<MODE> &sm, int64_t signalled, int pw, int lane,
                                                                    float (&bacc)[4])
 {
+    constexpr int kNStage = Ring<MODE>::kNStage;
     const int slot = (int)(signalled % kNStage);
-    if (MODE == kModeRows) {
+    if constexpr (MODE == kModeRows) {
         __syncwarp();      // every lane's copies of this stage have landed (each lane waited for its own)
         stage_rhs(sm, slot, pw, lane, bacc);
         const int last = sm.last_of_item[pw][slot];
@@ -171,8 +184,9 @@ template <int MODE> __device__ __forceinline__ void producer_signal(Smem &sm, in
     if (lane == 0) mbar_arrive(&sm.full[slot]);
 }
 
-template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int pw, int lane)
+template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
 {
+    constexpr int kNStage = Ring<MODE>::kNStage, kLag = Ring<MODE>::kLag;
     int64_t g = 0, signalled = 0, it = 0;
     const int c = lane & 15;                 // 16-byte chunk of the 256-byte row
     const int half = c >> 3, cc = c & 7;
@@ -258,8 +272,81 @@ template <int MODE> __device__ void producer_role(const Params &p, Smem &sm, int
     for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
 }
 
-template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane)
+// Streaming modes (chunks, Gramian pieces): producer warp pw fills the stages whose running number is pw modulo the
+// number of producer warps, whole stages of 32 rows each, and announces a stage once the next stage of its own has
+// been issued (or at once when it would otherwise block).
+template <int MODE> __device__ void stream_producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
 {
+    constexpr int kNStage = Ring<MODE>::kNStage, P = Cfg<MODE>::kProducers, kOwnLag = 1;
+    int64_t g = 0;                        // running number of the stage over all items of this block
+    int64_t issued = 0, announced = 0;    // own stages
+    const int c = lane & 15;              // 16-byte chunk of the 256-byte row
+    const int half = c >> 3, cc = c & 7;
+    bool alive = true;
+    auto announce = [&](int64_t n) {
+        const int slot = (int)((pw + P * n) % kNStage);
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.full[slot]);
+    };
+    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x) {
+        int64_t u, beg, end, slot_unused;
+        item_range<MODE>(p, t, u, beg, end, slot_unused);
+        for (int64_t e0 = beg; e0 < end; e0 += kStageRows, ++g) {
+            if ((int)(g % P) != pw) continue;
+            const int slot = (int)(g % kNStage);
+            const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+            // this lane's row of the stage
+            const int64_t e = e0 + lane;
+            int32_t my_idx = -1;
+            float my_y = 0.f;
+            if (e < end) {
+                my_idx = (MODE == kModeGramian) ? (int32_t)e : p.sv.idx[e];
+                my_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[e] : 1.f);
+            }
+            {
+                int free_now = 1;
+                if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
+                free_now = __shfl_sync(0xFFFFFFFFu, free_now, 0);
+                if (!free_now && announced < issued) {
+                    cp_async_wait<0>();
+                    for (; announced < issued; ++announced) announce(announced);
+                }
+            }
+            if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
+            const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
+            const int rc16 = (rc + 15) & ~15;
+            const uint32_t hbase = smem_u32(&sm.h[slot][0]) + half * kHalfBytes;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int r = (lane >> 4) + 2 * q;          // row inside the stage
+                const int32_t src = __shfl_sync(0xFFFFFFFFu, my_idx, r);
+                const uint32_t dst = hbase + r * 128 + ((cc ^ (r & 7)) << 4);
+                if (src >= 0) cp_async16(dst, p.X + (int64_t)src * D + c * 8);
+                else if (r < rc16) st_shared_zero16(dst);
+            }
+            if (MODE == kModeChunks && lane < rc16) {
+                const __nv_bfloat16 yhi = __float2bfloat16_rn(my_y);
+                const __nv_bfloat16 ylo = __float2bfloat16_rn(my_y - __bfloat162float(yhi));
+                const uint32_t packed = (uint32_t)__bfloat16_as_ushort(yhi) | ((uint32_t)__bfloat16_as_ushort(ylo) << 16);
+                st_shared_v4(smem_u32(&sm.y[slot][0]) + lane * 16, packed, 0u, 0u, 0u);
+            }
+            cp_async_commit();
+            ++issued;
+            if (issued - announced > kOwnLag) {
+                cp_async_wait<kOwnLag>();
+                announce(announced);
+                ++announced;
+            }
+        }
+    }
+    cp_async_wait<0>();
+    for (; announced < issued; ++announced) announce(announced);
+}
+
+template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, int lane)
+{
+    constexpr int kNStage = Ring<MODE>::kNStage;
     constexpr uint32_t kIdescMain = idesc_bf16_mn_major(128, 128);
     constexpr uint32_t kIdescY = idesc_bf16_mn_major(128, 16);
     const uint32_t tmem = sm.tmem_base;
@@ -305,7 +392,7 @@ template <int MODE> __device__ void mma_role(const Params &p, Smem &sm, int lane
 }
 
 template <int MODE>
-__device__ void copyout_role(const Params &p, Smem &sm, int gidx, int tid)
+__device__ void copyout_role(const Params &p, SmemT<MODE> &sm, int gidx, int tid)
 {
     constexpr int kAccStride = Cfg<MODE>::kAccStride;
     const int lane = tid & 31, w = tid >> 5;
@@ -793,13 +880,14 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
     // 1024-byte alignment for the swizzled stages; plain offset arithmetic on the shared array, so that the
     // compiler keeps every access below in the shared address space (no generic loads)
     unsigned char *aligned = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    Smem &sm = *reinterpret_cast<Smem *>(aligned);
-    float *Bs = reinterpret_cast<float *>(aligned + sizeof(Smem));
-    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(Smem) + sizeof(float) * D * kLdB);
+    constexpr int kNStage = Ring<MODE>::kNStage;
+    SmemT<MODE> &sm = *reinterpret_cast<SmemT<MODE> *>(aligned);
+    float *Bs = reinterpret_cast<float *>(aligned + sizeof(SmemT<MODE>));
+    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(SmemT<MODE>) + sizeof(float) * D * kLdB);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int s = 0; s < kNStage; ++s) { mbar_init(&sm.full[s], kProducerWarps); mbar_init(&sm.empty[s], 1); }
+        for (int s = 0; s < kNStage; ++s) { mbar_init(&sm.full[s], C::kFullArrivals); mbar_init(&sm.empty[s], 1); }
         for (int a = 0; a < kMaxGroups; ++a) { mbar_init(&sm.acc_full[a], 1); mbar_init(&sm.acc_empty[a], 1); }
         sm.abort_flag = 0;
         mbar_fence_init();
@@ -829,12 +917,13 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
 
     if (warp < C::kMmaWarp) {
         const int gidx = warp / (C::kGroupThreads / 32);
-        if (MODE == kModeRows) solver_rows_tmem(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
+        if constexpr (MODE == kModeRows) solver_rows_tmem(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
         else copyout_role<MODE>(p, sm, gidx, tid - gidx * C::kGroupThreads);
     } else if (warp == C::kMmaWarp) {
         mma_role<MODE>(p, sm, lane);
     } else {
-        producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
+        if constexpr (MODE == kModeRows) producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
+        else stream_producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
     }
 
     tc_fence_before();
@@ -888,16 +977,19 @@ __global__ void __launch_bounds__(kThreads, 2) k_split_solve_umma(SideView sv, i
     if (tid < 32) store_solution<D, __nv_bfloat16>(xq, ok, u, out, st);
 }
 
-size_t smem_bytes()
+template <int MODE> size_t smem_bytes()
 {
-    // the same (large) request in every mode: at most one block per SM, so two blocks never compete for
-    // the SM's 512 tensor-memory columns
-    return sizeof(Smem) + 1024 + sizeof(float) * D * kLdB + kMaxGroups * sizeof(RowGroupSmem);   // about 200 KB
+    // a large request in every mode (more than half of what an SM offers): at most one block per SM, so two
+    // blocks never compete for the SM's 512 tensor-memory columns
+    size_t b = sizeof(SmemT<MODE>) + 1024;
+    if (MODE == kModeRows) b += sizeof(float) * D * kLdB + kMaxGroups * sizeof(RowGroupSmem);
+    return b;
 }
+static_assert(sizeof(SmemT<1>) + 1024 <= 232448 && sizeof(SmemT<1>) > 116224, "ring depth of the streaming modes");
 
 template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStream_t s)
 {
-    const size_t smem = smem_bytes();
+    const size_t smem = smem_bytes<MODE>();
     cudaError_t e = cudaFuncSetAttribute(k_umma<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     k_umma<MODE><<<grid, Cfg<MODE>::kBlockThreads, smem, s>>>(p);
