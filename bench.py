@@ -309,14 +309,14 @@ def run_ours(args, w):
     main_ms = statistics.mean(half_ms["main_kernel"]) or rows_ms
     n_whole = [sum(st.rows_in_class[sd][1:11]) for sd in (0, 1)]
     n_split = [st.rows_in_class[sd][11] for sd in (0, 1)]
-    # dominant kernel: the whole-rows kernel (every row of more than 16 and at most `split` entries, plus the shorter
+    # dominant kernel: the whole-rows kernel (every row of more than 32 and at most `split` entries, plus the shorter
     # ones when the dual form stepped aside: gather, outer products, factor, solve, store).  Its algorithmic work per
     # launch, averaged over the two sides:
     split = w.get("split", 0) or 8192
     ent_whole = nnz - statistics.mean([st.n_chunks[sd] for sd in (0, 1)]) * split * 0.97   # entries outside split rows (approx.)
     dual_rows = statistics.mean(half_ms["dual_rows"])
     rows_whole = statistics.mean(n_whole) - dual_rows
-    ent_whole -= 4.0 * dual_rows          # rows of 1 .. 16 entries, about 4 on average under the rank-size law (approx.)
+    ent_whole -= 6.0 * dual_rows          # rows of 1 .. 32 entries, about 6 on average under the rank-size law (approx.)
     alu_main = rows_whole * (d ** 3 / 3.0 + 3.0 * d * d) + 2.0 * ent_whole * d
     bytes_main = ent_whole * (d * e + 4) + rows_whole * (d * e + 12)
     if t_bytes >= t_tensor + t_alu:
@@ -331,7 +331,7 @@ def run_ours(args, w):
     roof.update({"kernel": "k_umma<0>: whole rows (gather, tcgen05 outer products, Cholesky in tensor memory, solve, store)",
                  "main_kernel_ms": main_ms, "rows_per_launch": rows_whole,
                  "rows_in_dual_form": {"rows": half_ms["dual_rows"][0], "cols": half_ms["dual_rows"][1],
-                                       "note": "rows with at most 16 entries, solved by k_dual outside the dominant kernel"},
+                                       "note": "rows with at most 32 entries, solved by k_dual outside the dominant kernel"},
                  "peak_source": f"HBM and bf16 {peaks['source']} (sustained bf16); FP32 FMA measured in this run",
                  "half_epoch_ms": {"rows": half_ms["rows"][0], "cols": half_ms["cols"][0],
                                    "gramian": statistics.mean(half_ms["gramian"]), "row_kernels": rows_ms},

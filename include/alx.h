@@ -70,7 +70,7 @@ typedef struct alx_options {
     int64_t split;           /* rows longer than this are cut into chunks of this many entries that
                                 different thread blocks accumulate; 0 => ALX_DEFAULT_SPLIT; >= 16 */
     int32_t kernels;         /* 0 = best available for (d, storage): for d = 128 with bf16 tables the tensor-core
-                                kernels, rows with at most 16 observations solved in the dual (push-through) form
+                                kernels, rows with at most 32 observations solved in the dual (push-through) form
                                 of Eq. 4 while alpha0 G + lambda I is well conditioned; 1 = force the plain FP32-ALU
                                 kernels (reference path inside the library; every d, every storage); 2 = as 0 but
                                 every row in the primal form */

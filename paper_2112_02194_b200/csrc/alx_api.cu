@@ -45,7 +45,7 @@ struct alx_ctx {
     float *gram_partials = nullptr;
     float *split_partials = nullptr;
     void *dual_ws = nullptr;      // tensor path: B^-1 operand tiles and the flag of the dual form
-    int64_t dual_candidates = 0;  // rows of class 1 of the last half-epoch (solved in the dual form if the flag is set)
+    int64_t dual_candidates = 0;  // rows of classes 1 and 2 of the last half-epoch (solved in the dual form if the flag is set)
     double *loss_partials_buf = nullptr;
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
@@ -247,7 +247,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
                                      &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
-        c->dual_candidates = dual_form(c) ? c->class_offs[side][2] - c->class_offs[side][1] : 0;
+        c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;
     } else {
         ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side],
                                        c->n_split_rows[side], c->table[fixed], c->bf16, c->opt.d, c->Bmat,

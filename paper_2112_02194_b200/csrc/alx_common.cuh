@@ -135,12 +135,12 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host,
                              RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,
                              cudaEvent_t main_end, const void *dual_ws);
 
-// alx_dual.cu: rows with at most 16 observations in the dual form (d = 128, bf16 tables)
+// alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();
 cudaError_t launch_dual_prepare(const float *Bmat, void *ws, cudaStream_t s, int64_t *launches);
 const int *dual_flag_ptr(const void *ws);
-cudaError_t launch_rows_dual(const SideView &sv, int64_t first, int64_t count, const void *X, const void *ws, RowOut out,
-                             DevStatus *st, cudaStream_t s, int64_t *launches);
+cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
+                             const void *ws, RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches);
 
 // alx_loss.cu
 int64_t loss_partials(int64_t nnz);

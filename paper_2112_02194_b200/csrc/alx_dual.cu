@@ -1,18 +1,19 @@
-// Rows with at most 16 observations, d = 128, bfloat16 tables: Eq. 4 solved in its dual form.
+// Rows with at most 32 observations, d = 128, bfloat16 tables: Eq. 4 solved in its dual form.
 //
 // With B = alpha0 G + lambda I (the same for every row, Alg. 1 line 5) and H_u the k x d matrix of the row's
 // observed fixed-side embeddings, the push-through identity gives
 //     w_u = (B + H_u^T H_u)^-1 H_u^T y_u = B^-1 H_u^T (I_k + H_u B^-1 H_u^T)^-1 y_u ,
 // an exact restatement of Eq. 4 whose linear system is k x k instead of d x d.  B^-1 is computed once per
-// half-step (fp64, one block), the k x d products Z_u = H_u B^-1 of 8 rows at a time are one 128 x 128 x 128
-// tensor-core product (rows padded to 16 observations with zero embeddings, B^-1 split into three bfloat16
-// parts), and per row: S_u = I + Z_u H_u^T (FP32 FMAs), S_u t = y_u by the 16 x 16 Cholesky the primal kernel
-// uses for its diagonal blocks (padding rows are rows of the identity), w_u = Z_u^T t.
+// half-step (fp64, one block), the k x d products Z_u = H_u B^-1 of 8 (or 4) rows at a time are one
+// 128 x 128 x 128 tensor-core product (rows padded to 16 (or 32) observations with zero embeddings, B^-1 split
+// into three bfloat16 parts), and per row: S_u = I + Z_u H_u^T (FP32 FMAs), S_u t = y_u by the in-warp Cholesky
+// the primal kernel uses for its diagonal blocks (padding rows are rows of the identity), w_u = Z_u^T t.
+// Two instances: rows of 1 .. 16 observations (two rows per warp) and rows of 17 .. 32 (one row per warp).
 // The form is used only while B is well conditioned (its error grows with cond(B), which the primal form
 // avoids): k_binv_prepare sets a flag from ||B||_F ||B^-1||_F, the dual kernel does nothing when it is clear,
 // and the primal kernel then takes these rows as well.
 //
-// One persistent block per SM; three tiles of 8 rows in flight (shared-memory tile + 128 tensor-memory
+// One persistent block per SM; three tiles of 128 padded observations in flight (shared-memory tile + 128 tensor-memory
 // columns each); roles as in the primal kernel: 4 producer warps (gather, 16-byte cp.async into the K-major,
 // 128-byte-swizzled operand layout), 1 MMA warp, 3 solver groups of 128 threads (thread = tensor-memory lane =
 // one padded observation).  Every wait is bounded; a block that gives up sets a status flag and returns.
@@ -26,8 +27,7 @@ namespace {
 using namespace ptx;
 
 constexpr int D = 128;
-constexpr int kTileRows = 8;                  // matrix rows per tile
-constexpr int kPad = 16;                      // observations per matrix row after padding
+constexpr int kMaxTileRows = 8;               // matrix rows per tile: 128 / (observations per row after padding)
 constexpr int kSlots = 3;                     // tiles in flight
 constexpr int kTileBytes = 128 * D * 2;       // 128 padded observations x 128 features, bf16: two 64-feature panels
 constexpr int kPanelBytes = kTileBytes / 2;
@@ -153,8 +153,8 @@ struct __align__(1024) DualSmem {
     uint32_t tmem_base;
     int abort_flag;
     int stop[kSlots];
-    int row_u[kSlots][kTileRows];            // matrix row ids of the tile (-1: none)
-    int row_k[kSlots][kTileRows];            // their numbers of observations
+    int row_u[kSlots][kMaxTileRows];         // matrix row ids of the tile (-1: none)
+    int row_k[kSlots][kMaxTileRows];         // their numbers of observations
     float y[kSlots][128];                    // labels of the padded observations (0 for padding)
 };
 
@@ -165,16 +165,16 @@ __device__ __forceinline__ float rsqrt_fast(float x)
     return r;
 }
 
-// Cholesky of a 16 x 16 matrix held one row per lane of a half-warp (row l = lane & 15 in d[0 .. l]), both
-// half-warps of the warp at once on their own matrices; b is carried along as a 17th column.  Two pivots per
-// round; the two new columns go through shared memory (xch: 64 floats per half-warp, double buffered).
+// Cholesky of a KP x KP matrix held one row per lane (KP = 16: row l = lane & 15 in d[0 .. l], both half-warps of
+// the warp at once on their own matrices; KP = 32: row l = lane); b is carried along as one more column.  Two
+// pivots per round; the two new columns go through shared memory (xch: 4 KP floats per matrix, double buffered).
 // On return lane l holds row l of L in d[0 .. l], its component of L^-1 b in b and 1 / L[l][l] in my_inv.
-__device__ __forceinline__ bool factor16_pair(float (&d)[16], float &b, float &my_inv, int lane, float *xch)
+template <int KP> __device__ __forceinline__ bool factor_rows(float (&d)[KP], float &b, float &my_inv, int lane, float *xch)
 {
-    const int hb = lane & 16, l = lane & 15;
+    const int hb = (KP == 16) ? (lane & 16) : 0, l = lane & (KP - 1);
     bool all_ok = true;
 #pragma unroll
-    for (int j = 0; j < 16; j += 2) {
+    for (int j = 0; j < KP; j += 2) {
         const float p00 = __shfl_sync(0xFFFFFFFFu, d[j], hb + j);
         const float p10 = __shfl_sync(0xFFFFFFFFu, d[j], hb + j + 1);
         const float p11 = __shfl_sync(0xFFFFFFFFu, d[j + 1], hb + j + 1);
@@ -198,21 +198,22 @@ __device__ __forceinline__ bool factor16_pair(float (&d)[16], float &b, float &m
         const float m0 = below ? x0 : 0.f, m1 = below ? x1 : 0.f;
         const float bdown = fmaf(-m1, zj1, fmaf(-m0, zj, b));
         b = (l == j) ? zj : ((l == j + 1) ? zj1 : bdown);
-        if (j < 14) {
-            float *xb = &xch[(j & 2) * 16];
+        if (j < KP - 2) {
+            float *xb = &xch[(j & 2) * KP];
             xb[l] = x0;
-            xb[16 + l] = x1;
+            xb[KP + l] = x1;
             __syncwarp();
-            float c0[16], c1[16];
 #pragma unroll
-            for (int q4 = (j + 2) / 4; q4 < 4; ++q4) {
+            for (int q4 = (j + 2) / 4; q4 < KP / 4; ++q4) {
                 const float4 u4 = *reinterpret_cast<const float4 *>(&xb[4 * q4]);
-                const float4 v4 = *reinterpret_cast<const float4 *>(&xb[16 + 4 * q4]);
-                c0[4 * q4] = u4.x; c0[4 * q4 + 1] = u4.y; c0[4 * q4 + 2] = u4.z; c0[4 * q4 + 3] = u4.w;
-                c1[4 * q4] = v4.x; c1[4 * q4 + 1] = v4.y; c1[4 * q4 + 2] = v4.z; c1[4 * q4 + 3] = v4.w;
-            }
+                const float4 v4 = *reinterpret_cast<const float4 *>(&xb[KP + 4 * q4]);
+                const float c0[4] = {u4.x, u4.y, u4.z, u4.w}, c1[4] = {v4.x, v4.y, v4.z, v4.w};
 #pragma unroll
-            for (int c = j + 2; c < 16; ++c) d[c] = fmaf(-m1, c1[c], fmaf(-m0, c0[c], d[c]));
+                for (int e = 0; e < 4; ++e) {
+                    const int c = 4 * q4 + e;
+                    if (c >= j + 2) d[c] = fmaf(-m1, c1[e], fmaf(-m0, c0[e], d[c]));
+                }
+            }
         }
     }
     return all_ok;
@@ -251,32 +252,79 @@ __device__ __forceinline__ float halfwarp_reduce16(float (&v)[16], int lane)
     return keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
 }
 
-__device__ void dual_producer(const DualParams &p, DualSmem &sm, int pw, int lane)
+// Producer warp pw fills padded observations 32 pw .. 32 pw + 31 of every tile.  The index loads of a tile form a
+// chain of three dependent loads (row id from the order, its offsets, its column ids); they are issued one, two
+// and three tiles ahead, so that none of them is waited for.  A tile is announced once the next one has been
+// issued (or at once when the warp would otherwise block).
+template <int KP> __device__ void dual_producer(const DualParams &p, DualSmem &sm, int pw, int lane)
 {
+    constexpr int kTileRows = 128 / KP;
+    const int mr = (32 * pw + lane) / KP, j = lane & (KP - 1);     // my matrix row of the tile, my observation of it
+    const int c = lane & 15;                                        // 16-byte chunk of the 256-byte embedding
+    const int64_t stride = gridDim.x;
+    // pipeline registers: tile t+1 (ids loaded), tile t+2 (offsets loaded), tile t+3 (row id loaded)
+    int32_t u1 = -1, idx1 = -1, u2 = -1, u3 = -1;
+    int k1 = 0;
+    float y1 = 0.f;
+    int64_t beg2 = 0, end2 = 0;
+    auto load_u = [&](int64_t t) -> int32_t {
+        const int64_t r = t * kTileRows + mr;
+        return (t < p.n_tiles && r < p.count) ? p.sv.order[p.first + r] : -1;
+    };
+    auto load_ptr = [&](int32_t u, int64_t &beg, int64_t &end) {
+        beg = end = 0;
+        if (u >= 0) { beg = p.sv.ptr[u]; end = p.sv.ptr[u + 1]; }
+    };
+    auto load_idx = [&](int32_t u, int64_t beg, int64_t end, int32_t &idx, float &y, int &k) {
+        k = (int)(end - beg);
+        idx = -1;
+        y = 0.f;
+        if (u >= 0 && j < k) {
+            idx = p.sv.idx[beg + j];
+            y = p.sv.val ? p.sv.val[beg + j] : 1.f;
+        }
+    };
+    {   // fill the pipeline for the first tile of this block
+        const int64_t t0 = blockIdx.x;
+        u1 = load_u(t0);
+        int64_t b1, e1;
+        load_ptr(u1, b1, e1);
+        load_idx(u1, b1, e1, idx1, y1, k1);
+        u2 = load_u(t0 + stride);
+        load_ptr(u2, beg2, end2);
+        u3 = load_u(t0 + 2 * stride);
+    }
     int64_t it = 0;
-    for (int64_t t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ++it) {
+    int pending = -1;      // slot of the tile issued but not yet announced
+    for (int64_t t = blockIdx.x; t < p.n_tiles; t += stride, ++it) {
         const int slot = (int)(it % kSlots);
         const uint32_t ph = (uint32_t)((it / kSlots) & 1);
-        if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 110)) break;
-        // lane = padded observation 32 pw + lane of the tile: matrix row 2 pw + (lane >> 4), observation lane & 15
-        const int mr = 2 * pw + (lane >> 4), j = lane & 15;
-        const int64_t r = t * kTileRows + mr;
-        int32_t u = -1, my_idx = -1;
-        int k = 0;
-        float my_y = 0.f;
-        if (r < p.count) {
-            u = p.sv.order[p.first + r];
-            const int64_t beg = p.sv.ptr[u];
-            k = (int)(p.sv.ptr[u + 1] - beg);
-            if (j < k) {
-                my_idx = p.sv.idx[beg + j];
-                my_y = p.sv.val ? p.sv.val[beg + j] : 1.f;
+        // this tile's values, then advance the pipeline by one tile (nothing loaded here is used before the next trip)
+        const int32_t u = u1, my_idx = idx1;
+        const int k = k1;
+        const float my_y = y1;
+        u1 = u2;
+        load_idx(u2, beg2, end2, idx1, y1, k1);
+        u2 = u3;
+        load_ptr(u3, beg2, end2);
+        u3 = load_u(t + 3 * stride);
+
+        {
+            int free_now = 1;
+            if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
+            free_now = __shfl_sync(0xFFFFFFFFu, free_now, 0);
+            if (!free_now && pending >= 0) {
+                cp_async_wait<0>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.full[pending]);
+                pending = -1;
             }
         }
+        if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 110)) break;
         sm.y[slot][32 * pw + lane] = my_y;
         if (j == 0) { sm.row_u[slot][mr] = u; sm.row_k[slot][mr] = k; }
         const uint32_t tile = smem_u32(&sm.h[slot][0]);
-        const int c = lane & 15;                  // 16-byte chunk of the 256-byte embedding
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int rr = 2 * q + (lane >> 4);   // observation inside this warp's 32
@@ -286,10 +334,19 @@ __device__ void dual_producer(const DualParams &p, DualSmem &sm, int pw, int lan
             else st_shared_zero16(dst);
         }
         cp_async_commit();
-        cp_async_wait<0>();
+        if (pending >= 0) {
+            cp_async_wait<1>();
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.full[pending]);
+        }
+        pending = slot;
+    }
+    cp_async_wait<0>();
+    if (pending >= 0) {
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.full[slot]);
+        if (lane == 0) mbar_arrive(&sm.full[pending]);
     }
 }
 
@@ -322,11 +379,11 @@ __device__ void dual_mma(const DualParams &p, DualSmem &sm, int lane)
     }
 }
 
-__device__ void dual_solver(const DualParams &p, DualSmem &sm, int g, int tid)
+template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm, int g, int tid)
 {
     const int lane = tid & 31, w = tid >> 5;
     const int m = tid;                         // my padded observation = tensor-memory lane
-    const int mr = m >> 4, j = m & 15;         // matrix row of the tile, observation of that row
+    const int mr = m / KP, j = m & (KP - 1);   // matrix row of the tile, observation of that row
     const int bar_id = 1 + g;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + g * D;
     int64_t it = 0;
@@ -340,19 +397,19 @@ __device__ void dual_solver(const DualParams &p, DualSmem &sm, int g, int tid)
         const int u = sm.row_u[g][mr];
         const int k_u = sm.row_k[g][mr];
         const int k_other = __shfl_xor_sync(0xFFFFFFFFu, k_u, 16);
-        const int kmax = k_u > k_other ? k_u : k_other;       // warp-uniform: the two rows of this warp
+        const int kmax = k_u > k_other ? k_u : k_other;       // warp-uniform: the row(s) of this warp
         // S row: s[j'] = sum_f Z[me][f] H[row mr, observation j'][f]
-        float s[16];
+        float s[KP];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) s[c] = 0.f;
+        for (int c = 0; c < KP; ++c) s[c] = 0.f;
         const unsigned char *tile = &sm.h[g][0];
         for (int cf = 0; cf < D / 16; ++cf) {
             float z[16];
             tmem_ld16(trow + 16 * cf, z);
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
+            for (int jj = 0; jj < KP; ++jj) {
                 if (jj < kmax) {
-                    const int row = 16 * mr + jj;
+                    const int row = KP * mr + jj;
                     const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + tile_offset(row, 16 * cf));
                     const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + tile_offset(row, 16 * cf + 8));
                     const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
@@ -367,46 +424,55 @@ __device__ void dual_solver(const DualParams &p, DualSmem &sm, int g, int tid)
             }
         }
         // S = I + (the k x k block); padding observations are rows of the identity with a zero label
-        float d[16];
+        float d[KP];
         const bool mine = j < k_u;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) d[c] = ((mine && c < k_u) ? s[c] : 0.f) + ((c == j) ? 1.f : 0.f);
+        for (int c = 0; c < KP; ++c) d[c] = ((mine && c < k_u) ? s[c] : 0.f) + ((c == j) ? 1.f : 0.f);
         float b = sm.y[g][m];
         float my_inv = 0.f;
         // every thread of the group is past its reads of the tile: its memory now serves as scratch
         asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
         float *scratch = reinterpret_cast<float *>(&sm.h[g][0]);
-        float *xch = scratch + (tid >> 4) * 64;                 // per half-warp
-        float *Lrow = scratch + 8 * 64 + (tid >> 4) * 256;      // per matrix row: L, row-major
-        const bool ok = factor16_pair(d, b, my_inv, lane, xch);
+        float *xch = scratch + mr * (4 * KP);                   // per matrix row
+        float *Lrow = scratch + 8 * 128 + mr * (KP * KP);       // per matrix row: L, row-major
+        const bool ok = factor_rows<KP>(d, b, my_inv, lane, xch);
         // back substitution L^T t = z, column by column from the end
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4)
-            *reinterpret_cast<float4 *>(&Lrow[j * 16 + 4 * q4]) = make_float4(d[4 * q4], d[4 * q4 + 1], d[4 * q4 + 2], d[4 * q4 + 3]);
+        for (int q4 = 0; q4 < KP / 4; ++q4)
+            *reinterpret_cast<float4 *>(&Lrow[j * KP + 4 * q4]) = make_float4(d[4 * q4], d[4 * q4 + 1], d[4 * q4 + 2], d[4 * q4 + 3]);
         __syncwarp();
         float tj = 0.f;
-        const int hb = lane & 16;
+        const int hb = (KP == 16) ? (lane & 16) : 0;
 #pragma unroll
-        for (int c = 15; c >= 0; --c) {
+        for (int c = KP - 1; c >= 0; --c) {
             const float tc = __shfl_sync(0xFFFFFFFFu, b * my_inv, hb + c);
             if (j == c) tj = tc;
-            if (j < c) b = fmaf(-Lrow[c * 16 + j], tc, b);
+            if (j < c) b = fmaf(-Lrow[c * KP + j], tc, b);
         }
         // w = sum over my row's observations of t * Z[observation][:]
-        const bool row_ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, hb) != 0;    // the same for the 16 lanes of a row
+        const bool row_ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, hb) != 0;    // the same for the lanes of a row
         const bool store = (u >= 0);
         for (int cf = 0; cf < D / 16; ++cf) {
             float z[16];
             tmem_ld16(trow + 16 * cf, z);
 #pragma unroll
             for (int c = 0; c < 16; ++c) z[c] *= tj;
-            const float wr = halfwarp_reduce16(z, lane);       // feature 16 cf + j of row u
+            if (KP == 32) {
+                // the two halves of the row's 32 observations, lower half first
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const float other = __shfl_xor_sync(0xFFFFFFFFu, z[c], 16);
+                    z[c] = (lane & 16) ? other + z[c] : z[c] + other;
+                }
+            }
+            const float wr = halfwarp_reduce16(z, lane);       // feature 16 cf + (lane & 15) of row u
             const float wv = row_ok ? wr : 0.f;
-            if (store) {
-                reinterpret_cast<__nv_bfloat16 *>(p.out.table)[(int64_t)u * D + 16 * cf + j] = __float2bfloat16_rn(wv);
+            if (store && (KP == 16 || lane < 16)) {
+                const int f = 16 * cf + (lane & 15);
+                reinterpret_cast<__nv_bfloat16 *>(p.out.table)[(int64_t)u * D + f] = __float2bfloat16_rn(wv);
                 if (p.out.cap_slot) {
                     const int cs = p.out.cap_slot[u];
-                    if (cs >= 0) p.out.cap_out[(int64_t)cs * D + 16 * cf + j] = wv;
+                    if (cs >= 0) p.out.cap_out[(int64_t)cs * D + f] = wv;
                 }
             }
         }
@@ -421,7 +487,7 @@ __device__ void dual_solver(const DualParams &p, DualSmem &sm, int g, int tid)
     }
 }
 
-__global__ void __launch_bounds__(kBlockThreads, 1) k_dual(DualParams p)
+template <int KP> __global__ void __launch_bounds__(kBlockThreads, 1) k_dual(DualParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *aligned = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -450,9 +516,9 @@ __global__ void __launch_bounds__(kBlockThreads, 1) k_dual(DualParams p)
     __syncthreads();
     tc_fence_after();
 
-    if (warp < kMmaWarp) dual_solver(p, sm, warp / (kGroupThreads / 32), tid % kGroupThreads);
+    if (warp < kMmaWarp) dual_solver<KP>(p, sm, warp / (kGroupThreads / 32), tid % kGroupThreads);
     else if (warp == kMmaWarp) dual_mma(p, sm, lane);
-    else dual_producer(p, sm, warp - kMmaWarp - 1, lane);
+    else dual_producer<KP>(p, sm, warp - kMmaWarp - 1, lane);
 
     tc_fence_before();
     __syncthreads();
@@ -464,6 +530,19 @@ __global__ void __launch_bounds__(kBlockThreads, 1) k_dual(DualParams p)
 }
 
 static_assert(sizeof(DualSmem) + 1024 <= 232448, "shared memory of one block exceeds what an SM offers");
+
+template <int KP> cudaError_t launch_dual_instance(DualParams p, int sms, cudaStream_t s, int64_t *launches)
+{
+    if (p.count <= 0) return cudaSuccess;
+    p.n_tiles = (p.count + 128 / KP - 1) / (128 / KP);
+    const size_t smem = sizeof(DualSmem) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(k_dual<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int grid = (int)(p.n_tiles < sms ? p.n_tiles : (sms > 0 ? sms : 1));
+    k_dual<KP><<<grid, kBlockThreads, smem, s>>>(p);
+    ++*launches;
+    return cudaGetLastError();
+}
 
 }  // namespace
 
@@ -483,31 +562,28 @@ cudaError_t launch_dual_prepare(const float *Bmat, void *ws, cudaStream_t s, int
 
 const int *dual_flag_ptr(const void *ws) { return reinterpret_cast<const int *>(static_cast<const unsigned char *>(ws) + kBinvBytes); }
 
-// rows order[first .. first + count) of the solved side, each with 1 .. 16 observations
-cudaError_t launch_rows_dual(const SideView &sv, int64_t first, int64_t count, const void *X, const void *ws, RowOut out,
-                             DevStatus *st, cudaStream_t s, int64_t *launches)
+// rows order[first16 .. first16 + count16) of the solved side have 1 .. 16 observations each, the count32 rows after
+// them 17 .. 32
+cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
+                             const void *ws, RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches)
 {
-    if (count <= 0) return cudaSuccess;
     DualParams p{};
     p.sv = sv;
     p.X = reinterpret_cast<const __nv_bfloat16 *>(X);
     p.binv = static_cast<const unsigned char *>(ws);
     p.flag = dual_flag_ptr(ws);
-    p.first = first;
-    p.count = count;
-    p.n_tiles = (count + kTileRows - 1) / kTileRows;
     p.out = out;
     p.st = st;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const size_t smem = sizeof(DualSmem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(k_dual, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    p.first = first16;
+    p.count = count16;
+    cudaError_t e = launch_dual_instance<16>(p, sms, s, launches);
     if (e != cudaSuccess) return e;
-    const int grid = (int)(p.n_tiles < sms ? p.n_tiles : (sms > 0 ? sms : 1));
-    k_dual<<<grid, kBlockThreads, smem, s>>>(p);
-    ++*launches;
-    return cudaGetLastError();
+    p.first = first16 + count16;
+    p.count = count32;
+    return launch_dual_instance<32>(p, sms, s, launches);
 }
 
 }  // namespace alx

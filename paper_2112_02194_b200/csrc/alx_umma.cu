@@ -79,8 +79,8 @@ struct Params {
     int64_t last_item;           // rows mode: position in sv.order of item 0 (items walk downwards)
     int64_t n_fixed;             // Gramian mode: rows of the table
     const float *Bmat;           // alpha0 G + lambda I
-    const int *dual_flag;        // rows mode: set when the rows of class 1 are solved in the dual form elsewhere
-    int64_t n_items_primal;      // rows mode: items without the rows of class 1 (the last ones of the walk)
+    const int *dual_flag;        // rows mode: set when the rows of classes 1 and 2 are solved in the dual form elsewhere
+    int64_t n_items_primal;      // rows mode: items without the rows of classes 1 and 2 (the last ones of the walk)
     float *partials;             // chunks: [slot][D*D + D]; Gramian: [2 * kGramBlocks][D*D]
     RowOut out;
     DevStatus *st;
@@ -1047,12 +1047,12 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         ++*launches;
     }
     const int64_t n_whole = offs[kNClasses - 1] - offs[1];
-    if (dual_ws && offs[2] > offs[1]) {
-        // rows with 1 .. 16 observations: dual form, if the flag (set on the device) allows it
-        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], X, dual_ws, out, st, s, launches);
+    if (dual_ws && offs[3] > offs[1]) {
+        // rows with 1 .. 32 observations (classes 1 and 2): dual form, if the flag (set on the device) allows it
+        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], offs[3] - offs[2], X, dual_ws, out, st, s, launches);
         if (e != cudaSuccess) return e;
         p.dual_flag = dual_flag_ptr(dual_ws);
-        p.n_items_primal = offs[kNClasses - 1] - offs[2];
+        p.n_items_primal = offs[kNClasses - 1] - offs[3];
     }
     if (n_whole > 0) {
         p.n_items = n_whole;

@@ -266,12 +266,13 @@ def _problem(name):
 
 
 def _class1_rows(p):
+    """rows of 1 .. 32 observations: the ones the dual form takes"""
     deg = np.diff(p.rowptr)
-    return np.nonzero((deg >= 1) & (deg <= 16))[0].astype(np.int64)
+    return np.nonzero((deg >= 1) & (deg <= 32))[0].astype(np.int64)
 
 
 def test_dual_form_for_short_rows_matches_oracle_and_primal_form():
-    """Rows with at most 16 observations are solved through the push-through identity (a k x k system); the
+    """Rows with at most 32 observations are solved through the push-through identity (a k x k system); the
     result must satisfy the same residual gate as the primal form and agree with it."""
     p = _problem("local_d128_bf16")
     ids = _class1_rows(p)
