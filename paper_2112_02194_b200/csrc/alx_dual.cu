@@ -402,25 +402,36 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         float s[KP];
 #pragma unroll
         for (int c = 0; c < KP; ++c) s[c] = 0.f;
-        const unsigned char *tile = &sm.h[g][0];
+        // rows of my matrix row start at a multiple of 8 rows: the swizzle term of row KP mr + jj is jj & 7, known
+        // at compile time, and the row's offset is one runtime base plus constants
+        const unsigned char *tile = &sm.h[g][0] + (KP * mr / 8) * 1024;
+        float z[16], zn[16];
+        tmem_ld16(trow, z);
+        // not unrolled: the body is KP dot products of 16 terms; eight copies of it would not fit the instruction cache
+#pragma unroll 1
         for (int cf = 0; cf < D / 16; ++cf) {
-            float z[16];
-            tmem_ld16(trow + 16 * cf, z);
+            if (cf + 1 < D / 16) tmem_ld16_nowait(trow + 16 * (cf + 1), zn);      // lands while this chunk is used
 #pragma unroll
             for (int jj = 0; jj < KP; ++jj) {
                 if (jj < kmax) {
-                    const int row = KP * mr + jj;
-                    const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + tile_offset(row, 16 * cf));
-                    const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + tile_offset(row, 16 * cf + 8));
+                    const int base = (cf >> 2) * kPanelBytes + (jj >> 3) * 1024 + (jj & 7) * 128;
+                    const int c0 = (cf & 3) * 2;
+                    const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + base + ((c0 ^ (jj & 7)) << 4));
+                    const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + base + (((c0 + 1) ^ (jj & 7)) << 4));
                     const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-                    float acc = s[jj];
+                    // packed FP32 FMAs: even features in .x, odd features in .y (a bfloat16 pair unpacks to exactly that)
+                    float2 acc = make_float2(s[jj], 0.f);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        acc = fmaf(z[2 * e], __uint_as_float(hw[e] << 16), acc);
-                        acc = fmaf(z[2 * e + 1], __uint_as_float(hw[e] & 0xFFFF0000u), acc);
-                    }
-                    s[jj] = acc;
+                    for (int e = 0; e < 8; ++e)
+                        acc = __ffma2_rn(make_float2(z[2 * e], z[2 * e + 1]),
+                                         make_float2(__uint_as_float(hw[e] << 16), __uint_as_float(hw[e] & 0xFFFF0000u)), acc);
+                    s[jj] = acc.x + acc.y;
                 }
+            }
+            if (cf + 1 < D / 16) {
+                tmem_ld_wait();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) z[c] = zn[c];
             }
         }
         // S = I + (the k x k block); padding observations are rows of the identity with a zero label
@@ -452,6 +463,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         // w = sum over my row's observations of t * Z[observation][:]
         const bool row_ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, hb) != 0;    // the same for the lanes of a row
         const bool store = (u >= 0);
+#pragma unroll 1
         for (int cf = 0; cf < D / 16; ++cf) {
             float z[16];
             tmem_ld16(trow + 16 * cf, z);
