@@ -592,7 +592,9 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
 #pragma unroll
                 for (int c = 0; c < 16; c += 4) {
                     const float4 bb = *reinterpret_cast<const float4 *>(Brow + ck + c);
-                    a[c] += bb.x; a[c + 1] += bb.y; a[c + 2] += bb.z; a[c + 3] += bb.w;
+                    const float2 s01 = __fadd2_rn(make_float2(a[c], a[c + 1]), make_float2(bb.x, bb.y));
+                    const float2 s23 = __fadd2_rn(make_float2(a[c + 2], a[c + 3]), make_float2(bb.z, bb.w));
+                    a[c] = s01.x; a[c + 1] = s01.y; a[c + 2] = s23.x; a[c + 3] = s23.y;
                 }
             }
             PHASE_MARK(2);
@@ -644,7 +646,12 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                         c1[4 * q4] = v4.x; c1[4 * q4 + 1] = v4.y; c1[4 * q4 + 2] = v4.z; c1[4 * q4 + 3] = v4.w;
                     }
 #pragma unroll
-                    for (int c = j + 2; c < 16; ++c) a[c] = fmaf(-m1, c1[c], fmaf(-m0, c0[c], a[c]));
+                    for (int c = j + 2; c < 16; c += 2) {
+                        float2 r = __ffma2_rn(make_float2(-m0, -m0), make_float2(c0[c], c0[c + 1]), make_float2(a[c], a[c + 1]));
+                        r = __ffma2_rn(make_float2(-m1, -m1), make_float2(c1[c], c1[c + 1]), r);
+                        a[c] = r.x;
+                        a[c + 1] = r.y;
+                    }
                 }
                 if (!all_ok && lane == 0) gs.bad = 1;
                 if (is_diag) {
@@ -683,13 +690,25 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                         lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
                     }
                     a[pp] *= dv[pp];
+                    // packed FP32 FMAs on pairs of columns: half the issue slots, which the chains of the other
+                    // groups on this sub-partition need
+                    const float mneg = -a[pp];
+                    if ((pp + 1) & 1) a[pp + 1] = fmaf(mneg, lt[pp + 1], a[pp + 1]);
 #pragma unroll
-                    for (int c = pp + 1; c < 16; ++c) a[c] = fmaf(-a[pp], lt[c], a[c]);
+                    for (int c = (pp + 2) & ~1; c < 16; c += 2) {
+                        const float2 r = __ffma2_rn(make_float2(mneg, mneg), make_float2(lt[c], lt[c + 1]), make_float2(a[c], a[c + 1]));
+                        a[c] = r.x;
+                        a[c + 1] = r.y;
+                    }
                 }
-                float acc = 0.f;
+                float2 acc2 = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int c = 0; c < 16; ++c) acc = fmaf(a[c], gs.z[c], acc);
-                b -= acc;
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const float4 zz = *reinterpret_cast<const float4 *>(&gs.z[4 * q4]);
+                    acc2 = __ffma2_rn(make_float2(a[4 * q4], a[4 * q4 + 1]), make_float2(zz.x, zz.y), acc2);
+                    acc2 = __ffma2_rn(make_float2(a[4 * q4 + 2], a[4 * q4 + 3]), make_float2(zz.z, zz.w), acc2);
+                }
+                b -= acc2.x + acc2.y;
                 PHASE_MARK(11);
                 uint32_t w1[8], w2[8], w3[8];
 #pragma unroll
@@ -796,8 +815,13 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     const float4 v = *reinterpret_cast<const float4 *>(&Lb[cp * 16 + 4 * q4]);
                     lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
                 }
+                if ((cp + 1) & 1) tacc[cp + 1] = fmaf(lt[cp + 1], ycp, tacc[cp + 1]);
 #pragma unroll
-                for (int c = cp + 1; c < 16; ++c) tacc[c] = fmaf(lt[c], ycp, tacc[c]);
+                for (int c = (cp + 2) & ~1; c < 16; c += 2) {
+                    const float2 r = __ffma2_rn(make_float2(lt[c], lt[c + 1]), make_float2(ycp, ycp), make_float2(tacc[c], tacc[c + 1]));
+                    tacc[c] = r.x;
+                    tacc[c + 1] = r.y;
+                }
             }
         }
         // (4) back substitution L^T x = z; b now holds z_i
@@ -810,7 +834,11 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 tmem_ld16(trow + ck, wv);
                 const float xm = (pos >= k0 + 16) ? x : 0.f;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) wv[c] = (pos >= k0 + 16) ? wv[c] * xm : 0.f;
+                for (int c = 0; c < 16; c += 2) {
+                    const float2 r = __fmul2_rn(make_float2(wv[c], wv[c + 1]), make_float2(xm, xm));
+                    wv[c] = (pos >= k0 + 16) ? r.x : 0.f;
+                    wv[c + 1] = (pos >= k0 + 16) ? r.y : 0.f;
+                }
                 warp_reduce16(wv, lane);
             } else {
                 wv[0] = 0.f;
