@@ -324,10 +324,16 @@ def run_ours(args, w):
     else:
         roof = {"bound": "alu", "achieved": alu_main / (main_ms * 1e-3) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    # DRAM traffic of that kernel: measured with ncu on the 2M-row `medium` case (4.81 GB for 2.0M rows, L2 hit
-    # rate 90 %), scaled by the rows per launch; the window of +-1 % of the ids scales with the table, so this is
-    # an estimate, not a measurement at this size
-    roof["traffic"] = 4.81e9 / 2.0e6 * rows_whole if w["name"] == "cfg3" else None
+    # DRAM traffic of that kernel: dram__bytes_read + dram__bytes_write of one ncu capture of the 2M-row `medium`
+    # case, per row and per side (columns side: 4.63 GB for 2.00M rows at a 91 % L2 hit rate; rows side, rows of
+    # more than 32 entries: 11.31 GB for 0.359M rows at 46 %), scaled by the rows each launch of this workload
+    # solves and averaged over the two launches of an epoch.  The window of +-1 % of the ids (hence the L2 reuse)
+    # scales with the table, so this is an estimate, not a measurement at this size.
+    if w["name"] in ("cfg3", "medium"):
+        primal_rows = [n_whole[0] - half_ms["dual_rows"][0], n_whole[1] - half_ms["dual_rows"][1]]
+        roof["traffic"] = 0.5 * (primal_rows[0] * 11.31e9 / 0.359e6 + primal_rows[1] * 4.63e9 / 2.0e6)
+    else:
+        roof["traffic"] = None
     roof.update({"kernel": "k_umma<0>: whole rows (gather, tcgen05 outer products, Cholesky in tensor memory, solve, store)",
                  "main_kernel_ms": main_ms, "rows_per_launch": rows_whole,
                  "rows_in_dual_form": {"rows": half_ms["dual_rows"][0], "cols": half_ms["dual_rows"][1],

@@ -601,11 +601,16 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             // (1) diagonal block
             if (wpos == (k0 & ~31)) {
                 const int hb = k0 & 16;
-                const int l = lane - hb;
+                const int l = lane - hb;      // place relative to the block: < 0 eliminated earlier, 0 .. 15 the block,
+                                              // >= 16 the 16 rows after the block (when it is the first of its warp)
                 const bool is_diag = (l >= 0 && l < 16);
                 float my_inv = 0.f;
                 bool all_ok = true;
-                // two pivots per step; branch-free: lanes outside the block run the same code on zero multipliers
+                // Two pivots per round, no masks on the matrix entries: a row that is done only ever overwrites
+                // entries of its upper triangle (never read), and the rows after the block that share this warp get
+                // their forward substitution against the block for free (the same arithmetic in the same order as
+                // the substitution step below, which they then skip).  Only b needs guarding: rows that are done
+                // keep their component of L^-1 b.
 #pragma unroll
                 for (int j = 0; j < 16; j += 2) {
                     const float p00 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j);
@@ -613,26 +618,20 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     const float p11 = __shfl_sync(0xFFFFFFFFu, a[j + 1], hb + j + 1);
                     const float bj = __shfl_sync(0xFFFFFFFFu, b, hb + j);
                     const float bj1 = __shfl_sync(0xFFFFFFFFu, b, hb + j + 1);
-                    const bool ok0 = p00 > 0.f;
-                    const float inv0 = ok0 ? rsqrt_fast(p00) : 0.f;
+                    // a pivot <= 0 turns into NaN or infinity here and stays visible in 1 / L[row][row] (checked below)
+                    const float inv0 = rsqrt_fast(p00);
                     const float l10 = p10 * inv0;
                     const float q11 = fmaf(-l10, l10, p11);
-                    const bool ok1 = q11 > 0.f;
-                    const float inv1 = ok1 ? rsqrt_fast(q11) : 0.f;
-                    all_ok = all_ok && ok0 && ok1;
+                    const float inv1 = rsqrt_fast(q11);
                     const float zj = bj * inv0;
                     const float zj1 = fmaf(-l10, zj, bj1) * inv1;
-                    const float x0 = a[j] * inv0;                       // L[l][j] for rows below
-                    const float x1 = fmaf(-x0, l10, a[j + 1]) * inv1;   // L[l][j+1] for rows below
-                    const bool below = is_diag && l > j + 1;
-                    const float n0 = (l == j) ? p00 * inv0 : ((l == j + 1) ? l10 : x0);
-                    const float n1 = (l == j + 1) ? q11 * inv1 : x1;
-                    a[j] = is_diag ? n0 : a[j];
-                    a[j + 1] = is_diag ? n1 : a[j + 1];
+                    const float x0 = a[j] * inv0;                       // L[row][j]   (row j itself: sqrt of the pivot)
+                    const float x1 = fmaf(-x0, l10, a[j + 1]) * inv1;   // L[row][j+1] (row j+1 itself: sqrt of the second pivot)
+                    a[j] = x0;
+                    a[j + 1] = x1;
                     my_inv = (l == j) ? inv0 : ((l == j + 1) ? inv1 : my_inv);
-                    const float m0 = below ? x0 : 0.f, m1 = below ? x1 : 0.f;
-                    const float bdown = fmaf(-m1, zj1, fmaf(-m0, zj, b));
-                    b = (is_diag && l == j) ? zj : ((is_diag && l == j + 1) ? zj1 : bdown);
+                    const float bdown = fmaf(-x1, zj1, fmaf(-x0, zj, b));
+                    b = (l > j + 1) ? bdown : ((l == j + 1) ? zj1 : ((l == j) ? zj : b));
                     // the two new columns go through shared memory (shuffles are the slower path for 2 x 14 values)
                     float *xb = &gs.xch[(j & 2) * 16];
                     if (is_diag) { xb[l] = x0; xb[16 + l] = x1; }
@@ -647,12 +646,13 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     }
 #pragma unroll
                     for (int c = j + 2; c < 16; c += 2) {
-                        float2 r = __ffma2_rn(make_float2(-m0, -m0), make_float2(c0[c], c0[c + 1]), make_float2(a[c], a[c + 1]));
-                        r = __ffma2_rn(make_float2(-m1, -m1), make_float2(c1[c], c1[c + 1]), r);
+                        float2 r = __ffma2_rn(make_float2(-x0, -x0), make_float2(c0[c], c0[c + 1]), make_float2(a[c], a[c + 1]));
+                        r = __ffma2_rn(make_float2(-x1, -x1), make_float2(c1[c], c1[c + 1]), r);
                         a[c] = r.x;
                         a[c + 1] = r.y;
                     }
                 }
+                all_ok = __all_sync(0xFFFFFFFFu, !is_diag || (my_inv > 0.f && my_inv <= 3.0e38f));
                 if (!all_ok && lane == 0) gs.bad = 1;
                 if (is_diag) {
 #pragma unroll
@@ -673,6 +673,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             PHASE_MARK(4);
             // (2) rows after the block: forward substitution; diagonal threads: their column of the inverse
             if (pos >= k0 + 16) {
+              if (wpos != (k0 & ~31)) {      // (the rows after the block in its own warp are already done, see above)
                 float dv[16];
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
@@ -709,6 +710,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     acc2 = __ffma2_rn(make_float2(a[4 * q4 + 2], a[4 * q4 + 3]), make_float2(zz.z, zz.w), acc2);
                 }
                 b -= acc2.x + acc2.y;
+              }
                 PHASE_MARK(11);
                 uint32_t w1[8], w2[8], w3[8];
 #pragma unroll
