@@ -719,12 +719,16 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     // what is left, so p1 + p2 + p3 = p up to 2^-24
                     const __nv_bfloat162 hpair = __floats2bfloat162_rn(a[c], a[c + 1]);
                     const uint32_t hw = *reinterpret_cast<const uint32_t *>(&hpair);
-                    const float r0 = a[c] - __uint_as_float(hw << 16), r1 = a[c + 1] - __uint_as_float(hw & 0xFFFF0000u);
-                    const uint32_t m0 = __float_as_uint(r0) & 0xFFFF0000u, m1 = __float_as_uint(r1) & 0xFFFF0000u;
-                    const float s0 = r0 - __uint_as_float(m0), s1 = r1 - __uint_as_float(m1);
+                    // (packed arithmetic: x - y as fma(y, -1, x) on both lanes; the upper halves of two words are
+                    // gathered by one byte permutation)
+                    const float2 minus1 = make_float2(-1.f, -1.f);
+                    const float2 r = __ffma2_rn(make_float2(__uint_as_float(hw << 16), __uint_as_float(hw & 0xFFFF0000u)), minus1,
+                                                make_float2(a[c], a[c + 1]));
+                    const uint32_t m0 = __float_as_uint(r.x) & 0xFFFF0000u, m1 = __float_as_uint(r.y) & 0xFFFF0000u;
+                    const float2 sres = __ffma2_rn(make_float2(__uint_as_float(m0), __uint_as_float(m1)), minus1, r);
                     w1[c >> 1] = hw;
-                    w2[c >> 1] = (m0 >> 16) | m1;
-                    w3[c >> 1] = (__float_as_uint(s0) >> 16) | (__float_as_uint(s1) & 0xFFFF0000u);
+                    w2[c >> 1] = __byte_perm(m0, m1, 0x7632);
+                    w3[c >> 1] = __byte_perm(__float_as_uint(sres.x), __float_as_uint(sres.y), 0x7632);
                 }
                 const uint32_t roff = (uint32_t)((i >> 3) * 256 + (i & 7) * 16);
                 const uint32_t b1 = smem_u32(&gs.pop[0][0]) + roff, b2 = smem_u32(&gs.pop[1][0]) + roff,
