@@ -541,11 +541,10 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
     constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
     const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory (= the SM sub-partition)
     const int i = tid;                           // my row of the matrix (= feature index = tensor-memory lane)
-    // Group g eliminates in the cyclic order rot, rot+1, ..., 127, 0, ..., rot-1 (a symmetric permutation of the
-    // matrix): the rows that stay active longest then sit in a different lane quarter, hence on a different
-    // sub-partition's scheduler, for every group.
-    const int rot = (32 * gidx) & (D - 1);
-    const int pos = (i - rot) & (D - 1);         // my place in the elimination order
+    // Rows are eliminated in index order.  (A cyclic order shifted per group, which spreads the long-lived rows of
+    // the four groups over the four sub-partitions, was measured slower: the trailing columns then wrap around
+    // the end of the accumulator and every update takes two sets of tcgen05.mma instead of one.)
+    const int pos = i;                           // my place in the elimination order
     const int wpos = pos & ~31;                  // first place of my warp
     const int bar_id = 1 + gidx;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
@@ -578,7 +577,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
 
         for (int k = 0; k < D / 16; ++k) {
             const int k0 = 16 * k;
-            const int ck = (k0 + rot) & (D - 1);                   // tensor-memory columns of this block
+            const int ck = k0;                                     // tensor-memory columns of this block
             float a[16];
             const bool warp_live = (wpos + 31 >= k0);              // some row of my warp is at or after the block
             if (k > 0) {
@@ -750,7 +749,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             group128_sync(bar_id);
             PHASE_MARK(7);
             // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
-            // blocks of 32 rows further on in the elimination order, which never holds the next diagonal block.  It
+            // blocks of 32 rows further on (cyclically), which never holds the next diagonal block.  It
             // issues the 16 columns of the next panel, waits for them, releases the group through the barrier and
             // only then issues the remaining columns (a tcgen05.mma takes the issuing thread about 50 cycles).
             const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
@@ -773,7 +772,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 tc_fence_after();
 #pragma unroll
                 for (int q = 0; q < 3; ++q) da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
-                update((k0 + 16 + rot) & (D - 1), 16);
+                update(k0 + 16, 16);
                 umma_commit(&gs.trail_bar);
                 if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag, 70)) gs.stop = 1;
             }
@@ -782,12 +781,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 group128_sync(bar_id);
                 if (issuer) {
                     const int n_rest = D - k0 - 32;
-                    if (n_rest > 0) {
-                        const int cs = (k0 + 32 + rot) & (D - 1);
-                        const int n1 = (n_rest < D - cs) ? n_rest : D - cs;     // up to the wrap-around
-                        update(cs, n1);
-                        if (n_rest > n1) update(0, n_rest - n1);
-                    }
+                    if (n_rest > 0) update(k0 + 32, n_rest);
                     umma_commit(&gs.rest_bar);
                 }
             }
@@ -834,7 +828,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         float x = 0.f;
         for (int k = D / 16 - 1; k >= 0; --k) {
             const int k0 = 16 * k;
-            const int ck = (k0 + rot) & (D - 1);
+            const int ck = k0;
             float wv[16];
             if (wpos + 31 >= k0 + 16) {
                 tmem_ld16(trow + ck, wv);
