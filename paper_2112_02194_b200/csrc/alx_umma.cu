@@ -750,8 +750,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             PHASE_MARK(7);
             // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
             // blocks of 32 rows further on (cyclically), which never holds the next diagonal block.  It
-            // issues the 16 columns of the next panel, waits for them, releases the group through the barrier and
-            // only then issues the remaining columns (a tcgen05.mma takes the issuing thread about 50 cycles).
+            // issues the update and waits for it (a tcgen05.mma takes the issuing thread about 50 cycles).
             const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
             uint64_t da[3];
             const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
@@ -772,18 +771,16 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 tc_fence_after();
 #pragma unroll
                 for (int q = 0; q < 3; ++q) da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
-                update(k0 + 16, 16);
+                // all trailing columns in one set of six instructions: the tensor pipe takes about 50 cycles per
+                // instruction whatever its width, and it is shared by the four groups and the gather
+                update(k0 + 16, D - k0 - 16);
                 umma_commit(&gs.trail_bar);
+                umma_commit(&gs.rest_bar);
                 if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag, 70)) gs.stop = 1;
             }
             if (k < D / 16 - 1) {
                 trail_parity ^= 1u;
                 group128_sync(bar_id);
-                if (issuer) {
-                    const int n_rest = D - k0 - 32;
-                    if (n_rest > 0) update(k0 + 32, n_rest);
-                    umma_commit(&gs.rest_bar);
-                }
             }
             PHASE_MARK(8);
         }
