@@ -429,7 +429,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
                 }
             }
             if (cf + 1 < D / 16) {
-                tmem_ld_wait();
+                tmem_ld_wait16(zn);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) z[c] = zn[c];
             }

@@ -168,6 +168,16 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float (&v)[16])
 #pragma unroll
     for (int k = 0; k < 16; ++k) v[k] = __uint_as_float(r[k]);
 }
+// wait for the loads issued so far; the registers of a tmem_ld16_nowait are passed through so that no use of them
+// can be scheduled before the wait
+__device__ __forceinline__ void tmem_ld_wait16(float (&v)[16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]),
+                   "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15])
+                 :
+                 : "memory");
+}
 // thread t of the warp writes 16 consecutive 32-bit columns of lane (base lane + t)
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16])
 {
