@@ -98,8 +98,7 @@ struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver gr
     // three bfloat16 parts (p = p1 + p2 + p3 to 2^-24), each part a K-major 128 x 16 tile without swizzle:
     // groups of 8 rows take 256 bytes, the two 8-element K halves of a group are 128 bytes apart.
     unsigned char pop[3][D * 32];
-    uint64_t trail_bar;     // completion of the next-panel part of the trailing update of the current block step
-    uint64_t rest_bar;      // completion of the remaining part (the operand tiles may be rewritten after it)
+    uint64_t trail_bar;     // completion of the trailing update of the current block step (operand tiles free again)
     alignas(16) float Lt[16][16];    // transpose of the diagonal block's factor: Lt[p][c] = L[c][p] (read as float4)
     alignas(16) float xch[64];       // the two new columns of a diagonal-block step, double buffered
     alignas(16) float dinv[16];
@@ -569,7 +568,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         // right-hand side: the four producer warps' partial sums, in order
         const float *bp = &sm.bpart[it % kBRing][0][i];
         float b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
-        bool dead = false;
         float lrow[16];          // my row of my diagonal block's factor (kept for the block inverse at the end)
         float my_dinv = 0.f;     // 1 / L[i][i]
 #pragma unroll
@@ -581,9 +579,9 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             float a[16];
             const bool warp_live = (wpos + 31 >= k0);              // some row of my warp is at or after the block
             if (k > 0) {
-                // the previous step's tensor-core update of these columns has landed: the issuing thread waited
-                // for it before the group's barrier at the end of that step
-                if (gs.stop) { dead = true; break; }
+                // the previous step's tensor-core update has landed: every warp waits for it on its own (a wait that
+                // gives up only sets the group's stop flag; the group leaves together after the block loop)
+                if (!mbar_wait_warp(&gs.trail_bar, trail_parity ^ 1u, &sm.abort_flag, 70) && lane == 0) gs.stop = 1;
                 tc_fence_after();
             }
             if (warp_live) {
@@ -666,8 +664,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 }
             }
             PHASE_MARK(3);
-            // the previous step's whole tensor-core update has read its operand tiles before they are rewritten
-            if (k > 0 && lane == 0 && wpos == ((k0 + 64) & 96) && !mbar_wait(&gs.rest_bar, trail_parity ^ 1u, &sm.abort_flag, 80)) gs.stop = 1;
             group128_sync(bar_id);
             PHASE_MARK(4);
             // (2) rows after the block: forward substitution; diagonal threads: their column of the inverse
@@ -775,16 +771,12 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 // instruction whatever its width, and it is shared by the four groups and the gather
                 update(k0 + 16, D - k0 - 16);
                 umma_commit(&gs.trail_bar);
-                umma_commit(&gs.rest_bar);
-                if (!mbar_wait(&gs.trail_bar, trail_parity, &sm.abort_flag, 70)) gs.stop = 1;
             }
-            if (k < D / 16 - 1) {
-                trail_parity ^= 1u;
-                group128_sync(bar_id);
-            }
+            if (k < D / 16 - 1) trail_parity ^= 1u;
             PHASE_MARK(8);
         }
-        if (dead) break;
+        group128_sync(bar_id);
+        if (gs.stop) break;
         // my column of the inverse of my diagonal block.  The eight blocks go through shared memory, in the operand
         // tiles: every trailing update has completed (the last one was waited for before the last block step).
         float yinv[16];
@@ -925,7 +917,7 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
     if (MODE == kModeRows) {
         for (int e = tid; e < D * D; e += C::kBlockThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
         for (int g = 0; g < C::kGroups; ++g) {
-            if (tid == 0) { mbar_init(&rgs[g].trail_bar, 1); mbar_init(&rgs[g].rest_bar, 1); }
+            if (tid == 0) mbar_init(&rgs[g].trail_bar, 1);
             for (int k = tid; k < 3 * D * 32 / 16; k += C::kBlockThreads)
                 st_shared_zero16(smem_u32(&rgs[g].pop[0][0]) + k * 16);
         }
