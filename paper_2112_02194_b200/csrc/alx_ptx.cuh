@@ -52,6 +52,37 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return false;
 }
 
+// The suspending form of the wait, for the hand-over of accumulators between the MMA warp and the solver groups: the
+// hardware parks the thread until the phase completes or the time hint runs out, so the waiter takes no issue slots
+// and wakes up without the granularity of a sleep.  Same hard limit (2^16 tries of up to 16 us: about a second) and
+// give-up protocol as mbar_wait.
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1)
+{
+    for (uint32_t it = 0; it < (1u << 16); ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}\n"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(16000u)
+            : "memory");
+        if (ok) return true;
+        if (*abort_flag) return false;
+    }
+    if (*abort_flag == 0) *abort_flag = site;
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait_parked_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait_parked(bar, parity, abort_flag, site) ? 1 : 0;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    return ok != 0;
+}
+
 // One lane polls, the warp follows: keeps the polling traffic of a waiting warp to a single thread.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1)
 {

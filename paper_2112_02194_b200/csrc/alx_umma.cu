@@ -356,14 +356,14 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
         item_range<MODE>(p, t, u, beg, end, slot_unused);
         const int a = (int)(it % Cfg<MODE>::kGroups);
         const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
-        if (!mbar_wait_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
+        if (!mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
         tc_fence_after();
         const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
         bool first = true;
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
-            if (!mbar_wait_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) { alive = false; break; }
+            if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) { alive = false; break; }
             tc_fence_after();
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int nk = (rc + 15) >> 4;
@@ -558,7 +558,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         PHASE_MARK(0);
         // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
         if (tid == 0) {
-            gs.stop = mbar_wait(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
+            gs.stop = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
             gs.bad = 0;
         }
         group128_sync(bar_id);
