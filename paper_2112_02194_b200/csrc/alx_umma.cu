@@ -37,8 +37,8 @@ constexpr int kStageRows = 32;
 // ring of stages: rows mode shares shared memory with the solver groups' scratch and alpha0 G + lambda I, the two
 // streaming modes (chunks, Gramian) use that space for a deeper ring, which is what keeps HBM busy
 template <int MODE> struct Ring {
-    static constexpr int kNStage = (MODE == 0) ? 6 : 18;
-    static constexpr int kLag = (MODE == 0) ? 4 : 14;     // stages of copies in flight per producer warp
+    static constexpr int kNStage = (MODE == 0) ? 8 : 18;
+    static constexpr int kLag = (MODE == 0) ? 6 : 14;     // stages of copies in flight per producer warp
 };
 constexpr int kHalfBytes = kStageRows * 128;          // one 64-feature half of a stage
 constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
@@ -111,7 +111,7 @@ struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver gr
 template <int MODE> struct __align__(1024) SmemT {
     static constexpr int kNStage = Ring<MODE>::kNStage;
     unsigned char h[kNStage][kStageHBytes];
-    unsigned char y[kNStage][kStageYBytes];
+    unsigned char y[(MODE == 0) ? 1 : kNStage][kStageYBytes];      // label tiles (chunks mode only)
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
     uint32_t tmem_base;
     int abort_flag;
@@ -910,7 +910,7 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
         mbar_fence_init();
     }
     // label tiles start finite (all zero): rows beyond an item's end multiply zeros, never stale NaNs
-    for (int k = tid; k < kNStage * kStageYBytes / 16; k += C::kBlockThreads)
+    for (int k = tid; k < (int)sizeof(sm.y) / 16; k += C::kBlockThreads)
         st_shared_zero16(smem_u32(&sm.y[0][0]) + k * 16);
     for (int k = tid; k < kNStage * kStageHBytes / 16; k += C::kBlockThreads)
         st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
