@@ -54,11 +54,8 @@ constexpr int kGramBlocks = 148;                      // fixed, so that the orde
 enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2 };
 
 // thread layout per mode: solver groups (one accumulator each), then one MMA warp, then the producer warps
-#ifndef ALX_DEBUG_ACTIVE_GROUPS
-#define ALX_DEBUG_ACTIVE_GROUPS 4
-#endif
 template <int MODE> struct Cfg {
-    static constexpr int kGroups = (MODE == kModeRows) ? ALX_DEBUG_ACTIVE_GROUPS : 2;
+    static constexpr int kGroups = (MODE == kModeRows) ? 4 : 2;
     static constexpr int kGroupThreads = (MODE == kModeRows) ? 128 : 256;
     static constexpr int kAccStride = (MODE == kModeRows) ? 128 : 256;   // accumulator a: columns a * stride ..
     static constexpr int kSolverThreads = kGroups * kGroupThreads;
@@ -456,16 +453,21 @@ __device__ void copyout_role(const Params &p, SmemT<MODE> &sm, int gidx, int tid
 // ---------------------------------------------------------------------------------------------------------
 // Rows mode: factor and solve in place in tensor memory.  128 threads, thread i = row i = tensor-memory lane i.
 // Blocked right-looking Cholesky, 16 columns per step:
-//   (1) every live row reads its 16 panel values; the 16 threads that own the diagonal block factor it with
-//       shuffles (their warp-mates take part in the shuffles only) and carry b along as a 17th column;
-//   (2) rows below the block do their own forward substitution against the block (from shared memory),
-//       publish their panel row, and fold the block's part of L^-1 b into their b; meanwhile each diagonal
-//       thread computes its column of the block's inverse, which it keeps in registers for step (4);
+//   (1) every warp waits for the previous step's tensor-core update on its own, every live row reads its 16 panel
+//       values (adding alpha0 G + lambda I); the warp that holds the diagonal block factors it with shuffles, two
+//       pivots per round, b carried along as a 17th column; the rows after the block in the same warp get their
+//       forward substitution in the same rounds;
+//   (2) the other rows after the block do their forward substitution against the block (from shared memory) and
+//       fold the block's part of L^-1 b into their b; every row after the block publishes its panel row as three
+//       bfloat16 parts in the operand tiles and writes it back to tensor memory (back substitution reads it);
 //   (3) trailing update A22 -= P P^T on the tensor core, in place in tensor memory: six tcgen05.mma
-//       128 x N x 16 (N = columns right of the block) over the three-way bfloat16 split of P
+//       128 x N x 16 (N = all columns right of the block) over the three-way bfloat16 split of P
 //       (p1p1 + p1p2 + p2p1 + p1p3 + p3p1 + p2p2, the dropped terms are below 2^-26 relative),
-//       A operand negated by the instruction descriptor;
-//   (4) back substitution block by block from the end: per-block partial sums over the rows below are
+//       A operand negated by the instruction descriptor, issued by one thread of a warp that does not hold the
+//       next diagonal block;
+//   (4) after the last step every thread computes its column of the inverse of its own diagonal block (the
+//       eight blocks go through shared memory at once);
+//   (5) back substitution block by block from the end: per-block partial sums over the rows below are
 //       reduced in a fixed order (warp butterfly, then four warps in order), the diagonal threads apply
 //       their inverse columns.
 // alpha0 G + lambda I is added from shared memory when a panel is read (every element of the lower triangle
@@ -519,24 +521,10 @@ __device__ __forceinline__ void group128_sync(int bar_id)
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
 }
 
-#ifdef ALX_PHASE_TIMERS
-__device__ unsigned long long g_phase_cycles[16];
-#define PHASE_MARK(slot)                                                        \
-    do {                                                                        \
-        const long long now_ = clock64();                                       \
-        if (blockIdx.x == 0 && gidx == 0 && tid == 127) atomicAdd(&g_phase_cycles[slot], (unsigned long long)(now_ - t_prev_)); \
-        t_prev_ = now_;                                                         \
-    } while (0)
-#else
-#define PHASE_MARK(slot) do { } while (0)
-#endif
 
 __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, const float *__restrict__ Bs, int gidx,
                                  int tid)
 {
-#ifdef ALX_PHASE_TIMERS
-    long long t_prev_ = clock64();
-#endif
     constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
     const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory (= the SM sub-partition)
     const int i = tid;                           // my row of the matrix (= feature index = tensor-memory lane)
@@ -555,7 +543,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         int64_t u, beg, end, slot;
         item_range<kModeRows>(p, t, u, beg, end, slot);
         const uint32_t aph = (uint32_t)((it / kGroups) & 1);
-        PHASE_MARK(0);
         // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
         if (tid == 0) {
             gs.stop = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
@@ -564,7 +551,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         group128_sync(bar_id);
         if (gs.stop) break;
         tc_fence_after();
-        PHASE_MARK(1);
         // right-hand side: the four producer warps' partial sums, in order
         const float *bp = &sm.bpart[it % kBRing][0][i];
         float b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
@@ -594,7 +580,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     a[c] = s01.x; a[c + 1] = s01.y; a[c + 2] = s23.x; a[c + 3] = s23.y;
                 }
             }
-            PHASE_MARK(2);
             // (1) diagonal block
             if (wpos == (k0 & ~31)) {
                 const int hb = k0 & 16;
@@ -663,10 +648,8 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     my_dinv = my_inv;
                 }
             }
-            PHASE_MARK(3);
             group128_sync(bar_id);
-            PHASE_MARK(4);
-            // (2) rows after the block: forward substitution; diagonal threads: their column of the inverse
+            // (2) rows after the block: forward substitution, split, operand tiles
             if (pos >= k0 + 16) {
               if (wpos != (k0 & ~31)) {      // (the rows after the block in its own warp are already done, see above)
                 float dv[16];
@@ -706,7 +689,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 }
                 b -= acc2.x + acc2.y;
               }
-                PHASE_MARK(11);
                 uint32_t w1[8], w2[8], w3[8];
 #pragma unroll
                 for (int c = 0; c < 16; c += 2) {
@@ -731,19 +713,14 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 st_shared_v4(b1, w1[0], w1[1], w1[2], w1[3]); st_shared_v4(b1 + 128, w1[4], w1[5], w1[6], w1[7]);
                 st_shared_v4(b2, w2[0], w2[1], w2[2], w2[3]); st_shared_v4(b2 + 128, w2[4], w2[5], w2[6], w2[7]);
                 st_shared_v4(b3, w3[0], w3[1], w3[2], w3[3]); st_shared_v4(b3 + 128, w3[4], w3[5], w3[6], w3[7]);
-                PHASE_MARK(12);
                 fence_proxy_async();
-                PHASE_MARK(13);
             }
-            PHASE_MARK(5);
             if (warp_live) {
                 tmem_st16(trow + ck, a);      // L (rows before the block rewrite what they read)
                 tmem_st_wait();
             }
             tc_fence_before();
-            PHASE_MARK(6);
             group128_sync(bar_id);
-            PHASE_MARK(7);
             // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
             // blocks of 32 rows further on (cyclically), which never holds the next diagonal block.  It
             // issues the update and waits for it (a tcgen05.mma takes the issuing thread about 50 cycles).
@@ -773,7 +750,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 umma_commit(&gs.trail_bar);
             }
             if (k < D / 16 - 1) trail_parity ^= 1u;
-            PHASE_MARK(8);
         }
         group128_sync(bar_id);
         if (gs.stop) break;
@@ -849,7 +825,6 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                 if (is_diag) x = acc;
             }
         }
-        PHASE_MARK(9);
         // tensor memory is free again for the next item of this accumulator
         tc_fence_before();
         group128_sync(bar_id);
@@ -866,24 +841,10 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             raise_flag(p.st, kFlagNotSpd, u);
         }
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
-        PHASE_MARK(10);
     }
 }
 
 
-#ifdef ALX_PHASE_TIMERS
-}  // namespace
-extern "C" int alx_debug_phase_cycles(unsigned long long *out, int reset)
-{
-    cudaError_t e = cudaMemcpyFromSymbol(out, g_phase_cycles, sizeof(unsigned long long) * 16);
-    if (reset) {
-        unsigned long long z[16] = {};
-        cudaMemcpyToSymbol(g_phase_cycles, z, sizeof z);
-    }
-    return (int)e;
-}
-namespace {
-#endif
 
 template <int MODE>
 __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
