@@ -147,6 +147,26 @@ def test_alpha_zero_is_ridge_regression():
 
 # ---- the update is the exact minimiser: gradient of Eq. 3, all-pairs term summed explicitly -----
 
+def test_push_through_identity_gives_the_same_row():
+    """Eq. 4 restated for a row with k < d observations (the form the library uses for short rows):
+    (B + H^T H)^-1 H^T y = B^-1 H^T (I_k + H B^-1 H^T)^-1 y with B = alpha G + lambda I.  The oracle solves the
+    d x d form; the k x k form written out with numpy must give the same rows."""
+    rowptr, colidx, vals, W, H, _ = random_problem(9, 40, 12, 0.12, 31)
+    alpha, lam = 0.07, 0.3
+    got = ials.half_step(rowptr, colidx, vals, H, alpha, lam)
+    B = alpha * (H.T @ H) + lam * np.eye(H.shape[1])
+    Binv = np.linalg.inv(B)
+    for u in range(9):
+        idx = colidx[rowptr[u]:rowptr[u + 1]]
+        if idx.size == 0:
+            assert np.all(got[u] == 0)
+            continue
+        Hu, yu = H[idx], vals[rowptr[u]:rowptr[u + 1]]
+        Z = Hu @ Binv
+        t = np.linalg.solve(np.eye(idx.size) + Z @ Hu.T, yu)
+        np.testing.assert_allclose(got[u], Z.T @ t, rtol=1e-10, atol=1e-13)
+
+
 def test_gradient_of_objective_vanishes_at_the_update():
     n_rows, n_cols, d = 25, 18, 5
     rowptr, colidx, vals, W, H, mask = random_problem(n_rows, n_cols, d, 0.35, 9)
