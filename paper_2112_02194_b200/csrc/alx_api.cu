@@ -244,7 +244,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     if (tensor_path(c)) {
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
-                                     &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr));
+                                     &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed]));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
         c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;

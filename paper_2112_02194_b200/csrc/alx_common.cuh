@@ -133,7 +133,7 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                              int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
                              RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,
-                             cudaEvent_t main_end, const void *dual_ws);
+                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table);
 
 // alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();

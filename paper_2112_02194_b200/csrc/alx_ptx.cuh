@@ -105,6 +105,23 @@ template <int N> __device__ __forceinline__ void cp_async_wait()
 // makes this thread's earlier shared-memory writes (generic proxy) visible to the tensor core's reads (async proxy)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// ---- TMA row gather (tile::gather4): four rows of a 2-D tensor, one box width each, land as four consecutive
+// lines of the destination, swizzled as the tensor map says; completion is counted in bytes on an mbarrier.
+// x (first coordinate, in elements) times the element size must be a multiple of 16 bytes.  A row coordinate past the
+// tensor's extent is filled with zeros.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_gather4(uint32_t dst_smem, const void *tensor_map, int x, int r0, int r1, int r2, int r3,
+                                            uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst_smem), "l"(tensor_map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
+        : "memory");
+}
+
 __device__ __forceinline__ void st_shared_zero16(uint32_t dst_smem)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst_smem), "r"(0u) : "memory");

@@ -9,20 +9,23 @@
 //                    shared-memory stages, already in the operand layout the tensor core reads:
 //                    "MN-major, 128-byte swizzle" - a gathered row is one K index, its 128 features
 //                    are the M (and N) index, split into two 64-feature halves of 128 bytes;
-//   one MMA thread   issues tcgen05.mma 128 x 128 x 16 (A = B = the staged tile) into one of two
-//                    fp32 accumulators in tensor memory, plus a 128 x 16 x 16 product with a two-column
-//                    (high / low bfloat16 parts of the label) tile that yields sum y x_i;
-//   solver groups    rows: three groups of 128 threads, one per accumulator, thread i owning row i of
+//   one MMA thread   issues tcgen05.mma 128 x 128 x 16 (A = B = the staged tile) into one of the fp32
+//                    accumulators in tensor memory (four of 128 columns in rows mode, two of 256 otherwise);
+//                    chunks also get a 128 x 16 x 16 product with a two-column (high / low bfloat16 parts of
+//                    the label) tile that yields sum y x_i (whole rows: the producer warps sum it);
+//   solver groups    rows: four groups of 128 threads, one per accumulator, thread i owning row i of
 //                    the normal matrix.  The matrix never leaves tensor memory: the group adds
 //                    alpha0 G + lambda I on first touch, factors it in place with a blocked right-looking
-//                    Cholesky (tcgen05.ld / tcgen05.st of 16-column row segments), solves and stores the
-//                    row.  Gramian pieces and chunks: two groups of 256 threads copy the sums out.
+//                    Cholesky (tcgen05.ld / tcgen05.st of 16-column row segments, trailing updates on the
+//                    tensor core), solves and stores the row.  Gramian pieces and chunks: two groups of 256
+//                    threads copy the sums out.
 // Stage and accumulator hand-over is by mbarriers; every wait is bounded and a block that gives up
 // sets a status flag, releases its tensor memory and returns.
 #include "alx_chol.cuh"
 #include "alx_common.cuh"
 #include "alx_ptx.cuh"
 #include <cstring>
+#include <cuda.h>      // CUtensorMap and its enumerations (types only: the encoder is looked up at run time)
 
 namespace alx {
 
@@ -36,9 +39,14 @@ constexpr int D = 128;
 constexpr int kStageRows = 32;
 // ring of stages: rows mode shares shared memory with the solver groups' scratch and alpha0 G + lambda I, the two
 // streaming modes (chunks, Gramian) use that space for a deeper ring, which is what keeps HBM busy
+// (and stages of 64 gathered rows instead of 32: half the per-stage waits and commits of the MMA thread)
 template <int MODE> struct Ring {
-    static constexpr int kNStage = (MODE == 0) ? 8 : 18;
-    static constexpr int kLag = (MODE == 0) ? 6 : 14;     // stages of copies in flight per producer warp
+    static constexpr int kRows = (MODE == 0) ? 32 : 64;   // gathered rows per stage
+    static constexpr int kNStage = (MODE == 0) ? 8 : 12;
+    static constexpr int kLag = 6;                        // rows mode: stages of cp.async copies in flight per producer warp
+    static constexpr int kHalfBytes = kRows * 128;        // one 64-feature half of a stage
+    static constexpr int kStageHBytes = 2 * kHalfBytes;
+    static constexpr int kStageYBytes = 2 * kRows * 16;   // label tile, two 8-column chunks
 };
 constexpr int kHalfBytes = kStageRows * 128;          // one 64-feature half of a stage
 constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
@@ -61,10 +69,10 @@ template <int MODE> struct Cfg {
     static constexpr int kSolverThreads = kGroups * kGroupThreads;
     static constexpr int kMmaWarp = kSolverThreads / 32;
     static constexpr int kFirstProducerWarp = kMmaWarp + 1;
-    // rows mode: the four producer warps share every stage (8 rows each; their partial right-hand sides are summed in
-    // a fixed order); streaming modes: eight producer warps, each fills whole stages of its own (a stage costs a
-    // warp about 2000 cycles of waits, fences and address arithmetic whatever its share of the rows)
-    static constexpr int kProducers = (MODE == kModeRows) ? kProducerWarps : 8;
+    // rows mode: the four producer warps share every stage (8 rows each, by cp.async; their partial right-hand sides
+    // are summed in a fixed order); streaming modes: four producer warps, each fills whole stages of its own by TMA
+    // row gathers
+    static constexpr int kProducers = (MODE == kModeRows) ? kProducerWarps : 4;
     static constexpr int kFullArrivals = (MODE == kModeRows) ? kProducerWarps : 1;
     static constexpr int kBlockThreads = kSolverThreads + 32 + kProducers * 32;
 };
@@ -75,6 +83,7 @@ struct Params {
     int64_t n_items;             // rows of classes 1 .. 10 / chunk descriptors / 1024-row sub-pieces
     int64_t last_item;           // rows mode: position in sv.order of item 0 (items walk downwards)
     int64_t n_fixed;             // Gramian mode: rows of the table
+    int64_t n_table;             // rows of the fixed table (= the first row coordinate that a row gather fills with zeros)
     const float *Bmat;           // alpha0 G + lambda I
     const int *dual_flag;        // rows mode: set when the rows of classes 1 and 2 are solved in the dual form elsewhere
     int64_t n_items_primal;      // rows mode: items without the rows of classes 1 and 2 (the last ones of the walk)
@@ -107,8 +116,8 @@ struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver gr
 
 template <int MODE> struct __align__(1024) SmemT {
     static constexpr int kNStage = Ring<MODE>::kNStage;
-    unsigned char h[kNStage][kStageHBytes];
-    unsigned char y[(MODE == 0) ? 1 : kNStage][kStageYBytes];      // label tiles (chunks mode only)
+    unsigned char h[kNStage][Ring<MODE>::kStageHBytes];
+    unsigned char y[(MODE == 0) ? 1 : kNStage][Ring<MODE>::kStageYBytes];      // label tiles (chunks mode only)
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
     uint32_t tmem_base;
     int abort_flag;
@@ -117,7 +126,7 @@ template <int MODE> struct __align__(1024) SmemT {
     int stage_meta[kNStage];                     // K steps of the stage (1 or 2) | 4 if it ends its item; -1: no more work
     int rows_staged[kProducerWarps][kNStage];    // per producer warp: how many of its 8 rows of the stage are defined
     int last_of_item[kProducerWarps][kNStage];   // per producer warp: 1 + ring index of the item whose last stage this is, else 0
-    alignas(16) float bpart[kBRing][kProducerWarps][D];
+    alignas(16) float bpart[(MODE == 0) ? kBRing : 1][kProducerWarps][D];
 };
 
 template <int MODE> __device__ __forceinline__ void item_range(const Params &p, int64_t t, int64_t &u, int64_t &beg,
@@ -269,84 +278,84 @@ template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &
 }
 
 // Streaming modes (chunks, Gramian pieces): producer warp pw fills the stages whose running number is pw modulo the
-// number of producer warps, whole stages of 32 rows each, and announces a stage once the next stage of its own has
-// been issued (or at once when it would otherwise block).
-template <int MODE> __device__ void stream_producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
+// number of producer warps, whole stages of 64 rows each.  The rows come by TMA row gathers (four rows of one
+// 64-feature half per instruction, written with the 128-byte swizzle the tensor core reads), issued by lanes 0 .. 15 for
+// the 16 groups of four rows; the stage's mbarrier counts the bytes.  Rows past the end of the item take a row
+// coordinate past the end of the table, which the copy fills with zeros.
+template <int MODE>
+__device__ void stream_producer_role(const Params &p, const CUtensorMap *tmap, SmemT<MODE> &sm, int pw, int lane)
 {
-    constexpr int kNStage = Ring<MODE>::kNStage, P = Cfg<MODE>::kProducers, kOwnLag = 1;
+    constexpr int kNStage = Ring<MODE>::kNStage, kRows = Ring<MODE>::kRows, P = Cfg<MODE>::kProducers;
+    static_assert(kRows == 64, "two rows per lane, sixteen groups of four rows");
     int64_t g = 0;                        // running number of the stage over all items of this block
-    int64_t issued = 0, announced = 0;    // own stages
-    const int c = lane & 15;              // 16-byte chunk of the 256-byte row
-    const int half = c >> 3, cc = c & 7;
+    int ring_slot = 0;                    // ring position and phase of stage g
+    uint32_t ring_ph = 0;
+    const int32_t past_end = (int32_t)p.n_table;
     bool alive = true;
-    auto announce = [&](int64_t n) {
-        const int slot = (int)((pw + P * n) % kNStage);
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.full[slot]);
-    };
     for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x) {
         int64_t u, beg, end, slot_unused;
         item_range<MODE>(p, t, u, beg, end, slot_unused);
-        for (int64_t e0 = beg; e0 < end; e0 += kStageRows, ++g) {
+        for (int64_t e0 = beg; e0 < end; e0 += kRows, ++g) {
+            const int slot = ring_slot;
+            const uint32_t ph = ring_ph;
+            if (++ring_slot == kNStage) { ring_slot = 0; ring_ph ^= 1u; }
             if ((int)(g % P) != pw) continue;
-            const int slot = (int)(g % kNStage);
-            const uint32_t ph = (uint32_t)((g / kNStage) & 1);
-            // this lane's row of the stage
-            const int64_t e = e0 + lane;
-            int32_t my_idx = -1;
-            float my_y = 0.f;
-            if (e < end) {
-                my_idx = (MODE == kModeGramian) ? (int32_t)e : p.sv.idx[e];
-                my_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[e] : 1.f);
-            }
-            {
-                int free_now = 1;
-                if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
-                free_now = __shfl_sync(0xFFFFFFFFu, free_now, 0);
-                if (!free_now && announced < issued) {
-                    cp_async_wait<0>();
-                    for (; announced < issued; ++announced) announce(announced);
+            // this lane's two rows of the stage (lane and 32 + lane)
+            int32_t my_idx[2] = {past_end, past_end};
+            float my_y[2] = {0.f, 0.f};
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int64_t e = e0 + 32 * k + lane;
+                if (e < end) {
+                    my_idx[k] = (MODE == kModeGramian) ? (int32_t)e : p.sv.idx[e];
+                    my_y[k] = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[e] : 1.f);
                 }
             }
-            if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
-            const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
-            const int rc16 = (rc + 15) & ~15;
-            const uint32_t hbase = smem_u32(&sm.h[slot][0]) + half * kHalfBytes;
+            // rows 4 * lane .. 4 * lane + 3 of the stage (lanes 0 .. 15)
+            int32_t r4[4];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) {
-                const int r = (lane >> 4) + 2 * q;          // row inside the stage
-                const int32_t src = __shfl_sync(0xFFFFFFFFu, my_idx, r);
-                const uint32_t dst = hbase + r * 128 + ((cc ^ (r & 7)) << 4);
-                if (src >= 0) cp_async16(dst, p.X + (int64_t)src * D + c * 8);
-                else if (r < rc16) st_shared_zero16(dst);
+            for (int j = 0; j < 4; ++j) {
+                const int32_t v0 = __shfl_sync(0xFFFFFFFFu, my_idx[0], (4 * lane + j) & 31);
+                const int32_t v1 = __shfl_sync(0xFFFFFFFFu, my_idx[1], (4 * lane + j) & 31);
+                r4[j] = (lane < 8) ? v0 : v1;
             }
-            if (MODE == kModeChunks && lane < rc16) {
-                const __nv_bfloat16 yhi = __float2bfloat16_rn(my_y);
-                const __nv_bfloat16 ylo = __float2bfloat16_rn(my_y - __bfloat162float(yhi));
-                const uint32_t packed = (uint32_t)__bfloat16_as_ushort(yhi) | ((uint32_t)__bfloat16_as_ushort(ylo) << 16);
-                st_shared_v4(smem_u32(&sm.y[slot][0]) + lane * 16, packed, 0u, 0u, 0u);
+            if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
+            const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
+            const int rc16 = (rc + 15) & ~15;
+            if (MODE == kModeChunks) {
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    if (32 * k + lane < rc16) {
+                        const __nv_bfloat16 yhi = __float2bfloat16_rn(my_y[k]);
+                        const __nv_bfloat16 ylo = __float2bfloat16_rn(my_y[k] - __bfloat162float(yhi));
+                        const uint32_t packed = (uint32_t)__bfloat16_as_ushort(yhi) | ((uint32_t)__bfloat16_as_ushort(ylo) << 16);
+                        st_shared_v4(smem_u32(&sm.y[slot][0]) + (32 * k + lane) * 16, packed, 0u, 0u, 0u);
+                    }
+                }
+                fence_proxy_async();
             }
-            cp_async_commit();
-            ++issued;
-            if (issued - announced > kOwnLag) {
-                cp_async_wait<kOwnLag>();
-                announce(announced);
-                ++announced;
+            __syncwarp();
+            const int ngroups = rc16 >> 2;        // groups of four rows the tensor core will read
+            if (lane == 0) mbar_arrive_expect_tx(&sm.full[slot], (uint32_t)ngroups * 1024u);
+            if (lane < ngroups) {
+                const uint32_t dst = smem_u32(&sm.h[slot][0]) + lane * 512;
+                tma_gather4(dst, tmap, 0, r4[0], r4[1], r4[2], r4[3], &sm.full[slot]);
+                tma_gather4(dst + Ring<MODE>::kHalfBytes, tmap, 64, r4[0], r4[1], r4[2], r4[3], &sm.full[slot]);
             }
+            __syncwarp();
         }
     }
-    cp_async_wait<0>();
-    for (; announced < issued; ++announced) announce(announced);
 }
 
 template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, int lane)
 {
-    constexpr int kNStage = Ring<MODE>::kNStage;
+    constexpr int kNStage = Ring<MODE>::kNStage, kRows = Ring<MODE>::kRows;
     constexpr uint32_t kIdescMain = idesc_bf16_mn_major(128, 128);
     constexpr uint32_t kIdescY = idesc_bf16_mn_major(128, 16);
     const uint32_t tmem = sm.tmem_base;
-    int64_t g = 0, it = 0;
+    int64_t it = 0;
+    int slot = 0;             // ring position and phase of the next stage
+    uint32_t ph = 0;
     bool alive = true;
     for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
         int64_t u, beg, end, slot_unused;
@@ -357,22 +366,20 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
         tc_fence_after();
         const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
         bool first = true;
-        for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
-            const int slot = (int)(g % kNStage);
-            const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+        for (int64_t e0 = beg; e0 < end; e0 += kRows) {
             if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) { alive = false; break; }
             tc_fence_after();
-            const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
+            const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
             const int nk = (rc + 15) >> 4;
             if (lane == 0) {
                 const uint32_t hb = smem_u32(&sm.h[slot][0]);
                 const uint32_t yb = smem_u32(&sm.y[slot][0]);
                 for (int ks = 0; ks < nk; ++ks) {
                     // 16 gathered rows = two groups of 8 rows of 128 bytes; halves are kHalfBytes apart
-                    const uint64_t adesc = smem_desc(hb + ks * 2048, kHalfBytes, 1024, 2);
+                    const uint64_t adesc = smem_desc(hb + ks * 2048, Ring<MODE>::kHalfBytes, 1024, 2);
                     umma_f16(d_main, adesc, adesc, kIdescMain, !first);
                     if (MODE == kModeChunks) {
-                        const uint64_t ydesc = smem_desc(yb + ks * 256, 128, kStageRows * 16, 0);
+                        const uint64_t ydesc = smem_desc(yb + ks * 256, 128, kRows * 16, 0);
                         umma_f16(d_main + D, adesc, ydesc, kIdescY, !first);
                     }
                     first = false;
@@ -380,7 +387,7 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
                 umma_commit(&sm.empty[slot]);
             }
             __syncwarp();
-            ++g;
+            if (++slot == kNStage) { slot = 0; ph ^= 1u; }
         }
         if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
         __syncwarp();
@@ -847,7 +854,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
 
 
 template <int MODE>
-__global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
+__global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p, const __grid_constant__ CUtensorMap tmap)
 {
     using C = Cfg<MODE>;
     if (MODE == kModeRows && p.dual_flag && *p.dual_flag) {
@@ -873,7 +880,7 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
     // label tiles start finite (all zero): rows beyond an item's end multiply zeros, never stale NaNs
     for (int k = tid; k < (int)sizeof(sm.y) / 16; k += C::kBlockThreads)
         st_shared_zero16(smem_u32(&sm.y[0][0]) + k * 16);
-    for (int k = tid; k < kNStage * kStageHBytes / 16; k += C::kBlockThreads)
+    for (int k = tid; k < (int)sizeof(sm.h) / 16; k += C::kBlockThreads)
         st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
     if (MODE == kModeRows) {
         for (int e = tid; e < D * D; e += C::kBlockThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
@@ -901,7 +908,7 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p)
         mma_role<MODE>(p, sm, lane);
     } else {
         if constexpr (MODE == kModeRows) producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
-        else stream_producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
+        else stream_producer_role<MODE>(p, &tmap, sm, warp - C::kFirstProducerWarp, lane);
     }
 
     tc_fence_before();
@@ -965,12 +972,41 @@ template <int MODE> size_t smem_bytes()
 }
 static_assert(sizeof(SmemT<1>) + 1024 <= 232448 && sizeof(SmemT<1>) > 116224, "ring depth of the streaming modes");
 
+// Tensor map of a bfloat16 table [n x 128] for row gathers: boxes of one row by 64 features (128 bytes), 128-byte swizzle.
+// (The encoder is a driver entry point, looked up through the runtime so that the library needs no driver at link time.)
+cudaError_t table_tensor_map(const void *X, int64_t n, CUtensorMap *tm)
+{
+    typedef CUresult (*Encode)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                               const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static Encode encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return e;
+        if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<Encode>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)n};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * sizeof(__nv_bfloat16)};
+    const cuuint32_t box[2] = {64, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(X), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStream_t s)
 {
     const size_t smem = smem_bytes<MODE>();
     cudaError_t e = cudaFuncSetAttribute(k_umma<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_umma<MODE><<<grid, Cfg<MODE>::kBlockThreads, smem, s>>>(p);
+    CUtensorMap tm;
+    e = table_tensor_map(p.X, p.n_table, &tm);
+    if (e != cudaSuccess) return e;
+    k_umma<MODE><<<grid, Cfg<MODE>::kBlockThreads, smem, s>>>(p, tm);
     return cudaGetLastError();
 }
 
@@ -992,6 +1028,7 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
     Params p{};
     p.X = reinterpret_cast<const __nv_bfloat16 *>(X);
     p.n_fixed = n;
+    p.n_table = n;
     p.n_items = (n + kGramSubRows - 1) / kGramSubRows;
     p.partials = partials;
     cudaError_t e = launch_mode<kModeGramian>(p, kGramBlocks, s);
@@ -1002,12 +1039,13 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows,
                              const void *X, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
                              cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
-                             const void *dual_ws)
+                             const void *dual_ws, int64_t n_table)
 {
     const int sms = sm_count();
     Params p{};
     p.sv = sv;
     p.X = reinterpret_cast<const __nv_bfloat16 *>(X);
+    p.n_table = n_table;
     p.Bmat = Bmat;
     p.partials = split_partials;
     p.out = out;
