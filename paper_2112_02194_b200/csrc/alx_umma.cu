@@ -571,13 +571,8 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             const int ck = k0;                                     // tensor-memory columns of this block
             float a[16];
             const bool warp_live = (wpos + 31 >= k0);              // some row of my warp is at or after the block
-            if (k > 0) {
-                // the previous step's tensor-core update has landed: every warp waits for it on its own (a wait that
-                // gives up only sets the group's stop flag; the group leaves together after the block loop)
-                if (!mbar_wait_warp(&gs.trail_bar, trail_parity ^ 1u, &sm.abort_flag, 70) && lane == 0) gs.stop = 1;
-                tc_fence_after();
-            }
-            if (warp_live) {
+            const bool diag_warp = (wpos == (k0 & ~31));
+            auto load_panel = [&]() {
                 tmem_ld16(trow + ck, a);
 #pragma unroll
                 for (int c = 0; c < 16; c += 4) {
@@ -586,9 +581,19 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     const float2 s23 = __fadd2_rn(make_float2(a[c + 2], a[c + 3]), make_float2(bb.z, bb.w));
                     a[c] = s01.x; a[c + 1] = s01.y; a[c + 2] = s23.x; a[c + 3] = s23.y;
                 }
+            };
+            if (diag_warp) {
+                // the previous step's tensor-core update has landed: only the warp that holds the diagonal block waits
+                // for it (a wait that gives up only sets the group's stop flag; the group leaves together after the
+                // block loop); the other warps follow through the barrier below, at no cost in issue slots
+                if (k > 0) {
+                    if (!mbar_wait_warp(&gs.trail_bar, trail_parity ^ 1u, &sm.abort_flag, 70) && lane == 0) gs.stop = 1;
+                    tc_fence_after();
+                }
+                load_panel();
             }
             // (1) diagonal block
-            if (wpos == (k0 & ~31)) {
+            if (diag_warp) {
                 const int hb = k0 & 16;
                 const int l = lane - hb;      // place relative to the block: < 0 eliminated earlier, 0 .. 15 the block,
                                               // >= 16 the 16 rows after the block (when it is the first of its warp)
@@ -655,7 +660,12 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
                     my_dinv = my_inv;
                 }
             }
+            tc_fence_before();
             group128_sync(bar_id);
+            if (warp_live && !diag_warp) {
+                tc_fence_after();
+                load_panel();
+            }
             // (2) rows after the block: forward substitution, split, operand tiles
             if (pos >= k0 + 16) {
               if (wpos != (k0 & ~31)) {      // (the rows after the block in its own warp are already done, see above)
