@@ -414,7 +414,11 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     dev_free(c, scan_scratch);
 
     const int d = c->opt.d;
-    const int64_t max_chunks = c->n_chunks[0] > c->n_chunks[1] ? c->n_chunks[0] : c->n_chunks[1];
+    int64_t sums[2] = {c->n_chunks[0], c->n_chunks[1]};
+    if (tensor_path(c))      // one more sum per long whole row
+        for (int s = 0; s < 2; ++s)
+            sums[s] += c->class_offs[s][kNClasses - 1] - c->class_offs[s][long_class_begin(c->class_offs[s])];
+    const int64_t max_chunks = sums[0] > sums[1] ? sums[0] : sums[1];
     if (max_chunks > 0) ALX_ALLOC(c, c->split_partials, max_chunks * (int64_t)(d * d + d));
     ALX_ALLOC(c, c->loss_partials_buf, loss_partials(nnz));
     c->stats.nnz = nnz;

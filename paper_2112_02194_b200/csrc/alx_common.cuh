@@ -127,6 +127,17 @@ cudaError_t launch_rows_simple(const SideView &sv, const int64_t *class_offs_hos
                                float *split_partials, RowOut out, DevStatus *st, cudaStream_t s,
                                int64_t *launches);
 
+// Tensor-core path: the first degree class whose rows (with all longer whole rows) get their sums from the chunks
+// kernel instead of the rows kernel.  Classes 8 .. 10 (1025 .. 8192 observations at the default split) qualify, from
+// the top, as long as they hold at most kLongRowBudget rows together (one d x d + d sum of workspace each).
+constexpr int64_t kLongRowBudget = 65536;
+inline int long_class_begin(const int64_t *class_offs_host)
+{
+    int c = kNClasses - 1;
+    while (c > 8 && class_offs_host[kNClasses - 1] - class_offs_host[c - 1] <= kLongRowBudget) --c;
+    return c;
+}
+
 // alx_umma.cu: tensor-core path, d = 128 and bf16 tables only
 int64_t gramian_umma_partials();
 cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches);

@@ -84,18 +84,16 @@ struct Params {
     int64_t last_item;           // rows mode: position in sv.order of item 0 (items walk downwards)
     int64_t n_fixed;             // Gramian mode: rows of the table
     int64_t n_table;             // rows of the fixed table (= the first row coordinate that a row gather fills with zeros)
+    int64_t n_chunks;            // chunks mode: chunk descriptors; the items after them are the long whole rows
+    int64_t long_end;            // chunks mode and solve-from-sums: one past the position in sv.order of the last long row
+    int64_t split_begin;         // solve-from-sums: position in sv.order of the first split row
+    int64_t n_split_rows;        // solve-from-sums: split rows (items 0 .. n_split_rows - 1), then the long whole rows
     const float *Bmat;           // alpha0 G + lambda I
     const int *dual_flag;        // rows mode: set when the rows of classes 1 and 2 are solved in the dual form elsewhere
     int64_t n_items_primal;      // rows mode: items without the rows of classes 1 and 2 (the last ones of the walk)
     float *partials;             // chunks: [slot][D*D + D]; Gramian: [2 * kGramBlocks][D*D]
     RowOut out;
     DevStatus *st;
-};
-
-struct GroupSmem {   // split-row solve: one matrix in shared memory
-    float As[Geo<D>::A_FLOATS];
-    float Pt[Geo<D>::P_FLOATS];
-    float dinv[D];
 };
 
 constexpr int kLdB = D + 4;
@@ -138,8 +136,15 @@ template <int MODE> __device__ __forceinline__ void item_range(const Params &p, 
         end = p.sv.ptr[u + 1];
         slot = 0;
     } else if (MODE == kModeChunks) {
-        const int64_t *d = p.sv.chunk_desc + 4 * t;
-        u = d[0]; beg = d[1]; end = d[2]; slot = d[3];
+        if (t < p.n_chunks) {
+            const int64_t *d = p.sv.chunk_desc + 4 * t;
+            u = d[0]; beg = d[1]; end = d[2]; slot = d[3];
+        } else {      // a long whole row, longest class first: one sum of its own, stored after the chunks' sums
+            u = p.sv.order[p.long_end - 1 - (t - p.n_chunks)];
+            beg = p.sv.ptr[u];
+            end = p.sv.ptr[u + 1];
+            slot = t;
+        }
     } else {
         u = 0; slot = t;
         beg = t * kGramSubRows;
@@ -529,6 +534,10 @@ __device__ __forceinline__ void group128_sync(int bar_id)
 }
 
 
+// FROM_SUMS: the items are rows whose sums were formed by the chunks kernel (split rows: several chunks, added here
+// in ascending order; long whole rows: one sum each); the group loads them into its accumulator itself, no producer
+// or MMA warp takes part.
+template <bool FROM_SUMS>
 __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, const float *__restrict__ Bs, int gidx,
                                  int tid)
 {
@@ -548,19 +557,59 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
     for (int64_t t = blockIdx.x; t < p.n_items; t += gridDim.x, ++it) {
         if ((int)(it % kGroups) != gidx) continue;
         int64_t u, beg, end, slot;
-        item_range<kModeRows>(p, t, u, beg, end, slot);
-        const uint32_t aph = (uint32_t)((it / kGroups) & 1);
-        // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
-        if (tid == 0) {
-            gs.stop = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
-            gs.bad = 0;
+        float b;
+        if constexpr (FROM_SUMS) {
+            int64_t c0, c1;      // the row's sums: slots c0 .. c1 - 1 of the workspace
+            if (t < p.n_split_rows) {
+                u = p.sv.order[p.split_begin + t];
+                c0 = p.sv.split_first[t];
+                c1 = p.sv.split_first[t + 1];
+            } else {
+                const int64_t j = t - p.n_split_rows;
+                u = p.sv.order[p.long_end - 1 - j];
+                c0 = p.n_chunks + j;
+                c1 = c0 + 1;
+            }
+            if (tid == 0) { gs.stop = 0; gs.bad = 0; }
+            // my row of the lower triangle (16-column blocks up to my own) and my component of the right-hand side
+            constexpr int64_t kSum = (int64_t)D * D + D;
+            const float *base = p.partials + c0 * kSum;
+            b = 0.f;
+            for (int64_t c = c0; c < c1; ++c) b += p.partials[c * kSum + D * D + i];
+#pragma unroll 1
+            for (int cb = 0; cb <= (wpos + 31) / 16; ++cb) {
+                float acc[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+                const float *src = base + (int64_t)i * D + 16 * cb;
+                for (int64_t c = c0; c < c1; ++c, src += kSum) {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(src + 4 * q4);
+                        acc[4 * q4] += v.x; acc[4 * q4 + 1] += v.y; acc[4 * q4 + 2] += v.z; acc[4 * q4 + 3] += v.w;
+                    }
+                }
+                tmem_st16(trow + 16 * cb, acc);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            group128_sync(bar_id);
+            tc_fence_after();
+        } else {
+            item_range<kModeRows>(p, t, u, beg, end, slot);
+            const uint32_t aph = (uint32_t)((it / kGroups) & 1);
+            // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
+            if (tid == 0) {
+                gs.stop = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
+                gs.bad = 0;
+            }
+            group128_sync(bar_id);
+            if (gs.stop) break;
+            tc_fence_after();
+            // right-hand side: the four producer warps' partial sums, in order
+            const float *bp = &sm.bpart[it % kBRing][0][i];
+            b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
         }
-        group128_sync(bar_id);
-        if (gs.stop) break;
-        tc_fence_after();
-        // right-hand side: the four producer warps' partial sums, in order
-        const float *bp = &sm.bpart[it % kBRing][0][i];
-        float b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
         float lrow[16];          // my row of my diagonal block's factor (kept for the block inverse at the end)
         float my_dinv = 0.f;     // 1 / L[i][i]
 #pragma unroll
@@ -845,7 +894,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         // tensor memory is free again for the next item of this accumulator
         tc_fence_before();
         group128_sync(bar_id);
-        if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
+        if (!FROM_SUMS && tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
         const bool ok = gs.bad == 0;
         const float xo = ok ? x : 0.f;
         reinterpret_cast<__nv_bfloat16 *>(p.out.table)[u * D + i] = __float2bfloat16_rn(xo);
@@ -912,7 +961,7 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p, 
 
     if (warp < C::kMmaWarp) {
         const int gidx = warp / (C::kGroupThreads / 32);
-        if constexpr (MODE == kModeRows) solver_rows_tmem(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
+        if constexpr (MODE == kModeRows) solver_rows_tmem<false>(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
         else copyout_role<MODE>(p, sm, gidx, tid - gidx * C::kGroupThreads);
     } else if (warp == C::kMmaWarp) {
         mma_role<MODE>(p, sm, lane);
@@ -943,33 +992,39 @@ __global__ void k_zero_rows_bf16(const int32_t *__restrict__ rows, int64_t count
     }
 }
 
-// chunks of a split row added in ascending order, then factor / solve / store (one block of 256 per row)
-__global__ void __launch_bounds__(kThreads, 2) k_split_solve_umma(SideView sv, int64_t split_class_begin,
-                                                                  const float *__restrict__ partials,
-                                                                  const float *__restrict__ Bmat, RowOut out,
-                                                                  DevStatus *st)
+// Split rows and long whole rows: their sums come from the chunks kernel; four groups of 128 threads load them into
+// tensor memory (a split row's chunks added in ascending order) and factor / solve / store as in rows mode.
+__global__ void __launch_bounds__(4 * 128, 1) k_solve_sums(Params p)
 {
-    constexpr int LDA = Geo<D>::LDA;
-    extern __shared__ __align__(16) unsigned char smem_raw2[];
-    GroupSmem &gs = *reinterpret_cast<GroupSmem *>(smem_raw2);
-    __shared__ int s_bad;
-    const int tid = threadIdx.x;
-    const int64_t j = blockIdx.x;
-    const int64_t u = sv.order[split_class_begin + j];
-    const int64_t c0 = sv.split_first[j], c1 = sv.split_first[j + 1];
-    // lower triangle and right-hand side: element e of this thread summed over the chunks in order
-    for (int e = tid; e < D * D + D; e += kThreads) {
-        const int r = e >> 7, cidx = e & (D - 1);
-        if (e < D * D && cidx > r) continue;
-        float s = 0.f;
-        for (int64_t c = c0; c < c1; ++c) s += partials[c * (int64_t)(D * D + D) + e];
-        if (e < D * D) gs.As[r * LDA + cidx] = s + Bmat[e];
-        else gs.As[D * LDA + (e - D * D)] = s;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *aligned = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    Smem &sm = *reinterpret_cast<Smem *>(aligned);
+    float *Bs = reinterpret_cast<float *>(aligned + sizeof(Smem));
+    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(Smem) + sizeof(float) * D * kLdB);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) sm.abort_flag = 0;
+    for (int e = tid; e < D * D; e += blockDim.x) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
+    for (int g = 0; g < kMaxGroups; ++g) {
+        if (tid == 0) mbar_init(&rgs[g].trail_bar, 1);
+        for (int k = tid; k < 3 * D * 32 / 16; k += blockDim.x) st_shared_zero16(smem_u32(&rgs[g].pop[0][0]) + k * 16);
     }
+    if (tid == 0) mbar_fence_init();
+    fence_proxy_async();
+    if (warp == 0) {
+        tmem_alloc(&sm.tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
     __syncthreads();
-    float xq[D / 32];
-    const bool ok = cholesky_solve<D>(gs.As, gs.Pt, gs.dinv, xq, tid, 0, &s_bad);
-    if (tid < 32) store_solution<D, __nv_bfloat16>(xq, ok, u, out, st);
+    tc_fence_after();
+    solver_rows_tmem<true>(p, sm, rgs[warp >> 2], Bs, warp >> 2, tid & 127);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(sm.tmem_base, kTmemCols);
+    }
+    if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, (long long)sm.abort_flag * 1000000 + blockIdx.x);
 }
 
 template <int MODE> size_t smem_bytes()
@@ -1061,28 +1116,40 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
     p.out = out;
     p.st = st;
     cudaError_t e;
-    if (n_chunks > 0) {
-        p.n_items = n_chunks;
-        e = launch_mode<kModeChunks>(p, (int)(n_chunks < sms ? n_chunks : sms), s);
+    // Rows of more than 1024 observations (as many classes from the top as the workspace budget allows) do not go
+    // through the rows kernel, whose gather holds 64 KB in flight per SM: the chunks kernel (192 KB in flight)
+    // forms their sums, one per row, behind the sums of the split rows' chunks.
+    const int c_long = long_class_begin(offs);
+    const int64_t n_long = offs[kNClasses - 1] - offs[c_long];
+    if (n_chunks + n_long > 0) {
+        p.n_chunks = n_chunks;
+        p.long_end = offs[kNClasses - 1];
+        p.n_items = n_chunks + n_long;
+        e = launch_mode<kModeChunks>(p, (int)(p.n_items < sms ? p.n_items : sms), s);
         ++*launches;
         if (e != cudaSuccess) return e;
-        const size_t smem = sizeof(GroupSmem);
-        e = cudaFuncSetAttribute(k_split_solve_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        p.split_begin = offs[kNClasses - 1];
+        p.n_split_rows = n_split_rows;
+        p.n_items = n_split_rows + n_long;
+        const size_t smem = smem_bytes<kModeRows>();
+        e = cudaFuncSetAttribute(k_solve_sums, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_split_solve_umma<<<(unsigned)n_split_rows, kThreads, smem, s>>>(sv, offs[kNClasses - 1], split_partials, Bmat, out, st);
+        k_solve_sums<<<(int)(p.n_items < sms ? p.n_items : sms), 4 * 128, smem, s>>>(p);
         ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
     }
-    const int64_t n_whole = offs[kNClasses - 1] - offs[1];
+    const int64_t n_whole = offs[c_long] - offs[1];
     if (dual_ws && offs[3] > offs[1]) {
         // rows with 1 .. 32 observations (classes 1 and 2): dual form, if the flag (set on the device) allows it
         e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], offs[3] - offs[2], X, dual_ws, out, st, s, launches);
         if (e != cudaSuccess) return e;
         p.dual_flag = dual_flag_ptr(dual_ws);
-        p.n_items_primal = offs[kNClasses - 1] - offs[3];
+        p.n_items_primal = offs[c_long] - offs[3];
     }
     if (n_whole > 0) {
         p.n_items = n_whole;
-        p.last_item = offs[kNClasses - 1] - 1;
+        p.last_item = offs[c_long] - 1;
         if (main_begin) cudaEventRecord(main_begin, s);
         e = launch_mode<kModeRows>(p, (int)(n_whole < sms ? n_whole : sms), s);
         if (main_end) cudaEventRecord(main_end, s);

@@ -68,7 +68,8 @@ def powerlaw(name, n, nnz, s, cap, d, lam, alpha, storage, law, seed, split=0, v
 
 def small_suite():
     """Problems the oracle finishes in seconds; together they span every degree class, both storage types,
-    every supported d, labelled entries, empty rows, alpha0 = 0 and rows longer than the split threshold."""
+    every supported d, labelled entries (on both kernel paths), empty rows, alpha0 = 0 and rows longer than the split
+    threshold."""
     return [
         tiny,
         lambda: powerlaw("zipf_d64_f32", 6000, 180000, 1.2, 3000, 64, 0.05, 0.001, "f32", "zipf", 11, empty_rows=5),
@@ -80,4 +81,10 @@ def small_suite():
         lambda: powerlaw("alpha0_d16_bf16", 1500, 30000, 1.0, 600, 16, 0.1, 0.0, "bf16", "uniform", 15, n_cols=1300),
         lambda: powerlaw("default_split_d64_bf16", 1200, 120000, 1.3, 9500, 64, 0.02, 0.001, "bf16", "uniform", 16,
                          n_cols=20000),
+        # labelled entries on the tensor-core path: whole rows of more than 1024 observations (their sums come from the
+        # chunks kernel), and the same matrix with rows split at 512
+        lambda: powerlaw("long_labels_d128_bf16", 1500, 120000, 1.0, 3000, 128, 0.02, 0.001, "bf16", "zipf", 17,
+                         values=True, n_cols=8000),
+        lambda: powerlaw("split_labels_d128_bf16", 1500, 120000, 1.0, 3000, 128, 0.02, 0.001, "bf16", "zipf", 17,
+                         split=512, values=True, n_cols=8000),
     ]

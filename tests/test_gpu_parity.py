@@ -32,7 +32,7 @@ def row_rel(x, ref):
 
 SUITE = problems.small_suite()
 IDS = ["tiny", "zipf_d64_f32", "local_d128_bf16", "split_d128_bf16", "split_d32_f32_labels", "alpha0_d16_bf16",
-       "default_split_d64_bf16"]
+       "default_split_d64_bf16", "long_labels_d128_bf16", "split_labels_d128_bf16"]
 
 
 @pytest.fixture(scope="module", params=list(range(len(SUITE))), ids=IDS)
