@@ -317,6 +317,9 @@ def run_ours(args, w):
     dual_rows = statistics.mean(half_ms["dual_rows"])
     rows_whole = statistics.mean(n_whole) - dual_rows
     ent_whole -= 6.0 * dual_rows          # rows of 1 .. 32 entries, about 6 on average under the rank-size law (approx.)
+    # whole rows of more than 1024 entries get their sums from the chunks kernel and their solve from k_solve_sums
+    rows_whole -= statistics.mean(st.long_rows)
+    ent_whole -= statistics.mean(st.long_entries)
     alu_main = rows_whole * (d ** 3 / 3.0 + 3.0 * d * d) + 2.0 * ent_whole * d
     bytes_main = ent_whole * (d * e + 4) + rows_whole * (d * e + 12)
     if t_bytes >= t_tensor + t_alu:
@@ -325,19 +328,22 @@ def run_ours(args, w):
         roof = {"bound": "alu", "achieved": alu_main / (main_ms * 1e-3) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     # DRAM traffic of that kernel: dram__bytes_read + dram__bytes_write of one ncu capture of the 2M-row `medium`
-    # case, per row and per side (columns side: 4.72 GB for 2.00M rows at a 91 % L2 hit rate; rows side, rows of
-    # more than 32 entries: 11.17 GB for 0.359M rows at 46 %), scaled by the rows each launch of this workload
+    # case, per row and per side (columns side: 4.44 GB for 2.00M rows at a 91 % L2 hit rate; rows side, rows of
+    # 33 .. 1024 entries: 5.00 GB for 0.372M rows at 56 %), scaled by the rows each launch of this workload
     # solves and averaged over the two launches of an epoch.  The window of +-1 % of the ids (hence the L2 reuse)
     # scales with the table, so this is an estimate, not a measurement at this size.
     if w["name"] in ("cfg3", "medium"):
-        primal_rows = [n_whole[0] - half_ms["dual_rows"][0], n_whole[1] - half_ms["dual_rows"][1]]
-        roof["traffic"] = 0.5 * (primal_rows[0] * 11.17e9 / 0.359e6 + primal_rows[1] * 4.72e9 / 2.0e6)
+        primal_rows = [n_whole[sd] - half_ms["dual_rows"][sd] - st.long_rows[sd] for sd in (0, 1)]
+        roof["traffic"] = 0.5 * (primal_rows[0] * 5.00e9 / 0.372e6 + primal_rows[1] * 4.44e9 / 2.0e6)
     else:
         roof["traffic"] = None
     roof.update({"kernel": "k_umma<0>: whole rows (gather, tcgen05 outer products, Cholesky in tensor memory, solve, store)",
                  "main_kernel_ms": main_ms, "rows_per_launch": rows_whole,
                  "rows_in_dual_form": {"rows": half_ms["dual_rows"][0], "cols": half_ms["dual_rows"][1],
                                        "note": "rows with at most 32 entries, solved by k_dual outside the dominant kernel"},
+                 "long_rows": {"rows": list(st.long_rows), "entries": list(st.long_entries),
+                               "note": "whole rows of more than 1024 entries: sums by the chunks kernel, solve by "
+                                       "k_solve_sums, outside the dominant kernel"},
                  "peak_source": f"HBM and bf16 {peaks['source']} (sustained bf16); FP32 FMA measured in this run",
                  "half_epoch_ms": {"rows": half_ms["rows"][0], "cols": half_ms["cols"][0],
                                    "gramian": statistics.mean(half_ms["gramian"]), "row_kernels": rows_ms},

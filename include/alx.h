@@ -89,6 +89,9 @@ typedef struct alx_stats {
     double ms_main_kernel;                   /* tensor path: device time of the whole-rows kernel of the LAST half-epoch, else 0 */
     int64_t dual_rows;                       /* rows the LAST half-epoch solved in the dual form of Eq. 4 (0: none, or the
                                                 form stepped aside because alpha0 G + lambda I was ill conditioned) */
+    int64_t long_rows[2];                    /* [side], tensor-core kernels only: whole rows of more than 1024 entries
+                                                whose sums the chunks kernel forms (as it does for the split rows) */
+    int64_t long_entries[2];                 /* [side]: the entries those rows hold */
 } alx_stats;
 
 /* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.

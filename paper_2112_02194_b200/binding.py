@@ -39,7 +39,8 @@ class alx_stats(Structure):
     _fields_ = [("nnz", c_int64), ("rows_in_class", (c_int64 * ALX_N_CLASSES) * 2), ("n_chunks", c_int64 * 2),
                 ("not_spd", c_int64), ("ms_gramian", c_double), ("ms_rows", c_double),
                 ("ms_half_epoch", c_double), ("kernel_launches", c_int64), ("workspace_bytes", c_int64),
-                ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double), ("dual_rows", c_int64)]
+                ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double), ("dual_rows", c_int64),
+                ("long_rows", c_int64 * 2), ("long_entries", c_int64 * 2)]
 
 
 EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_set_embedding_rows",

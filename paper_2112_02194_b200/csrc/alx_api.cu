@@ -415,9 +415,21 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
 
     const int d = c->opt.d;
     int64_t sums[2] = {c->n_chunks[0], c->n_chunks[1]};
-    if (tensor_path(c))      // one more sum per long whole row
-        for (int s = 0; s < 2; ++s)
-            sums[s] += c->class_offs[s][kNClasses - 1] - c->class_offs[s][long_class_begin(c->class_offs[s])];
+    for (int s = 0; s < 2; ++s) c->stats.long_rows[s] = c->stats.long_entries[s] = 0;
+    if (tensor_path(c)) {    // one more sum per long whole row
+        int64_t *total = nullptr;
+        ALX_ALLOC(c, total, 2);
+        for (int s = 0; s < 2; ++s) {
+            const int64_t first = c->class_offs[s][long_class_begin(c->class_offs[s])];
+            const int64_t n_long = c->class_offs[s][kNClasses - 1] - first;
+            sums[s] += n_long;
+            c->stats.long_rows[s] = n_long;
+            ALX_CUDA(c, launch_sum_row_lengths(c->ptr[s], c->order[s] + first, n_long, total + s, c->stream, &c->launches));
+        }
+        ALX_CUDA(c, cudaMemcpyAsync(c->stats.long_entries, total, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
+        ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        dev_free(c, total);
+    }
     const int64_t max_chunks = sums[0] > sums[1] ? sums[0] : sums[1];
     if (max_chunks > 0) ALX_ALLOC(c, c->split_partials, max_chunks * (int64_t)(d * d + d));
     ALX_ALLOC(c, c->loss_partials_buf, loss_partials(nnz));

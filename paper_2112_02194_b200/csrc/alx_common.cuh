@@ -90,6 +90,8 @@ int64_t scan_scratch_elems(int64_t n);
 cudaError_t launch_validate(const int64_t *rowptr, const int32_t *colidx, int64_t n_rows, int64_t n_cols,
                             int64_t nnz, DevStatus *st, cudaStream_t s, int64_t *launches);
 cudaError_t launch_degrees(const int64_t *ptr, int64_t n, int32_t *deg, cudaStream_t s, int64_t *launches);
+cudaError_t launch_sum_row_lengths(const int64_t *ptr, const int32_t *rows, int64_t count, int64_t *out, cudaStream_t s,
+                                   int64_t *launches);
 cudaError_t launch_count_cols(const int32_t *colidx, int64_t nnz, int32_t *counts, cudaStream_t s, int64_t *launches);
 cudaError_t launch_fill_transpose(const int64_t *rowptr, const int32_t *colidx, int64_t n_rows, int64_t nnz,
                                   const int64_t *colptr, int32_t *cursor, int32_t *rowidx, cudaStream_t s,

@@ -391,6 +391,33 @@ cudaError_t launch_validate(const int64_t *rowptr, const int32_t *colidx, int64_
     return cudaGetLastError();
 }
 
+// total length of the listed rows (one block; a few ten thousand rows at most)
+__global__ void k_sum_row_lengths(const int64_t *__restrict__ ptr, const int32_t *__restrict__ rows, int64_t count,
+                                  int64_t *__restrict__ out)
+{
+    __shared__ long long part[256];
+    long long s = 0;
+    for (int64_t k = threadIdx.x; k < count; k += 256) {
+        const int32_t u = rows[k];
+        s += ptr[u + 1] - ptr[u];
+    }
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int h = 128; h > 0; h >>= 1) {
+        if ((int)threadIdx.x < h) part[threadIdx.x] += part[threadIdx.x + h];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = part[0];
+}
+
+cudaError_t launch_sum_row_lengths(const int64_t *ptr, const int32_t *rows, int64_t count, int64_t *out, cudaStream_t s,
+                                   int64_t *launches)
+{
+    k_sum_row_lengths<<<1, 256, 0, s>>>(ptr, rows, count, out);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_degrees(const int64_t *ptr, int64_t n, int32_t *deg, cudaStream_t s, int64_t *launches)
 {
     k_degrees<<<grid_for(n, 256), 256, 0, s>>>(ptr, n, deg);
