@@ -357,7 +357,7 @@ __device__ void dual_mma(const DualParams &p, DualSmem &sm, int lane)
     for (int64_t t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ++it) {
         const int slot = (int)(it % kSlots);
         const uint32_t ph = (uint32_t)((it / kSlots) & 1);
-        if (!mbar_wait_warp(&sm.full[slot], ph, &sm.abort_flag, 120)) break;
+        if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 120)) break;
         tc_fence_after();
         if (lane == 0) {
             const uint32_t hb = smem_u32(&sm.h[slot][0]);
@@ -390,7 +390,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
     for (int64_t t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ++it) {
         if ((int)(it % kSlots) != g) continue;
         const uint32_t ph = (uint32_t)((it / kSlots) & 1);
-        if (tid == 0) sm.stop[g] = mbar_wait(&sm.acc_full[g], ph, &sm.abort_flag, 130) ? 0 : 1;
+        if (tid == 0) sm.stop[g] = mbar_wait_parked(&sm.acc_full[g], ph, &sm.abort_flag, 130) ? 0 : 1;
         asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
         if (sm.stop[g]) break;
         tc_fence_after();
