@@ -58,6 +58,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 // give-up protocol as mbar_wait.
 __device__ __forceinline__ bool mbar_wait_parked(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int site = 1)
 {
+    // a phase that has completed already costs no suspend / resume round trip (measured: about 350 cycles per stage
+    // for the MMA warp when the producers are ahead of it)
+    if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < (1u << 16); ++it) {
         uint32_t ok;
         asm volatile(
