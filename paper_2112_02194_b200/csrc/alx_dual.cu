@@ -321,7 +321,7 @@ template <int KP> __device__ void dual_producer(const DualParams &p, DualSmem &s
                 pending = -1;
             }
         }
-        if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 110)) break;
+        if (!mbar_wait_parked_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 110)) break;
         sm.y[slot][32 * pw + lane] = my_y;
         if (j == 0) { sm.row_u[slot][mr] = u; sm.row_k[slot][mr] = k; }
         const uint32_t tile = smem_u32(&sm.h[slot][0]);
