@@ -137,6 +137,23 @@ alx_status alx_half_epoch(alx_ctx *ctx, alx_side solved_side);
 alx_status alx_epoch(alx_ctx *ctx);
 
 /*
+ * The same work as alx_set_csr followed by alx_set_embeddings of both tables, from HOST arrays, with the
+ * copies overlapped: W (n_rows x d) and H (n_cols x d), row-major, elements of the context's STORAGE
+ * type, follow S over the bus on a second stream while the integer work of alx_set_csr runs.  The
+ * overlap needs page-locked host memory (pageable memory works, without overlap).  The arrays are not
+ * referenced after the call returns.  Synchronises.  Errors as alx_set_csr.
+ */
+alx_status alx_load_host(alx_ctx *ctx, const int64_t *rowptr, const int32_t *colidx, const float *values,
+                         int64_t nnz, const void *W, const void *H);
+
+/*
+ * The same work as alx_epoch followed by alx_get_embeddings of both whole tables into HOST arrays of the
+ * storage type (W_dst: n_rows x d, H_dst: n_cols x d): the new W is read back on a second stream while
+ * the column pass, which only reads it, runs.  Page-locked destinations overlap.  Synchronises.
+ */
+alx_status alx_epoch_to_host(alx_ctx *ctx, void *W_dst, void *H_dst);
+
+/*
  * As alx_half_epoch, and additionally returns, for the k listed rows of the solved side, the
  * float32 solution BEFORE it is rounded to the storage type (x_out: k x d floats, host memory).
  * Used to check the residual |A x - b| / |b| of the solver itself.  Synchronises.

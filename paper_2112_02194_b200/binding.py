@@ -44,7 +44,7 @@ class alx_stats(Structure):
 
 
 EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_set_embedding_rows",
-           "alx_half_epoch",
+           "alx_half_epoch", "alx_load_host", "alx_epoch_to_host",
            "alx_epoch", "alx_half_epoch_capture", "alx_loss", "alx_get_embeddings", "alx_get_gramian",
            "alx_gramian", "alx_fp32_peak_tflops", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
            "alx_last_error", "alx_version", "alx_gramian_noalloc", "alx_gramian_noalloc_max_rows",
@@ -71,6 +71,8 @@ def load_library() -> ctypes.CDLL:
     lib.alx_set_embedding_rows.argtypes = [P, c_int, c_int64, c_int64, P, c_int, c_int]
     lib.alx_half_epoch.argtypes = [P, c_int]
     lib.alx_epoch.argtypes = [P]
+    lib.alx_load_host.argtypes = [P, P, P, P, c_int64, P, P]
+    lib.alx_epoch_to_host.argtypes = [P, P, P]
     lib.alx_half_epoch_capture.argtypes = [P, c_int, P, c_int64, P]
     lib.alx_loss.argtypes = [P, POINTER(c_double), POINTER(c_double)]
     lib.alx_get_embeddings.argtypes = [P, c_int, P, c_int, c_int64, c_int64, c_int]
@@ -231,6 +233,27 @@ class Alx:
 
     def epoch(self):
         self._check(self.lib.alx_epoch(self.ctx))
+
+    def load_host(self, rowptr, colidx, values, W, H):
+        """set_csr + set_embeddings of both tables from host numpy arrays (tables in the storage type: float32, or
+        uint16 bf16 bit patterns), with the table uploads overlapped with the set-up kernels."""
+        import numpy as np
+        rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+        colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+        vals = None if values is None else np.ascontiguousarray(values, dtype=np.float32)
+        want = np.uint16 if self.storage == "bf16" else np.float32
+        assert W.dtype == want and H.dtype == want and W.flags.c_contiguous and H.flags.c_contiguous
+        self._check(self.lib.alx_load_host(self.ctx, rowptr.ctypes.data, colidx.ctypes.data,
+                                           None if vals is None else vals.ctypes.data, colidx.size,
+                                           W.ctypes.data, H.ctypes.data))
+
+    def epoch_to_host(self, W_out, H_out):
+        """epoch + download of both tables into host numpy arrays of the storage type; W is read back during the
+        column pass."""
+        import numpy as np
+        want = np.uint16 if self.storage == "bf16" else np.float32
+        assert W_out.dtype == want and H_out.dtype == want and W_out.flags.c_contiguous and H_out.flags.c_contiguous
+        self._check(self.lib.alx_epoch_to_host(self.ctx, W_out.ctypes.data, H_out.ctypes.data))
 
     def half_epoch_capture(self, side, row_ids):
         ids = np.ascontiguousarray(row_ids, dtype=np.int64)

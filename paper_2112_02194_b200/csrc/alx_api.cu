@@ -50,6 +50,11 @@ struct alx_ctx {
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
 
+    // second stream for the host copies that alx_load_host / alx_epoch_to_host overlap with kernels
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copy_ev = nullptr;
+    const void *upload_after_csr[2] = {nullptr, nullptr};   // alx_load_host: tables to upload behind the upload of S
+
     cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     bool main_timed = false;
     alx_stats stats{};
@@ -345,6 +350,8 @@ alx_status alx_destroy(alx_ctx *c)
     DeviceGuard guard(c->device);
     cudaStreamSynchronize(c->stream);
     for (auto &e : c->ev) if (e) cudaEventDestroy(e);
+    if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaStreamDestroy(c->copy_stream); }
+    if (c->copy_ev) cudaEventDestroy(c->copy_ev);
     std::vector<std::pair<void *, size_t>> owned = c->owned;
     for (auto &p : owned) dev_free(c, p.first);
     delete c;
@@ -369,6 +376,15 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     if (values) {
         ALX_ALLOC(c, c->val[0], nz);
         if (nnz > 0) ALX_CUDA(c, cudaMemcpyAsync(c->val[0], values, sizeof(float) * nnz, kind, c->stream));
+    }
+    if (c->upload_after_csr[0] || c->upload_after_csr[1]) {
+        // alx_load_host: the tables follow S over the bus on the second stream, while the kernels below run
+        ALX_CUDA(c, cudaEventRecord(c->copy_ev, c->stream));
+        ALX_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->copy_ev, 0));
+        for (int sd = 0; sd < 2; ++sd)
+            if (c->upload_after_csr[sd])
+                ALX_CUDA(c, cudaMemcpyAsync(c->table[sd], c->upload_after_csr[sd], (size_t)c->n[sd] * c->opt.d * c->elem,
+                                            cudaMemcpyHostToDevice, c->copy_stream));
     }
     // validate before anything indexes with these arrays
     ALX_CUDA(c, launch_validate(c->ptr[0], c->idx[0], n_rows, n_cols, nnz, c->status, c->stream, &c->launches));
@@ -543,6 +559,61 @@ alx_status alx_epoch(alx_ctx *c)
     alx_status st = alx_half_epoch(c, ALX_ROWS);
     if (st != ALX_OK) return st;
     return alx_half_epoch(c, ALX_COLS);
+}
+
+namespace {
+alx_status ensure_copy_stream(alx_ctx *c)
+{
+    if (!c->copy_stream) ALX_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+    if (!c->copy_ev) ALX_CUDA(c, cudaEventCreateWithFlags(&c->copy_ev, cudaEventDisableTiming));
+    return ALX_OK;
+}
+}  // namespace
+
+alx_status alx_load_host(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx, const float *values, int64_t nnz,
+                         const void *W, const void *H)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!W || !H) return fail(c, ALX_ERR_INVALID_ARG, "null table");
+    DeviceGuard guard(c->device);
+    alx_status st = ensure_copy_stream(c);
+    if (st != ALX_OK) return st;
+    c->upload_after_csr[ALX_ROWS] = W;
+    c->upload_after_csr[ALX_COLS] = H;
+    st = alx_set_csr(c, rowptr, colidx, values, nnz, 0);
+    c->upload_after_csr[0] = c->upload_after_csr[1] = nullptr;
+    const cudaError_t e = cudaStreamSynchronize(c->copy_stream);     // whatever alx_set_csr returned, the copies have ended
+    if (st != ALX_OK) return st;
+    ALX_CUDA(c, e);
+    for (int sd = 0; sd < 2; ++sd) {
+        c->have_table[sd] = true;
+        c->have_gram[sd] = false;
+    }
+    return ALX_OK;
+}
+
+alx_status alx_epoch_to_host(alx_ctx *c, void *W_dst, void *H_dst)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (!W_dst || !H_dst) return fail(c, ALX_ERR_INVALID_ARG, "null destination");
+    DeviceGuard guard(c->device);
+    alx_status st = ensure_copy_stream(c);
+    if (st != ALX_OK) return st;
+    st = half_epoch_impl(c, ALX_ROWS, nullptr, nullptr);
+    if (st != ALX_OK) return st;
+    // the new W goes to the host on the second stream while the column pass (which only reads it) runs
+    ALX_CUDA(c, cudaEventRecord(c->copy_ev, c->stream));
+    ALX_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->copy_ev, 0));
+    ALX_CUDA(c, cudaMemcpyAsync(W_dst, c->table[ALX_ROWS], (size_t)c->n[ALX_ROWS] * c->opt.d * c->elem, cudaMemcpyDeviceToHost,
+                                c->copy_stream));
+    st = half_epoch_impl(c, ALX_COLS, nullptr, nullptr);
+    if (st == ALX_OK)
+        ALX_CUDA(c, cudaMemcpyAsync(H_dst, c->table[ALX_COLS], (size_t)c->n[ALX_COLS] * c->opt.d * c->elem,
+                                    cudaMemcpyDeviceToHost, c->stream));
+    const cudaError_t e = cudaStreamSynchronize(c->copy_stream);
+    if (st != ALX_OK) return st;
+    ALX_CUDA(c, e);
+    return check_device_status(c);
 }
 
 alx_status alx_half_epoch_capture(alx_ctx *c, alx_side side, const int64_t *row_ids, int64_t k, float *x_out)

@@ -186,6 +186,41 @@ def test_device_pointers_and_ranged_reads():
     a.destroy(); b.destroy()
 
 
+@pytest.mark.parametrize("which", [1, 2, 7])
+def test_overlapped_host_calls_match_the_separate_calls(which):
+    """alx_load_host + alx_epoch_to_host (copies overlapped with kernels on a second stream) give, bit for bit, what
+    alx_set_csr + alx_set_embeddings x2 + alx_epoch + alx_get_embeddings x2 give; page-locked buffers, labelled or not."""
+    import torch
+    p = SUITE[which]()
+    dt = "bf16" if p.storage == "bf16" else "f32"
+    a = make_ctx(p)
+    a.epoch()
+    W_ref, H_ref = a.get_embeddings(ROWS, dtype=dt), a.get_embeddings(COLS, dtype=dt)
+    a.destroy()
+    from paper_2112_02194_b200 import Alx
+
+    def pinned(x):
+        t = torch.empty(x.shape, dtype=torch.int16 if x.dtype == np.uint16 else torch.float32, pin_memory=True)
+        arr = t.numpy().view(x.dtype)
+        arr[...] = x
+        return t, arr
+    b = Alx(p.n_rows, p.n_cols, p.d, p.lam, p.alpha, storage=p.storage, split=p.split)
+    keepW, W0 = pinned(p.W0)
+    keepH, H0 = pinned(p.H0)
+    keepWo, W_out = pinned(np.zeros_like(p.W0))
+    keepHo, H_out = pinned(np.zeros_like(p.H0))
+    b.load_host(p.rowptr, p.colidx, p.values, W0, H0)
+    b.epoch_to_host(W_out, H_out)
+    np.testing.assert_array_equal(W_out, W_ref)
+    np.testing.assert_array_equal(H_out, H_ref)
+    # and once more on the same context (the second stream and its event are reused)
+    b.load_host(p.rowptr, p.colidx, p.values, W0, H0)
+    b.epoch_to_host(W_out, H_out)
+    np.testing.assert_array_equal(W_out, W_ref)
+    np.testing.assert_array_equal(H_out, H_ref)
+    b.destroy()
+
+
 def test_error_paths_return_status_codes():
     from paper_2112_02194_b200 import Alx, AlxError
     with pytest.raises(AlxError) as e:
