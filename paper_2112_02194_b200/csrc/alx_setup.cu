@@ -197,6 +197,38 @@ __global__ void k_sort_small(const int64_t *__restrict__ colptr, int32_t *__rest
     if (lane < len) rowidx[beg + rank] = v;
 }
 
+// columns of 33 .. 128 entries (classes 3 and 4): one warp each, four keys per lane, rank by counting over shuffles
+// (about 1200 warp instructions per column; a block-wide network with a barrier per stage took ten times as long)
+__global__ void k_sort_warp128(const int64_t *__restrict__ colptr, int32_t *__restrict__ rowidx,
+                               const int32_t *__restrict__ cols, int64_t n_cols_in_class)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_cols_in_class) return;
+    const int32_t c = cols[w];
+    const int64_t beg = colptr[c];
+    const int len = (int)(colptr[c + 1] - beg);
+    int32_t v[4];
+    int rank[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) v[q] = (32 * q + lane < len) ? rowidx[beg + 32 * q + lane] : 0x7FFFFFFF;
+#pragma unroll
+    for (int q2 = 0; q2 < 4; ++q2) {
+        if (32 * q2 < len) {            // warp-uniform
+#pragma unroll 8
+            for (int o = 0; o < 32; ++o) {
+                const int32_t other = __shfl_sync(0xFFFFFFFFu, v[q2], o);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) rank[q] += (other < v[q]) ? 1 : 0;
+            }
+        }
+    }
+    // every lane has read its keys before any lane writes (the shuffles above need all lanes); ids are distinct
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        if (32 * q + lane < len) rowidx[beg + rank[q]] = v[q];
+}
+
 constexpr int kSortMediumMax = 4096;
 
 __global__ void __launch_bounds__(256) k_sort_medium(const int64_t *__restrict__ colptr,
@@ -448,17 +480,22 @@ cudaError_t launch_fill_transpose(const int64_t *rowptr, const int32_t *colidx, 
 cudaError_t launch_sort_segments(const int64_t *colptr, int32_t *rowidx, const int32_t *order,
                                  const int64_t *offs, cudaStream_t s, int64_t *launches)
 {
-    // classes 1-2: at most 32 entries; 3-9: at most 4096; 10-11: anything longer (class 11 starts at
+    // classes 1-2: at most 32 entries; 3-4: at most 128; 5-9: at most 4096; 10-11: anything longer (class 11 starts at
     // split + 1, which a small split can put below 4096: the global-memory network handles any length)
     const int64_t n_small = offs[3] - offs[1];
-    const int64_t n_medium = offs[10] - offs[3];
+    const int64_t n_warp = offs[5] - offs[3];        // classes 3 and 4: 33 .. 128 entries
+    const int64_t n_medium = offs[10] - offs[5];
     const int64_t n_large = offs[12] - offs[10];
     if (n_small > 0) {
         k_sort_small<<<grid_for(n_small * 32, 256), 256, 0, s>>>(colptr, rowidx, order + offs[1], n_small);
         ++*launches;
     }
+    if (n_warp > 0) {
+        k_sort_warp128<<<grid_for(n_warp * 32, 256), 256, 0, s>>>(colptr, rowidx, order + offs[3], n_warp);
+        ++*launches;
+    }
     if (n_medium > 0) {
-        k_sort_medium<<<(unsigned)n_medium, 256, 0, s>>>(colptr, rowidx, order + offs[3]);
+        k_sort_medium<<<(unsigned)n_medium, 256, 0, s>>>(colptr, rowidx, order + offs[5]);
         ++*launches;
     }
     if (n_large > 0) {
