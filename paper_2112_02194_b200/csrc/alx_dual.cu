@@ -411,21 +411,52 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
 #pragma unroll 1
         for (int cf = 0; cf < D / 16; ++cf) {
             if (cf + 1 < D / 16) tmem_ld16_nowait(trow + 16 * (cf + 1), zn);      // lands while this chunk is used
+            if constexpr (KP == 16) {
 #pragma unroll
-            for (int jj = 0; jj < KP; ++jj) {
-                if (jj < kmax) {
-                    const int base = (cf >> 2) * kPanelBytes + (jj >> 3) * 1024 + (jj & 7) * 128;
-                    const int c0 = (cf & 3) * 2;
-                    const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + base + ((c0 ^ (jj & 7)) << 4));
-                    const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + base + (((c0 + 1) ^ (jj & 7)) << 4));
-                    const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-                    // packed FP32 FMAs: even features in .x, odd features in .y (a bfloat16 pair unpacks to exactly that)
-                    float2 acc = make_float2(s[jj], 0.f);
+                for (int jj = 0; jj < KP; jj += 2) {
+                    // two observations per trip and two partial sums each: four independent chains of packed FMAs (one
+                    // chain of eight per observation left the warp waiting on its own results); an odd kmax spends one
+                    // product on a padding row, which holds zeros
+                    if (jj < kmax) {
+                        float2 acc[2][2];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        acc = __ffma2_rn(make_float2(z[2 * e], z[2 * e + 1]),
-                                         make_float2(__uint_as_float(hw[e] << 16), __uint_as_float(hw[e] & 0xFFFF0000u)), acc);
-                    s[jj] = acc.x + acc.y;
+                        for (int t = 0; t < 2; ++t) {
+                            const int jt = jj + t;
+                            const int base = (cf >> 2) * kPanelBytes + (jt >> 3) * 1024 + (jt & 7) * 128;
+                            const int c0 = (cf & 3) * 2;
+                            const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + base + ((c0 ^ (jt & 7)) << 4));
+                            const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + base + (((c0 + 1) ^ (jt & 7)) << 4));
+                            const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+                            // packed FP32 FMAs: even features in .x, odd features in .y (a bfloat16 pair unpacks to exactly that)
+                            acc[t][0] = make_float2(s[jt], 0.f);
+                            acc[t][1] = make_float2(0.f, 0.f);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                acc[t][e & 1] = __ffma2_rn(make_float2(z[2 * e], z[2 * e + 1]),
+                                                           make_float2(__uint_as_float(hw[e] << 16), __uint_as_float(hw[e] & 0xFFFF0000u)),
+                                                           acc[t][e & 1]);
+                        }
+#pragma unroll
+                        for (int t = 0; t < 2; ++t) s[jj + t] = (acc[t][0].x + acc[t][1].x) + (acc[t][0].y + acc[t][1].y);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int jj = 0; jj < KP; ++jj) {
+                    if (jj < kmax) {
+                        const int base = (cf >> 2) * kPanelBytes + (jj >> 3) * 1024 + (jj & 7) * 128;
+                        const int c0 = (cf & 3) * 2;
+                        const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + base + ((c0 ^ (jj & 7)) << 4));
+                        const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + base + (((c0 + 1) ^ (jj & 7)) << 4));
+                        const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+                        // packed FP32 FMAs: even features in .x, odd features in .y (a bfloat16 pair unpacks to exactly that)
+                        float2 acc = make_float2(s[jj], 0.f);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            acc = __ffma2_rn(make_float2(z[2 * e], z[2 * e + 1]),
+                                             make_float2(__uint_as_float(hw[e] << 16), __uint_as_float(hw[e] & 0xFFFF0000u)), acc);
+                        s[jj] = acc.x + acc.y;
+                    }
                 }
             }
             if (cf + 1 < D / 16) {
