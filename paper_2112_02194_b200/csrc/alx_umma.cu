@@ -465,11 +465,12 @@ __device__ void copyout_role(const Params &p, SmemT<MODE> &sm, int gidx, int tid
 // ---------------------------------------------------------------------------------------------------------
 // Rows mode: factor and solve in place in tensor memory.  128 threads, thread i = row i = tensor-memory lane i.
 // Blocked right-looking Cholesky, 16 columns per step:
-//   (1) every warp waits for the previous step's tensor-core update on its own, every live row reads its 16 panel
-//       values (adding alpha0 G + lambda I); the warp that holds the diagonal block factors it with shuffles, two
-//       pivots per round, b carried along as a 17th column; the rows after the block in the same warp get their
-//       forward substitution in the same rounds;
-//   (2) the other rows after the block do their forward substitution against the block (from shared memory) and
+//   (1) the warp that holds the diagonal block waits for the previous step's tensor-core update, reads its 16 panel
+//       values (adding alpha0 G + lambda I) and factors the block with shuffles, two pivots per round, b carried
+//       along as a 17th column; the rows after the block in the same warp get their forward substitution in the
+//       same rounds;
+//   (2) after the group's barrier the other live rows read their panel values, those after the block do their
+//       forward substitution against the block (from shared memory) and
 //       fold the block's part of L^-1 b into their b; every row after the block publishes its panel row as three
 //       bfloat16 parts in the operand tiles and writes it back to tensor memory (back substitution reads it);
 //   (3) trailing update A22 -= P P^T on the tensor core, in place in tensor memory: six tcgen05.mma
@@ -789,7 +790,8 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             group128_sync(bar_id);
             // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
             // blocks of 32 rows further on (cyclically), which never holds the next diagonal block.  It
-            // issues the update and waits for it (a tcgen05.mma takes the issuing thread about 50 cycles).
+            // issues the update and commits it to the group's mbarrier (a tcgen05.mma takes the issuing thread about
+            // 50 cycles); the next step's diagonal warp waits for it.
             const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
             uint64_t da[3];
             const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
