@@ -149,7 +149,11 @@ struct DualParams {
 struct __align__(1024) DualSmem {
     unsigned char binv[kBinvBytes];
     unsigned char h[kSlots][kTileBytes];     // after a tile's S matrices are formed: scratch of its solver group
-    uint64_t full[kSlots], empty[kSlots], acc_full[kSlots];
+    uint64_t full[kSlots], empty[kSlots], acc_full[kSlots], acc_empty[kSlots];
+    // KP = 16: scratch of a solver group's factorisation (exchange buffers and L), apart from the tile, so that the
+    // tile's slot is refilled while the group factors, solves and forms w (KP = 32 needs 18 KB per group, which does
+    // not fit: there the scratch takes the tile's place after the S products, and the slot is released at the end)
+    float scratch16[kSlots][8 * 64 + 8 * 256];
     uint32_t tmem_base;
     int abort_flag;
     int stop[kSlots];
@@ -358,6 +362,7 @@ __device__ void dual_mma(const DualParams &p, DualSmem &sm, int lane)
         const int slot = (int)(it % kSlots);
         const uint32_t ph = (uint32_t)((it / kSlots) & 1);
         if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 120)) break;
+        if (!mbar_wait_parked_warp(&sm.acc_empty[slot], ph ^ 1u, &sm.abort_flag, 121)) break;    // the slot's accumulator is free
         tc_fence_after();
         if (lane == 0) {
             const uint32_t hb = smem_u32(&sm.h[slot][0]);
@@ -474,9 +479,10 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         float my_inv = 0.f;
         // every thread of the group is past its reads of the tile: its memory now serves as scratch
         asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-        float *scratch = reinterpret_cast<float *>(&sm.h[g][0]);
+        if (KP == 16 && tid == 0) mbar_arrive(&sm.empty[g]);    // the tile, its labels and row ids are not read again
+        float *scratch = (KP == 16) ? &sm.scratch16[g][0] : reinterpret_cast<float *>(&sm.h[g][0]);
         float *xch = scratch + mr * (4 * KP);                   // per matrix row
-        float *Lrow = scratch + 8 * 128 + mr * (KP * KP);       // per matrix row: L, row-major
+        float *Lrow = scratch + (128 / KP) * (4 * KP) + mr * (KP * KP);       // per matrix row: L, row-major
         const bool ok = factor_rows<KP>(d, b, my_inv, lane, xch);
         // back substitution L^T t = z, column by column from the end
 #pragma unroll
@@ -526,7 +532,10 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         // the tile's shared memory and tensor-memory columns are free again
         tc_fence_before();
         asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-        if (tid == 0) mbar_arrive(&sm.empty[g]);
+        if (tid == 0) {
+            mbar_arrive(&sm.acc_empty[g]);
+            if (KP != 16) mbar_arrive(&sm.empty[g]);
+        }
     }
 }
 
@@ -543,6 +552,7 @@ template <int KP> __global__ void __launch_bounds__(kBlockThreads, 1) k_dual(Dua
             mbar_init(&sm.full[s], kProducerWarps);
             mbar_init(&sm.empty[s], 1);
             mbar_init(&sm.acc_full[s], 1);
+            mbar_init(&sm.acc_empty[s], 1);
             sm.stop[s] = 0;
         }
         sm.abort_flag = 0;
