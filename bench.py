@@ -328,13 +328,13 @@ def run_ours(args, w):
         roof = {"bound": "alu", "achieved": alu_main / (main_ms * 1e-3) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     # DRAM traffic of that kernel: dram__bytes_read + dram__bytes_write of one ncu capture of the 2M-row `medium`
-    # case, per row and per side (columns side: 4.44 GB for 2.00M rows at a 91 % L2 hit rate; rows side, rows of
-    # 33 .. 1024 entries: 5.00 GB for 0.372M rows at 56 %), scaled by the rows each launch of this workload
+    # case, per row and per side (columns side: 4.48 GB for 2.00M rows at a 91 % L2 hit rate; rows side, rows of
+    # 33 .. 1024 entries: 5.30 GB for 0.372M rows at 55 %), scaled by the rows each launch of this workload
     # solves and averaged over the two launches of an epoch.  The window of +-1 % of the ids (hence the L2 reuse)
     # scales with the table, so this is an estimate, not a measurement at this size.
     if w["name"] in ("cfg3", "medium"):
         primal_rows = [n_whole[sd] - half_ms["dual_rows"][sd] - st.long_rows[sd] for sd in (0, 1)]
-        roof["traffic"] = 0.5 * (primal_rows[0] * 5.00e9 / 0.372e6 + primal_rows[1] * 4.44e9 / 2.0e6)
+        roof["traffic"] = 0.5 * (primal_rows[0] * 5.30e9 / 0.372e6 + primal_rows[1] * 4.48e9 / 2.0e6)
     else:
         roof["traffic"] = None
     roof.update({"kernel": "k_umma<0>: whole rows (gather, tcgen05 outer products, Cholesky in tensor memory, solve, store)",
