@@ -43,14 +43,12 @@ constexpr int kStageRows = 32;
 template <int MODE> struct Ring {
     static constexpr int kRows = (MODE == 0) ? 32 : 64;   // gathered rows per stage
     static constexpr int kNStage = (MODE == 0) ? 8 : 12;
-    static constexpr int kLag = 6;                        // rows mode: stages of cp.async copies in flight per producer warp
     static constexpr int kHalfBytes = kRows * 128;        // one 64-feature half of a stage
     static constexpr int kStageHBytes = 2 * kHalfBytes;
     static constexpr int kStageYBytes = 2 * kRows * 16;   // label tile, two 8-column chunks
 };
-constexpr int kHalfBytes = kStageRows * 128;          // one 64-feature half of a stage
-constexpr int kStageHBytes = 2 * kHalfBytes;          // 8192
-constexpr int kStageYBytes = 2 * kStageRows * 16;     // 1024: label tile, two 8-column chunks
+constexpr int kHalfBytes = kStageRows * 128;          // rows mode: one 64-feature half of a stage
+constexpr int kRowsLag = 6;                           // rows mode: stages of cp.async copies in flight per producer warp
 constexpr int kProducerWarps = 4;
 constexpr int kTmemCols = 512;
 constexpr int kMaxGroups = 4;
@@ -196,7 +194,7 @@ template <int MODE> __device__ __forceinline__ void producer_signal(SmemT<MODE> 
 
 template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
 {
-    constexpr int kNStage = Ring<MODE>::kNStage, kLag = Ring<MODE>::kLag;
+    constexpr int kNStage = Ring<MODE>::kNStage, kLag = kRowsLag;
     int64_t g = 0, signalled = 0, it = 0;
     const int c = lane & 15;                 // 16-byte chunk of the 256-byte row
     const int half = c >> 3, cc = c & 7;
@@ -793,7 +791,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             // issues the update and commits it to the group's mbarrier (a tcgen05.mma takes the issuing thread about
             // 50 cycles); the next step's diagonal warp waits for it.
             const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
-            uint64_t da[3];
+            uint64_t da[3] = {0, 0, 0};
             const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
             // columns [c_lo, c_lo + n) of the matrix (= panel rows c_lo ..) -= P P^T restricted to them
             auto update = [&](int c_lo, int n) {
