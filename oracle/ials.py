@@ -46,6 +46,8 @@ def lib():
         _lib.alxo_degree_class.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32]
         _lib.alxo_chunks.restype = ctypes.c_int64
         _lib.alxo_half_step_rows.restype = ctypes.c_int
+        _lib.alxo_cg.restype = ctypes.c_int
+        _lib.alxo_half_step_rows_cg.restype = ctypes.c_int
     return _lib
 
 
@@ -110,6 +112,40 @@ def half_step(rowptr, colidx, values, X_fixed, alpha, lam, storage="f64", row_id
     if cnt[2]:
         raise FloatingPointError("oracle: normal matrix not positive definite")
     return (Y, Yraw) if return_raw else Y
+
+
+def cg(A, b, tol=1e-5, max_iter=64, return_iterates=False):
+    """Conjugate gradients on A x = b (Sec. 4.5; textbook form, x_0 = 0, stop at |r_k| <= tol |b| or max_iter)."""
+    A, b = _f64(A), _f64(b)
+    d = b.size
+    x = np.empty(d)
+    its = np.empty((max_iter, d)) if return_iterates else None
+    work = np.empty(3 * d)
+    k = lib().alxo_cg(ctypes.c_int(d), _p(A), _p(b), ctypes.c_double(tol), ctypes.c_int(max_iter), _p(x), _p(its),
+                      _p(work))
+    return (x, k, its[:k]) if return_iterates else (x, k)
+
+
+def half_step_cg(rowptr, colidx, values, X_fixed, alpha, lam, storage="f64", row_ids=None, G=None, tol=1e-5,
+                 max_iter=64):
+    """Eq. 4 with the solve by conjugate gradients; returns (rows rounded to storage, unrounded, steps per row)."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    vals = None if values is None else _f64(values)
+    X = _f64(X_fixed)
+    N, d = X.shape
+    n = rowptr.size - 1
+    G = _f64(gramian(X) if G is None else G)
+    ids = None if row_ids is None else np.ascontiguousarray(row_ids, dtype=np.int64)
+    count = n if ids is None else ids.size
+    Y = np.empty((count, d))
+    Yraw = np.empty((count, d))
+    iters = np.empty(count, dtype=np.int32)
+    lib().alxo_half_step_rows_cg(
+        ctypes.c_int64(n), ctypes.c_int64(N), ctypes.c_int(d), _p(rowptr), _p(colidx), _p(vals), _p(X), _p(G),
+        ctypes.c_double(alpha), ctypes.c_double(lam), ctypes.c_int(STORAGE[storage]), _p(ids), ctypes.c_int64(count),
+        ctypes.c_double(tol), ctypes.c_int(max_iter), _p(Y), _p(Yraw), _p(iters))
+    return Y, Yraw, iters
 
 
 def row_system(rowptr, colidx, values, X_fixed, G, alpha, lam, u):

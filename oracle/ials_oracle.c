@@ -29,8 +29,14 @@
  * closed forms (d = 1, single observation with and without the all-pairs term, orthogonal
  * fixed side), ridge regression for alpha = 0, gradient of Eq. 3 by explicit all-pairs
  * sums, monotone objective, permutation equivariance, operation counters.
- * The conjugate-gradient variant the paper uses for its results is not stated in enough
- * detail to reproduce (no iteration count or tolerance): not implemented here.
+ *   - alxo_cg / alxo_half_step_rows_cg : the conjugate-gradient solve of Sec. 4.5 (the solver the
+ *                           paper's results use).  The paper states no start vector, iteration count or
+ *                           tolerance; the reading taken here: the textbook method (Hestenes-Stiefel),
+ *                           start x = 0, stop as soon as |r_k| <= tol |b| or after max_iter steps.
+ *                           Pins: converges to the Cholesky answer, exact after k steps when A has k
+ *                           distinct eigenvalues, error decreasing in the A-norm, residuals mutually
+ *                           orthogonal.  The iterates themselves have nothing in the paper to be compared
+ *                           with: parity unpinned for the iterate sequence, pinned for the limit.
  */
 #include <math.h>
 #include <stdint.h>
@@ -38,6 +44,9 @@
 #include <string.h>
 
 enum { ALXO_F64 = 0, ALXO_F32 = 1, ALXO_BF16 = 2 };
+
+void alxo_row_system(int d, int64_t beg, int64_t end, const int32_t *colidx, const double *values,
+                     const double *X, const double *G, double alpha, double lambda, double *A, double *b);
 
 /* ---- storage rounding (Sec. 4.4: tables in bfloat16, solve in float32 or wider) ---- */
 
@@ -209,6 +218,72 @@ int alxo_half_step_rows(int64_t n, int64_t N, int d, const int64_t *rowptr, cons
         counters[2] += tot_fail;
     }
     return tot_fail ? 1 : 0;
+}
+
+/* ---- conjugate gradients (Sec. 4.5), textbook form, fp64, x_0 = 0 ----
+ * Solves A x = b for a symmetric positive definite d x d matrix.  Stops at the first k with |r_k| <= tol |b|
+ * (r_k by the recurrence) or after max_iter steps; returns the number of steps taken.  When `iterates` is not
+ * NULL it receives x_1 .. x_k, d values each (room for max_iter of them).  work holds 3 d doubles.
+ */
+int alxo_cg(int d, const double *A, const double *b, double tol, int max_iter, double *x, double *iterates,
+            double *work)
+{
+    double *r = work, *p = work + d, *q = work + 2 * d;
+    double bb = 0.0;
+    for (int a = 0; a < d; ++a) { x[a] = 0.0; r[a] = b[a]; p[a] = b[a]; bb += b[a] * b[a]; }
+    double rr = bb;
+    if (bb == 0.0) return 0;
+    int k = 0;
+    while (k < max_iter && rr > tol * tol * bb) {
+        double pq = 0.0;
+        for (int a = 0; a < d; ++a) {                                  /* q <- A p */
+            double t = 0.0;
+            for (int c = 0; c < d; ++c) t += A[a * d + c] * p[c];
+            q[a] = t;
+            pq += p[a] * t;
+        }
+        const double step = rr / pq;
+        double rr_new = 0.0;
+        for (int a = 0; a < d; ++a) {
+            x[a] += step * p[a];
+            r[a] -= step * q[a];
+            rr_new += r[a] * r[a];
+        }
+        const double beta = rr_new / rr;
+        for (int a = 0; a < d; ++a) p[a] = r[a] + beta * p[a];
+        rr = rr_new;
+        if (iterates) memcpy(iterates + (size_t)k * d, x, sizeof(double) * (size_t)d);
+        ++k;
+    }
+    return k;
+}
+
+/* alxo_half_step_rows with the solve of Alg. 1 line 10 done by alxo_cg; iters_out[k] (may be NULL) = steps of row k */
+int alxo_half_step_rows_cg(int64_t n, int64_t N, int d, const int64_t *rowptr, const int32_t *colidx,
+                           const double *values, const double *X, const double *G, double alpha,
+                           double lambda, int storage, const int64_t *row_ids, int64_t n_ids, double tol,
+                           int max_iter, double *Y_out, double *Y_raw, int32_t *iters_out)
+{
+    (void)N;
+    int64_t count = row_ids ? n_ids : n;
+#pragma omp parallel
+    {
+        double *A = (double *)malloc(sizeof(double) * ((size_t)d * d + 5 * (size_t)d));
+        double *b = A + (size_t)d * d, *w = b + d, *work = w + d;
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t k = 0; k < count; ++k) {
+            int64_t u = row_ids ? row_ids[k] : k;
+            alxo_row_system(d, rowptr[u], rowptr[u + 1], colidx, values, X, G, alpha, lambda, A, b);
+            int it = alxo_cg(d, A, b, tol, max_iter, w, NULL, work);
+            if (iters_out) iters_out[k] = it;
+            for (int a = 0; a < d; ++a) {
+                if (Y_raw) Y_raw[k * d + a] = w[a];
+                Y_out[k * d + a] = alxo_round_storage(w[a], storage);
+            }
+        }
+        free(A);
+    }
+    return 0;
 }
 
 /* normal matrix and right-hand side of one row, for residual checks of someone else's solution */

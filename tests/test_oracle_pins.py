@@ -366,3 +366,86 @@ def test_bucket_and_chunk_invariants():
         assert np.all(d[:, 0] == u) and d[0, 1] == rowptr[u] and d[-1, 2] == rowptr[u + 1]
         assert np.all(d[1:, 1] == d[:-1, 2]) and np.all(d[:-1, 2] - d[:-1, 1] == split)
         assert 0 < d[-1, 2] - d[-1, 1] <= split
+
+
+# ---- streamed Gramian (used by the full-size parity tests) ---------------------------------------------
+
+def test_gramian_stream_equals_gramian_on_a_ragged_table():
+    rng = np.random.default_rng(5)
+    X = rng.normal(0, 0.3, (1003, 7))
+    calls = []
+
+    def block(r0, cnt):
+        calls.append((r0, cnt))
+        return X[r0:r0 + cnt]
+    G = ials.gramian_stream(block, 1003, 7, block_rows=250)
+    assert calls == [(0, 250), (250, 250), (500, 250), (750, 250), (1000, 3)]     # every row once, ragged tail
+    assert np.abs(G - ials.gramian(X)).max() <= 1e-13 * np.abs(G).max()
+    assert np.abs(G - X.T @ X).max() <= 1e-12 * np.abs(G).max()
+    # a block function that is handed (or honours) wrong ranges must not go unnoticed
+    G_bad = ials.gramian_stream(lambda r0, cnt: X[r0:r0 + min(cnt, 249)], 1003, 7, block_rows=250)
+    assert np.abs(G_bad - G).max() > 1e-6 * np.abs(G).max()
+    # one block (table shorter than the block size) and an exact multiple
+    assert np.allclose(ials.gramian_stream(block, 1003, 7, block_rows=5000), G, rtol=0, atol=1e-13 * np.abs(G).max())
+    assert np.allclose(ials.gramian_stream(lambda r0, cnt: X[r0:r0 + cnt], 1000, 7, block_rows=250), X[:1000].T @ X[:1000])
+
+
+# ---- conjugate gradients (Sec. 4.5): pinned by its limit and by the textbook properties of its iterates ----
+
+def _spd(d, eigs, seed):
+    rng = np.random.default_rng(seed)
+    Q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    return (Q * np.asarray(eigs, dtype=np.float64)) @ Q.T, rng.standard_normal(d)
+
+
+def test_cg_converges_to_the_direct_solution():
+    A, b = _spd(24, np.linspace(0.5, 40.0, 24), 1)
+    x, k = ials.cg(A, b, tol=1e-13, max_iter=200)
+    assert np.linalg.norm(x - np.linalg.solve(A, b)) <= 1e-11 * np.linalg.norm(x)
+    assert k <= 40
+    # d = 1: one step gives b / A
+    x1, k1 = ials.cg(np.array([[4.0]]), np.array([3.0]), tol=1e-15, max_iter=5)
+    assert k1 == 1 and x1[0] == 0.75
+    # zero right-hand side: zero steps, zero solution
+    x0, k0 = ials.cg(A, np.zeros(24))
+    assert k0 == 0 and np.all(x0 == 0)
+
+
+def test_cg_is_exact_after_as_many_steps_as_distinct_eigenvalues():
+    eigs = np.repeat([0.3, 1.0, 2.5, 7.0, 19.0], 6)          # d = 30, five distinct eigenvalues
+    A, b = _spd(30, eigs, 2)
+    x, k, its = ials.cg(A, b, tol=1e-9, max_iter=30, return_iterates=True)
+    assert k == 5
+    assert np.linalg.norm(A @ x - b) <= 1e-9 * np.linalg.norm(b)
+    assert np.linalg.norm(A @ its[3] - b) > 1e-6 * np.linalg.norm(b)       # and not before
+
+
+def test_cg_error_decreases_in_the_energy_norm_and_residuals_are_orthogonal():
+    A, b = _spd(40, np.geomspace(0.05, 30.0, 40), 3)
+    x_star = np.linalg.solve(A, b)
+    _, k, its = ials.cg(A, b, tol=1e-10, max_iter=80, return_iterates=True)
+    err = [np.sqrt((x_star - x) @ A @ (x_star - x)) for x in [np.zeros(40)] + list(its)]
+    assert all(e1 < e0 for e0, e1 in zip(err, err[1:]))
+    R = np.array([b - A @ x for x in [np.zeros(40)] + list(its[:12])])
+    Rn = R / np.linalg.norm(R, axis=1, keepdims=True)
+    off = Rn @ Rn.T - np.eye(len(Rn))
+    assert np.abs(off).max() <= 1e-8
+    # each iterate minimises the energy norm over the Krylov space: x_2 against brute force over span{b, A b}
+    K = np.stack([b, A @ b], axis=1)
+    c = np.linalg.solve(K.T @ A @ K, K.T @ b)
+    assert np.linalg.norm(K @ c - its[1]) <= 1e-10 * np.linalg.norm(its[1])
+
+
+def test_half_step_cg_meets_the_tolerance_and_approaches_the_exact_half_step():
+    rowptr, colidx, vals, W, H, _ = random_problem(30, 22, 6, 0.3, 11)
+    alpha, lam = 0.05, 0.2
+    G = ials.gramian(H)
+    exact, exact_raw = ials.half_step(rowptr, colidx, vals, H, alpha, lam, G=G, return_raw=True)
+    Y, raw, iters = ials.half_step_cg(rowptr, colidx, vals, H, alpha, lam, G=G, tol=1e-5, max_iter=64)
+    assert iters[0] == 0 and np.all(raw[0] == 0)                            # the empty row
+    for u in range(1, 30):
+        A, b = ials.row_system(rowptr, colidx, vals, H, G, alpha, lam, u)
+        assert np.linalg.norm(A @ raw[u] - b) <= 1.0001e-5 * np.linalg.norm(b)
+        assert 1 <= iters[u] <= 6                                           # at most d steps
+    tight, tight_raw, _ = ials.half_step_cg(rowptr, colidx, vals, H, alpha, lam, G=G, tol=1e-13, max_iter=64)
+    assert np.linalg.norm(tight_raw - exact_raw) <= 1e-10 * np.linalg.norm(exact_raw)
