@@ -245,7 +245,8 @@ def run_ours(args, w):
     nnz = int(colidx.numel())
     t_gen = time.perf_counter() - t_gen
 
-    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0))
+    a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0), solver=args.solver,
+            cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol)
     t_set = time.perf_counter()
     a.set_csr(rowptr, colidx)
     torch.cuda.synchronize()
@@ -270,7 +271,8 @@ def run_ours(args, w):
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    half_ms = {"rows": [], "cols": [], "gramian": [], "row_kernels": [], "main_kernel": [], "dual_rows": []}
+    half_ms = {"rows": [], "cols": [], "gramian": [], "row_kernels": [], "main_kernel": [], "dual_rows": [],
+               "cg_rows": [], "cg_products": [], "cg_fallbacks": []}
     ev[0].record()
     for k in range(args.steps):
         a.half_epoch(ALX_ROWS)
@@ -293,6 +295,9 @@ def run_ours(args, w):
         half_ms["row_kernels"].append(s2.ms_rows)
         half_ms["main_kernel"].append(s2.ms_main_kernel)
         half_ms["dual_rows"].append(s2.dual_rows)
+        half_ms["cg_rows"].append(s2.cg_rows)
+        half_ms["cg_products"].append(s2.cg_products)
+        half_ms["cg_fallbacks"].append(s2.cg_fallbacks)
     fp32_peak = a.fp32_peak_tflops()
     loss = a.loss()[0]
     ms, units = aggregate_over_ranks(ms_local, float(nnz), world, dev)
@@ -371,7 +376,8 @@ def run_ours(args, w):
         torch.cuda.empty_cache()
         o_W = torch.empty_like(h_W, pin_memory=True)
         o_H = torch.empty_like(h_H, pin_memory=True)
-        b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0))
+        b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0), solver=args.solver,
+                cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol)
         reps = 2 if w["name"] != "small" else 3
         times = []
         for r in range(reps):
@@ -409,7 +415,10 @@ def run_ours(args, w):
                           "paper_context": "about 20 min/epoch for 365M nodes / 29.9B edges on 256 TPU v3 cores"},
                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
                "cpu_baseline": cpu_baseline,
-               "extra": {"epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
+               "extra": {"solver": {"option": args.solver, "cg_rows": half_ms["cg_rows"], "cg_products": half_ms["cg_products"],
+                                    "cg_fallbacks": half_ms["cg_fallbacks"],
+                                    "note": "[rows half-epoch, columns half-epoch] of the half-epoch pair after the timed region"},
+                         "epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
                          "setup_s": {"generate": t_gen, "alx_set_csr_device": t_set},
                          "rows_in_class": [list(st.rows_in_class[0]), list(st.rows_in_class[1])],
                          "n_chunks": list(st.n_chunks), "workspace_gb": st.workspace_bytes / 1e9}}
@@ -425,6 +434,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--solver", type=int, default=0, choices=[0, 1],
+                    help="alx_options.solver: 0 = conjugate gradients where available (Cholesky otherwise), 1 = Cholesky")
+    ap.add_argument("--cg-max-iter", type=int, default=0, help="alx_options.cg_max_iter (0 = the library's default)")
+    ap.add_argument("--cg-tol", type=float, default=0.0, help="alx_options.cg_tol (0 = the library's default)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")
     args = ap.parse_args()

@@ -47,6 +47,10 @@ typedef enum {
 typedef enum { ALX_ROWS = 0, ALX_COLS = 1 } alx_side; /* which table is SOLVED; the other is held fixed */
 typedef enum { ALX_F32 = 0, ALX_BF16 = 1 } alx_dtype;
 
+typedef enum { ALX_SOLVER_AUTO = 0, ALX_SOLVER_CHOLESKY = 1 } alx_solver;
+#define ALX_DEFAULT_CG_MAX_ITER 48
+#define ALX_DEFAULT_CG_TOL 1e-5f
+
 /* number of degree classes and the default split threshold, see alx_get_buckets */
 #define ALX_N_CLASSES 12
 #define ALX_DEFAULT_SPLIT 8192
@@ -74,6 +78,13 @@ typedef struct alx_options {
                                 of Eq. 4 while alpha0 G + lambda I is well conditioned; 1 = force the plain FP32-ALU
                                 kernels (reference path inside the library; every d, every storage); 2 = as 0 but
                                 every row in the primal form */
+    int32_t solver;          /* how the d x d system of Eq. 4 is solved (Sec. 4.5 compares the choices):
+                                ALX_SOLVER_AUTO (0): conjugate gradients where the library has them (the whole-rows
+                                tensor-core kernel), started at x = 0 and stopped at |r| <= cg_tol |b|; a row that has not
+                                converged after cg_max_iter steps, and every row elsewhere, is solved by Cholesky.
+                                ALX_SOLVER_CHOLESKY (1): Cholesky for every row */
+    int32_t cg_max_iter;     /* 0 => ALX_DEFAULT_CG_MAX_ITER */
+    float cg_tol;            /* 0 => ALX_DEFAULT_CG_TOL; at most 1e-2 */
     int32_t reserved;
 } alx_options;
 
@@ -92,6 +103,9 @@ typedef struct alx_stats {
     int64_t long_rows[2];                    /* [side], tensor-core kernels only: whole rows of more than 1024 entries
                                                 whose sums the chunks kernel forms (as it does for the split rows) */
     int64_t long_entries[2];                 /* [side]: the entries those rows hold */
+    int64_t cg_rows;                         /* LAST half-epoch: rows the conjugate-gradient solve took, */
+    int64_t cg_products;                     /* the matrix-vector products it spent on them (steps + 1 per row), */
+    int64_t cg_fallbacks;                    /* and how many of those rows went on to the Cholesky solve (not converged) */
 } alx_stats;
 
 /* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.

@@ -3,6 +3,7 @@
 // happens on the host.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -49,6 +50,8 @@ struct alx_ctx {
     double *loss_partials_buf = nullptr;
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
+    unsigned long long *cg_counters = nullptr;   // tensor path: rows solved by conjugate gradients, products, fall-backs (last half-epoch)
+    int32_t *cg_fallback_list = nullptr;         // tensor path with conjugate gradients: the rows left to the Cholesky solve
 
     // second stream for the host copies that alx_load_host / alx_epoch_to_host overlap with kernels
     cudaStream_t copy_stream = nullptr;
@@ -219,6 +222,16 @@ void release_matrix(alx_ctx *c)
 
 bool tensor_path(const alx_ctx *c) { return c->bf16 && c->opt.d == 128 && c->opt.kernels != 1; }
 bool dual_form(const alx_ctx *c) { return tensor_path(c) && c->opt.kernels == 0; }
+CgOptions cg_options(const alx_ctx *c)
+{
+    CgOptions o;
+    o.enabled = c->opt.solver == ALX_SOLVER_AUTO;
+    o.max_iter = c->opt.cg_max_iter > 0 ? c->opt.cg_max_iter : ALX_DEFAULT_CG_MAX_ITER;
+    o.tol = c->opt.cg_tol > 0.f ? c->opt.cg_tol : ALX_DEFAULT_CG_TOL;
+    o.counters = c->cg_counters;
+    o.fallback_list = c->cg_fallback_list;
+    return o;
+}
 
 alx_status gramian_of(alx_ctx *c, int table_side)
 {
@@ -247,9 +260,11 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
     RowOut out{c->table[side], cap_slot, cap_out};
     if (tensor_path(c)) {
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 32 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
-                                     &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed]));
+                                     &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed],
+                                     cg_options(c)));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
         c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;
@@ -280,7 +295,7 @@ alx_status alx_create(int64_t n_rows, int64_t n_cols, int32_t d, float lambda, f
     memset(&o, 0, sizeof o);
     o.n_rows = n_rows; o.n_cols = n_cols; o.d = d; o.lambda = lambda; o.alpha0 = alpha0;
     o.storage = ALX_F32; o.device = -1;
-    return alx_create_ex(&o, out);
+    return alx_create_ex(&o, out);   /* solver, cg_max_iter, cg_tol = 0: the defaults */
 }
 
 alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
@@ -294,6 +309,8 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
     if (opt->storage != ALX_F32 && opt->storage != ALX_BF16) return ALX_ERR_INVALID_ARG;
     if ((opt->alloc == nullptr) != (opt->free == nullptr)) return ALX_ERR_INVALID_ARG;
     if (opt->split != 0 && opt->split < 16) return ALX_ERR_INVALID_ARG;
+    if (opt->solver != ALX_SOLVER_AUTO && opt->solver != ALX_SOLVER_CHOLESKY) return ALX_ERR_INVALID_ARG;
+    if (opt->cg_max_iter < 0 || opt->cg_max_iter > 1024 || !(opt->cg_tol >= 0.f) || opt->cg_tol > 1e-2f) return ALX_ERR_INVALID_ARG;
     int dev = opt->device;
     if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return ALX_ERR_CUDA;
     int count = 0;
@@ -331,6 +348,9 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
         ALX_ALLOC(c, c->loss_result, 4);
         ALX_ALLOC(c, c->status, 1);
         ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));
+        ALX_ALLOC(c, c->cg_counters, 32);
+        if (tensor_path(c) && c->opt.solver == ALX_SOLVER_AUTO) ALX_ALLOC(c, c->cg_fallback_list, nmax);
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 32 * sizeof(unsigned long long), c->stream));
         for (auto &e : c->ev) ALX_CUDA(c, cudaEventCreate(&e));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
         return ALX_OK;
@@ -746,6 +766,17 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
         int flag = 0;
         ALX_CUDA(c, cudaMemcpy(&flag, dual_flag_ptr(c->dual_ws), sizeof flag, cudaMemcpyDeviceToHost));
         c->stats.dual_rows = flag ? c->dual_candidates : 0;
+    }
+    {
+        unsigned long long h[32] = {};
+        ALX_CUDA(c, cudaMemcpy(h, c->cg_counters, sizeof h, cudaMemcpyDeviceToHost));
+        if (getenv("ALX_PROBE_PRINT"))
+            fprintf(stderr, "alx probe: rows %llu products %llu | cycles other %llu wait-acc %llu pre %llu first-mv %llu mv %llu shfl %llu bar %llu tail %llu | mma warp: other %llu wait-acc %llu wait-full %llu mma-issue %llu commit %llu acc-commit %llu syncwarp %llu item-top %llu | producer 0: other %llu item-top %llu wait-empty %llu issue %llu wait-landed %llu rhs %llu test %llu\n",
+                    h[0], h[1], h[8], h[9], h[10], h[11], h[12], h[13], h[14], h[15], h[16], h[17], h[18], h[19], h[20], h[21], h[22], h[23],
+                    h[24], h[25], h[26], h[27], h[28], h[29], h[30]);
+        c->stats.cg_rows = (int64_t)h[0];
+        c->stats.cg_products = (int64_t)h[1];
+        c->stats.cg_fallbacks = (int64_t)h[2];
     }
     c->stats.kernel_launches = c->launches;
     c->stats.workspace_bytes = c->bytes_held;

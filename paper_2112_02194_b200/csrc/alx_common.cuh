@@ -140,13 +140,22 @@ inline int long_class_begin(const int64_t *class_offs_host)
     return c;
 }
 
+// conjugate-gradient solve of the whole-rows tensor-core kernel (Sec. 4.5)
+struct CgOptions {
+    bool enabled;
+    int max_iter;                  // a row that has not converged by then is solved by the in-place Cholesky instead
+    float tol;                     // stop at |r| <= tol |b|
+    unsigned long long *counters;  // device, [3]: rows, matrix-vector products, rows that fell back
+    int32_t *fallback_list;        // device, one entry per row of the larger side: the rows left to the Cholesky solve
+};
+
 // alx_umma.cu: tensor-core path, d = 128 and bf16 tables only
 int64_t gramian_umma_partials();
 cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches);
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                              int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
                              RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,
-                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table);
+                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table, const CgOptions &cg);
 
 // alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();

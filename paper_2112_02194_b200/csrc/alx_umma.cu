@@ -25,6 +25,7 @@
 #include "alx_common.cuh"
 #include "alx_ptx.cuh"
 #include <cstring>
+#include <type_traits>
 #include <cuda.h>      // CUtensorMap and its enumerations (types only: the encoder is looked up at run time)
 
 namespace alx {
@@ -41,37 +42,57 @@ constexpr int kStageRows = 32;
 // streaming modes (chunks, Gramian) use that space for a deeper ring, which is what keeps HBM busy
 // (and stages of 64 gathered rows instead of 32: half the per-stage waits and commits of the MMA thread)
 template <int MODE> struct Ring {
-    static constexpr int kRows = (MODE == 0) ? 32 : 64;   // gathered rows per stage
-    static constexpr int kNStage = (MODE == 0) ? 8 : 12;
+    static constexpr int kRows = (MODE == 0 || MODE == 3) ? 32 : 64;   // gathered rows per stage
+    // (the conjugate-gradient rows kernel needs no operand tiles for a factorisation: their space deepens its ring,
+    // and a gather is bound by latency times bytes in flight)
+    static constexpr int kNStage = (MODE == 0) ? 8 : ((MODE == 3) ? 13 : 12);
     static constexpr int kHalfBytes = kRows * 128;        // one 64-feature half of a stage
     static constexpr int kStageHBytes = 2 * kHalfBytes;
     static constexpr int kStageYBytes = 2 * kRows * 16;   // label tile, two 8-column chunks
+    // rows modes: ring of per-item right-hand sides.  A slot is read when a solver group starts its item j; by then the
+    // MMA warp is at item j + 3 at most (item j + 4 needs the accumulator of j) and the producers at most one ring of
+    // stages, hence as many items, further: slots j .. j + kNStage + 3 are live at most
+    static constexpr int kBRing = kNStage + 4;
+    // rows modes: stages of cp.async copies in flight per producer warp (a gather is bound by latency times bytes in flight)
+    static constexpr int kLag = 6;
 };
 constexpr int kHalfBytes = kStageRows * 128;          // rows mode: one 64-feature half of a stage
-constexpr int kRowsLag = 6;                           // rows mode: stages of cp.async copies in flight per producer warp
 constexpr int kProducerWarps = 4;
 constexpr int kTmemCols = 512;
 constexpr int kMaxGroups = 4;
-constexpr int kBRing = 16;                            // rows mode: ring of per-item right-hand sides
 constexpr int kGramSubRows = 256;                     // rows per tensor-memory accumulation of the Gramian (the
                                                       // accumulator truncates: fewer steps, smaller bias)
 constexpr int kGramBlocks = 148;                      // fixed, so that the order of sums depends on sizes only
 
-enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2 };
+// kModeRowsCg: whole rows as kModeRows, solved by conjugate gradients instead of the in-place Cholesky
+enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2, kModeRowsCg = 3 };
+__host__ __device__ constexpr bool is_rows(int mode) { return mode == kModeRows || mode == kModeRowsCg; }
+
+// Development aid (-DALX_PROBE): thread 0 of every solver group sums clock cycles per phase into cg_counters[3 ..].
+struct Probe {
+#ifdef ALX_PROBE
+    long long t0 = 0, acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    __device__ __forceinline__ void start() { t0 = clock64(); }
+    __device__ __forceinline__ void lap(int k) { const long long t = clock64(); acc[k] += t - t0; t0 = t; }
+#else
+    __device__ __forceinline__ void start() {}
+    __device__ __forceinline__ void lap(int) {}
+#endif
+};
 
 // thread layout per mode: solver groups (one accumulator each), then one MMA warp, then the producer warps
 template <int MODE> struct Cfg {
-    static constexpr int kGroups = (MODE == kModeRows) ? 4 : 2;
-    static constexpr int kGroupThreads = (MODE == kModeRows) ? 128 : 256;
-    static constexpr int kAccStride = (MODE == kModeRows) ? 128 : 256;   // accumulator a: columns a * stride ..
+    static constexpr int kGroups = is_rows(MODE) ? 4 : 2;
+    static constexpr int kGroupThreads = is_rows(MODE) ? 128 : 256;
+    static constexpr int kAccStride = is_rows(MODE) ? 128 : 256;   // accumulator a: columns a * stride ..
     static constexpr int kSolverThreads = kGroups * kGroupThreads;
     static constexpr int kMmaWarp = kSolverThreads / 32;
     static constexpr int kFirstProducerWarp = kMmaWarp + 1;
     // rows mode: the four producer warps share every stage (8 rows each, by cp.async; their partial right-hand sides
     // are summed in a fixed order); streaming modes: four producer warps, each fills whole stages of its own by TMA
     // row gathers
-    static constexpr int kProducers = (MODE == kModeRows) ? kProducerWarps : 4;
-    static constexpr int kFullArrivals = (MODE == kModeRows) ? kProducerWarps : 1;
+    static constexpr int kProducers = is_rows(MODE) ? kProducerWarps : 4;
+    static constexpr int kFullArrivals = is_rows(MODE) ? kProducerWarps : 1;
     static constexpr int kBlockThreads = kSolverThreads + 32 + kProducers * 32;
 };
 
@@ -92,9 +113,22 @@ struct Params {
     float *partials;             // chunks: [slot][D*D + D]; Gramian: [2 * kGramBlocks][D*D]
     RowOut out;
     DevStatus *st;
+    const int32_t *item_list;    // rows mode, second launch: the rows to solve (instead of the walk through sv.order) ...
+    const unsigned long long *item_count;   // ... and how many of them (device)
+    int32_t *fallback_list;      // conjugate gradients: rows that did not converge are appended here (any order) ...
+    unsigned long long *fallback_count;     // ... and counted here; a second launch solves them by Cholesky
+    int solver;                  // rows mode: 0 = in-place Cholesky, 1 = conjugate gradients
+    int cg_max_iter;             // conjugate gradients: steps after which a row goes to the Cholesky solve instead
+    float cg_tol2;               // conjugate gradients: stop at |r|^2 <= cg_tol2 |b|^2
+    unsigned long long *cg_counters;   // [3]: rows solved by conjugate gradients, their matrix-vector products, rows that fell back
 };
 
 constexpr int kLdB = D + 4;
+// conjugate gradients read the matrix with the 16x128b tensor-memory shape (a thread holds four rows, every fourth
+// column): alpha0 G + lambda I and the vector of a product are kept in shared memory by column class (column mod 4),
+// 36 floats per class so that the four classes of a quarter-warp's 16-byte loads fall into different banks
+constexpr int kQStride = 36;
+constexpr int kLdBq = 4 * kQStride;      // floats per row of alpha0 G + lambda I in that layout
 struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver group
     // Panel of the current block step as tensor-core operands: row i = what thread i computed, split into
     // three bfloat16 parts (p = p1 + p2 + p3 to 2^-24), each part a K-major 128 x 16 tile without swizzle:
@@ -110,10 +144,18 @@ struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver gr
     int stop;               // set by the polling thread when a wait gave up; read by the group after its barrier
 };
 
+// scratch of one conjugate-gradient solver group: the vector of the next product by column class, the four warps' partial
+// sums of a step's reduction, and the flags the group shares
+struct __align__(128) CgGroupSmem {
+    alignas(16) float pop[1][4 * 36 + 16];
+    int bad;
+    int stop;
+};
+
 template <int MODE> struct __align__(1024) SmemT {
     static constexpr int kNStage = Ring<MODE>::kNStage;
     unsigned char h[kNStage][Ring<MODE>::kStageHBytes];
-    unsigned char y[(MODE == 0) ? 1 : kNStage][Ring<MODE>::kStageYBytes];      // label tiles (chunks mode only)
+    unsigned char y[is_rows(MODE) ? 1 : kNStage][Ring<MODE>::kStageYBytes];      // label tiles (chunks mode only)
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
     uint32_t tmem_base;
     int abort_flag;
@@ -122,14 +164,14 @@ template <int MODE> struct __align__(1024) SmemT {
     int stage_meta[kNStage];                     // K steps of the stage (1 or 2) | 4 if it ends its item; -1: no more work
     int rows_staged[kProducerWarps][kNStage];    // per producer warp: how many of its 8 rows of the stage are defined
     int last_of_item[kProducerWarps][kNStage];   // per producer warp: 1 + ring index of the item whose last stage this is, else 0
-    alignas(16) float bpart[(MODE == 0) ? kBRing : 1][kProducerWarps][D];
+    alignas(16) float bpart[is_rows(MODE) ? Ring<MODE>::kBRing : 1][kProducerWarps][D];
 };
 
 template <int MODE> __device__ __forceinline__ void item_range(const Params &p, int64_t t, int64_t &u, int64_t &beg,
                                                                int64_t &end, int64_t &slot)
 {
-    if (MODE == kModeRows) {
-        u = p.sv.order[p.last_item - t];
+    if (is_rows(MODE)) {
+        u = p.item_list ? p.item_list[t] : p.sv.order[p.last_item - t];
         beg = p.sv.ptr[u];
         end = p.sv.ptr[u + 1];
         slot = 0;
@@ -154,7 +196,8 @@ template <int MODE> __device__ __forceinline__ void item_range(const Params &p, 
 // rows mode: sum y x over this warp's 8 rows of a landed stage (lane = features 4*lane .. 4*lane+3)
 using Smem = SmemT<0>;       // rows mode
 
-__device__ __forceinline__ void stage_rhs(Smem &sm, int slot, int pw, int lane, float (&bacc)[4])
+template <class SmemRows>
+__device__ __forceinline__ void stage_rhs(SmemRows &sm, int slot, int pw, int lane, float (&bacc)[4])
 {
     const int f = 4 * lane;
     const int half = f >> 6, cc = (f & 63) >> 3, inner = (f & 7) * 2;
@@ -178,7 +221,7 @@ template <int MODE> __device__ __forceinline__ void producer_signal(SmemT<MODE> 
 {
     constexpr int kNStage = Ring<MODE>::kNStage;
     const int slot = (int)(signalled % kNStage);
-    if constexpr (MODE == kModeRows) {
+    if constexpr (is_rows(MODE)) {
         __syncwarp();      // every lane's copies of this stage have landed (each lane waited for its own)
         stage_rhs(sm, slot, pw, lane, bacc);
         const int last = sm.last_of_item[pw][slot];
@@ -192,27 +235,71 @@ template <int MODE> __device__ __forceinline__ void producer_signal(SmemT<MODE> 
     if (lane == 0) mbar_arrive(&sm.full[slot]);
 }
 
-template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
+// Rows modes: the offsets of the block's next 32 items, one item per lane, fetched together every 32 items (a row's
+// offsets hang on a chain of dependent loads, order -> ptr; walked item by item, that latency would be paid per item,
+// which rows of a hundred entries cannot afford).  Item `it` of the block is row order[last_item - (blockIdx.x + it grid)].
+struct ItemWindow {
+    int64_t beg = 0, end = 0;      // this lane's item of the window (empty range past the last item)
+    __device__ __forceinline__ void load(const Params &p, int64_t it0, int lane)
+    {
+        const int64_t t = (int64_t)blockIdx.x + (it0 + lane) * gridDim.x;
+        beg = end = 0;
+        if (t < p.n_items) {
+            const int64_t u = p.item_list ? p.item_list[t] : p.sv.order[p.last_item - t];
+            beg = p.sv.ptr[u];
+            end = p.sv.ptr[u + 1];
+        }
+    }
+    __device__ __forceinline__ void get(int k, int64_t &b, int64_t &e) const
+    {
+        b = __shfl_sync(0xFFFFFFFFu, beg, k);
+        e = __shfl_sync(0xFFFFFFFFu, end, k);
+    }
+};
+
+// PARK: wait for a free stage suspended (no issue slots taken) instead of polling: for the kernel whose solver
+// groups, not the gather, set the pace
+template <int MODE, bool PARK> __device__ void producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
 {
-    constexpr int kNStage = Ring<MODE>::kNStage, kLag = kRowsLag;
+    constexpr int kNStage = Ring<MODE>::kNStage, kLag = Ring<MODE>::kLag;
     int64_t g = 0, signalled = 0, it = 0;
     const int c = lane & 15;                 // 16-byte chunk of the 256-byte row
     const int half = c >> 3, cc = c & 7;
     float bacc[4] = {0.f, 0.f, 0.f, 0.f};
     bool alive = true;
-    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
-        int64_t u, beg, end, slot_unused;
-        item_range<MODE>(p, t, u, beg, end, slot_unused);
-        // ids (and labels) of this warp's 8 rows of a stage are fetched one stage ahead by lanes 0..7
-        int32_t nxt_idx = -1;
-        float nxt_y = 0.f;
-        {
-            const int64_t e = beg + pw * 8 + (lane & 7);
-            if (lane < 8 && e < end) {
-                nxt_idx = (MODE == kModeGramian) ? (int32_t)e : p.sv.idx[e];
-                nxt_y = (MODE == kModeGramian) ? 0.f : (p.sv.val ? p.sv.val[e] : 1.f);
-            }
+    ItemWindow win;
+    // ids (and labels) of this warp's 8 rows of a stage are fetched one stage ahead by lanes 0..7; those of an item's
+    // first stage while the item before it is gathered (except across a window's end)
+    int32_t pre_idx = -1;
+    float pre_y = 0.f;
+    bool have_pre = false;
+    auto first_ids = [&](int64_t beg, int64_t end, int32_t &idx, float &y) {
+        idx = -1;
+        y = 0.f;
+        const int64_t e = beg + pw * 8 + (lane & 7);
+        if (lane < 8 && e < end) {
+            idx = p.sv.idx[e];
+            y = p.sv.val ? p.sv.val[e] : 1.f;
         }
+    };
+    Probe pr;
+    pr.start();
+    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
+        pr.lap(0);
+        if ((it & 31) == 0) win.load(p, it, lane);
+        int64_t beg, end;
+        win.get((int)(it & 31), beg, end);
+        int32_t nxt_idx;
+        float nxt_y;
+        if (have_pre) { nxt_idx = pre_idx; nxt_y = pre_y; }
+        else first_ids(beg, end, nxt_idx, nxt_y);
+        have_pre = (it & 31) != 31;
+        if (have_pre) {
+            int64_t nbeg, nend;
+            win.get((int)(it & 31) + 1, nbeg, nend);
+            first_ids(nbeg, nend, pre_idx, pre_y);
+        }
+        pr.lap(1);
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
@@ -229,6 +316,7 @@ template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &
             }
             // No free slot yet: the copies in flight have time to land, so hand over every stage issued so far
             // before blocking (otherwise up to kLag landed stages would stay unannounced until the next issue).
+            pr.lap(0);
             {
                 int free_now = 1;
                 if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
@@ -238,13 +326,16 @@ template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &
                     for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
                 }
             }
-            if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
+            pr.lap(5);
+            if (!(PARK ? mbar_wait_parked_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)
+                       : mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE))) { alive = false; break; }
+            pr.lap(2);
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int rc16 = (rc + 15) & ~15;
-            if (MODE == kModeRows) {
+            if (is_rows(MODE)) {
                 if (lane < 8) sm.ylab[slot][pw * 8 + lane] = my_y;
                 if (lane == 0) {
-                    sm.last_of_item[pw][slot] = (e0 + kStageRows >= end) ? 1 + (int)(it % kBRing) : 0;
+                    sm.last_of_item[pw][slot] = (e0 + kStageRows >= end) ? 1 + (int)(it % Ring<MODE>::kBRing) : 0;
                     const int mine = rc16 - pw * 8;
                     sm.rows_staged[pw][slot] = mine < 0 ? 0 : (mine > 8 ? 8 : mine);
                 }
@@ -269,15 +360,22 @@ template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &
             }
             cp_async_commit();
             ++g;
+            pr.lap(3);
             if (g - signalled > kLag) {     // the oldest unannounced stage is kLag issues back: its copies have landed
                 cp_async_wait<kLag>();
+                pr.lap(4);
                 producer_signal<MODE>(sm, signalled, pw, lane, bacc);
                 ++signalled;
+                pr.lap(6);
             }
         }
     }
     cp_async_wait<0>();
     for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
+#ifdef ALX_PROBE
+    if (lane == 0 && pw == 0 && p.cg_counters)
+        for (int k = 0; k < 7; ++k) atomicAdd(&p.cg_counters[24 + k], (unsigned long long)pr.acc[k]);
+#endif
 }
 
 // Streaming modes (chunks, Gramian pieces): producer warp pw fills the stages whose running number is pw modulo the
@@ -360,20 +458,33 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
     int slot = 0;             // ring position and phase of the next stage
     uint32_t ph = 0;
     bool alive = true;
+    Probe pr;
+    pr.start();
+    ItemWindow win;
     for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
         int64_t u, beg, end, slot_unused;
-        item_range<MODE>(p, t, u, beg, end, slot_unused);
+        if constexpr (is_rows(MODE)) {
+            if ((it & 31) == 0) win.load(p, it, lane);
+            win.get((int)(it & 31), beg, end);
+        } else {
+            item_range<MODE>(p, t, u, beg, end, slot_unused);
+        }
         const int a = (int)(it % Cfg<MODE>::kGroups);
         const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
+        pr.lap(7);
         if (!mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
         tc_fence_after();
+        pr.lap(1);
         const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
         bool first = true;
         for (int64_t e0 = beg; e0 < end; e0 += kRows) {
+            pr.lap(0);
             if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) { alive = false; break; }
             tc_fence_after();
+            pr.lap(2);
             const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
             const int nk = (rc + 15) >> 4;
+            pr.lap(0);
             if (lane == 0) {
                 const uint32_t hb = smem_u32(&sm.h[slot][0]);
                 const uint32_t yb = smem_u32(&sm.y[slot][0]);
@@ -387,14 +498,23 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
                     }
                     first = false;
                 }
+                pr.lap(3);
                 umma_commit(&sm.empty[slot]);
+                pr.lap(4);
             }
-            __syncwarp();
             if (++slot == kNStage) { slot = 0; ph ^= 1u; }
         }
+        pr.lap(0);
         if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
+        pr.lap(5);
         __syncwarp();
+        pr.lap(6);
     }
+#ifdef ALX_PROBE
+    pr.lap(0);
+    if (lane == 0 && p.cg_counters)
+        for (int k = 0; k < 8; ++k) atomicAdd(&p.cg_counters[16 + k], (unsigned long long)pr.acc[k]);
+#endif
 }
 
 template <int MODE>
@@ -533,28 +653,465 @@ __device__ __forceinline__ void group128_sync(int bar_id)
 }
 
 
+// The in-place factor / solve of one matrix held in tensor memory (steps (1) .. (5) above); returns x_i.  add_b: alpha0 G +
+// lambda I is still to be added (from shared memory, as the panels are read); b: my component of the right-hand side.
+// A wait that gave up leaves gs.stop set (the caller leaves its loop); a non-positive pivot leaves gs.bad set.
+template <class SmemRows>
+__device__ __forceinline__ float chol_in_tmem(SmemRows &sm, RowGroupSmem &gs, const float *Brow, uint32_t trow, uint32_t d_base,
+                                              int bar_id, int tid, float b, bool add_b, uint32_t &trail_parity)
+{
+    const int lane = tid & 31, w = tid >> 5;
+    const int i = tid, pos = tid, wpos = pos & ~31;
+    float lrow[16];          // my row of my diagonal block's factor (kept for the block inverse at the end)
+    float my_dinv = 0.f;     // 1 / L[i][i]
+#pragma unroll
+    for (int c = 0; c < 16; ++c) lrow[c] = 0.f;
+
+    for (int k = 0; k < D / 16; ++k) {
+        const int k0 = 16 * k;
+        const int ck = k0;                                     // tensor-memory columns of this block
+        float a[16];
+        const bool warp_live = (wpos + 31 >= k0);              // some row of my warp is at or after the block
+        const bool diag_warp = (wpos == (k0 & ~31));
+        auto load_panel = [&]() {
+            tmem_ld16(trow + ck, a);
+#pragma unroll
+            for (int c = 0; c < 16; c += 4) {
+                if (!add_b) break;
+                const float4 bb = *reinterpret_cast<const float4 *>(Brow + ck + c);
+                const float2 s01 = __fadd2_rn(make_float2(a[c], a[c + 1]), make_float2(bb.x, bb.y));
+                const float2 s23 = __fadd2_rn(make_float2(a[c + 2], a[c + 3]), make_float2(bb.z, bb.w));
+                a[c] = s01.x; a[c + 1] = s01.y; a[c + 2] = s23.x; a[c + 3] = s23.y;
+            }
+        };
+        if (diag_warp) {
+            // the previous step's tensor-core update has landed: only the warp that holds the diagonal block waits
+            // for it (a wait that gives up only sets the group's stop flag; the group leaves together after the
+            // block loop); the other warps follow through the barrier below, at no cost in issue slots
+            if (k > 0) {
+                if (!mbar_wait_warp(&gs.trail_bar, trail_parity ^ 1u, &sm.abort_flag, 70) && lane == 0) gs.stop = 1;
+                tc_fence_after();
+            }
+            load_panel();
+        }
+        // (1) diagonal block
+        if (diag_warp) {
+            const int hb = k0 & 16;
+            const int l = lane - hb;      // place relative to the block: < 0 eliminated earlier, 0 .. 15 the block,
+                                          // >= 16 the 16 rows after the block (when it is the first of its warp)
+            const bool is_diag = (l >= 0 && l < 16);
+            float my_inv = 0.f;
+            bool all_ok = true;
+            // Two pivots per round, no masks on the matrix entries: a row that is done only ever overwrites
+            // entries of its upper triangle (never read), and the rows after the block that share this warp get
+            // their forward substitution against the block for free (the same arithmetic in the same order as
+            // the substitution step below, which they then skip).  Only b needs guarding: rows that are done
+            // keep their component of L^-1 b.
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+                const float p00 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j);
+                const float p10 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j + 1);
+                const float p11 = __shfl_sync(0xFFFFFFFFu, a[j + 1], hb + j + 1);
+                const float bj = __shfl_sync(0xFFFFFFFFu, b, hb + j);
+                const float bj1 = __shfl_sync(0xFFFFFFFFu, b, hb + j + 1);
+                // a pivot <= 0 turns into NaN or infinity here and stays visible in 1 / L[row][row] (checked below)
+                const float inv0 = rsqrt_fast(p00);
+                const float l10 = p10 * inv0;
+                const float q11 = fmaf(-l10, l10, p11);
+                const float inv1 = rsqrt_fast(q11);
+                const float zj = bj * inv0;
+                const float zj1 = fmaf(-l10, zj, bj1) * inv1;
+                const float x0 = a[j] * inv0;                       // L[row][j]   (row j itself: sqrt of the pivot)
+                const float x1 = fmaf(-x0, l10, a[j + 1]) * inv1;   // L[row][j+1] (row j+1 itself: sqrt of the second pivot)
+                a[j] = x0;
+                a[j + 1] = x1;
+                my_inv = (l == j) ? inv0 : ((l == j + 1) ? inv1 : my_inv);
+                const float bdown = fmaf(-x1, zj1, fmaf(-x0, zj, b));
+                b = (l > j + 1) ? bdown : ((l == j + 1) ? zj1 : ((l == j) ? zj : b));
+                // the two new columns go through shared memory (shuffles are the slower path for 2 x 14 values)
+                float *xb = &gs.xch[(j & 2) * 16];
+                if (is_diag) { xb[l] = x0; xb[16 + l] = x1; }
+                __syncwarp();
+                float c0[16], c1[16];
+#pragma unroll
+                for (int q4 = (j + 2) / 4; q4 < 4; ++q4) {
+                    const float4 u4 = *reinterpret_cast<const float4 *>(&xb[4 * q4]);
+                    const float4 v4 = *reinterpret_cast<const float4 *>(&xb[16 + 4 * q4]);
+                    c0[4 * q4] = u4.x; c0[4 * q4 + 1] = u4.y; c0[4 * q4 + 2] = u4.z; c0[4 * q4 + 3] = u4.w;
+                    c1[4 * q4] = v4.x; c1[4 * q4 + 1] = v4.y; c1[4 * q4 + 2] = v4.z; c1[4 * q4 + 3] = v4.w;
+                }
+#pragma unroll
+                for (int c = j + 2; c < 16; c += 2) {
+                    float2 r = __ffma2_rn(make_float2(-x0, -x0), make_float2(c0[c], c0[c + 1]), make_float2(a[c], a[c + 1]));
+                    r = __ffma2_rn(make_float2(-x1, -x1), make_float2(c1[c], c1[c + 1]), r);
+                    a[c] = r.x;
+                    a[c + 1] = r.y;
+                }
+            }
+            all_ok = __all_sync(0xFFFFFFFFu, !is_diag || (my_inv > 0.f && my_inv <= 3.0e38f));
+            if (!all_ok && lane == 0) gs.bad = 1;
+            if (is_diag) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const float v = (c <= l) ? a[c] : 0.f;
+                    gs.Lt[c][l] = v;
+                    lrow[c] = v;
+                }
+                gs.dinv[l] = my_inv;
+                gs.z[l] = b;
+                my_dinv = my_inv;
+            }
+        }
+        tc_fence_before();
+        group128_sync(bar_id);
+        if (warp_live && !diag_warp) {
+            tc_fence_after();
+            load_panel();
+        }
+        // (2) rows after the block: forward substitution, split, operand tiles
+        if (pos >= k0 + 16) {
+          if (wpos != (k0 & ~31)) {      // (the rows after the block in its own warp are already done, see above)
+            float dv[16];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const float4 v = *reinterpret_cast<const float4 *>(&gs.dinv[4 * q4]);
+                dv[4 * q4] = v.x; dv[4 * q4 + 1] = v.y; dv[4 * q4 + 2] = v.z; dv[4 * q4 + 3] = v.w;
+            }
+            // column-oriented: once a[pp] is final it is eliminated from the later entries, which are
+            // independent of each other
+#pragma unroll
+            for (int pp = 0; pp < 16; ++pp) {
+                float lt[16];
+#pragma unroll
+                for (int q4 = (pp + 1) / 4; q4 < 4; ++q4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[pp][4 * q4]);
+                    lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
+                }
+                a[pp] *= dv[pp];
+                // packed FP32 FMAs on pairs of columns: half the issue slots, which the chains of the other
+                // groups on this sub-partition need
+                const float mneg = -a[pp];
+                if ((pp + 1) & 1) a[pp + 1] = fmaf(mneg, lt[pp + 1], a[pp + 1]);
+#pragma unroll
+                for (int c = (pp + 2) & ~1; c < 16; c += 2) {
+                    const float2 r = __ffma2_rn(make_float2(mneg, mneg), make_float2(lt[c], lt[c + 1]), make_float2(a[c], a[c + 1]));
+                    a[c] = r.x;
+                    a[c + 1] = r.y;
+                }
+            }
+            float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const float4 zz = *reinterpret_cast<const float4 *>(&gs.z[4 * q4]);
+                acc2 = __ffma2_rn(make_float2(a[4 * q4], a[4 * q4 + 1]), make_float2(zz.x, zz.y), acc2);
+                acc2 = __ffma2_rn(make_float2(a[4 * q4 + 2], a[4 * q4 + 3]), make_float2(zz.z, zz.w), acc2);
+            }
+            b -= acc2.x + acc2.y;
+          }
+            uint32_t w1[8], w2[8], w3[8];
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) {
+                // part 1 rounds to nearest (one packed conversion); parts 2 and 3 keep the leading 8 bits of
+                // what is left, so p1 + p2 + p3 = p up to 2^-24
+                const __nv_bfloat162 hpair = __floats2bfloat162_rn(a[c], a[c + 1]);
+                const uint32_t hw = *reinterpret_cast<const uint32_t *>(&hpair);
+                // (packed arithmetic: x - y as fma(y, -1, x) on both lanes; the upper halves of two words are
+                // gathered by one byte permutation)
+                const float2 minus1 = make_float2(-1.f, -1.f);
+                const float2 r = __ffma2_rn(make_float2(__uint_as_float(hw << 16), __uint_as_float(hw & 0xFFFF0000u)), minus1,
+                                            make_float2(a[c], a[c + 1]));
+                const uint32_t m0 = __float_as_uint(r.x) & 0xFFFF0000u, m1 = __float_as_uint(r.y) & 0xFFFF0000u;
+                const float2 sres = __ffma2_rn(make_float2(__uint_as_float(m0), __uint_as_float(m1)), minus1, r);
+                w1[c >> 1] = hw;
+                w2[c >> 1] = __byte_perm(m0, m1, 0x7632);
+                w3[c >> 1] = __byte_perm(__float_as_uint(sres.x), __float_as_uint(sres.y), 0x7632);
+            }
+            const uint32_t roff = (uint32_t)((i >> 3) * 256 + (i & 7) * 16);
+            const uint32_t b1 = smem_u32(&gs.pop[0][0]) + roff, b2 = smem_u32(&gs.pop[1][0]) + roff,
+                           b3 = smem_u32(&gs.pop[2][0]) + roff;
+            st_shared_v4(b1, w1[0], w1[1], w1[2], w1[3]); st_shared_v4(b1 + 128, w1[4], w1[5], w1[6], w1[7]);
+            st_shared_v4(b2, w2[0], w2[1], w2[2], w2[3]); st_shared_v4(b2 + 128, w2[4], w2[5], w2[6], w2[7]);
+            st_shared_v4(b3, w3[0], w3[1], w3[2], w3[3]); st_shared_v4(b3 + 128, w3[4], w3[5], w3[6], w3[7]);
+            fence_proxy_async();
+        }
+        if (warp_live) {
+            tmem_st16(trow + ck, a);      // L (rows before the block rewrite what they read)
+            tmem_st_wait();
+        }
+        tc_fence_before();
+        group128_sync(bar_id);
+        // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
+        // blocks of 32 rows further on (cyclically), which never holds the next diagonal block.  It
+        // issues the update and commits it to the group's mbarrier (a tcgen05.mma takes the issuing thread about
+        // 50 cycles); the next step's diagonal warp waits for it.
+        const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
+        uint64_t da[3] = {0, 0, 0};
+        // columns [c_lo, c_lo + n) of the matrix (= panel rows c_lo ..) -= P P^T restricted to them
+        auto update = [&](int c_lo, int n) {
+            const uint32_t idesc = idesc_bf16_k_major_negA(128, n);
+            uint64_t db[3];
+#pragma unroll
+            for (int q = 0; q < 3; ++q) db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + (uint32_t)(c_lo * 32), 128, 256, 0);
+            umma_f16(d_base + c_lo, da[0], db[0], idesc, true);
+            umma_f16(d_base + c_lo, da[0], db[1], idesc, true);
+            umma_f16(d_base + c_lo, da[1], db[0], idesc, true);
+            umma_f16(d_base + c_lo, da[0], db[2], idesc, true);
+            umma_f16(d_base + c_lo, da[2], db[0], idesc, true);
+            umma_f16(d_base + c_lo, da[1], db[1], idesc, true);
+        };
+        if (k < D / 16 - 1 && issuer) {
+            tc_fence_after();
+#pragma unroll
+            for (int q = 0; q < 3; ++q) da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
+            // all trailing columns in one set of six instructions: the tensor pipe takes about 50 cycles per
+            // instruction whatever its width, and it is shared by the four groups and the gather
+            update(k0 + 16, D - k0 - 16);
+            umma_commit(&gs.trail_bar);
+        }
+        if (k < D / 16 - 1) trail_parity ^= 1u;
+    }
+    group128_sync(bar_id);
+    if (gs.stop) return 0.f;
+    // my column of the inverse of my diagonal block.  The eight blocks go through shared memory, in the operand
+    // tiles: every trailing update has completed (the last one was waited for before the last block step).
+    float yinv[16];
+    {
+        float *Lall = reinterpret_cast<float *>(&gs.pop[0][0]);      // [8 blocks][16][16], transposed
+        float *dall = Lall + 8 * 256;                                 // [128] reciprocals of the diagonal
+        float *Lb = Lall + (pos >> 4) * 256;
+        const int l = pos & 15;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) Lb[c * 16 + l] = lrow[c];
+        dall[pos] = my_dinv;
+        __syncwarp();
+        const float *dvb = dall + (pos & ~15);
+        float tacc[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) tacc[c] = 0.f;
+#pragma unroll
+        for (int cp = 0; cp < 16; ++cp) {
+            // y[cp] of the solve L y = e_l
+            const float ycp = (cp < l) ? 0.f : ((cp == l) ? dvb[cp] : -tacc[cp] * dvb[cp]);
+            yinv[cp] = ycp;
+            float lt[16];
+#pragma unroll
+            for (int q4 = (cp + 1) / 4; q4 < 4; ++q4) {
+                const float4 v = *reinterpret_cast<const float4 *>(&Lb[cp * 16 + 4 * q4]);
+                lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
+            }
+            if ((cp + 1) & 1) tacc[cp + 1] = fmaf(lt[cp + 1], ycp, tacc[cp + 1]);
+#pragma unroll
+            for (int c = (cp + 2) & ~1; c < 16; c += 2) {
+                const float2 r = __ffma2_rn(make_float2(lt[c], lt[c + 1]), make_float2(ycp, ycp), make_float2(tacc[c], tacc[c + 1]));
+                tacc[c] = r.x;
+                tacc[c + 1] = r.y;
+            }
+        }
+    }
+    // (4) back substitution L^T x = z; b now holds z_i
+    float x = 0.f;
+    for (int k = D / 16 - 1; k >= 0; --k) {
+        const int k0 = 16 * k;
+        const int ck = k0;
+        float wv[16];
+        if (wpos + 31 >= k0 + 16) {
+            tmem_ld16(trow + ck, wv);
+            const float xm = (pos >= k0 + 16) ? x : 0.f;
+#pragma unroll
+            for (int c = 0; c < 16; c += 2) {
+                const float2 r = __fmul2_rn(make_float2(wv[c], wv[c + 1]), make_float2(xm, xm));
+                wv[c] = (pos >= k0 + 16) ? r.x : 0.f;
+                wv[c + 1] = (pos >= k0 + 16) ? r.y : 0.f;
+            }
+            warp_reduce16(wv, lane);
+        } else {
+            wv[0] = 0.f;
+        }
+        if ((lane & 1) == 0) gs.red[k & 1][w][lane >> 1] = wv[0];
+        group128_sync(bar_id);
+        if (wpos == (k0 & ~31)) {
+            const int hb = k0 & 16;
+            const int l = lane - hb;
+            const bool is_diag = (l >= 0 && l < 16);
+            float rhs = 0.f;
+            if (is_diag) rhs = b - (((gs.red[k & 1][0][l] + gs.red[k & 1][1][l]) + gs.red[k & 1][2][l]) + gs.red[k & 1][3][l]);
+            float acc = 0.f;
+#pragma unroll
+            for (int cp = 0; cp < 16; ++cp) {
+                const float r = __shfl_sync(0xFFFFFFFFu, rhs, hb + cp);
+                acc = fmaf(yinv[cp], r, acc);     // yinv[cp] = Linv[cp][l], zero for cp < l
+            }
+            if (is_diag) x = acc;
+        }
+    }
+    return x;
+}
+
+// The 16x128b tensor-memory shape as the conjugate-gradient solve uses it: thread (g, q) = (lane / 4, lane % 4) of warp w
+// sees rows 32w + g + 8k (k = 0 .. 3) of the matrix at the columns of its class, q + 4j.  One load brings 32 columns by
+// 16 lanes: cur[2j] = (row k = 2h, column 32cb + q + 4j), cur[2j + 1] = (row k = 2h + 1, same column), j = 0 .. 7.
+//
+// Adds alpha0 G + lambda I to the matrix in tensor memory (every column: the products read both triangles).
+// Bq[row * kLdBq + q * kQStride + j] = B[row][q + 4j].
+__device__ __forceinline__ void cg_add_base(uint32_t twarp, const float *Bq, int row0, int q)
+{
+#pragma unroll 2
+    for (int step = 0; step < 8; ++step) {
+        const int h = step & 1, cb = step >> 1;
+        const uint32_t taddr = twarp + ((uint32_t)(h * 16) << 16) + 32 * cb;
+        float cur[16];
+        tmem_ld_16x128b_x8(taddr, cur);
+        const float *b0 = Bq + (row0 + 16 * h) * kLdBq + q * kQStride + 8 * cb, *b1 = b0 + 8 * kLdBq;
+#pragma unroll
+        for (int j4 = 0; j4 < 2; ++j4) {
+            const float4 u = *reinterpret_cast<const float4 *>(b0 + 4 * j4), v = *reinterpret_cast<const float4 *>(b1 + 4 * j4);
+            cur[8 * j4 + 0] += u.x; cur[8 * j4 + 1] += v.x; cur[8 * j4 + 2] += u.y; cur[8 * j4 + 3] += v.y;
+            cur[8 * j4 + 4] += u.z; cur[8 * j4 + 5] += v.z; cur[8 * j4 + 6] += u.w; cur[8 * j4 + 7] += v.w;
+        }
+        tmem_st_16x128b_x8(taddr, cur);
+    }
+    tmem_st_wait();
+}
+
+// Partial sums of the product A v for this thread's four rows over its column class: acc01 = rows k = 0, 1; acc23 =
+// rows k = 2, 3.  The next load is in flight while the current one is multiplied.  vq: the vector by column class,
+// vq[q * kQStride + j] = v[q + 4j].
+__device__ __forceinline__ void cg_matvec(uint32_t twarp, const float *vq, int q, float2 &acc01, float2 &acc23)
+{
+    float a[2][16];
+    float2 vv[8];
+    float2 s01[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, s23[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    tmem_ld_16x128b_x8_nowait(twarp, a[0]);
+#pragma unroll
+    for (int step = 0; step < 8; ++step) {
+        const int h = step & 1, cb = step >> 1;         // lane half (rows k = 2h, 2h + 1), block of 32 columns
+        float (&cur)[16] = a[step & 1];
+        float (&nxt)[16] = a[(step + 1) & 1];
+        if (h == 0) {       // the eight vector entries of this block of columns serve both lane halves
+            const float4 v0 = *reinterpret_cast<const float4 *>(vq + q * kQStride + 8 * cb);
+            const float4 v1 = *reinterpret_cast<const float4 *>(vq + q * kQStride + 8 * cb + 4);
+            vv[0] = make_float2(v0.x, v0.x); vv[1] = make_float2(v0.y, v0.y); vv[2] = make_float2(v0.z, v0.z);
+            vv[3] = make_float2(v0.w, v0.w); vv[4] = make_float2(v1.x, v1.x); vv[5] = make_float2(v1.y, v1.y);
+            vv[6] = make_float2(v1.z, v1.z); vv[7] = make_float2(v1.w, v1.w);
+        }
+        tmem_ld_wait16(cur);
+        if (step + 1 < 8)
+            tmem_ld_16x128b_x8_nowait(twarp + ((uint32_t)(((step + 1) & 1) * 16) << 16) + 32 * ((step + 1) >> 1), nxt);
+        float2 (&dst)[2] = h ? s23 : s01;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            dst[j & 1] = __ffma2_rn(make_float2(cur[2 * j], cur[2 * j + 1]), vv[j], dst[j & 1]);
+    }
+    acc01 = __fadd2_rn(s01[0], s01[1]);
+    acc23 = __fadd2_rn(s23[0], s23[1]);
+}
+
+// Conjugate gradients on (A' + alpha0 G + lambda I) x = b with the matrix in tensor memory (Sec. 4.5: the solver of the
+// paper's results), start x = 0.  The matrix is read through the 16x128b shape: thread (g, q) = (lane / 4, lane % 4) of
+// warp w multiplies rows 32w + g + 8k (k = 0 .. 3) by the vector's entries of its column class q, the four threads of a
+// quad exchange their partial sums so that thread (g, q) ends up with the product's component of row 32w + g + 8q: the
+// row it owns (component of x, r, p and A p).  The vector of the next product goes through shared memory, stored by
+// column class.  One fused reduction per step: the recurrences are arranged so that the product is taken with the
+// residual (w = A r; p and s = A p follow by recurrence), and |r|^2 and r.w are reduced together (warp butterfly, then
+// the four warps in order: a fixed order).  alpha0 G + lambda I is added to the matrix in tensor memory first.
+// Returns true with the owned component of x when
+// |r| <= tol |b|; false when the step limit is reached or a step length is not positive (the matrix is left complete
+// in tensor memory, and the caller solves it directly).
+__device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, const float *Bq, uint32_t twarp, int bar_id,
+                                           int tid, float b, float &x_out, int &matvecs, Probe &pr)
+{
+    const int lane = tid & 31, w = tid >> 5, g = lane >> 2, q = lane & 3;
+    const int own = 32 * w + g + 8 * q;                          // the row this thread owns
+    float *vq = reinterpret_cast<float *>(&gs.pop[0][0]);       // the vector of the next product (the operand tiles are idle)
+    float *red = vq + 4 * kQStride;                              // [4 warps][2]
+    float *vslot = vq + (own & 3) * kQStride + (own >> 2);
+    float x = 0.f, r = b, pdir = 0.f, sdir = 0.f;
+    float rg_old = 0.f, inv_alpha_old = 0.f, bb = 0.f;
+    *vslot = r;
+    cg_add_base(twarp, Bq, 32 * w + g, q);
+    pr.lap(3);
+    group128_sync(bar_id);
+    bool ok = false;
+    int it = 0;
+    for (;; ++it) {
+        float2 acc01, acc23;
+        pr.lap(2);
+        cg_matvec(twarp, vq, q, acc01, acc23);
+        pr.lap(4);
+        // quad exchange: after two rounds thread q holds the sum over the quad of the partial sums of row k = q
+        float wv;
+        {
+            const bool hi = (q & 2) != 0;                           // keeps rows 2, 3 and sends rows 0, 1
+            const float send0 = hi ? acc01.x : acc23.x, send1 = hi ? acc01.y : acc23.y;
+            const float keep0 = hi ? acc23.x : acc01.x, keep1 = hi ? acc23.y : acc01.y;
+            const float t0 = keep0 + __shfl_xor_sync(0xFFFFFFFFu, send0, 2);
+            const float t1 = keep1 + __shfl_xor_sync(0xFFFFFFFFu, send1, 2);
+            const bool odd = (q & 1) != 0;                          // keeps the odd row of its pair
+            const float send = odd ? t0 : t1, keep = odd ? t1 : t0;
+            wv = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+        }
+        float gsum = r * r, dl = r * wv;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, o);
+            dl += __shfl_xor_sync(0xFFFFFFFFu, dl, o);
+        }
+        pr.lap(5);
+        if (lane == 0) *reinterpret_cast<float2 *>(red + 2 * w) = make_float2(gsum, dl);
+        group128_sync(bar_id);
+        pr.lap(6);
+        {
+            const float4 r01 = *reinterpret_cast<const float4 *>(red), r23 = *reinterpret_cast<const float4 *>(red + 4);
+            gsum = ((r01.x + r01.z) + r23.x) + r23.z;
+            dl = ((r01.y + r01.w) + r23.y) + r23.w;
+        }
+        if (it == 0) bb = gsum;
+        if (gsum <= p.cg_tol2 * bb) { ok = true; break; }        // (also b = 0: x = 0)
+        if (it >= p.cg_max_iter) break;
+        const float rg = __fdividef(1.f, gsum);
+        const float beta = gsum * rg_old;                        // 0 at the first step
+        const float inv_alpha = dl * rg - beta * inv_alpha_old;  // p.A p / |r|^2
+        if (!(inv_alpha > 0.f) || !(inv_alpha <= 3.0e38f)) break;
+        const float alpha = __fdividef(1.f, inv_alpha);
+        pdir = fmaf(beta, pdir, r);
+        sdir = fmaf(beta, sdir, wv);
+        x = fmaf(alpha, pdir, x);
+        r = fmaf(-alpha, sdir, r);
+        rg_old = rg;
+        inv_alpha_old = inv_alpha;
+        *vslot = r;
+        group128_sync(bar_id);
+    }
+    // (every thread took the same branch: the reduced values are the same in all of them)
+    matvecs = it + 1;
+    x_out = x;
+    return ok;
+}
+
 // FROM_SUMS: the items are rows whose sums were formed by the chunks kernel (split rows: several chunks, added here
 // in ascending order; long whole rows: one sum each); the group loads them into its accumulator itself, no producer
 // or MMA warp takes part.
-template <bool FROM_SUMS>
-__device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, const float *__restrict__ Bs, int gidx,
+template <bool FROM_SUMS, bool CG, class SmemRows, class GroupSmem>
+__device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, const float *__restrict__ Bs, int gidx,
                                  int tid)
 {
+    static_assert(!(FROM_SUMS && CG), "the rows whose sums come from the chunks kernel are solved directly");
     constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
     const int lane = tid & 31, w = tid >> 5;     // w = lane quarter of tensor memory (= the SM sub-partition)
     const int i = tid;                           // my row of the matrix (= feature index = tensor-memory lane)
-    // Rows are eliminated in index order.  (A cyclic order shifted per group, which spreads the long-lived rows of
-    // the four groups over the four sub-partitions, was measured slower: the trailing columns then wrap around
-    // the end of the accumulator and every update takes two sets of tcgen05.mma instead of one.)
-    const int pos = i;                           // my place in the elimination order
-    const int wpos = pos & ~31;                  // first place of my warp
+    const int wpos = i & ~31;                    // first row of my warp
     const int bar_id = 1 + gidx;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
     const float *Brow = Bs + i * kLdB;
+    constexpr bool use_cg = CG;                           // (then Bs holds alpha0 G + lambda I by column class, see kLdBq)
+    const int own_cg = 32 * w + (lane >> 2) + 8 * (lane & 3);
     uint32_t trail_parity = 0;
-    int64_t it = 0;
-    for (int64_t t = blockIdx.x; t < p.n_items; t += gridDim.x, ++it) {
-        if ((int)(it % kGroups) != gidx) continue;
+    unsigned cg_rows = 0, cg_matvecs = 0;      // thread 0 of the group counts (per block: far below 2^32)
+    Probe pr;
+    pr.start();
+    for (int it = gidx;; it += kGroups) {      // this group's items: every fourth of the block's
+        const int64_t t = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
+        if (t >= p.n_items) break;
         int64_t u, beg, end, slot;
         float b;
         if constexpr (FROM_SUMS) {
@@ -595,7 +1152,7 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             group128_sync(bar_id);
             tc_fence_after();
         } else {
-            item_range<kModeRows>(p, t, u, beg, end, slot);
+            item_range<CG ? kModeRowsCg : kModeRows>(p, t, u, beg, end, slot);
             const uint32_t aph = (uint32_t)((it / kGroups) & 1);
             // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
             if (tid == 0) {
@@ -605,291 +1162,27 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
             group128_sync(bar_id);
             if (gs.stop) break;
             tc_fence_after();
+            pr.lap(1);
             // right-hand side: the four producer warps' partial sums, in order
-            const float *bp = &sm.bpart[it % kBRing][0][i];
+            const float *bp = &sm.bpart[it % Ring<CG ? kModeRowsCg : kModeRows>::kBRing][0][use_cg ? own_cg : i];
             b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
         }
-        float lrow[16];          // my row of my diagonal block's factor (kept for the block inverse at the end)
-        float my_dinv = 0.f;     // 1 / L[i][i]
-#pragma unroll
-        for (int c = 0; c < 16; ++c) lrow[c] = 0.f;
-
-        for (int k = 0; k < D / 16; ++k) {
-            const int k0 = 16 * k;
-            const int ck = k0;                                     // tensor-memory columns of this block
-            float a[16];
-            const bool warp_live = (wpos + 31 >= k0);              // some row of my warp is at or after the block
-            const bool diag_warp = (wpos == (k0 & ~31));
-            auto load_panel = [&]() {
-                tmem_ld16(trow + ck, a);
-#pragma unroll
-                for (int c = 0; c < 16; c += 4) {
-                    const float4 bb = *reinterpret_cast<const float4 *>(Brow + ck + c);
-                    const float2 s01 = __fadd2_rn(make_float2(a[c], a[c + 1]), make_float2(bb.x, bb.y));
-                    const float2 s23 = __fadd2_rn(make_float2(a[c + 2], a[c + 3]), make_float2(bb.z, bb.w));
-                    a[c] = s01.x; a[c + 1] = s01.y; a[c + 2] = s23.x; a[c + 3] = s23.y;
-                }
-            };
-            if (diag_warp) {
-                // the previous step's tensor-core update has landed: only the warp that holds the diagonal block waits
-                // for it (a wait that gives up only sets the group's stop flag; the group leaves together after the
-                // block loop); the other warps follow through the barrier below, at no cost in issue slots
-                if (k > 0) {
-                    if (!mbar_wait_warp(&gs.trail_bar, trail_parity ^ 1u, &sm.abort_flag, 70) && lane == 0) gs.stop = 1;
-                    tc_fence_after();
-                }
-                load_panel();
-            }
-            // (1) diagonal block
-            if (diag_warp) {
-                const int hb = k0 & 16;
-                const int l = lane - hb;      // place relative to the block: < 0 eliminated earlier, 0 .. 15 the block,
-                                              // >= 16 the 16 rows after the block (when it is the first of its warp)
-                const bool is_diag = (l >= 0 && l < 16);
-                float my_inv = 0.f;
-                bool all_ok = true;
-                // Two pivots per round, no masks on the matrix entries: a row that is done only ever overwrites
-                // entries of its upper triangle (never read), and the rows after the block that share this warp get
-                // their forward substitution against the block for free (the same arithmetic in the same order as
-                // the substitution step below, which they then skip).  Only b needs guarding: rows that are done
-                // keep their component of L^-1 b.
-#pragma unroll
-                for (int j = 0; j < 16; j += 2) {
-                    const float p00 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j);
-                    const float p10 = __shfl_sync(0xFFFFFFFFu, a[j], hb + j + 1);
-                    const float p11 = __shfl_sync(0xFFFFFFFFu, a[j + 1], hb + j + 1);
-                    const float bj = __shfl_sync(0xFFFFFFFFu, b, hb + j);
-                    const float bj1 = __shfl_sync(0xFFFFFFFFu, b, hb + j + 1);
-                    // a pivot <= 0 turns into NaN or infinity here and stays visible in 1 / L[row][row] (checked below)
-                    const float inv0 = rsqrt_fast(p00);
-                    const float l10 = p10 * inv0;
-                    const float q11 = fmaf(-l10, l10, p11);
-                    const float inv1 = rsqrt_fast(q11);
-                    const float zj = bj * inv0;
-                    const float zj1 = fmaf(-l10, zj, bj1) * inv1;
-                    const float x0 = a[j] * inv0;                       // L[row][j]   (row j itself: sqrt of the pivot)
-                    const float x1 = fmaf(-x0, l10, a[j + 1]) * inv1;   // L[row][j+1] (row j+1 itself: sqrt of the second pivot)
-                    a[j] = x0;
-                    a[j + 1] = x1;
-                    my_inv = (l == j) ? inv0 : ((l == j + 1) ? inv1 : my_inv);
-                    const float bdown = fmaf(-x1, zj1, fmaf(-x0, zj, b));
-                    b = (l > j + 1) ? bdown : ((l == j + 1) ? zj1 : ((l == j) ? zj : b));
-                    // the two new columns go through shared memory (shuffles are the slower path for 2 x 14 values)
-                    float *xb = &gs.xch[(j & 2) * 16];
-                    if (is_diag) { xb[l] = x0; xb[16 + l] = x1; }
-                    __syncwarp();
-                    float c0[16], c1[16];
-#pragma unroll
-                    for (int q4 = (j + 2) / 4; q4 < 4; ++q4) {
-                        const float4 u4 = *reinterpret_cast<const float4 *>(&xb[4 * q4]);
-                        const float4 v4 = *reinterpret_cast<const float4 *>(&xb[16 + 4 * q4]);
-                        c0[4 * q4] = u4.x; c0[4 * q4 + 1] = u4.y; c0[4 * q4 + 2] = u4.z; c0[4 * q4 + 3] = u4.w;
-                        c1[4 * q4] = v4.x; c1[4 * q4 + 1] = v4.y; c1[4 * q4 + 2] = v4.z; c1[4 * q4 + 3] = v4.w;
-                    }
-#pragma unroll
-                    for (int c = j + 2; c < 16; c += 2) {
-                        float2 r = __ffma2_rn(make_float2(-x0, -x0), make_float2(c0[c], c0[c + 1]), make_float2(a[c], a[c + 1]));
-                        r = __ffma2_rn(make_float2(-x1, -x1), make_float2(c1[c], c1[c + 1]), r);
-                        a[c] = r.x;
-                        a[c + 1] = r.y;
-                    }
-                }
-                all_ok = __all_sync(0xFFFFFFFFu, !is_diag || (my_inv > 0.f && my_inv <= 3.0e38f));
-                if (!all_ok && lane == 0) gs.bad = 1;
-                if (is_diag) {
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float v = (c <= l) ? a[c] : 0.f;
-                        gs.Lt[c][l] = v;
-                        lrow[c] = v;
-                    }
-                    gs.dinv[l] = my_inv;
-                    gs.z[l] = b;
-                    my_dinv = my_inv;
-                }
-            }
-            tc_fence_before();
-            group128_sync(bar_id);
-            if (warp_live && !diag_warp) {
-                tc_fence_after();
-                load_panel();
-            }
-            // (2) rows after the block: forward substitution, split, operand tiles
-            if (pos >= k0 + 16) {
-              if (wpos != (k0 & ~31)) {      // (the rows after the block in its own warp are already done, see above)
-                float dv[16];
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const float4 v = *reinterpret_cast<const float4 *>(&gs.dinv[4 * q4]);
-                    dv[4 * q4] = v.x; dv[4 * q4 + 1] = v.y; dv[4 * q4 + 2] = v.z; dv[4 * q4 + 3] = v.w;
-                }
-                // column-oriented: once a[pp] is final it is eliminated from the later entries, which are
-                // independent of each other
-#pragma unroll
-                for (int pp = 0; pp < 16; ++pp) {
-                    float lt[16];
-#pragma unroll
-                    for (int q4 = (pp + 1) / 4; q4 < 4; ++q4) {
-                        const float4 v = *reinterpret_cast<const float4 *>(&gs.Lt[pp][4 * q4]);
-                        lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
-                    }
-                    a[pp] *= dv[pp];
-                    // packed FP32 FMAs on pairs of columns: half the issue slots, which the chains of the other
-                    // groups on this sub-partition need
-                    const float mneg = -a[pp];
-                    if ((pp + 1) & 1) a[pp + 1] = fmaf(mneg, lt[pp + 1], a[pp + 1]);
-#pragma unroll
-                    for (int c = (pp + 2) & ~1; c < 16; c += 2) {
-                        const float2 r = __ffma2_rn(make_float2(mneg, mneg), make_float2(lt[c], lt[c + 1]), make_float2(a[c], a[c + 1]));
-                        a[c] = r.x;
-                        a[c + 1] = r.y;
-                    }
-                }
-                float2 acc2 = make_float2(0.f, 0.f);
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const float4 zz = *reinterpret_cast<const float4 *>(&gs.z[4 * q4]);
-                    acc2 = __ffma2_rn(make_float2(a[4 * q4], a[4 * q4 + 1]), make_float2(zz.x, zz.y), acc2);
-                    acc2 = __ffma2_rn(make_float2(a[4 * q4 + 2], a[4 * q4 + 3]), make_float2(zz.z, zz.w), acc2);
-                }
-                b -= acc2.x + acc2.y;
-              }
-                uint32_t w1[8], w2[8], w3[8];
-#pragma unroll
-                for (int c = 0; c < 16; c += 2) {
-                    // part 1 rounds to nearest (one packed conversion); parts 2 and 3 keep the leading 8 bits of
-                    // what is left, so p1 + p2 + p3 = p up to 2^-24
-                    const __nv_bfloat162 hpair = __floats2bfloat162_rn(a[c], a[c + 1]);
-                    const uint32_t hw = *reinterpret_cast<const uint32_t *>(&hpair);
-                    // (packed arithmetic: x - y as fma(y, -1, x) on both lanes; the upper halves of two words are
-                    // gathered by one byte permutation)
-                    const float2 minus1 = make_float2(-1.f, -1.f);
-                    const float2 r = __ffma2_rn(make_float2(__uint_as_float(hw << 16), __uint_as_float(hw & 0xFFFF0000u)), minus1,
-                                                make_float2(a[c], a[c + 1]));
-                    const uint32_t m0 = __float_as_uint(r.x) & 0xFFFF0000u, m1 = __float_as_uint(r.y) & 0xFFFF0000u;
-                    const float2 sres = __ffma2_rn(make_float2(__uint_as_float(m0), __uint_as_float(m1)), minus1, r);
-                    w1[c >> 1] = hw;
-                    w2[c >> 1] = __byte_perm(m0, m1, 0x7632);
-                    w3[c >> 1] = __byte_perm(__float_as_uint(sres.x), __float_as_uint(sres.y), 0x7632);
-                }
-                const uint32_t roff = (uint32_t)((i >> 3) * 256 + (i & 7) * 16);
-                const uint32_t b1 = smem_u32(&gs.pop[0][0]) + roff, b2 = smem_u32(&gs.pop[1][0]) + roff,
-                               b3 = smem_u32(&gs.pop[2][0]) + roff;
-                st_shared_v4(b1, w1[0], w1[1], w1[2], w1[3]); st_shared_v4(b1 + 128, w1[4], w1[5], w1[6], w1[7]);
-                st_shared_v4(b2, w2[0], w2[1], w2[2], w2[3]); st_shared_v4(b2 + 128, w2[4], w2[5], w2[6], w2[7]);
-                st_shared_v4(b3, w3[0], w3[1], w3[2], w3[3]); st_shared_v4(b3 + 128, w3[4], w3[5], w3[6], w3[7]);
-                fence_proxy_async();
-            }
-            if (warp_live) {
-                tmem_st16(trow + ck, a);      // L (rows before the block rewrite what they read)
-                tmem_st_wait();
-            }
-            tc_fence_before();
-            group128_sync(bar_id);
-            // (3) trailing update on the tensor core.  The issuing thread changes with the step: lane 0 of the warp two
-            // blocks of 32 rows further on (cyclically), which never holds the next diagonal block.  It
-            // issues the update and commits it to the group's mbarrier (a tcgen05.mma takes the issuing thread about
-            // 50 cycles); the next step's diagonal warp waits for it.
-            const bool issuer = (lane == 0) && (wpos == ((k0 + 16 + 64) & 96));
-            uint64_t da[3] = {0, 0, 0};
-            const uint32_t d_base = sm.tmem_base + gidx * kAccStride;
-            // columns [c_lo, c_lo + n) of the matrix (= panel rows c_lo ..) -= P P^T restricted to them
-            auto update = [&](int c_lo, int n) {
-                const uint32_t idesc = idesc_bf16_k_major_negA(128, n);
-                uint64_t db[3];
-#pragma unroll
-                for (int q = 0; q < 3; ++q) db[q] = smem_desc(smem_u32(&gs.pop[q][0]) + (uint32_t)(c_lo * 32), 128, 256, 0);
-                umma_f16(d_base + c_lo, da[0], db[0], idesc, true);
-                umma_f16(d_base + c_lo, da[0], db[1], idesc, true);
-                umma_f16(d_base + c_lo, da[1], db[0], idesc, true);
-                umma_f16(d_base + c_lo, da[0], db[2], idesc, true);
-                umma_f16(d_base + c_lo, da[2], db[0], idesc, true);
-                umma_f16(d_base + c_lo, da[1], db[1], idesc, true);
-            };
-            if (k < D / 16 - 1 && issuer) {
-                tc_fence_after();
-#pragma unroll
-                for (int q = 0; q < 3; ++q) da[q] = smem_desc(smem_u32(&gs.pop[q][0]), 128, 256, 0);
-                // all trailing columns in one set of six instructions: the tensor pipe takes about 50 cycles per
-                // instruction whatever its width, and it is shared by the four groups and the gather
-                update(k0 + 16, D - k0 - 16);
-                umma_commit(&gs.trail_bar);
-            }
-            if (k < D / 16 - 1) trail_parity ^= 1u;
-        }
-        group128_sync(bar_id);
-        if (gs.stop) break;
-        // my column of the inverse of my diagonal block.  The eight blocks go through shared memory, in the operand
-        // tiles: every trailing update has completed (the last one was waited for before the last block step).
-        float yinv[16];
-        {
-            float *Lall = reinterpret_cast<float *>(&gs.pop[0][0]);      // [8 blocks][16][16], transposed
-            float *dall = Lall + 8 * 256;                                 // [128] reciprocals of the diagonal
-            float *Lb = Lall + (pos >> 4) * 256;
-            const int l = pos & 15;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) Lb[c * 16 + l] = lrow[c];
-            dall[pos] = my_dinv;
-            __syncwarp();
-            const float *dvb = dall + (pos & ~15);
-            float tacc[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) tacc[c] = 0.f;
-#pragma unroll
-            for (int cp = 0; cp < 16; ++cp) {
-                // y[cp] of the solve L y = e_l
-                const float ycp = (cp < l) ? 0.f : ((cp == l) ? dvb[cp] : -tacc[cp] * dvb[cp]);
-                yinv[cp] = ycp;
-                float lt[16];
-#pragma unroll
-                for (int q4 = (cp + 1) / 4; q4 < 4; ++q4) {
-                    const float4 v = *reinterpret_cast<const float4 *>(&Lb[cp * 16 + 4 * q4]);
-                    lt[4 * q4] = v.x; lt[4 * q4 + 1] = v.y; lt[4 * q4 + 2] = v.z; lt[4 * q4 + 3] = v.w;
-                }
-                if ((cp + 1) & 1) tacc[cp + 1] = fmaf(lt[cp + 1], ycp, tacc[cp + 1]);
-#pragma unroll
-                for (int c = (cp + 2) & ~1; c < 16; c += 2) {
-                    const float2 r = __ffma2_rn(make_float2(lt[c], lt[c + 1]), make_float2(ycp, ycp), make_float2(tacc[c], tacc[c + 1]));
-                    tacc[c] = r.x;
-                    tacc[c + 1] = r.y;
-                }
-            }
-        }
-        // (4) back substitution L^T x = z; b now holds z_i
         float x = 0.f;
-        for (int k = D / 16 - 1; k >= 0; --k) {
-            const int k0 = 16 * k;
-            const int ck = k0;
-            float wv[16];
-            if (wpos + 31 >= k0 + 16) {
-                tmem_ld16(trow + ck, wv);
-                const float xm = (pos >= k0 + 16) ? x : 0.f;
-#pragma unroll
-                for (int c = 0; c < 16; c += 2) {
-                    const float2 r = __fmul2_rn(make_float2(wv[c], wv[c + 1]), make_float2(xm, xm));
-                    wv[c] = (pos >= k0 + 16) ? r.x : 0.f;
-                    wv[c + 1] = (pos >= k0 + 16) ? r.y : 0.f;
-                }
-                warp_reduce16(wv, lane);
-            } else {
-                wv[0] = 0.f;
+        int own = i;                  // the row whose solution this thread holds at the end
+        bool solved = true;
+        if constexpr (CG) {
+            int matvecs = 0;
+            solved = cg_in_tmem(p, gs, Bs, sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride, bar_id, tid, b, x,
+                                matvecs, pr);
+            own = own_cg;
+            if (tid == 0) {
+                ++cg_rows;
+                cg_matvecs += matvecs;
+                if (!solved) p.fallback_list[atomicAdd(p.fallback_count, 1ull)] = (int32_t)u;    // left to the direct solve
             }
-            if ((lane & 1) == 0) gs.red[k & 1][w][lane >> 1] = wv[0];
-            group128_sync(bar_id);
-            if (wpos == (k0 & ~31)) {
-                const int hb = k0 & 16;
-                const int l = lane - hb;
-                const bool is_diag = (l >= 0 && l < 16);
-                float rhs = 0.f;
-                if (is_diag) rhs = b - (((gs.red[k & 1][0][l] + gs.red[k & 1][1][l]) + gs.red[k & 1][2][l]) + gs.red[k & 1][3][l]);
-                float acc = 0.f;
-#pragma unroll
-                for (int cp = 0; cp < 16; ++cp) {
-                    const float r = __shfl_sync(0xFFFFFFFFu, rhs, hb + cp);
-                    acc = fmaf(yinv[cp], r, acc);     // yinv[cp] = Linv[cp][l], zero for cp < l
-                }
-                if (is_diag) x = acc;
-            }
+        } else {
+            x = chol_in_tmem(sm, gs, Brow, trow, sm.tmem_base + gidx * kAccStride, bar_id, tid, b, true, trail_parity);
+            if (gs.stop) break;
         }
         // tensor memory is free again for the next item of this accumulator
         tc_fence_before();
@@ -897,28 +1190,49 @@ __device__ void solver_rows_tmem(const Params &p, Smem &sm, RowGroupSmem &gs, co
         if (!FROM_SUMS && tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
         const bool ok = gs.bad == 0;
         const float xo = ok ? x : 0.f;
-        reinterpret_cast<__nv_bfloat16 *>(p.out.table)[u * D + i] = __float2bfloat16_rn(xo);
-        if (p.out.cap_slot) {
-            const int cs = p.out.cap_slot[u];
-            if (cs >= 0) p.out.cap_out[(int64_t)cs * D + i] = xo;
+        if (solved) {
+            reinterpret_cast<__nv_bfloat16 *>(p.out.table)[u * D + own] = __float2bfloat16_rn(xo);
+            if (p.out.cap_slot) {
+                const int cs = p.out.cap_slot[u];
+                if (cs >= 0) p.out.cap_out[(int64_t)cs * D + own] = xo;
+            }
         }
         if (!ok && tid == 0) {
             atomicAdd(&p.st->not_spd, 1ull);
             raise_flag(p.st, kFlagNotSpd, u);
         }
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
+        pr.lap(7);
+    }
+#ifdef ALX_PROBE
+    if (tid == 0 && p.cg_counters)
+        for (int k = 0; k < 8; ++k) atomicAdd(&p.cg_counters[8 + k], (unsigned long long)pr.acc[k]);
+#endif
+    if (tid == 0 && cg_rows && p.cg_counters) {
+        atomicAdd(&p.cg_counters[0], (unsigned long long)cg_rows);
+        atomicAdd(&p.cg_counters[1], (unsigned long long)cg_matvecs);
     }
 }
 
 
 
+// The conjugate-gradient variant runs 24 warps: the 21 of the roles and three idle ones that complete the last
+// warpgroup, so that registers can move between warpgroups (setmaxnreg): the four producer warps form one warpgroup
+// (64 registers per thread), the MMA warp and the idle warps the next (32), and the solver warps take 96 (their
+// matrix-vector product holds two loads of 16 matrix entries, 8 duplicated vector entries and four packed sums).
+template <int MODE> constexpr int block_threads() { return MODE == kModeRowsCg ? 768 : Cfg<MODE>::kBlockThreads; }
+
 template <int MODE>
-__global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p, const __grid_constant__ CUtensorMap tmap)
+__global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, const __grid_constant__ CUtensorMap tmap)
 {
     using C = Cfg<MODE>;
-    if (MODE == kModeRows && p.dual_flag && *p.dual_flag) {
-        p.n_items = p.n_items_primal;
+    constexpr bool CG = MODE == kModeRowsCg;
+    if (MODE == kModeRows && p.item_count) {
+        p.n_items = (int64_t)*p.item_count;                 // the rows conjugate gradients left over
         if ((int64_t)blockIdx.x >= p.n_items) return;      // block-uniform, before any barrier or allocation
+    } else if (is_rows(MODE) && p.dual_flag && *p.dual_flag) {
+        p.n_items = p.n_items_primal;
+        if ((int64_t)blockIdx.x >= p.n_items) return;
     }
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled stages; plain offset arithmetic on the shared array, so that the
@@ -927,7 +1241,8 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p, 
     constexpr int kNStage = Ring<MODE>::kNStage;
     SmemT<MODE> &sm = *reinterpret_cast<SmemT<MODE> *>(aligned);
     float *Bs = reinterpret_cast<float *>(aligned + sizeof(SmemT<MODE>));
-    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(SmemT<MODE>) + sizeof(float) * D * kLdB);
+    using GroupSmem = typename std::conditional<CG, CgGroupSmem, RowGroupSmem>::type;
+    GroupSmem *rgs = reinterpret_cast<GroupSmem *>(aligned + sizeof(SmemT<MODE>) + sizeof(float) * D * kLdBq);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
@@ -937,21 +1252,33 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p, 
         mbar_fence_init();
     }
     // label tiles start finite (all zero): rows beyond an item's end multiply zeros, never stale NaNs
-    for (int k = tid; k < (int)sizeof(sm.y) / 16; k += C::kBlockThreads)
+    constexpr int kThreads = block_threads<MODE>();
+    for (int k = tid; k < (int)sizeof(sm.y) / 16; k += kThreads)
         st_shared_zero16(smem_u32(&sm.y[0][0]) + k * 16);
-    for (int k = tid; k < (int)sizeof(sm.h) / 16; k += C::kBlockThreads)
+    for (int k = tid; k < (int)sizeof(sm.h) / 16; k += kThreads)
         st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
-    if (MODE == kModeRows) {
-        for (int e = tid; e < D * D; e += C::kBlockThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
+    if constexpr (CG) {
+        for (int e = tid; e < D * D; e += kThreads)
+            Bs[(e >> 7) * kLdBq + (e & 3) * kQStride + ((e & (D - 1)) >> 2)] = p.Bmat[e];
+    } else if constexpr (MODE == kModeRows) {
+        for (int e = tid; e < D * D; e += kThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
         for (int g = 0; g < C::kGroups; ++g) {
             if (tid == 0) mbar_init(&rgs[g].trail_bar, 1);
-            for (int k = tid; k < 3 * D * 32 / 16; k += C::kBlockThreads)
+            for (int k = tid; k < 3 * D * 32 / 16; k += kThreads)
                 st_shared_zero16(smem_u32(&rgs[g].pop[0][0]) + k * 16);
         }
         if (tid == 0) mbar_fence_init();
     }
     fence_proxy_async();
-    if (warp == C::kMmaWarp) {
+    // Roles by warp.  The conjugate-gradient variant puts the producers (one warpgroup), then the MMA warp with three idle
+    // warps (the next warpgroup), in front of the sixteen solver warps: the warp scheduler favours low warp numbers when
+    // several warps are ready, and the few instructions of the roles that feed the solvers must not queue behind them.
+    // `rw` is the warp's number in the order solvers, MMA / producers as the other modes have it.
+    constexpr int kMmaWarp = CG ? C::kFirstProducerWarp + C::kProducers - 1 : C::kMmaWarp;      // CG: after the producers
+    constexpr int kFirstProducerWarp = CG ? C::kMmaWarp : C::kFirstProducerWarp;
+    const int rw = CG ? (warp < 8 ? warp + C::kMmaWarp : warp - 8) : warp;
+    const int rtid = rw * 32 + lane;
+    if (rw == kMmaWarp) {
         tmem_alloc(&sm.tmem_base, kTmemCols);
         tmem_relinquish();
     }
@@ -959,20 +1286,25 @@ __global__ void __launch_bounds__(Cfg<MODE>::kBlockThreads, 1) k_umma(Params p, 
     __syncthreads();
     tc_fence_after();
 
-    if (warp < C::kMmaWarp) {
-        const int gidx = warp / (C::kGroupThreads / 32);
-        if constexpr (MODE == kModeRows) solver_rows_tmem<false>(p, sm, rgs[gidx], Bs, gidx, tid - gidx * C::kGroupThreads);
-        else copyout_role<MODE>(p, sm, gidx, tid - gidx * C::kGroupThreads);
-    } else if (warp == C::kMmaWarp) {
+    if (rw < C::kMmaWarp) {
+        const int gidx = rw / (C::kGroupThreads / 32);
+        if constexpr (CG) setmaxnreg_inc<96>();
+        if constexpr (is_rows(MODE)) solver_rows_tmem<false, CG>(p, sm, rgs[gidx], Bs, gidx, rtid - gidx * C::kGroupThreads);
+        else copyout_role<MODE>(p, sm, gidx, rtid - gidx * C::kGroupThreads);
+    } else if (CG && rw > kMmaWarp) {
+        setmaxnreg_dec<32>();       // idle warps of the last warpgroup
+    } else if (rw == kMmaWarp) {
+        if constexpr (CG) setmaxnreg_dec<32>();
         mma_role<MODE>(p, sm, lane);
     } else {
-        if constexpr (MODE == kModeRows) producer_role<MODE>(p, sm, warp - C::kFirstProducerWarp, lane);
-        else stream_producer_role<MODE>(p, &tmap, sm, warp - C::kFirstProducerWarp, lane);
+        if constexpr (CG) setmaxnreg_dec<64>();
+        if constexpr (is_rows(MODE)) producer_role<MODE, CG>(p, sm, rw - kFirstProducerWarp, lane);
+        else stream_producer_role<MODE>(p, &tmap, sm, rw - kFirstProducerWarp, lane);
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == C::kMmaWarp) {
+    if (rw == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(sm.tmem_base, kTmemCols);
     }
@@ -1000,7 +1332,7 @@ __global__ void __launch_bounds__(4 * 128, 1) k_solve_sums(Params p)
     unsigned char *aligned = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     Smem &sm = *reinterpret_cast<Smem *>(aligned);
     float *Bs = reinterpret_cast<float *>(aligned + sizeof(Smem));
-    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(Smem) + sizeof(float) * D * kLdB);
+    RowGroupSmem *rgs = reinterpret_cast<RowGroupSmem *>(aligned + sizeof(Smem) + sizeof(float) * D * kLdBq);
     const int tid = threadIdx.x, warp = tid >> 5;
     if (tid == 0) sm.abort_flag = 0;
     for (int e = tid; e < D * D; e += blockDim.x) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
@@ -1017,7 +1349,7 @@ __global__ void __launch_bounds__(4 * 128, 1) k_solve_sums(Params p)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    solver_rows_tmem<true>(p, sm, rgs[warp >> 2], Bs, warp >> 2, tid & 127);
+    solver_rows_tmem<true, false>(p, sm, rgs[warp >> 2], Bs, warp >> 2, tid & 127);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -1032,10 +1364,13 @@ template <int MODE> size_t smem_bytes()
     // a large request in every mode (more than half of what an SM offers): at most one block per SM, so two
     // blocks never compete for the SM's 512 tensor-memory columns
     size_t b = sizeof(SmemT<MODE>) + 1024;
-    if (MODE == kModeRows) b += sizeof(float) * D * kLdB + kMaxGroups * sizeof(RowGroupSmem);
+    if (MODE == kModeRows) b += sizeof(float) * D * kLdBq + kMaxGroups * sizeof(RowGroupSmem);
+    if (MODE == kModeRowsCg) b += sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem);
     return b;
 }
 static_assert(sizeof(SmemT<1>) + 1024 <= 232448 && sizeof(SmemT<1>) > 116224, "ring depth of the streaming modes");
+static_assert(sizeof(SmemT<0>) + 1024 + sizeof(float) * D * kLdBq + kMaxGroups * sizeof(RowGroupSmem) <= 232448, "rows mode");
+static_assert(sizeof(SmemT<3>) + 1024 + sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem) <= 232448, "rows mode, CG");
 
 // Tensor map of a bfloat16 table [n x 128] for row gathers: boxes of one row by 64 features (128 bytes), 128-byte swizzle.
 // (The encoder is a driver entry point, looked up through the runtime so that the library needs no driver at link time.)
@@ -1071,7 +1406,7 @@ template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStrea
     CUtensorMap tm;
     e = table_tensor_map(p.X, p.n_table, &tm);
     if (e != cudaSuccess) return e;
-    k_umma<MODE><<<grid, Cfg<MODE>::kBlockThreads, smem, s>>>(p, tm);
+    k_umma<MODE><<<grid, block_threads<MODE>(), smem, s>>>(p, tm);
     return cudaGetLastError();
 }
 
@@ -1104,7 +1439,7 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows,
                              const void *X, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
                              cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
-                             const void *dual_ws, int64_t n_table)
+                             const void *dual_ws, int64_t n_table, const CgOptions &cg)
 {
     const int sms = sm_count();
     Params p{};
@@ -1150,11 +1485,27 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
     if (n_whole > 0) {
         p.n_items = n_whole;
         p.last_item = offs[c_long] - 1;
+        p.solver = cg.enabled ? 1 : 0;
+        p.cg_max_iter = cg.max_iter;
+        p.cg_tol2 = cg.tol * cg.tol;
+        p.cg_counters = cg.counters;
+        p.fallback_list = cg.fallback_list;
+        p.fallback_count = cg.counters + 2;
+        const int grid = (int)(n_whole < sms ? n_whole : sms);
         if (main_begin) cudaEventRecord(main_begin, s);
-        e = launch_mode<kModeRows>(p, (int)(n_whole < sms ? n_whole : sms), s);
-        if (main_end) cudaEventRecord(main_end, s);
+        e = cg.enabled ? launch_mode<kModeRowsCg>(p, grid, s) : launch_mode<kModeRows>(p, grid, s);
         ++*launches;
         if (e != cudaSuccess) return e;
+        if (cg.enabled) {
+            // the rows conjugate gradients did not finish (none, as a rule: the blocks then return at once)
+            p.item_list = cg.fallback_list;
+            p.item_count = cg.counters + 2;
+            p.dual_flag = nullptr;
+            e = launch_mode<kModeRows>(p, grid, s);
+            ++*launches;
+            if (e != cudaSuccess) return e;
+        }
+        if (main_end) cudaEventRecord(main_end, s);
     }
     const int64_t n_zero = offs[1] - offs[0];
     if (n_zero > 0) {

@@ -10,9 +10,9 @@ pytestmark = pytest.mark.gpu
 ROWS, COLS = 0, 1
 
 
-def make_ctx(p, kernels=0):
+def make_ctx(p, kernels=0, **kw):
     from paper_2112_02194_b200 import Alx
-    a = Alx(p.n_rows, p.n_cols, p.d, p.lam, p.alpha, storage=p.storage, split=p.split, kernels=kernels)
+    a = Alx(p.n_rows, p.n_cols, p.d, p.lam, p.alpha, storage=p.storage, split=p.split, kernels=kernels, **kw)
     a.set_csr(p.rowptr, p.colidx, p.values)
     a.set_embeddings(ROWS, p.W0)
     a.set_embeddings(COLS, p.H0)
@@ -352,6 +352,75 @@ def test_dual_form_steps_aside_when_base_matrix_is_ill_conditioned():
     assert np.linalg.cond(p.alpha * G + p.lam * np.eye(p.d)) > 1e4
     worst = 0.0
     for n in range(0, ids.size, 7):
+        A, b = ials.row_system(p.rowptr, p.colidx, None, H0r, G, p.alpha, p.lam, int(ids[n]))
+        worst = max(worst, np.linalg.norm(A @ x32[n] - b) / np.linalg.norm(b))
+    assert worst <= 1e-4, worst
+
+
+def _whole_rows(p):
+    """rows of 33 .. 1024 observations: the ones the whole-rows tensor-core kernel solves"""
+    deg = np.diff(p.rowptr)
+    return np.nonzero((deg >= 33) & (deg <= 1024))[0].astype(np.int64)
+
+
+@pytest.mark.parametrize("name", ["local_d128_bf16", "long_labels_d128_bf16"])
+def test_conjugate_gradient_solve_meets_the_gates_and_tracks_the_oracle(name):
+    """Sec. 4.5: conjugate gradients (the default solve of the whole-rows tensor-core kernel), started at 0 and
+    stopped at |r| <= 1e-5 |b|.  Judged by the residual of the fp32 solution and its distance to the exact row update;
+    the number of products is compared with the oracle's textbook iteration (the iterates themselves are unpinned)."""
+    p = _problem(name)
+    ids = _whole_rows(p)
+    assert ids.size > 200
+    H0 = p.f64(p.H0)
+    G = ials.gramian(H0)
+    vals64 = None if p.values is None else p.values.astype(np.float64)
+    sols, stats = {}, {}
+    for label, kw in (("cg", dict()), ("chol", dict(solver=1)), ("fallback", dict(cg_max_iter=2))):
+        a = make_ctx(p, **kw)
+        sols[label] = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+        stats[label] = a.get_stats()
+        assert stats[label].not_spd == 0
+        a.destroy()
+    assert stats["cg"].cg_rows == ids.size and stats["cg"].cg_fallbacks == 0
+    assert stats["chol"].cg_rows == 0
+    assert stats["fallback"].cg_rows == ids.size and stats["fallback"].cg_fallbacks > 0.9 * ids.size
+    _, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G, return_raw=True)
+    _, _, o_iters = ials.half_step_cg(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G,
+                                     tol=1e-5, max_iter=48)
+    # products = steps + 1 (the product of the step at which convergence is seen); fp32 may need a step more or less
+    mean_products = stats["cg"].cg_products / stats["cg"].cg_rows
+    assert abs(mean_products - (o_iters.mean() + 1)) <= 1.0, (mean_products, o_iters.mean())
+    for label in ("cg", "chol", "fallback"):
+        assert rel_fro(sols[label], W_raw) <= 1e-4, label
+        assert row_rel(sols[label], W_raw).max() <= 1e-3, label
+    worst = 0.0
+    for n in range(0, ids.size, 3):
+        A, b = ials.row_system(p.rowptr, p.colidx, vals64, H0, G, p.alpha, p.lam, int(ids[n]))
+        for label in ("cg", "fallback"):
+            worst = max(worst, np.linalg.norm(A @ sols[label][n] - b) / np.linalg.norm(b))
+    assert worst <= 1e-4, worst
+
+
+def test_conjugate_gradients_hand_over_ill_conditioned_rows_to_cholesky():
+    """alpha0 G + lambda I with a condition number of about 4e4: conjugate gradients do not reach 1e-5 within the step
+    limit, so those rows must come out of the Cholesky solve, and meet the residual gate all the same."""
+    from synth import graphs
+    p = _problem("local_d128_bf16")
+    rng = np.random.Generator(np.random.PCG64(78))
+    H0 = 0.05 + 0.002 * rng.standard_normal((p.n_cols, p.d))
+    p.H0 = graphs.to_storage_bits(H0, p.storage)
+    p.alpha, p.lam = 0.5, 0.01
+    ids = _whole_rows(p)
+    a = make_ctx(p)
+    x32 = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+    st = a.get_stats()
+    a.destroy()
+    # (the dual form steps aside on this matrix, so the rows of at most 32 observations take the same route)
+    assert st.not_spd == 0 and st.cg_rows >= ids.size and 0 < st.cg_fallbacks <= st.cg_rows
+    H0r = p.f64(p.H0)
+    G = ials.gramian(H0r)
+    worst = 0.0
+    for n in range(0, ids.size, 5):
         A, b = ials.row_system(p.rowptr, p.colidx, None, H0r, G, p.alpha, p.lam, int(ids[n]))
         worst = max(worst, np.linalg.norm(A @ x32[n] - b) / np.linalg.norm(b))
     assert worst <= 1e-4, worst
