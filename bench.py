@@ -246,7 +246,7 @@ def run_ours(args, w):
     t_gen = time.perf_counter() - t_gen
 
     a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0), solver=args.solver,
-            cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol)
+            cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol, cg_start=args.cg_start)
     t_set = time.perf_counter()
     a.set_csr(rowptr, colidx)
     torch.cuda.synchronize()
@@ -377,7 +377,7 @@ def run_ours(args, w):
         o_W = torch.empty_like(h_W, pin_memory=True)
         o_H = torch.empty_like(h_H, pin_memory=True)
         b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0), solver=args.solver,
-                cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol)
+                cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol, cg_start=args.cg_start)
         reps = 2 if w["name"] != "small" else 3
         times = []
         for r in range(reps):
@@ -437,6 +437,8 @@ def main():
     ap.add_argument("--solver", type=int, default=0, choices=[0, 1],
                     help="alx_options.solver: 0 = conjugate gradients where available (Cholesky otherwise), 1 = Cholesky")
     ap.add_argument("--cg-max-iter", type=int, default=0, help="alx_options.cg_max_iter (0 = the library's default)")
+    ap.add_argument("--cg-start", type=int, default=0, choices=[0, 1],
+                    help="alx_options.cg_start: 0 = the stored embedding, 1 = zero")
     ap.add_argument("--cg-tol", type=float, default=0.0, help="alx_options.cg_tol (0 = the library's default)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")

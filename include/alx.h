@@ -48,6 +48,7 @@ typedef enum { ALX_ROWS = 0, ALX_COLS = 1 } alx_side; /* which table is SOLVED; 
 typedef enum { ALX_F32 = 0, ALX_BF16 = 1 } alx_dtype;
 
 typedef enum { ALX_SOLVER_AUTO = 0, ALX_SOLVER_CHOLESKY = 1 } alx_solver;
+typedef enum { ALX_CG_START_STORED = 0, ALX_CG_START_ZERO = 1 } alx_cg_start;
 #define ALX_DEFAULT_CG_MAX_ITER 48
 #define ALX_DEFAULT_CG_TOL 1e-5f
 
@@ -80,12 +81,15 @@ typedef struct alx_options {
                                 every row in the primal form */
     int32_t solver;          /* how the d x d system of Eq. 4 is solved (Sec. 4.5 compares the choices):
                                 ALX_SOLVER_AUTO (0): conjugate gradients where the library has them (the whole-rows
-                                tensor-core kernel), started at x = 0 and stopped at |r| <= cg_tol |b|; a row that has not
+                                tensor-core kernel), started as cg_start says and stopped at |r| <= cg_tol |b|; a row that has not
                                 converged after cg_max_iter steps, and every row elsewhere, is solved by Cholesky.
                                 ALX_SOLVER_CHOLESKY (1): Cholesky for every row */
     int32_t cg_max_iter;     /* 0 => ALX_DEFAULT_CG_MAX_ITER */
     float cg_tol;            /* 0 => ALX_DEFAULT_CG_TOL; at most 1e-2 */
-    int32_t reserved;
+    int32_t cg_start;        /* start vector of the conjugate gradients (the paper states none): ALX_CG_START_STORED (0): the
+                                row's embedding as stored in the table being solved (close to the solution once training
+                                is under way; costs one product for r = b - A x0, and falls back to zero when |r| > |b|);
+                                ALX_CG_START_ZERO (1): x = 0, so that a row's work does not depend on the table's history */
 } alx_options;
 
 typedef struct alx_stats {

@@ -222,9 +222,11 @@ void release_matrix(alx_ctx *c)
 
 bool tensor_path(const alx_ctx *c) { return c->bf16 && c->opt.d == 128 && c->opt.kernels != 1; }
 bool dual_form(const alx_ctx *c) { return tensor_path(c) && c->opt.kernels == 0; }
-CgOptions cg_options(const alx_ctx *c)
+CgOptions cg_options(const alx_ctx *c, int solved_side)
 {
     CgOptions o;
+    // the start vector of a row is its stored embedding once that table holds something (set by the caller or solved)
+    o.warm_start = c->opt.cg_start == ALX_CG_START_STORED && c->have_table[solved_side];
     o.enabled = c->opt.solver == ALX_SOLVER_AUTO;
     o.max_iter = c->opt.cg_max_iter > 0 ? c->opt.cg_max_iter : ALX_DEFAULT_CG_MAX_ITER;
     o.tol = c->opt.cg_tol > 0.f ? c->opt.cg_tol : ALX_DEFAULT_CG_TOL;
@@ -264,7 +266,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
                                      &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed],
-                                     cg_options(c)));
+                                     cg_options(c, side)));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
         c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;
@@ -310,6 +312,7 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
     if ((opt->alloc == nullptr) != (opt->free == nullptr)) return ALX_ERR_INVALID_ARG;
     if (opt->split != 0 && opt->split < 16) return ALX_ERR_INVALID_ARG;
     if (opt->solver != ALX_SOLVER_AUTO && opt->solver != ALX_SOLVER_CHOLESKY) return ALX_ERR_INVALID_ARG;
+    if (opt->cg_start != ALX_CG_START_STORED && opt->cg_start != ALX_CG_START_ZERO) return ALX_ERR_INVALID_ARG;
     if (opt->cg_max_iter < 0 || opt->cg_max_iter > 1024 || !(opt->cg_tol >= 0.f) || opt->cg_tol > 1e-2f) return ALX_ERR_INVALID_ARG;
     int dev = opt->device;
     if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return ALX_ERR_CUDA;

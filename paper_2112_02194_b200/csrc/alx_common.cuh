@@ -145,6 +145,7 @@ struct CgOptions {
     bool enabled;
     int max_iter;                  // a row that has not converged by then is solved by the in-place Cholesky instead
     float tol;                     // stop at |r| <= tol |b|
+    bool warm_start;               // start from the row's stored embedding (the solved table holds trained values)
     unsigned long long *counters;  // device, [3]: rows, matrix-vector products, rows that fell back
     int32_t *fallback_list;        // device, one entry per row of the larger side: the rows left to the Cholesky solve
 };

@@ -42,10 +42,9 @@ constexpr int kStageRows = 32;
 // streaming modes (chunks, Gramian) use that space for a deeper ring, which is what keeps HBM busy
 // (and stages of 64 gathered rows instead of 32: half the per-stage waits and commits of the MMA thread)
 template <int MODE> struct Ring {
-    static constexpr int kRows = (MODE == 0 || MODE == 3) ? 32 : 64;   // gathered rows per stage
-    // (the conjugate-gradient rows kernel needs no operand tiles for a factorisation: their space deepens its ring,
-    // and a gather is bound by latency times bytes in flight)
-    static constexpr int kNStage = (MODE == 0) ? 8 : ((MODE == 3) ? 13 : 12);
+    static constexpr int kRows = (MODE == 0) ? 32 : 64;   // gathered rows per stage
+    // (the conjugate-gradient rows kernel needs no operand tiles for a factorisation: their space goes to its ring)
+    static constexpr int kNStage = (MODE == 0 || MODE == 3) ? 8 : 12;
     static constexpr int kHalfBytes = kRows * 128;        // one 64-feature half of a stage
     static constexpr int kStageHBytes = 2 * kHalfBytes;
     static constexpr int kStageYBytes = 2 * kRows * 16;   // label tile, two 8-column chunks
@@ -69,6 +68,20 @@ enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2, kModeRowsCg = 3 };
 __host__ __device__ constexpr bool is_rows(int mode) { return mode == kModeRows || mode == kModeRowsCg; }
 
 // Development aid (-DALX_PROBE): thread 0 of every solver group sums clock cycles per phase into cg_counters[3 ..].
+#ifdef ALX_PROBE
+// event trace of block 0: g_trace[role][item][event] = clock64 at the event (items kTraceFirst .. kTraceFirst + 15 of the block)
+constexpr int kTraceFirst = 64;
+__device__ unsigned long long g_trace[8][16][16];
+__device__ __forceinline__ void trace_ev(int role, long long item, int ev)
+{
+    if (blockIdx.x == 0 && item >= kTraceFirst && item < kTraceFirst + 16 && ev < 16)
+        g_trace[role][item - kTraceFirst][ev] = (unsigned long long)clock64();
+}
+#define TRACE(role, item, ev) trace_ev(role, item, ev)
+#else
+#define TRACE(role, item, ev)
+#endif
+
 struct Probe {
 #ifdef ALX_PROBE
     long long t0 = 0, acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -92,7 +105,10 @@ template <int MODE> struct Cfg {
     // are summed in a fixed order); streaming modes: four producer warps, each fills whole stages of its own by TMA
     // row gathers
     static constexpr int kProducers = is_rows(MODE) ? kProducerWarps : 4;
-    static constexpr int kFullArrivals = is_rows(MODE) ? kProducerWarps : 1;
+    static constexpr int kFullArrivals = (MODE == kModeRows) ? kProducerWarps : 1;
+    // a stage is free again when the tensor core has read it -- and, in the conjugate-gradient rows kernel, when the
+    // producer warp that gathered it has summed y x over its rows
+    static constexpr int kEmptyArrivals = (MODE == kModeRowsCg) ? 2 : 1;
     static constexpr int kBlockThreads = kSolverThreads + 32 + kProducers * 32;
 };
 
@@ -120,6 +136,7 @@ struct Params {
     int solver;                  // rows mode: 0 = in-place Cholesky, 1 = conjugate gradients
     int cg_max_iter;             // conjugate gradients: steps after which a row goes to the Cholesky solve instead
     float cg_tol2;               // conjugate gradients: stop at |r|^2 <= cg_tol2 |b|^2
+    int cg_warm;                 // conjugate gradients: start from the row's stored embedding instead of zero
     unsigned long long *cg_counters;   // [3]: rows solved by conjugate gradients, their matrix-vector products, rows that fell back
 };
 
@@ -157,14 +174,18 @@ template <int MODE> struct __align__(1024) SmemT {
     unsigned char h[kNStage][Ring<MODE>::kStageHBytes];
     unsigned char y[is_rows(MODE) ? 1 : kNStage][Ring<MODE>::kStageYBytes];      // label tiles (chunks mode only)
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
+    uint64_t rhs_done[MODE == kModeRowsCg ? Ring<MODE>::kBRing : 1];   // conjugate-gradient rows kernel: an item's right-hand side is written
     uint32_t tmem_base;
     int abort_flag;
-    // rows mode: the producer warps also sum y x_i of the rows they staged (four partial sums per item)
-    float ylab[kNStage][kStageRows];          // labels of the staged rows
+    // rows modes: the producer warps also sum y x_i of the rows they staged.  kModeRows: the four warps share every stage
+    // (four partial sums per item); kModeRowsCg: a warp gathers whole items (one sum per item)
+    static constexpr int kRhsParts = (MODE == kModeRowsCg) ? 1 : kProducerWarps;
+    float ylab[kNStage][Ring<MODE>::kRows];      // labels of the staged rows
     int stage_meta[kNStage];                     // K steps of the stage (1 or 2) | 4 if it ends its item; -1: no more work
-    int rows_staged[kProducerWarps][kNStage];    // per producer warp: how many of its 8 rows of the stage are defined
-    int last_of_item[kProducerWarps][kNStage];   // per producer warp: 1 + ring index of the item whose last stage this is, else 0
-    alignas(16) float bpart[is_rows(MODE) ? Ring<MODE>::kBRing : 1][kProducerWarps][D];
+    int rows_staged[kProducerWarps][kNStage];    // kModeRows, per producer warp: how many of its 8 rows of the stage are defined
+    int last_of_item[kProducerWarps][kNStage];   // kModeRows, per producer warp: 1 + ring index of the item whose last stage this is, else 0
+    int own_queue[kProducerWarps][kNStage];      // kModeRowsCg, per producer warp: its stages in flight (slot, rows, last-of-item mark)
+    alignas(16) float bpart[is_rows(MODE) ? Ring<MODE>::kBRing : 1][kRhsParts][D];
 };
 
 template <int MODE> __device__ __forceinline__ void item_range(const Params &p, int64_t t, int64_t &u, int64_t &beg,
@@ -378,6 +399,199 @@ template <int MODE, bool PARK> __device__ void producer_role(const Params &p, Sm
 #endif
 }
 
+// Producer of the conjugate-gradient rows kernel.  Producer warp pw gathers every fourth item of the block, whole: all its
+// stages of 64 rows, by TMA row gathers (four rows of one 64-feature half per instruction, written with the 128-byte
+// swizzle the tensor core reads; lanes 0 .. 15 issue them, the stage's mbarrier counts the bytes, rows past the item's end
+// take a row coordinate past the end of the table and are filled with zeros).  The four warps thus work on four items at
+// a time: what bounds a gather of short rows is the chain of loads, waits and hand-overs per stage, and four chains run
+// side by side.  Every warp walks all items (their offsets come in windows of 32) to number the stages: stage g of the
+// block sits in slot g mod ring, whichever warp fills it; the MMA warp takes the stages in that order.
+// Stages are ISSUED in order too: a warp issues stage g after stage g - 1 has been issued (a counter in shared memory
+// passes the turn).  An mbarrier tells its phases apart by parity only; a warp that jumped ahead by a lap of the ring
+// would take a slot's release of two laps ago for the one it needs.  With the turn, the slot of stage g is in one of two
+// states when its warp looks: stage g - ring released, or not yet.  The turn covers only the wait for the slot and the
+// copy instructions; the index loads before and the sums after run in parallel.
+// Once a stage has landed its warp adds the rows' y x to the item's right-hand side and releases the slot (a slot is
+// free again after the tensor core and that warp are done with it); after an item's last stage it publishes the sum
+// and arrives on the item's right-hand-side barrier, which the solver group waits for.
+template <int MODE>
+__device__ void producer_role_items(const Params &p, const CUtensorMap *tmap, SmemT<MODE> &sm, int pw, int lane)
+{
+    constexpr int kNStage = Ring<MODE>::kNStage, kRows = Ring<MODE>::kRows, kBRing = Ring<MODE>::kBRing;
+    static_assert(kRows == 64, "two rows per lane, sixteen groups of four rows");
+    const int32_t past_end = (int32_t)p.n_table;
+    volatile int *turn = &sm.stage_meta[0];  // stages issued so far by the four warps together
+    int g_run = 0;                           // stages of the items walked so far (the same count in every warp)
+    int head = 0, tail = 0;                  // this warp's stages handed over / issued
+    uint32_t q_parity = 0;                   // bit k: parity of the `full` phase of this warp's stage number k (modulo 32)
+    float bacc[4] = {0.f, 0.f, 0.f, 0.f};
+    bool alive = true;
+    ItemWindow win;
+    const int f = 4 * lane;                  // this lane's four features in the sums of y x
+    const int fhalf = f >> 6, fcc = (f & 63) >> 3, finner = (f & 7) * 2;
+    // the oldest stage of this warp not handed over yet has landed (the caller made sure): sum y x over its rows, release it
+    auto hand_over = [&]() {
+        const int e = sm.own_queue[pw][head % kNStage];
+        const int slot = e & 0xFF, nrows = (e >> 8) & 0xFF, last = e >> 16;
+        // every lane reads the copied rows, so every lane observes the completed phase itself
+        for (int k = 0; k < 64 && !mbar_test_wait(&sm.full[slot], (q_parity >> (head & 31)) & 1u); ++k) { }
+        const unsigned char *base = &sm.h[slot][0] + fhalf * Ring<MODE>::kHalfBytes;
+        if (p.sv.val) {
+#pragma unroll 4
+            for (int j = 0; j < nrows; ++j) {
+                const uint2 v = *reinterpret_cast<const uint2 *>(base + j * 128 + ((fcc ^ (j & 7)) << 4) + finner);
+                const float y = sm.ylab[slot][j];
+                bacc[0] = fmaf(y, __uint_as_float(v.x << 16), bacc[0]);
+                bacc[1] = fmaf(y, __uint_as_float(v.x & 0xFFFF0000u), bacc[1]);
+                bacc[2] = fmaf(y, __uint_as_float(v.y << 16), bacc[2]);
+                bacc[3] = fmaf(y, __uint_as_float(v.y & 0xFFFF0000u), bacc[3]);
+            }
+        } else {        // every label is 1: eight rows (one 1024-byte group of the tile) per trip, loads first
+            for (int j0 = 0; j0 < nrows; j0 += 8) {
+                uint2 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = *reinterpret_cast<const uint2 *>(base + (j0 + j) * 128 + ((fcc ^ j) << 4) + finner);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    bacc[0] += __uint_as_float(v[j].x << 16);
+                    bacc[1] += __uint_as_float(v[j].x & 0xFFFF0000u);
+                    bacc[2] += __uint_as_float(v[j].y << 16);
+                    bacc[3] += __uint_as_float(v[j].y & 0xFFFF0000u);
+                }
+            }
+        }
+        if (last) {
+            *reinterpret_cast<float4 *>(&sm.bpart[last - 1][0][f]) = make_float4(bacc[0], bacc[1], bacc[2], bacc[3]);
+            bacc[0] = bacc[1] = bacc[2] = bacc[3] = 0.f;
+        }
+        __syncwarp();
+        if (lane == 0) {
+            if (last) mbar_arrive(&sm.rhs_done[last - 1]);
+            mbar_arrive(&sm.empty[slot]);
+        }
+        ++head;
+    };
+    // has this warp's oldest stage in flight landed?  (lane 0 looks, the warp follows)
+    auto oldest_landed = [&]() {
+        int yes = 0;
+        if (lane == 0)
+            yes = mbar_test_wait(&sm.full[sm.own_queue[pw][head % kNStage] & 0xFF], (q_parity >> (head & 31)) & 1u) ? 1 : 0;
+        return __shfl_sync(0xFFFFFFFFu, yes, 0) != 0;
+    };
+    auto wait_oldest = [&]() {
+        return mbar_wait_parked_warp(&sm.full[sm.own_queue[pw][head % kNStage] & 0xFF], (q_parity >> (head & 31)) & 1u,
+                                     &sm.abort_flag, 20);
+    };
+    int64_t it = 0;
+    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
+        if ((it & 31) == 0) win.load(p, it, lane);
+        int64_t beg, end;
+        win.get((int)(it & 31), beg, end);
+        const int nst = (int)((end - beg + kRows - 1) / kRows);
+        const int g0 = g_run;
+        g_run += nst;
+        if ((int)(it & 3) != pw) continue;
+        // ids and labels of a stage's rows: this lane's two rows (lane and 32 + lane), fetched one stage ahead
+        int32_t nxt_idx[2];
+        float nxt_y[2];
+        auto fetch_ids = [&](int64_t e0) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int64_t e = e0 + 32 * k + lane;
+                nxt_idx[k] = past_end;
+                nxt_y[k] = 0.f;
+                if (e < end) {
+                    nxt_idx[k] = p.sv.idx[e];
+                    nxt_y[k] = p.sv.val ? p.sv.val[e] : 1.f;
+                }
+            }
+        };
+        fetch_ids(beg);
+        for (int s = 0; s < nst && alive; ++s) {
+            const int g = g0 + s;
+            const int64_t e0 = beg + (int64_t)s * kRows;
+            const int slot = g % kNStage;
+            const uint32_t ph = (uint32_t)((g / kNStage) & 1);
+            const int32_t my_idx[2] = {nxt_idx[0], nxt_idx[1]};
+            const float my_y[2] = {nxt_y[0], nxt_y[1]};
+            if (s + 1 < nst) fetch_ids(e0 + kRows);
+            if (lane == 0) TRACE(5, it, 0 + 5 * s);
+            // (1) wait for the turn; the hand-overs fill the wait (one stage at a time, the turn is looked at first: while this
+            // warp holds the turn the other three wait for it)
+            for (uint32_t spin = 0;; ++spin) {
+                int mine = 0;
+                if (lane == 0) mine = (*turn >= g) ? 1 : 0;
+                if (__shfl_sync(0xFFFFFFFFu, mine, 0)) break;
+                if (head < tail && oldest_landed()) {
+                    hand_over();
+                    spin = 0;
+                    continue;
+                }
+                if (spin > (1u << 22) || ((spin & 63u) == 63u && sm.abort_flag)) {
+                    if (lane == 0 && sm.abort_flag == 0) sm.abort_flag = 12;
+                    alive = false;
+                    break;
+                }
+                if (spin > 8u) __nanosleep(spin < 128u ? 64u : 256u);
+            }
+            if (!alive) break;
+            if (lane == 0) TRACE(5, it, 1 + 5 * s);
+            // (2) the slot: stage g - ring must have been released.  While it is not, this warp's own stages in flight go
+            // first (their release may be what the ring's turn-over waits for), then the warp waits suspended.
+            for (;;) {
+                int free_now = 0;
+                if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
+                if (__shfl_sync(0xFFFFFFFFu, free_now, 0)) break;
+                if (head < tail) {
+                    if (!wait_oldest()) { alive = false; break; }
+                    hand_over();
+                } else {
+                    if (!mbar_wait_parked_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10)) alive = false;
+                    break;
+                }
+            }
+            if (!alive) break;
+            if (lane == 0) TRACE(5, it, 2 + 5 * s);
+            // (3) issue the stage and pass the turn on
+            const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
+            const int rc16 = (rc + 15) & ~15;
+            if (p.sv.val) {
+                sm.ylab[slot][lane] = my_y[0];
+                sm.ylab[slot][32 + lane] = my_y[1];
+            }
+            if (lane == 0) sm.own_queue[pw][tail % kNStage] = slot | (rc16 << 8) | ((s + 1 == nst) ? ((1 + (int)(it % kBRing)) << 16) : 0);
+            q_parity = (q_parity & ~(1u << (tail & 31))) | (ph << (tail & 31));
+            // rows 4 * lane .. 4 * lane + 3 of the stage (lanes 0 .. 15)
+            int32_t r4[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int32_t v0 = __shfl_sync(0xFFFFFFFFu, my_idx[0], (4 * lane + j) & 31);
+                const int32_t v1 = __shfl_sync(0xFFFFFFFFu, my_idx[1], (4 * lane + j) & 31);
+                r4[j] = (lane < 8) ? v0 : v1;
+            }
+            __syncwarp();
+            const int ngroups = rc16 >> 2;        // groups of four rows the tensor core will read
+            if (lane == 0) mbar_arrive_expect_tx(&sm.full[slot], (uint32_t)ngroups * 1024u);
+            if (lane < ngroups) {
+                const uint32_t dst = smem_u32(&sm.h[slot][0]) + lane * 512;
+                tma_gather4(dst, tmap, 0, r4[0], r4[1], r4[2], r4[3], &sm.full[slot]);
+                tma_gather4(dst + Ring<MODE>::kHalfBytes, tmap, 64, r4[0], r4[1], r4[2], r4[3], &sm.full[slot]);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence_block();
+                *turn = g + 1;
+                TRACE(5, it, 3 + 5 * s);
+            }
+            ++tail;
+        }
+    }
+    while (alive && head < tail) {
+        if (!wait_oldest()) break;
+        hand_over();
+    }
+}
+
 // Streaming modes (chunks, Gramian pieces): producer warp pw fills the stages whose running number is pw modulo the
 // number of producer warps, whole stages of 64 rows each.  The rows come by TMA row gathers (four rows of one
 // 64-feature half per instruction, written with the 128-byte swizzle the tensor core reads), issued by lanes 0 .. 15 for
@@ -454,67 +668,85 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
     constexpr uint32_t kIdescMain = idesc_bf16_mn_major(128, 128);
     constexpr uint32_t kIdescY = idesc_bf16_mn_major(128, 16);
     const uint32_t tmem = sm.tmem_base;
-    int64_t it = 0;
     int slot = 0;             // ring position and phase of the next stage
     uint32_t ph = 0;
     bool alive = true;
-    Probe pr;
-    pr.start();
-    ItemWindow win;
-    for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
-        int64_t u, beg, end, slot_unused;
-        if constexpr (is_rows(MODE)) {
-            if ((it & 31) == 0) win.load(p, it, lane);
-            win.get((int)(it & 31), beg, end);
-        } else {
-            item_range<MODE>(p, t, u, beg, end, slot_unused);
-        }
-        const int a = (int)(it % Cfg<MODE>::kGroups);
-        const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
-        pr.lap(7);
-        if (!mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
+    // one stage: wait for it, issue its K steps of 16 rows, release it when they have completed
+    auto stage = [&](uint32_t d_main, int nk, bool &first, long long item, int s) -> bool {
+        if (lane == 0 && MODE == kModeRowsCg) TRACE(0, item, 2 + 3 * s);
+        if (!(MODE == kModeRowsCg ? mbar_wait_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)
+                                  : mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE))) return false;
         tc_fence_after();
-        pr.lap(1);
-        const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
-        bool first = true;
-        for (int64_t e0 = beg; e0 < end; e0 += kRows) {
-            pr.lap(0);
-            if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) { alive = false; break; }
-            tc_fence_after();
-            pr.lap(2);
-            const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
-            const int nk = (rc + 15) >> 4;
-            pr.lap(0);
-            if (lane == 0) {
-                const uint32_t hb = smem_u32(&sm.h[slot][0]);
-                const uint32_t yb = smem_u32(&sm.y[slot][0]);
-                for (int ks = 0; ks < nk; ++ks) {
-                    // 16 gathered rows = two groups of 8 rows of 128 bytes; halves are kHalfBytes apart
-                    const uint64_t adesc = smem_desc(hb + ks * 2048, Ring<MODE>::kHalfBytes, 1024, 2);
-                    umma_f16(d_main, adesc, adesc, kIdescMain, !first);
-                    if (MODE == kModeChunks) {
-                        const uint64_t ydesc = smem_desc(yb + ks * 256, 128, kRows * 16, 0);
-                        umma_f16(d_main + D, adesc, ydesc, kIdescY, !first);
-                    }
-                    first = false;
+        if (lane == 0 && MODE == kModeRowsCg) TRACE(0, item, 3 + 3 * s);
+        if (lane == 0) {
+            const uint32_t hb = smem_u32(&sm.h[slot][0]);
+            const uint32_t yb = smem_u32(&sm.y[slot][0]);
+            for (int ks = 0; ks < nk; ++ks) {
+                // 16 gathered rows = two groups of 8 rows of 128 bytes; halves are kHalfBytes apart
+                const uint64_t adesc = smem_desc(hb + ks * 2048, Ring<MODE>::kHalfBytes, 1024, 2);
+                umma_f16(d_main, adesc, adesc, kIdescMain, !first);
+                if (MODE == kModeChunks) {
+                    const uint64_t ydesc = smem_desc(yb + ks * 256, 128, kRows * 16, 0);
+                    umma_f16(d_main + D, adesc, ydesc, kIdescY, !first);
                 }
-                pr.lap(3);
-                umma_commit(&sm.empty[slot]);
-                pr.lap(4);
+                first = false;
             }
-            if (++slot == kNStage) { slot = 0; ph ^= 1u; }
+            umma_commit(&sm.empty[slot]);
+            if (MODE == kModeRowsCg) TRACE(0, item, 4 + 3 * s);
         }
-        pr.lap(0);
-        if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
-        pr.lap(5);
-        __syncwarp();
-        pr.lap(6);
+        if (++slot == kNStage) { slot = 0; ph ^= 1u; }
+        return true;
+    };
+    if constexpr (is_rows(MODE)) {
+        // rows modes: all this warp needs of an item is its number of stages and the K steps of the last one; they come
+        // for 32 items at a time, one item per lane (the offsets hang on a chain of dependent loads, see ItemWindow)
+        const int n_mine = (int)((p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x);      // items of this block
+        int info = 0;
+        for (int it = 0; it < n_mine && alive; ++it) {
+            if ((it & 31) == 0) {
+                ItemWindow win;
+                win.load(p, it, lane);
+                const int len = (int)(win.end - win.beg);
+                const int nst = (len + kRows - 1) / kRows;
+                const int tail_rows = len - (nst - 1) * kRows;
+                info = (nst << 8) | ((tail_rows + 15) >> 4);
+            }
+            const int mine = __shfl_sync(0xFFFFFFFFu, info, it & 31);
+            const int nst = mine >> 8, nk_last = mine & 0xFF;
+            const int a = it % Cfg<MODE>::kGroups;
+            const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
+            if (lane == 0 && MODE == kModeRowsCg) TRACE(0, it, 0);
+            if (!(MODE == kModeRowsCg ? mbar_wait_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)
+                                      : mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE))) break;
+            tc_fence_after();
+            if (lane == 0 && MODE == kModeRowsCg) TRACE(0, it, 1);
+            const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
+            bool first = true;
+            for (int s = 0; s < nst; ++s)
+                if (!stage(d_main, s + 1 < nst ? kRows / 16 : nk_last, first, it, s)) { alive = false; break; }
+            if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
+            if (lane == 0 && MODE == kModeRowsCg) TRACE(0, it, 15);
+            __syncwarp();
+        }
+    } else {
+        int64_t it = 0;
+        for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
+            int64_t u, beg, end, slot_unused;
+            item_range<MODE>(p, t, u, beg, end, slot_unused);
+            const int a = (int)(it % Cfg<MODE>::kGroups);
+            const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
+            if (!mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
+            tc_fence_after();
+            const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
+            bool first = true;
+            for (int64_t e0 = beg; e0 < end; e0 += kRows) {
+                const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
+                if (!stage(d_main, (rc + 15) >> 4, first, it, 0)) { alive = false; break; }
+            }
+            if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
+            __syncwarp();
+        }
     }
-#ifdef ALX_PROBE
-    pr.lap(0);
-    if (lane == 0 && p.cg_counters)
-        for (int k = 0; k < 8; ++k) atomicAdd(&p.cg_counters[16 + k], (unsigned long long)pr.acc[k]);
-#endif
 }
 
 template <int MODE>
@@ -1007,7 +1239,8 @@ __device__ __forceinline__ void cg_matvec(uint32_t twarp, const float *vq, int q
 }
 
 // Conjugate gradients on (A' + alpha0 G + lambda I) x = b with the matrix in tensor memory (Sec. 4.5: the solver of the
-// paper's results), start x = 0.  The matrix is read through the 16x128b shape: thread (g, q) = (lane / 4, lane % 4) of
+// paper's results).  Start: x = 0, or (cg_warm) the row's stored embedding x0 -- one more product for r = b - A x0, taken
+// back to x = 0 when |r| > |b|.  The matrix is read through the 16x128b shape: thread (g, q) = (lane / 4, lane % 4) of
 // warp w multiplies rows 32w + g + 8k (k = 0 .. 3) by the vector's entries of its column class q, the four threads of a
 // quad exchange their partial sums so that thread (g, q) ends up with the product's component of row 32w + g + 8q: the
 // row it owns (component of x, r, p and A p).  The vector of the next product goes through shared memory, stored by
@@ -1018,54 +1251,77 @@ __device__ __forceinline__ void cg_matvec(uint32_t twarp, const float *vq, int q
 // |r| <= tol |b|; false when the step limit is reached or a step length is not positive (the matrix is left complete
 // in tensor memory, and the caller solves it directly).
 __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, const float *Bq, uint32_t twarp, int bar_id,
-                                           int tid, float b, float &x_out, int &matvecs, Probe &pr)
+                                           int tid, float b, float x0, float &x_out, int &matvecs, Probe &pr)
 {
     const int lane = tid & 31, w = tid >> 5, g = lane >> 2, q = lane & 3;
     const int own = 32 * w + g + 8 * q;                          // the row this thread owns
-    float *vq = reinterpret_cast<float *>(&gs.pop[0][0]);       // the vector of the next product (the operand tiles are idle)
-    float *red = vq + 4 * kQStride;                              // [4 warps][2]
+    float *vq = reinterpret_cast<float *>(&gs.pop[0][0]);       // the vector of the next product
+    float *red = vq + 4 * kQStride;                              // [4 warps][4]
     float *vslot = vq + (own & 3) * kQStride + (own >> 2);
-    float x = 0.f, r = b, pdir = 0.f, sdir = 0.f;
+    // product with the vector in shared memory; this thread's component of the result
+    auto product = [&]() {
+        float2 acc01, acc23;
+        cg_matvec(twarp, vq, q, acc01, acc23);
+        // quad exchange: after two rounds thread q holds the sum over the quad of the partial sums of row k = q
+        const bool hi = (q & 2) != 0;                           // keeps rows 2, 3 and sends rows 0, 1
+        const float send0 = hi ? acc01.x : acc23.x, send1 = hi ? acc01.y : acc23.y;
+        const float keep0 = hi ? acc23.x : acc01.x, keep1 = hi ? acc23.y : acc01.y;
+        const float t0 = keep0 + __shfl_xor_sync(0xFFFFFFFFu, send0, 2);
+        const float t1 = keep1 + __shfl_xor_sync(0xFFFFFFFFu, send1, 2);
+        const bool odd = (q & 1) != 0;                          // keeps the odd row of its pair
+        const float send = odd ? t0 : t1, keep = odd ? t1 : t0;
+        return keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+    };
+    bool warm = p.cg_warm != 0;
+    float x = warm ? x0 : 0.f, r = b, pdir = 0.f, sdir = 0.f;
     float rg_old = 0.f, inv_alpha_old = 0.f, bb = 0.f;
-    *vslot = r;
+    int products = 0;
+    *vslot = warm ? x0 : b;
     cg_add_base(twarp, Bq, 32 * w + g, q);
     pr.lap(3);
     group128_sync(bar_id);
+    if (warm) {                 // r = b - A x0
+        r = b - product();
+        ++products;
+        group128_sync(bar_id);  // every thread has read the vector
+        *vslot = r;
+        group128_sync(bar_id);
+    }
     bool ok = false;
-    int it = 0;
-    for (;; ++it) {
-        float2 acc01, acc23;
+    for (int it = 0;; ++it) {
         pr.lap(2);
-        cg_matvec(twarp, vq, q, acc01, acc23);
+        const float wv = product();
+        ++products;
         pr.lap(4);
-        // quad exchange: after two rounds thread q holds the sum over the quad of the partial sums of row k = q
-        float wv;
-        {
-            const bool hi = (q & 2) != 0;                           // keeps rows 2, 3 and sends rows 0, 1
-            const float send0 = hi ? acc01.x : acc23.x, send1 = hi ? acc01.y : acc23.y;
-            const float keep0 = hi ? acc23.x : acc01.x, keep1 = hi ? acc23.y : acc01.y;
-            const float t0 = keep0 + __shfl_xor_sync(0xFFFFFFFFu, send0, 2);
-            const float t1 = keep1 + __shfl_xor_sync(0xFFFFFFFFu, send1, 2);
-            const bool odd = (q & 1) != 0;                          // keeps the odd row of its pair
-            const float send = odd ? t0 : t1, keep = odd ? t1 : t0;
-            wv = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
-        }
-        float gsum = r * r, dl = r * wv;
+        float gsum = r * r, dl = r * wv, bsum = b * b;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, o);
             dl += __shfl_xor_sync(0xFFFFFFFFu, dl, o);
+            if (it == 0) bsum += __shfl_xor_sync(0xFFFFFFFFu, bsum, o);
         }
         pr.lap(5);
-        if (lane == 0) *reinterpret_cast<float2 *>(red + 2 * w) = make_float2(gsum, dl);
+        if (lane == 0) *reinterpret_cast<float4 *>(red + 4 * w) = make_float4(gsum, dl, bsum, 0.f);
         group128_sync(bar_id);
         pr.lap(6);
         {
-            const float4 r01 = *reinterpret_cast<const float4 *>(red), r23 = *reinterpret_cast<const float4 *>(red + 4);
-            gsum = ((r01.x + r01.z) + r23.x) + r23.z;
-            dl = ((r01.y + r01.w) + r23.y) + r23.w;
+            const float4 r0 = *reinterpret_cast<const float4 *>(red), r1 = *reinterpret_cast<const float4 *>(red + 4),
+                         r2 = *reinterpret_cast<const float4 *>(red + 8), r3 = *reinterpret_cast<const float4 *>(red + 12);
+            gsum = ((r0.x + r1.x) + r2.x) + r3.x;
+            dl = ((r0.y + r1.y) + r2.y) + r3.y;
+            if (it == 0) bb = ((r0.z + r1.z) + r2.z) + r3.z;
         }
-        if (it == 0) bb = gsum;
+        if (it == 0 && warm && !(gsum <= bb)) {
+            // the start vector is further from the solution than zero is (tables not trained yet): start again from zero
+            warm = false;
+            x = 0.f;
+            r = b;
+            group128_sync(bar_id);
+            *vslot = r;
+            group128_sync(bar_id);
+            it = -1;
+            continue;
+        }
         if (gsum <= p.cg_tol2 * bb) { ok = true; break; }        // (also b = 0: x = 0)
         if (it >= p.cg_max_iter) break;
         const float rg = __fdividef(1.f, gsum);
@@ -1082,8 +1338,8 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
         *vslot = r;
         group128_sync(bar_id);
     }
-    // (every thread took the same branch: the reduced values are the same in all of them)
-    matvecs = it + 1;
+    // (every thread took the same branches: the reduced values are the same in all of them)
+    matvecs = products;
     x_out = x;
     return ok;
 }
@@ -1113,7 +1369,7 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
         const int64_t t = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
         if (t >= p.n_items) break;
         int64_t u, beg, end, slot;
-        float b;
+        float b, x0 = 0.f;
         if constexpr (FROM_SUMS) {
             int64_t c0, c1;      // the row's sums: slots c0 .. c1 - 1 of the workspace
             if (t < p.n_split_rows) {
@@ -1153,27 +1409,42 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
             tc_fence_after();
         } else {
             item_range<CG ? kModeRowsCg : kModeRows>(p, t, u, beg, end, slot);
+            if constexpr (CG) {       // the start vector: the row's stored embedding (read before the wait for the sums)
+                if (p.cg_warm) x0 = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(p.out.table)[u * D + own_cg]);
+            }
             const uint32_t aph = (uint32_t)((it / kGroups) & 1);
             // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
             if (tid == 0) {
-                gs.stop = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60) ? 0 : 1;
+                TRACE(1 + gidx, it, 0);
+                bool ok = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60);
+                TRACE(1 + gidx, it, 1);
+                if constexpr (CG) {       // (the right-hand side follows the stages' landing on a barrier of its own)
+                    constexpr int kBRing = Ring<kModeRowsCg>::kBRing;
+                    ok = ok && mbar_wait_parked(&sm.rhs_done[it % kBRing], (uint32_t)((it / kBRing) & 1), &sm.abort_flag, 61);
+                }
+                TRACE(1 + gidx, it, 2);
+                gs.stop = ok ? 0 : 1;
                 gs.bad = 0;
             }
             group128_sync(bar_id);
             if (gs.stop) break;
             tc_fence_after();
+            if (tid == 0) TRACE(1 + gidx, it, 3);
             pr.lap(1);
-            // right-hand side: the four producer warps' partial sums, in order
-            const float *bp = &sm.bpart[it % Ring<CG ? kModeRowsCg : kModeRows>::kBRing][0][use_cg ? own_cg : i];
-            b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
+            if constexpr (CG) {
+                b = sm.bpart[it % Ring<kModeRowsCg>::kBRing][0][own_cg];
+            } else {      // right-hand side: the four producer warps' partial sums, in order
+                const float *bp = &sm.bpart[it % Ring<kModeRows>::kBRing][0][i];
+                b = ((bp[0] + bp[D]) + bp[2 * D]) + bp[3 * D];
+            }
         }
         float x = 0.f;
         int own = i;                  // the row whose solution this thread holds at the end
         bool solved = true;
         if constexpr (CG) {
             int matvecs = 0;
-            solved = cg_in_tmem(p, gs, Bs, sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride, bar_id, tid, b, x,
-                                matvecs, pr);
+            solved = cg_in_tmem(p, gs, Bs, sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride, bar_id, tid, b, x0,
+                                x, matvecs, pr);
             own = own_cg;
             if (tid == 0) {
                 ++cg_rows;
@@ -1185,9 +1456,11 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
             if (gs.stop) break;
         }
         // tensor memory is free again for the next item of this accumulator
+        if (CG && tid == 0) TRACE(1 + gidx, it, 4);
         tc_fence_before();
         group128_sync(bar_id);
         if (!FROM_SUMS && tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
+        if (CG && tid == 0) TRACE(1 + gidx, it, 5);
         const bool ok = gs.bad == 0;
         const float xo = ok ? x : 0.f;
         if (solved) {
@@ -1202,6 +1475,7 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
             raise_flag(p.st, kFlagNotSpd, u);
         }
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
+        if (CG && tid == 0) TRACE(1 + gidx, it, 6);
         pr.lap(7);
     }
 #ifdef ALX_PROBE
@@ -1246,9 +1520,11 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int s = 0; s < kNStage; ++s) { mbar_init(&sm.full[s], C::kFullArrivals); mbar_init(&sm.empty[s], 1); }
+        for (int s = 0; s < kNStage; ++s) { mbar_init(&sm.full[s], C::kFullArrivals); mbar_init(&sm.empty[s], C::kEmptyArrivals); }
+        if (CG) for (int s = 0; s < Ring<MODE>::kBRing; ++s) mbar_init(&sm.rhs_done[s], 1);
         for (int a = 0; a < kMaxGroups; ++a) { mbar_init(&sm.acc_full[a], 1); mbar_init(&sm.acc_empty[a], 1); }
         sm.abort_flag = 0;
+        sm.stage_meta[0] = 0;      // (conjugate-gradient rows kernel: the producers' turn counter)
         mbar_fence_init();
     }
     // label tiles start finite (all zero): rows beyond an item's end multiply zeros, never stale NaNs
@@ -1298,7 +1574,8 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
         mma_role<MODE>(p, sm, lane);
     } else {
         if constexpr (CG) setmaxnreg_dec<64>();
-        if constexpr (is_rows(MODE)) producer_role<MODE, CG>(p, sm, rw - kFirstProducerWarp, lane);
+        if constexpr (CG) producer_role_items<MODE>(p, &tmap, sm, rw - kFirstProducerWarp, lane);
+        else if constexpr (is_rows(MODE)) producer_role<MODE, false>(p, sm, rw - kFirstProducerWarp, lane);
         else stream_producer_role<MODE>(p, &tmap, sm, rw - kFirstProducerWarp, lane);
     }
 
@@ -1420,6 +1697,15 @@ int sm_count()
 
 }  // namespace
 
+#ifdef ALX_PROBE
+}  // namespace alx
+extern "C" int alx_debug_trace(unsigned long long *out)
+{
+    return (int)cudaMemcpyFromSymbol(out, alx::g_trace, sizeof(unsigned long long) * 8 * 16 * 16);
+}
+namespace alx {
+#endif
+
 int64_t gramian_umma_partials() { return (int64_t)kGramBlocks * Cfg<kModeGramian>::kGroups; }
 
 // Gramian of a bf16 table with d = 128 on the tensor cores; partials must hold gramian_umma_partials() * d * d floats
@@ -1488,6 +1774,7 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         p.solver = cg.enabled ? 1 : 0;
         p.cg_max_iter = cg.max_iter;
         p.cg_tol2 = cg.tol * cg.tol;
+        p.cg_warm = cg.warm_start ? 1 : 0;
         p.cg_counters = cg.counters;
         p.fallback_list = cg.fallback_list;
         p.fallback_count = cg.counters + 2;
