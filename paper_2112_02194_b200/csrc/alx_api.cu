@@ -3,7 +3,6 @@
 // happens on the host.
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -262,7 +261,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
     RowOut out{c->table[side], cap_slot, cap_out};
     if (tensor_path(c)) {
-        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 32 * sizeof(unsigned long long), c->stream));
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
                                      &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed],
@@ -351,9 +350,9 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
         ALX_ALLOC(c, c->loss_result, 4);
         ALX_ALLOC(c, c->status, 1);
         ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));
-        ALX_ALLOC(c, c->cg_counters, 32);
+        ALX_ALLOC(c, c->cg_counters, 3);
         if (tensor_path(c) && c->opt.solver == ALX_SOLVER_AUTO) ALX_ALLOC(c, c->cg_fallback_list, nmax);
-        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 32 * sizeof(unsigned long long), c->stream));
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
         for (auto &e : c->ev) ALX_CUDA(c, cudaEventCreate(&e));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
         return ALX_OK;
@@ -771,12 +770,8 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
         c->stats.dual_rows = flag ? c->dual_candidates : 0;
     }
     {
-        unsigned long long h[32] = {};
+        unsigned long long h[3] = {0, 0, 0};
         ALX_CUDA(c, cudaMemcpy(h, c->cg_counters, sizeof h, cudaMemcpyDeviceToHost));
-        if (getenv("ALX_PROBE_PRINT"))
-            fprintf(stderr, "alx probe: rows %llu products %llu | cycles other %llu wait-acc %llu pre %llu first-mv %llu mv %llu shfl %llu bar %llu tail %llu | mma warp: other %llu wait-acc %llu wait-full %llu mma-issue %llu commit %llu acc-commit %llu syncwarp %llu item-top %llu | producer 0: other %llu item-top %llu wait-empty %llu issue %llu wait-landed %llu rhs %llu test %llu\n",
-                    h[0], h[1], h[8], h[9], h[10], h[11], h[12], h[13], h[14], h[15], h[16], h[17], h[18], h[19], h[20], h[21], h[22], h[23],
-                    h[24], h[25], h[26], h[27], h[28], h[29], h[30]);
         c->stats.cg_rows = (int64_t)h[0];
         c->stats.cg_products = (int64_t)h[1];
         c->stats.cg_fallbacks = (int64_t)h[2];

@@ -61,9 +61,6 @@ __device__ __forceinline__ bool mbar_wait_parked(uint64_t *bar, uint32_t parity,
     // a phase that has completed already costs no suspend / resume round trip (measured: about 350 cycles per stage
     // for the MMA warp when the producers are ahead of it)
     if (mbar_test_wait(bar, parity)) return true;
-#ifdef ALX_DBG_NO_PARK
-    return mbar_wait(bar, parity, abort_flag, site);
-#endif
     for (uint32_t it = 0; it < (1u << 16); ++it) {
         uint32_t ok;
         asm volatile(

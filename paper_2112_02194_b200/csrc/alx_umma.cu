@@ -1,21 +1,24 @@
 // Tensor-core (tcgen05 / tensor memory) kernels for d = 128 with bfloat16 tables:
 //   - the Gramian X^T X of the fixed table                                   (Alg. 1 line 2)
 //   - per row: sum x_i (x) x_i and sum y x_i over the row's observations      (Alg. 1 lines 6-9),
-//     then the same factor / solve / store as the FP32-ALU path               (Alg. 1 line 10, Eq. 4)
+//     then the solve of Eq. 4 and the store                                   (Alg. 1 line 10)
 //   - partial sums of the chunks of rows longer than `split`
 //
 // One persistent block per SM, three roles:
-//   producer warps   gather the fixed-side rows of an item with 16-byte cp.async into a ring of
-//                    shared-memory stages, already in the operand layout the tensor core reads:
-//                    "MN-major, 128-byte swizzle" - a gathered row is one K index, its 128 features
-//                    are the M (and N) index, split into two 64-feature halves of 128 bytes;
+//   producer warps   gather the fixed-side rows of an item into a ring of shared-memory stages, already in the
+//                    operand layout the tensor core reads: "MN-major, 128-byte swizzle" - a gathered row is one
+//                    K index, its 128 features are the M (and N) index, split into two 64-feature halves of 128
+//                    bytes.  By TMA row gathers (chunks, Gramian, conjugate-gradient rows kernel) or 16-byte
+//                    cp.async (Cholesky rows kernel);
 //   one MMA thread   issues tcgen05.mma 128 x 128 x 16 (A = B = the staged tile) into one of the fp32
-//                    accumulators in tensor memory (four of 128 columns in rows mode, two of 256 otherwise);
+//                    accumulators in tensor memory (four of 128 columns in the rows modes, two of 256 otherwise);
 //                    chunks also get a 128 x 16 x 16 product with a two-column (high / low bfloat16 parts of
 //                    the label) tile that yields sum y x_i (whole rows: the producer warps sum it);
-//   solver groups    rows: four groups of 128 threads, one per accumulator, thread i owning row i of
-//                    the normal matrix.  The matrix never leaves tensor memory: the group adds
-//                    alpha0 G + lambda I on first touch, factors it in place with a blocked right-looking
+//   solver groups    rows: four groups of 128 threads, one per accumulator.  The matrix never leaves tensor
+//                    memory.  kModeRowsCg (the default): conjugate gradients, the matrix read through the 16x128b
+//                    tensor-memory shape for every product (Sec. 4.5: the paper's solver); a row that does not
+//                    converge is left to a second launch.  kModeRows: thread i owns row i, the group adds
+//                    alpha0 G + lambda I on first touch and factors in place with a blocked right-looking
 //                    Cholesky (tcgen05.ld / tcgen05.st of 16-column row segments, trailing updates on the
 //                    tensor core), solves and stores the row.  Gramian pieces and chunks: two groups of 256
 //                    threads copy the sums out.
@@ -52,8 +55,6 @@ template <int MODE> struct Ring {
     // MMA warp is at item j + 3 at most (item j + 4 needs the accumulator of j) and the producers at most one ring of
     // stages, hence as many items, further: slots j .. j + kNStage + 3 are live at most
     static constexpr int kBRing = kNStage + 4;
-    // rows modes: stages of cp.async copies in flight per producer warp (a gather is bound by latency times bytes in flight)
-    static constexpr int kLag = 6;
 };
 constexpr int kHalfBytes = kStageRows * 128;          // rows mode: one 64-feature half of a stage
 constexpr int kProducerWarps = 4;
@@ -66,32 +67,6 @@ constexpr int kGramBlocks = 148;                      // fixed, so that the orde
 // kModeRowsCg: whole rows as kModeRows, solved by conjugate gradients instead of the in-place Cholesky
 enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2, kModeRowsCg = 3 };
 __host__ __device__ constexpr bool is_rows(int mode) { return mode == kModeRows || mode == kModeRowsCg; }
-
-// Development aid (-DALX_PROBE): thread 0 of every solver group sums clock cycles per phase into cg_counters[3 ..].
-#ifdef ALX_PROBE
-// event trace of block 0: g_trace[role][item][event] = clock64 at the event (items kTraceFirst .. kTraceFirst + 15 of the block)
-constexpr int kTraceFirst = 64;
-__device__ unsigned long long g_trace[8][16][16];
-__device__ __forceinline__ void trace_ev(int role, long long item, int ev)
-{
-    if (blockIdx.x == 0 && item >= kTraceFirst && item < kTraceFirst + 16 && ev < 16)
-        g_trace[role][item - kTraceFirst][ev] = (unsigned long long)clock64();
-}
-#define TRACE(role, item, ev) trace_ev(role, item, ev)
-#else
-#define TRACE(role, item, ev)
-#endif
-
-struct Probe {
-#ifdef ALX_PROBE
-    long long t0 = 0, acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    __device__ __forceinline__ void start() { t0 = clock64(); }
-    __device__ __forceinline__ void lap(int k) { const long long t = clock64(); acc[k] += t - t0; t0 = t; }
-#else
-    __device__ __forceinline__ void start() {}
-    __device__ __forceinline__ void lap(int) {}
-#endif
-};
 
 // thread layout per mode: solver groups (one accumulator each), then one MMA warp, then the producer warps
 template <int MODE> struct Cfg {
@@ -278,11 +253,9 @@ struct ItemWindow {
     }
 };
 
-// PARK: wait for a free stage suspended (no issue slots taken) instead of polling: for the kernel whose solver
-// groups, not the gather, set the pace
-template <int MODE, bool PARK> __device__ void producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
+template <int MODE> __device__ void producer_role(const Params &p, SmemT<MODE> &sm, int pw, int lane)
 {
-    constexpr int kNStage = Ring<MODE>::kNStage, kLag = Ring<MODE>::kLag;
+    constexpr int kNStage = Ring<MODE>::kNStage, kLag = 6;      // kLag: stages of cp.async copies in flight per producer warp
     int64_t g = 0, signalled = 0, it = 0;
     const int c = lane & 15;                 // 16-byte chunk of the 256-byte row
     const int half = c >> 3, cc = c & 7;
@@ -303,10 +276,7 @@ template <int MODE, bool PARK> __device__ void producer_role(const Params &p, Sm
             y = p.sv.val ? p.sv.val[e] : 1.f;
         }
     };
-    Probe pr;
-    pr.start();
     for (int64_t t = blockIdx.x; t < p.n_items && alive; t += gridDim.x, ++it) {
-        pr.lap(0);
         if ((it & 31) == 0) win.load(p, it, lane);
         int64_t beg, end;
         win.get((int)(it & 31), beg, end);
@@ -320,7 +290,6 @@ template <int MODE, bool PARK> __device__ void producer_role(const Params &p, Sm
             win.get((int)(it & 31) + 1, nbeg, nend);
             first_ids(nbeg, nend, pre_idx, pre_y);
         }
-        pr.lap(1);
         for (int64_t e0 = beg; e0 < end; e0 += kStageRows) {
             const int slot = (int)(g % kNStage);
             const uint32_t ph = (uint32_t)((g / kNStage) & 1);
@@ -337,7 +306,6 @@ template <int MODE, bool PARK> __device__ void producer_role(const Params &p, Sm
             }
             // No free slot yet: the copies in flight have time to land, so hand over every stage issued so far
             // before blocking (otherwise up to kLag landed stages would stay unannounced until the next issue).
-            pr.lap(0);
             {
                 int free_now = 1;
                 if (lane == 0) free_now = mbar_test_wait(&sm.empty[slot], ph ^ 1u) ? 1 : 0;
@@ -347,10 +315,7 @@ template <int MODE, bool PARK> __device__ void producer_role(const Params &p, Sm
                     for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
                 }
             }
-            pr.lap(5);
-            if (!(PARK ? mbar_wait_parked_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)
-                       : mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE))) { alive = false; break; }
-            pr.lap(2);
+            if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
             const int rc = (int)((end - e0 < kStageRows) ? end - e0 : kStageRows);
             const int rc16 = (rc + 15) & ~15;
             if (is_rows(MODE)) {
@@ -381,22 +346,15 @@ template <int MODE, bool PARK> __device__ void producer_role(const Params &p, Sm
             }
             cp_async_commit();
             ++g;
-            pr.lap(3);
             if (g - signalled > kLag) {     // the oldest unannounced stage is kLag issues back: its copies have landed
                 cp_async_wait<kLag>();
-                pr.lap(4);
                 producer_signal<MODE>(sm, signalled, pw, lane, bacc);
                 ++signalled;
-                pr.lap(6);
             }
         }
     }
     cp_async_wait<0>();
     for (; signalled < g; ++signalled) producer_signal<MODE>(sm, signalled, pw, lane, bacc);
-#ifdef ALX_PROBE
-    if (lane == 0 && pw == 0 && p.cg_counters)
-        for (int k = 0; k < 7; ++k) atomicAdd(&p.cg_counters[24 + k], (unsigned long long)pr.acc[k]);
-#endif
 }
 
 // Producer of the conjugate-gradient rows kernel.  Producer warp pw gathers every fourth item of the block, whole: all its
@@ -515,7 +473,6 @@ __device__ void producer_role_items(const Params &p, const CUtensorMap *tmap, Sm
             const int32_t my_idx[2] = {nxt_idx[0], nxt_idx[1]};
             const float my_y[2] = {nxt_y[0], nxt_y[1]};
             if (s + 1 < nst) fetch_ids(e0 + kRows);
-            if (lane == 0) TRACE(5, it, 0 + 5 * s);
             // (1) wait for the turn; the hand-overs fill the wait (one stage at a time, the turn is looked at first: while this
             // warp holds the turn the other three wait for it)
             for (uint32_t spin = 0;; ++spin) {
@@ -535,7 +492,6 @@ __device__ void producer_role_items(const Params &p, const CUtensorMap *tmap, Sm
                 if (spin > 8u) __nanosleep(spin < 128u ? 64u : 256u);
             }
             if (!alive) break;
-            if (lane == 0) TRACE(5, it, 1 + 5 * s);
             // (2) the slot: stage g - ring must have been released.  While it is not, this warp's own stages in flight go
             // first (their release may be what the ring's turn-over waits for), then the warp waits suspended.
             for (;;) {
@@ -551,7 +507,6 @@ __device__ void producer_role_items(const Params &p, const CUtensorMap *tmap, Sm
                 }
             }
             if (!alive) break;
-            if (lane == 0) TRACE(5, it, 2 + 5 * s);
             // (3) issue the stage and pass the turn on
             const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
             const int rc16 = (rc + 15) & ~15;
@@ -581,7 +536,6 @@ __device__ void producer_role_items(const Params &p, const CUtensorMap *tmap, Sm
             if (lane == 0) {
                 __threadfence_block();
                 *turn = g + 1;
-                TRACE(5, it, 3 + 5 * s);
             }
             ++tail;
         }
@@ -672,12 +626,9 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
     uint32_t ph = 0;
     bool alive = true;
     // one stage: wait for it, issue its K steps of 16 rows, release it when they have completed
-    auto stage = [&](uint32_t d_main, int nk, bool &first, long long item, int s) -> bool {
-        if (lane == 0 && MODE == kModeRowsCg) TRACE(0, item, 2 + 3 * s);
-        if (!(MODE == kModeRowsCg ? mbar_wait_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)
-                                  : mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE))) return false;
+    auto stage = [&](uint32_t d_main, int nk, bool &first) -> bool {
+        if (!mbar_wait_parked_warp(&sm.full[slot], ph, &sm.abort_flag, 30 + MODE)) return false;
         tc_fence_after();
-        if (lane == 0 && MODE == kModeRowsCg) TRACE(0, item, 3 + 3 * s);
         if (lane == 0) {
             const uint32_t hb = smem_u32(&sm.h[slot][0]);
             const uint32_t yb = smem_u32(&sm.y[slot][0]);
@@ -692,7 +643,6 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
                 first = false;
             }
             umma_commit(&sm.empty[slot]);
-            if (MODE == kModeRowsCg) TRACE(0, item, 4 + 3 * s);
         }
         if (++slot == kNStage) { slot = 0; ph ^= 1u; }
         return true;
@@ -715,17 +665,13 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
             const int nst = mine >> 8, nk_last = mine & 0xFF;
             const int a = it % Cfg<MODE>::kGroups;
             const uint32_t aph = (uint32_t)((it / Cfg<MODE>::kGroups) & 1);
-            if (lane == 0 && MODE == kModeRowsCg) TRACE(0, it, 0);
-            if (!(MODE == kModeRowsCg ? mbar_wait_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)
-                                      : mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE))) break;
+            if (!mbar_wait_parked_warp(&sm.acc_empty[a], aph ^ 1u, &sm.abort_flag, 40 + MODE)) break;
             tc_fence_after();
-            if (lane == 0 && MODE == kModeRowsCg) TRACE(0, it, 1);
             const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
             bool first = true;
             for (int s = 0; s < nst; ++s)
-                if (!stage(d_main, s + 1 < nst ? kRows / 16 : nk_last, first, it, s)) { alive = false; break; }
+                if (!stage(d_main, s + 1 < nst ? kRows / 16 : nk_last, first)) { alive = false; break; }
             if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
-            if (lane == 0 && MODE == kModeRowsCg) TRACE(0, it, 15);
             __syncwarp();
         }
     } else {
@@ -741,7 +687,7 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
             bool first = true;
             for (int64_t e0 = beg; e0 < end; e0 += kRows) {
                 const int rc = (int)((end - e0 < kRows) ? end - e0 : kRows);
-                if (!stage(d_main, (rc + 15) >> 4, first, it, 0)) { alive = false; break; }
+                if (!stage(d_main, (rc + 15) >> 4, first)) { alive = false; break; }
             }
             if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
             __syncwarp();
@@ -1251,7 +1197,7 @@ __device__ __forceinline__ void cg_matvec(uint32_t twarp, const float *vq, int q
 // |r| <= tol |b|; false when the step limit is reached or a step length is not positive (the matrix is left complete
 // in tensor memory, and the caller solves it directly).
 __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, const float *Bq, uint32_t twarp, int bar_id,
-                                           int tid, float b, float x0, float &x_out, int &matvecs, Probe &pr)
+                                           int tid, float b, float x0, float &x_out, int &matvecs)
 {
     const int lane = tid & 31, w = tid >> 5, g = lane >> 2, q = lane & 3;
     const int own = 32 * w + g + 8 * q;                          // the row this thread owns
@@ -1278,7 +1224,6 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
     int products = 0;
     *vslot = warm ? x0 : b;
     cg_add_base(twarp, Bq, 32 * w + g, q);
-    pr.lap(3);
     group128_sync(bar_id);
     if (warm) {                 // r = b - A x0
         r = b - product();
@@ -1289,10 +1234,8 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
     }
     bool ok = false;
     for (int it = 0;; ++it) {
-        pr.lap(2);
         const float wv = product();
         ++products;
-        pr.lap(4);
         float gsum = r * r, dl = r * wv, bsum = b * b;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -1300,10 +1243,8 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
             dl += __shfl_xor_sync(0xFFFFFFFFu, dl, o);
             if (it == 0) bsum += __shfl_xor_sync(0xFFFFFFFFu, bsum, o);
         }
-        pr.lap(5);
         if (lane == 0) *reinterpret_cast<float4 *>(red + 4 * w) = make_float4(gsum, dl, bsum, 0.f);
         group128_sync(bar_id);
-        pr.lap(6);
         {
             const float4 r0 = *reinterpret_cast<const float4 *>(red), r1 = *reinterpret_cast<const float4 *>(red + 4),
                          r2 = *reinterpret_cast<const float4 *>(red + 8), r3 = *reinterpret_cast<const float4 *>(red + 12);
@@ -1359,12 +1300,10 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
     const int bar_id = 1 + gidx;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
     const float *Brow = Bs + i * kLdB;
-    constexpr bool use_cg = CG;                           // (then Bs holds alpha0 G + lambda I by column class, see kLdBq)
+    // (CG: Bs holds alpha0 G + lambda I by column class, see kLdBq)
     const int own_cg = 32 * w + (lane >> 2) + 8 * (lane & 3);
     uint32_t trail_parity = 0;
     unsigned cg_rows = 0, cg_matvecs = 0;      // thread 0 of the group counts (per block: far below 2^32)
-    Probe pr;
-    pr.start();
     for (int it = gidx;; it += kGroups) {      // this group's items: every fourth of the block's
         const int64_t t = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
         if (t >= p.n_items) break;
@@ -1415,22 +1354,17 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
             const uint32_t aph = (uint32_t)((it / kGroups) & 1);
             // one thread polls, the group follows through its barrier (a failed wait sets the block's abort flag)
             if (tid == 0) {
-                TRACE(1 + gidx, it, 0);
                 bool ok = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 60);
-                TRACE(1 + gidx, it, 1);
                 if constexpr (CG) {       // (the right-hand side follows the stages' landing on a barrier of its own)
                     constexpr int kBRing = Ring<kModeRowsCg>::kBRing;
                     ok = ok && mbar_wait_parked(&sm.rhs_done[it % kBRing], (uint32_t)((it / kBRing) & 1), &sm.abort_flag, 61);
                 }
-                TRACE(1 + gidx, it, 2);
                 gs.stop = ok ? 0 : 1;
                 gs.bad = 0;
             }
             group128_sync(bar_id);
             if (gs.stop) break;
             tc_fence_after();
-            if (tid == 0) TRACE(1 + gidx, it, 3);
-            pr.lap(1);
             if constexpr (CG) {
                 b = sm.bpart[it % Ring<kModeRowsCg>::kBRing][0][own_cg];
             } else {      // right-hand side: the four producer warps' partial sums, in order
@@ -1444,7 +1378,7 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
         if constexpr (CG) {
             int matvecs = 0;
             solved = cg_in_tmem(p, gs, Bs, sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride, bar_id, tid, b, x0,
-                                x, matvecs, pr);
+                                x, matvecs);
             own = own_cg;
             if (tid == 0) {
                 ++cg_rows;
@@ -1456,11 +1390,9 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
             if (gs.stop) break;
         }
         // tensor memory is free again for the next item of this accumulator
-        if (CG && tid == 0) TRACE(1 + gidx, it, 4);
         tc_fence_before();
         group128_sync(bar_id);
         if (!FROM_SUMS && tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
-        if (CG && tid == 0) TRACE(1 + gidx, it, 5);
         const bool ok = gs.bad == 0;
         const float xo = ok ? x : 0.f;
         if (solved) {
@@ -1475,13 +1407,7 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
             raise_flag(p.st, kFlagNotSpd, u);
         }
         group128_sync(bar_id);      // gs.bad is reset at the top of the next item
-        if (CG && tid == 0) TRACE(1 + gidx, it, 6);
-        pr.lap(7);
     }
-#ifdef ALX_PROBE
-    if (tid == 0 && p.cg_counters)
-        for (int k = 0; k < 8; ++k) atomicAdd(&p.cg_counters[8 + k], (unsigned long long)pr.acc[k]);
-#endif
     if (tid == 0 && cg_rows && p.cg_counters) {
         atomicAdd(&p.cg_counters[0], (unsigned long long)cg_rows);
         atomicAdd(&p.cg_counters[1], (unsigned long long)cg_matvecs);
@@ -1575,7 +1501,7 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
     } else {
         if constexpr (CG) setmaxnreg_dec<64>();
         if constexpr (CG) producer_role_items<MODE>(p, &tmap, sm, rw - kFirstProducerWarp, lane);
-        else if constexpr (is_rows(MODE)) producer_role<MODE, false>(p, sm, rw - kFirstProducerWarp, lane);
+        else if constexpr (is_rows(MODE)) producer_role<MODE>(p, sm, rw - kFirstProducerWarp, lane);
         else stream_producer_role<MODE>(p, &tmap, sm, rw - kFirstProducerWarp, lane);
     }
 
@@ -1697,14 +1623,6 @@ int sm_count()
 
 }  // namespace
 
-#ifdef ALX_PROBE
-}  // namespace alx
-extern "C" int alx_debug_trace(unsigned long long *out)
-{
-    return (int)cudaMemcpyFromSymbol(out, alx::g_trace, sizeof(unsigned long long) * 8 * 16 * 16);
-}
-namespace alx {
-#endif
 
 int64_t gramian_umma_partials() { return (int64_t)kGramBlocks * Cfg<kModeGramian>::kGroups; }
 
