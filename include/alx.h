@@ -234,9 +234,10 @@ const char *alx_last_error(const alx_ctx *ctx);
  * Gramian of a table without allocating anything (the paper has no counterpart; this is an addition for
  * callers that cannot allocate device memory when they call: inside a frozen memory pool, on a thread
  * that must not take an allocator lock, under a memory budget fixed at start-up).
- *   table   : device pointer, n x d row-major, float32 or bfloat16 (dtype)
- *   gramian : device pointer, d x d doubles, receives table^T table; written on `stream` (cudaStream_t,
- *             NULL = legacy default stream); the call does not synchronise
+ *   table   : device pointer, 16-byte aligned, n x d row-major, float32 or bfloat16 (dtype)
+ *   gramian : device pointer, 8-byte aligned, d x d doubles, receives table^T table; written on `stream`
+ *             (cudaStream_t, NULL = legacy default stream); the call does not synchronise
+ * A pointer that is not aligned as stated is refused with ALX_ERR_INVALID_ARG before anything is launched.
  * Same kernels and the same fixed summation order as alx_gramian on a context created with kernels = 1
  * (the FP32-ALU kernels), so those results agree to the last bit.
  * The piece sums go to a fixed array inside the library image (16 MiB + 64 KiB on every GPU that loads
@@ -245,7 +246,10 @@ const char *alx_last_error(const alx_ctx *ctx);
  * are refused with ALX_ERR_UNSUPPORTED and a message in alx_noalloc_last_error().  No cudaMalloc, cudaFree
  * or other allocating routine is called.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
- * device current; make that first call outside any stream capture.  The device that owns `table` must be
+ * device current; make that first call outside any stream capture.  The first use of the library's Gramian
+ * kernels on a device is also when the driver loads the module that carries the array, so that is when the
+ * 16 MiB are taken from the device: a caller whose memory is frozen later should make one warm-up call per
+ * device before the freeze.  The device that owns `table` must be
  * the current device.  All calls share the one array and it keeps the previous call's contents (each call
  * overwrites every piece it later reads, so nothing needs clearing): two calls whose kernels overlap on
  * the GPU -- different streams, or different host threads -- race; order them on one stream.

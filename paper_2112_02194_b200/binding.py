@@ -333,6 +333,8 @@ def gramian_noalloc(table, out):
     import torch
     lib = load_library()
     assert table.is_cuda and table.is_contiguous() and table.dim() == 2
+    if table.dtype not in (torch.bfloat16, torch.float32):     # any other element size would make the kernel read past the buffer
+        raise TypeError(f"gramian_noalloc: table must be float32 or bfloat16, not {table.dtype}")
     assert out.is_cuda and out.is_contiguous() and out.dtype == torch.float64 and out.numel() == table.shape[1] ** 2
     dt = ALX_BF16 if table.dtype == torch.bfloat16 else ALX_F32
     st = lib.alx_gramian_noalloc(table.data_ptr(), dt, table.shape[0], table.shape[1], out.data_ptr(),

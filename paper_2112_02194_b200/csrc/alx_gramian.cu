@@ -227,6 +227,11 @@ alx_status alx_gramian_noalloc(const void *table, alx_dtype dtype, int64_t n, in
         return noalloc_fail(ALX_ERR_INVALID_ARG, "alx_gramian_noalloc: null pointer, n < 1 or unknown dtype");
     if (d != 16 && d != 32 && d != 64 && d != 128)
         return noalloc_fail(ALX_ERR_UNSUPPORTED, "alx_gramian_noalloc: d must be 16, 32, 64 or 128");
+    // the kernels read the table in 16-byte pieces and write doubles: a pointer that is not aligned for that would
+    // fault on the device instead of being refused here
+    if ((reinterpret_cast<uintptr_t>(table) & 15u) != 0 || (reinterpret_cast<uintptr_t>(gramian) & 7u) != 0)
+        return noalloc_fail(ALX_ERR_INVALID_ARG,
+                            "alx_gramian_noalloc: table must be 16-byte aligned and gramian 8-byte aligned");
     const int64_t max_rows = alx_gramian_noalloc_max_rows(d);
     if (n > max_rows)
         return noalloc_fail(ALX_ERR_UNSUPPORTED,

@@ -32,17 +32,28 @@ static inline uint16_t f32_to_bf16_rne(float f)
 }
 
 /* rows[n_rows] (or NULL: rows row_begin .. row_begin + n_rows - 1) of a table with d columns; out is float32
- * (bf16 = 0) or uint16 bfloat16 bit patterns (bf16 = 1), n_rows x d */
+ * (bf16 = 0) or uint16 bfloat16 bit patterns (bf16 = 1), n_rows x d; with as_f64 the same stored values widened to
+ * double (exact), which is what the fp64 checker reads */
 void synth_host_rows(uint64_t key, const int64_t *table, const int64_t *rows, int64_t row_begin, int64_t n_rows, int d,
-                     double scale, int bf16, void *out)
+                     double scale, int bf16, int as_f64, void *out)
 {
 #pragma omp parallel for schedule(static)
     for (int64_t k = 0; k < n_rows; ++k) {
         const int64_t r = rows ? rows[k] : row_begin + k;
         for (int c = 0; c < d; ++c) {
             const float f = draw(key, table, r * d + c, scale);
-            if (bf16) ((uint16_t *)out)[k * d + c] = f32_to_bf16_rne(f);
-            else ((float *)out)[k * d + c] = f;
+            if (as_f64) {
+                float stored = f;
+                if (bf16) {
+                    const uint32_t b = (uint32_t)f32_to_bf16_rne(f) << 16;
+                    memcpy(&stored, &b, 4);
+                }
+                ((double *)out)[k * d + c] = (double)stored;
+            } else if (bf16) {
+                ((uint16_t *)out)[k * d + c] = f32_to_bf16_rne(f);
+            } else {
+                ((float *)out)[k * d + c] = f;
+            }
         }
     }
 }

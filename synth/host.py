@@ -30,9 +30,10 @@ def _get():
 
 
 def embedding_rows(d: int, seed: int, stream: int, storage: str, rows=None, row_begin: int = 0,
-                   row_count: int = 0, sigma: float | None = None) -> np.ndarray:
+                   row_count: int = 0, sigma: float | None = None, as_f64: bool = False) -> np.ndarray:
     """Rows of the table ``graphs.init_embeddings(n, d, seed, stream, storage)``: either the ids in ``rows`` or the
-    block row_begin .. row_begin + row_count - 1.  float32 or uint16 (bf16 bits)."""
+    block row_begin .. row_begin + row_count - 1.  float32 or uint16 (bf16 bits); with ``as_f64`` the stored values
+    widened to float64 (the same as ``graphs.storage_to_f64`` of the bits, without the detour)."""
     if sigma is None:
         sigma = 0.1 / np.sqrt(d)
     table = np.ascontiguousarray(graphs.normal_table(), dtype=np.int64)
@@ -45,8 +46,8 @@ def embedding_rows(d: int, seed: int, stream: int, storage: str, rows=None, row_
     else:
         n = int(row_count)
         rp = None
-    out = np.empty((n, d), dtype=np.uint16 if storage == "bf16" else np.float32)
+    out = np.empty((n, d), dtype=np.float64 if as_f64 else (np.uint16 if storage == "bf16" else np.float32))
     _get().synth_host_rows(ctypes.c_uint64(key), table.ctypes.data_as(ctypes.c_void_p), rp, ctypes.c_int64(row_begin),
                            ctypes.c_int64(n), ctypes.c_int(d), ctypes.c_double(scale), ctypes.c_int(storage == "bf16"),
-                           out.ctypes.data_as(ctypes.c_void_p))
+                           ctypes.c_int(1 if as_f64 else 0), out.ctypes.data_as(ctypes.c_void_p))
     return out

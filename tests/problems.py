@@ -46,7 +46,7 @@ def tiny():
 
 
 def powerlaw(name, n, nnz, s, cap, d, lam, alpha, storage, law, seed, split=0, values=False, n_cols=None,
-             empty_rows=0):
+             empty_rows=0, zero_labels=0.0):
     n_cols = n if n_cols is None else n_cols
     deg = graphs.zipf_degrees(n, nnz, s, min(cap, n_cols // 2), seed)
     if empty_rows:
@@ -62,6 +62,10 @@ def powerlaw(name, n, nnz, s, cap, d, lam, alpha, storage, law, seed, split=0, v
     if values:
         rng = np.random.Generator(np.random.PCG64(seed + 2))
         vals = rng.uniform(0.5, 2.0, colidx.size).astype(np.float32)
+        if zero_labels:       # y = 0 is a legal observation: it adds x (x) x to the row's matrix and nothing to its right-hand side
+            vals[rng.random(colidx.size) < zero_labels] = 0.0
+            for u in (5, 17, 33):       # and a few rows whose every label is 0
+                vals[rowptr[u]:rowptr[u + 1]] = 0.0
     W0, H0 = _tables(n, n_cols, d, seed + 3, storage)
     return Problem(name, n, n_cols, d, lam, alpha, storage, rowptr, colidx, vals, W0, H0, split)
 
@@ -87,4 +91,10 @@ def small_suite():
                          values=True, n_cols=8000),
         lambda: powerlaw("split_labels_d128_bf16", 1500, 120000, 1.0, 3000, 128, 0.02, 0.001, "bf16", "zipf", 17,
                          split=512, values=True, n_cols=8000),
+        # the remaining (d, storage) pairs: d = 128 with fp32 tables, labels of which a fifth are 0 (some rows hold nothing
+        # but zeros: their right-hand side is 0 and so is their solution); d = 32 with bfloat16 tables
+        lambda: powerlaw("zero_labels_d128_f32", 1200, 40000, 1.0, 700, 128, 0.02, 0.001, "f32", "zipf", 18,
+                         split=256, values=True, n_cols=2500, zero_labels=0.2),
+        lambda: powerlaw("uniform_d32_bf16", 2000, 50000, 1.1, 900, 32, 0.05, 0.002, "bf16", "uniform", 19, n_cols=1700,
+                         empty_rows=2),
     ]

@@ -48,3 +48,21 @@ def test_synth_library_builds():
     from synth import device
     lib = ctypes.CDLL(device.build())
     assert hasattr(lib, "synth_edges") and hasattr(lib, "synth_normal")
+
+
+def test_noalloc_gramian_refuses_bad_pointers_without_a_gpu():
+    """The argument checks of alx_gramian_noalloc come before any CUDA call: misaligned or null pointers, unknown
+    sizes and types are refused with a status code on a machine without a GPU too (nothing is ever dereferenced)."""
+    import ctypes
+    from paper_2112_02194_b200 import binding
+    lib = binding.load_library()
+    buf = ctypes.create_string_buffer(4096)
+    base = (ctypes.addressof(buf) + 255) & ~255
+    assert lib.alx_gramian_noalloc(None, 0, 16, 128, base, None) == 1
+    assert lib.alx_gramian_noalloc(base, 7, 16, 128, base, None) == 1                     # unknown dtype
+    assert lib.alx_gramian_noalloc(base, 0, 16, 48, base, None) == 7                      # unsupported d
+    assert lib.alx_gramian_noalloc(base + 4, 0, 16, 128, base, None) == 1                 # table not 16-byte aligned
+    assert b"aligned" in lib.alx_noalloc_last_error()
+    assert lib.alx_gramian_noalloc(base, 0, 16, 128, base + 4, None) == 1                 # gramian not 8-byte aligned
+    assert lib.alx_gramian_noalloc(base, 0, (1 << 20) + 1, 128, base, None) == 7          # beyond the fixed array
+    assert b"exceed" in lib.alx_noalloc_last_error()
