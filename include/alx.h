@@ -19,7 +19,10 @@
  *     synchronising call (alx_synchronize, alx_loss, alx_get_*) turns into an error code.
  *     Nothing traps or asserts on the device.
  *   - Results are run-to-run deterministic: no floating-point atomics, all partial sums are
- *     combined in a fixed order that depends only on the problem sizes.
+ *     combined in a fixed order that depends only on the problem sizes.  The same sequence of calls on
+ *     a fresh context gives the same bits.  (With ALX_SOLVER_AUTO a half-epoch's solver depends on what
+ *     the side's previous half-epoch on that context cost, so repeating one call on a used context may
+ *     give the same solution in other bits.)
  */
 #ifndef ALX_H_
 #define ALX_H_
@@ -51,6 +54,7 @@ typedef enum { ALX_SOLVER_AUTO = 0, ALX_SOLVER_CHOLESKY = 1 } alx_solver;
 typedef enum { ALX_CG_START_STORED = 0, ALX_CG_START_ZERO = 1 } alx_cg_start;
 #define ALX_DEFAULT_CG_MAX_ITER 48
 #define ALX_DEFAULT_CG_TOL 1e-5f
+#define ALX_DEFAULT_CG_SWITCH_PRODUCTS 28.f
 
 /* number of degree classes and the default split threshold, see alx_get_buckets */
 #define ALX_N_CLASSES 12
@@ -82,10 +86,16 @@ typedef struct alx_options {
     int32_t solver;          /* how the d x d system of Eq. 4 is solved (Sec. 4.5 compares the choices):
                                 ALX_SOLVER_AUTO (0): conjugate gradients where the library has them (the whole-rows
                                 tensor-core kernel), started as cg_start says and stopped at |r| <= cg_tol |b|; a row that has not
-                                converged after cg_max_iter steps, and every row elsewhere, is solved by Cholesky.
+                                converged after cg_max_iter steps, and every row elsewhere, is solved by Cholesky.  A side
+                                whose conjugate-gradient half-epoch spent more than cg_switch_products (28) products per row on average (where
+                                the in-place Cholesky is the faster solve on B200) takes Cholesky for its next half-epochs,
+                                with one conjugate-gradient half-epoch in every eight to look again; the choice is made
+                                on the device from the counts of the side's last run.
                                 ALX_SOLVER_CHOLESKY (1): Cholesky for every row */
     int32_t cg_max_iter;     /* 0 => ALX_DEFAULT_CG_MAX_ITER */
     float cg_tol;            /* 0 => ALX_DEFAULT_CG_TOL; at most 1e-2 */
+    float cg_switch_products; /* the mean number of products per row beyond which a side's next half-epochs take Cholesky
+                                (see solver); 0 => ALX_DEFAULT_CG_SWITCH_PRODUCTS */
     int32_t cg_start;        /* start vector of the conjugate gradients (the paper states none): ALX_CG_START_STORED (0): the
                                 row's embedding as stored in the table being solved (close to the solution once training
                                 is under way; costs one product for r = b - A x0, and falls back to zero when |r| > |b|);
@@ -110,6 +120,8 @@ typedef struct alx_stats {
     int64_t cg_rows;                         /* LAST half-epoch: rows the conjugate-gradient solve took, */
     int64_t cg_products;                     /* the matrix-vector products it spent on them (steps + 1 per row), */
     int64_t cg_fallbacks;                    /* and how many of those rows went on to the Cholesky solve (not converged) */
+    int32_t cholesky_by_policy[2];           /* [side]: 1 if the side's LAST half-epoch took Cholesky for every row because
+                                                its conjugate-gradient run before that spent too many products per row */
 } alx_stats;
 
 /* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.

@@ -33,7 +33,7 @@ class alx_options(Structure):
                 ("alpha0", c_float), ("storage", c_int32), ("device", c_int32), ("stream", c_void_p),
                 ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_user", c_void_p), ("split", c_int64),
                 ("kernels", c_int32), ("solver", c_int32), ("cg_max_iter", c_int32), ("cg_tol", c_float),
-                ("cg_start", c_int32)]
+                ("cg_switch_products", c_float), ("cg_start", c_int32)]
 
 
 class alx_stats(Structure):
@@ -42,7 +42,7 @@ class alx_stats(Structure):
                 ("ms_half_epoch", c_double), ("kernel_launches", c_int64), ("workspace_bytes", c_int64),
                 ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double), ("dual_rows", c_int64),
                 ("long_rows", c_int64 * 2), ("long_entries", c_int64 * 2), ("cg_rows", c_int64),
-                ("cg_products", c_int64), ("cg_fallbacks", c_int64)]
+                ("cg_products", c_int64), ("cg_fallbacks", c_int64), ("cholesky_by_policy", c_int32 * 2)]
 
 
 EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_set_embedding_rows",
@@ -113,7 +113,7 @@ class Alx:
     """One context.  Methods carry the C names without the ``alx_`` prefix and only marshal arguments."""
 
     def __init__(self, n_rows, n_cols, d, lam, alpha0, storage="f32", split=0, kernels=0, device=None,
-                 use_torch_allocator=True, solver=0, cg_max_iter=0, cg_tol=0.0, cg_start=0):
+                 use_torch_allocator=True, solver=0, cg_max_iter=0, cg_tol=0.0, cg_start=0, cg_switch_products=0.0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("alx needs a CUDA device (B200, sm_100a); there is no CPU path")
@@ -133,6 +133,7 @@ class Alx:
         opt.kernels = kernels
         opt.solver, opt.cg_max_iter, opt.cg_tol = int(solver), int(cg_max_iter), float(cg_tol)
         opt.cg_start = int(cg_start)
+        opt.cg_switch_products = float(cg_switch_products)
         if use_torch_allocator:
             dev = torch.device("cuda", self.device)
 

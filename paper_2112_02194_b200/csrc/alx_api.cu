@@ -51,6 +51,7 @@ struct alx_ctx {
     DevStatus *status = nullptr;
     unsigned long long *cg_counters = nullptr;   // tensor path: rows solved by conjugate gradients, products, fall-backs (last half-epoch)
     int32_t *cg_fallback_list = nullptr;         // tensor path with conjugate gradients: the rows left to the Cholesky solve
+    CgPolicy *cg_policy = nullptr;               // [2]: per side, what the solver choice of its next half-epoch rests on
 
     // second stream for the host copies that alx_load_host / alx_epoch_to_host overlap with kernels
     cudaStream_t copy_stream = nullptr;
@@ -231,6 +232,8 @@ CgOptions cg_options(const alx_ctx *c, int solved_side)
     o.tol = c->opt.cg_tol > 0.f ? c->opt.cg_tol : ALX_DEFAULT_CG_TOL;
     o.counters = c->cg_counters;
     o.fallback_list = c->cg_fallback_list;
+    o.policy = c->cg_policy ? c->cg_policy + solved_side : nullptr;
+    o.switch_products = c->opt.cg_switch_products > 0.f ? c->opt.cg_switch_products : ALX_DEFAULT_CG_SWITCH_PRODUCTS;
     return o;
 }
 
@@ -312,6 +315,7 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
     if (opt->split != 0 && opt->split < 16) return ALX_ERR_INVALID_ARG;
     if (opt->solver != ALX_SOLVER_AUTO && opt->solver != ALX_SOLVER_CHOLESKY) return ALX_ERR_INVALID_ARG;
     if (opt->cg_start != ALX_CG_START_STORED && opt->cg_start != ALX_CG_START_ZERO) return ALX_ERR_INVALID_ARG;
+    if (!(opt->cg_switch_products >= 0.f)) return ALX_ERR_INVALID_ARG;
     if (opt->cg_max_iter < 0 || opt->cg_max_iter > 1024 || !(opt->cg_tol >= 0.f) || opt->cg_tol > 1e-2f) return ALX_ERR_INVALID_ARG;
     int dev = opt->device;
     if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return ALX_ERR_CUDA;
@@ -351,7 +355,11 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
         ALX_ALLOC(c, c->status, 1);
         ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));
         ALX_ALLOC(c, c->cg_counters, 3);
-        if (tensor_path(c) && c->opt.solver == ALX_SOLVER_AUTO) ALX_ALLOC(c, c->cg_fallback_list, nmax);
+        if (tensor_path(c) && c->opt.solver == ALX_SOLVER_AUTO) {
+            ALX_ALLOC(c, c->cg_fallback_list, nmax);
+            ALX_ALLOC(c, c->cg_policy, 2);
+            ALX_CUDA(c, cudaMemsetAsync(c->cg_policy, 0, 2 * sizeof(CgPolicy), c->stream));
+        }
         ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
         for (auto &e : c->ev) ALX_CUDA(c, cudaEventCreate(&e));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
@@ -775,6 +783,12 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
         c->stats.cg_rows = (int64_t)h[0];
         c->stats.cg_products = (int64_t)h[1];
         c->stats.cg_fallbacks = (int64_t)h[2];
+        c->stats.cholesky_by_policy[0] = c->stats.cholesky_by_policy[1] = 0;
+        if (c->cg_policy) {
+            CgPolicy pol[2];
+            ALX_CUDA(c, cudaMemcpy(pol, c->cg_policy, sizeof pol, cudaMemcpyDeviceToHost));
+            for (int sd = 0; sd < 2; ++sd) c->stats.cholesky_by_policy[sd] = pol[sd].use_cholesky;
+        }
     }
     c->stats.kernel_launches = c->launches;
     c->stats.workspace_bytes = c->bytes_held;

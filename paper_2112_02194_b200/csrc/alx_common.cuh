@@ -140,6 +140,20 @@ inline int long_class_begin(const int64_t *class_offs_host)
     return c;
 }
 
+// What the library remembers, per side, of the conjugate-gradient solve's cost, on the device (so that choosing the
+// solver of a half-epoch needs no host round trip): rows and products of the side's last conjugate-gradient run, the
+// choice for the run being launched, and how many half-epochs of the side have been launched.
+struct CgPolicy {
+    unsigned long long rows, products;
+    int use_cholesky;     // this half-epoch: 1 = the in-place Cholesky takes every row of the whole-rows kernel
+    int calls;
+};
+// Conjugate gradients pay while a row takes fewer than about 28 products on average (measured on B200: about 2900 + 300
+// per product cycles of an SM per row, against 12 600 for the in-place Cholesky; alx_options.cg_switch_products); beyond
+// that the side's next half-epochs go to Cholesky, with one conjugate-gradient half-epoch every kCgReprobe to see whether
+// the matrices have improved
+constexpr int kCgReprobe = 8;
+
 // conjugate-gradient solve of the whole-rows tensor-core kernel (Sec. 4.5)
 struct CgOptions {
     bool enabled;
@@ -148,6 +162,8 @@ struct CgOptions {
     bool warm_start;               // start from the row's stored embedding (the solved table holds trained values)
     unsigned long long *counters;  // device, [3]: rows, matrix-vector products, rows that fell back
     int32_t *fallback_list;        // device, one entry per row of the larger side: the rows left to the Cholesky solve
+    CgPolicy *policy;              // device, this side's record
+    float switch_products;         // mean products per row beyond which the side's next half-epochs take Cholesky
 };
 
 // alx_umma.cu: tensor-core path, d = 128 and bf16 tables only

@@ -108,6 +108,7 @@ struct Params {
     const unsigned long long *item_count;   // ... and how many of them (device)
     int32_t *fallback_list;      // conjugate gradients: rows that did not converge are appended here (any order) ...
     unsigned long long *fallback_count;     // ... and counted here; a second launch solves them by Cholesky
+    const CgPolicy *policy;      // rows modes: the side's solver choice for this half-epoch (nullptr: none, the launch decides)
     int solver;                  // rows mode: 0 = in-place Cholesky, 1 = conjugate gradients
     int cg_max_iter;             // conjugate gradients: steps after which a row goes to the Cholesky solve instead
     float cg_tol2;               // conjugate gradients: stop at |r|^2 <= cg_tol2 |b|^2
@@ -1427,12 +1428,15 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
 {
     using C = Cfg<MODE>;
     constexpr bool CG = MODE == kModeRowsCg;
-    if (MODE == kModeRows && p.item_count) {
+    // which rows this launch takes (block-uniform decisions, before any barrier or allocation)
+    if (MODE == kModeRowsCg && p.policy && p.policy->use_cholesky) return;      // the Cholesky launch takes them all
+    if (MODE == kModeRows && p.item_count && !(p.policy && p.policy->use_cholesky)) {
         p.n_items = (int64_t)*p.item_count;                 // the rows conjugate gradients left over
-        if ((int64_t)blockIdx.x >= p.n_items) return;      // block-uniform, before any barrier or allocation
-    } else if (is_rows(MODE) && p.dual_flag && *p.dual_flag) {
-        p.n_items = p.n_items_primal;
         if ((int64_t)blockIdx.x >= p.n_items) return;
+    } else {
+        if (MODE == kModeRows) p.item_list = nullptr;       // (every row: the walk through the degree classes)
+        if (is_rows(MODE) && p.dual_flag && *p.dual_flag) p.n_items = p.n_items_primal;
+        if (is_rows(MODE) && (int64_t)blockIdx.x >= p.n_items) return;
     }
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzled stages; plain offset arithmetic on the shared array, so that the
@@ -1512,6 +1516,26 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
         tmem_dealloc(sm.tmem_base, kTmemCols);
     }
     if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, (long long)sm.abort_flag * 1000000 + blockIdx.x);
+}
+
+// Before a side's whole-rows launches: choose the solver from the side's last conjugate-gradient run.
+__global__ void k_cg_policy(CgPolicy *pol, float switch_products)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const int calls = pol->calls++;
+    int use = 0;
+    if (pol->rows > 0 && (float)pol->products > switch_products * (float)pol->rows) use = 1;
+    if (use && (calls % kCgReprobe) == kCgReprobe - 1) use = 0;
+    pol->use_cholesky = use;
+}
+// After them: keep the run's counts (they are cleared at the start of every half-epoch).
+__global__ void k_cg_record(CgPolicy *pol, const unsigned long long *counters)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (!pol->use_cholesky) {
+        pol->rows = counters[0];
+        pol->products = counters[1];
+    }
 }
 
 __global__ void k_zero_rows_bf16(const int32_t *__restrict__ rows, int64_t count, RowOut out)
@@ -1698,18 +1722,24 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         p.fallback_count = cg.counters + 2;
         const int grid = (int)(n_whole < sms ? n_whole : sms);
         if (main_begin) cudaEventRecord(main_begin, s);
-        e = cg.enabled ? launch_mode<kModeRowsCg>(p, grid, s) : launch_mode<kModeRows>(p, grid, s);
-        ++*launches;
-        if (e != cudaSuccess) return e;
         if (cg.enabled) {
-            // the rows conjugate gradients did not finish (none, as a rule: the blocks then return at once)
+            // solver of this half-epoch: conjugate gradients unless the side's last run took too many products
+            k_cg_policy<<<1, 32, 0, s>>>(cg.policy, cg.switch_products);
+            p.policy = cg.policy;
+            e = launch_mode<kModeRowsCg>(p, grid, s);
+            if (e != cudaSuccess) return e;
+            k_cg_record<<<1, 32, 0, s>>>(cg.policy, cg.counters);
+            // the Cholesky kernel: the rows conjugate gradients did not finish (none, as a rule: its blocks then return at
+            // once), or every row when the choice above fell on it
             p.item_list = cg.fallback_list;
             p.item_count = cg.counters + 2;
-            p.dual_flag = nullptr;
+            e = launch_mode<kModeRows>(p, grid, s);
+            *launches += 4;
+        } else {
             e = launch_mode<kModeRows>(p, grid, s);
             ++*launches;
-            if (e != cudaSuccess) return e;
         }
+        if (e != cudaSuccess) return e;
         if (main_end) cudaEventRecord(main_end, s);
     }
     const int64_t n_zero = offs[1] - offs[0];
