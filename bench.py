@@ -175,6 +175,20 @@ def dist_env():
     return rank, world, local
 
 
+def replica_command(argv, gpus: int, port: int):
+    """Command that runs this script as `gpus` replica processes, one per GPU of this node (replicas only: every rank
+    runs the whole workload on its own GPU; the ranks meet at the barriers and in the max/sum of the result line)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
 def aggregate_over_ranks(ms_local: float, units_local: float, world: int, device=None):
     """(max over ranks of the time, sum over ranks of the units) -- replicas only, no data-path collective."""
     if world == 1:
@@ -312,38 +326,47 @@ def run_ours(args, w):
     t_roof = max(t_bytes, t_tensor + t_alu)
     rows_ms = statistics.mean(half_ms["row_kernels"])
     main_ms = statistics.mean(half_ms["main_kernel"]) or rows_ms
-    n_whole = [sum(st.rows_in_class[sd][1:11]) for sd in (0, 1)]
+    # dominant kernels: the whole-rows launches (every row of more than 32 and at most 1024 entries, plus the shorter
+    # ones when the dual form stepped aside: gather, outer products, solve, store).  Rows and entries per launch are
+    # exact: per-class counts from alx_stats minus what the dual-form kernel and the chunks kernel took.
     n_split = [st.rows_in_class[sd][11] for sd in (0, 1)]
-    # dominant kernel: the whole-rows kernel (every row of more than 32 and at most `split` entries, plus the shorter
-    # ones when the dual form stepped aside: gather, outer products, factor, solve, store).  Its algorithmic work per
-    # launch, averaged over the two sides:
-    split = w.get("split", 0) or 8192
-    ent_whole = nnz - statistics.mean([st.n_chunks[sd] for sd in (0, 1)]) * split * 0.97   # entries outside split rows (approx.)
-    dual_rows = statistics.mean(half_ms["dual_rows"])
-    rows_whole = statistics.mean(n_whole) - dual_rows
-    ent_whole -= 6.0 * dual_rows          # rows of 1 .. 32 entries, about 6 on average under the rank-size law (approx.)
-    # whole rows of more than 1024 entries get their sums from the chunks kernel and their solve from k_solve_sums
-    rows_whole -= statistics.mean(st.long_rows)
-    ent_whole -= statistics.mean(st.long_entries)
-    alu_main = rows_whole * (d ** 3 / 3.0 + 3.0 * d * d) + 2.0 * ent_whole * d
+    rows_side, ent_side, alu_side = [], [], []
+    chol_row = d ** 3 / 3.0 + 3.0 * d * d
+    for sd in (0, 1):
+        rows_sd = sum(st.rows_in_class[sd][1:11]) - st.long_rows[sd]
+        ent_sd = sum(st.entries_in_class[sd][1:11]) - st.long_entries[sd]
+        if half_ms["dual_rows"][sd] > 0:
+            rows_sd -= st.rows_in_class[sd][1] + st.rows_in_class[sd][2]
+            ent_sd -= st.entries_in_class[sd][1] + st.entries_in_class[sd][2]
+        rows_side.append(rows_sd)
+        ent_side.append(ent_sd)
+        # solve work of the launch: the cheaper of Cholesky and the products conjugate gradients really spent
+        cg_r, cg_p, cg_f = half_ms["cg_rows"][sd], half_ms["cg_products"][sd], half_ms["cg_fallbacks"][sd]
+        solve = (rows_sd - cg_r + cg_f) * chol_row + min(cg_r * chol_row, cg_p * (2.0 * d * d + 10.0 * d) + cg_r * d * d)
+        alu_side.append(solve + 2.0 * ent_sd * d)
+    rows_whole = statistics.mean(rows_side)
+    ent_whole = statistics.mean(ent_side)
+    alu_main = statistics.mean(alu_side)
     bytes_main = ent_whole * (d * e + 4) + rows_whole * (d * e + 12)
     if t_bytes >= t_tensor + t_alu:
         roof = {"bound": "hbm", "achieved": bytes_main / (main_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     else:
         roof = {"bound": "alu", "achieved": alu_main / (main_ms * 1e-3) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    # DRAM traffic of that kernel: dram__bytes_read + dram__bytes_write of one ncu capture of the 2M-row `medium`
-    # case, per row and per side (columns side: 4.48 GB for 2.00M rows at a 91 % L2 hit rate; rows side, rows of
-    # 33 .. 1024 entries: 5.30 GB for 0.372M rows at 55 %), scaled by the rows each launch of this workload
-    # solves and averaged over the two launches of an epoch.  The window of +-1 % of the ids (hence the L2 reuse)
-    # scales with the table, so this is an estimate, not a measurement at this size.
-    if w["name"] in ("cfg3", "medium"):
-        primal_rows = [n_whole[sd] - half_ms["dual_rows"][sd] - st.long_rows[sd] for sd in (0, 1)]
-        roof["traffic"] = 0.5 * (primal_rows[0] * 5.30e9 / 0.372e6 + primal_rows[1] * 4.48e9 / 2.0e6)
-    else:
-        roof["traffic"] = None
-    roof.update({"kernel": "k_umma<0>: whole rows (gather, tcgen05 outer products, Cholesky in tensor memory, solve, store)",
-                 "main_kernel_ms": main_ms, "rows_per_launch": rows_whole,
+    # DRAM traffic of these launches is not measured in this run (it needs a profiler pass); the committed profile
+    # summaries hold dram bytes of one capture on the 2M-row `medium` case
+    roof["traffic"] = None
+    # the half-epoch roofline with the solve counted at what conjugate gradients really spent (never above Cholesky)
+    alu_cg_half = statistics.mean([alu_half - rows_side[sd] * chol_row - 2.0 * ent_side[sd] * d + alu_side[sd] for sd in (0, 1)])
+    t_alu_cg = alu_cg_half / (fp32_peak * 1e12)
+    t_roof_cg = max(t_bytes, t_tensor + t_alu_cg)
+    kernel_txt = ("k_umma<3> + k_umma<0>: whole rows (item gather by TMA, tcgen05 outer products into tensor memory, "
+                  "conjugate gradients on the matrix in tensor memory, Cholesky in tensor memory for rows that do not "
+                  "converge or sides the policy moved, store)" if st.kernel_path[0] == 1 else
+                  "k_rows_simple: whole rows on the FP32 ALUs (gather, outer products, Cholesky in shared memory, store)")
+    roof.update({"kernel": kernel_txt,
+                 "main_kernel_ms": main_ms, "rows_per_launch": rows_whole, "entries_per_launch": ent_whole,
+                 "per_side": {"rows": rows_side, "entries": ent_side, "alu_flop": alu_side},
                  "rows_in_dual_form": {"rows": half_ms["dual_rows"][0], "cols": half_ms["dual_rows"][1],
                                        "note": "rows with at most 32 entries, solved by k_dual outside the dominant kernel"},
                  "long_rows": {"rows": list(st.long_rows), "entries": list(st.long_entries),
@@ -355,6 +378,9 @@ def run_ours(args, w):
                  "roofline_half_epoch_ms": {"bytes": t_bytes * 1e3, "tensor": t_tensor * 1e3, "alu": t_alu * 1e3,
                                             "max(bytes, tensor+alu)": t_roof * 1e3},
                  "frac_of_roofline_time": t_roof * 1e3 / statistics.mean([half_ms["rows"][0], half_ms["cols"][0]]),
+                 "roofline_half_epoch_ms_solve_as_spent": {"alu": t_alu_cg * 1e3, "max(bytes, tensor+alu)": t_roof_cg * 1e3,
+                                                           "frac": t_roof_cg * 1e3 / statistics.mean([half_ms["rows"][0], half_ms["cols"][0]]),
+                                                           "note": "solve counted as min(Cholesky, products x (2d^2 + 10d)) on the rows conjugate gradients took"},
                  "split_rows": n_split})
 
     # ---- end to end from host buffers: upload S and both tables, one epoch, download both tables
@@ -406,8 +432,9 @@ def run_ours(args, w):
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-               "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-               "config": {"workload": w["name"], "description": w["desc"], "nnz": nnz, "n_rows": n, "n_cols": n,
+               "vs_baseline": None, "dtype": storage if storage == "bf16" else "f32", "data": "synthetic",
+               "config": {"workload": w["name"], "arithmetic": ("bf16 products into f32 sums on the tensor cores, f32 solve"
+                                                              if st.kernel_path[0] == 1 else "f32 throughout"), "description": w["desc"], "nnz": nnz, "n_rows": n, "n_cols": n,
                           "d": d, "storage": storage, "lambda": w["lam"], "alpha0": w["alpha"],
                           "step": "one epoch = rows half-epoch + columns half-epoch",
                           "l2": "inputs larger than L2 (tables and index arrays are GBs)",
@@ -421,6 +448,8 @@ def run_ours(args, w):
                          "epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
                          "setup_s": {"generate": t_gen, "alx_set_csr_device": t_set},
                          "rows_in_class": [list(st.rows_in_class[0]), list(st.rows_in_class[1])],
+                         "entries_in_class": [list(st.entries_in_class[0]), list(st.entries_in_class[1])],
+                         "cholesky_by_policy": list(st.cholesky_by_policy),
                          "n_chunks": list(st.n_chunks), "workspace_gb": st.workspace_bytes / 1e9}}
         print(json.dumps(out))
     if world > 1:
@@ -444,6 +473,9 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload], name=args.workload)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: become the launcher of one replica process per GPU
+        sys.exit(subprocess.call(replica_command(sys.argv[1:], args.gpus, free_port())))
     if args.impl == "reference":
         run_reference(args, w)
     else:

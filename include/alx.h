@@ -122,6 +122,8 @@ typedef struct alx_stats {
     int64_t cg_fallbacks;                    /* and how many of those rows went on to the Cholesky solve (not converged) */
     int32_t cholesky_by_policy[2];           /* [side]: 1 if the side's LAST half-epoch took Cholesky for every row because
                                                 its conjugate-gradient run before that spent too many products per row */
+    int64_t entries_in_class[2][ALX_N_CLASSES]; /* [side][class]: the observed entries held by the rows of each degree class
+                                                   (sums to nnz over the classes of a side) */
 } alx_stats;
 
 /* Create a context for an n_rows x n_cols problem: fp32 tables, defaults for everything else.
@@ -135,8 +137,8 @@ alx_status alx_destroy(alx_ctx *ctx);
  * rowptr[n_rows + 1] (int64, rowptr[0] = 0, rowptr[n_rows] = nnz), colidx[nnz] (int32, strictly
  * ascending inside each row: S is a set of pairs), values[nnz] (float labels y, or NULL: y = 1).
  * The call copies the arrays, validates them on the device (ALX_ERR_BAD_CSR, never a trap), builds
- * the transpose (CSC, row ids ascending inside each column; "a similar pass over the item side",
- * Alg. 1 line 11, needs it), and for both orientations the degree-class order of the rows and the
+ * the transpose (CSC, row ids ascending inside each column: the item-side pass of Alg. 1 line 11
+ * reads the entries column by column), and for both orientations the degree-class order of the rows and the
  * chunk descriptors of the rows longer than `split`.  Integer work only; synchronises.
  */
 alx_status alx_set_csr(alx_ctx *ctx, const int64_t *rowptr, const int32_t *colidx, const float *values,

@@ -42,7 +42,8 @@ class alx_stats(Structure):
                 ("ms_half_epoch", c_double), ("kernel_launches", c_int64), ("workspace_bytes", c_int64),
                 ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double), ("dual_rows", c_int64),
                 ("long_rows", c_int64 * 2), ("long_entries", c_int64 * 2), ("cg_rows", c_int64),
-                ("cg_products", c_int64), ("cg_fallbacks", c_int64), ("cholesky_by_policy", c_int32 * 2)]
+                ("cg_products", c_int64), ("cg_fallbacks", c_int64), ("cholesky_by_policy", c_int32 * 2),
+                ("entries_in_class", (c_int64 * ALX_N_CLASSES) * 2)]
 
 
 EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set_embeddings", "alx_set_embedding_rows",

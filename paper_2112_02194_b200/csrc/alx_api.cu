@@ -46,6 +46,7 @@ struct alx_ctx {
     float *split_partials = nullptr;
     void *dual_ws = nullptr;      // tensor path: B^-1 operand tiles and the flag of the dual form
     int64_t dual_candidates = 0;  // rows of classes 1 and 2 of the last half-epoch (solved in the dual form if the flag is set)
+    int dual_flag_latched = 0;    // that flag as the last half-epoch's kernels saw it (the loss and the Gramian calls rewrite it)
     double *loss_partials_buf = nullptr;
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
@@ -138,6 +139,34 @@ template <typename T> bool alloc_into(alx_ctx *c, T *&dst, size_t count)
                         (size_t)(count) * sizeof(*(dst)));                                         \
     } while (0)
 
+// Temporaries of one call: whatever is still registered when the call returns, on any path, goes back to the allocator
+// (after the stream has drained, since kernels in flight may still use it).
+struct Scratch {
+    alx_ctx *c;
+    std::vector<void *> held;
+    explicit Scratch(alx_ctx *ctx) : c(ctx) {}
+    Scratch(const Scratch &) = delete;
+    Scratch &operator=(const Scratch &) = delete;
+    template <typename T> T *keep(T *p) { if (p) held.push_back(p); return p; }
+    void release(void *p)
+    {
+        for (size_t k = 0; k < held.size(); ++k)
+            if (held[k] == p) { held.erase(held.begin() + k); dev_free(c, p); return; }
+    }
+    ~Scratch()
+    {
+        if (held.empty()) return;
+        cudaStreamSynchronize(c->stream);
+        for (void *p : held) dev_free(c, p);
+    }
+};
+
+#define ALX_TMP(c, scratch, dst, count)                                                            \
+    do {                                                                                           \
+        ALX_ALLOC(c, dst, count);                                                                  \
+        (scratch).keep(dst);                                                                       \
+    } while (0)
+
 // read and clear the device status word (after a stream synchronise)
 alx_status check_device_status(alx_ctx *c)
 {
@@ -150,8 +179,11 @@ alx_status check_device_status(alx_ctx *c)
     if (h.flags & kFlagBadRowptr) return fail(c, ALX_ERR_BAD_CSR, "rowptr is not a monotone offset array (near row %lld)", h.first_bad);
     if (h.flags & kFlagBadCol) return fail(c, ALX_ERR_BAD_CSR, "column index out of range at entry %lld", h.first_bad);
     if (h.flags & kFlagUnsorted) return fail(c, ALX_ERR_BAD_CSR, "column indices not strictly ascending inside a row at entry %lld", h.first_bad);
+    // a wait that ran out leaves rows unsolved, which matters more than rows set to zero: report it first
+    if (h.flags & kFlagTimeout)
+        return fail(c, ALX_ERR_CUDA, "a bounded wait inside a kernel ran out (wait site %lld, block %lld)%s", h.first_bad / 1000000,
+                    h.first_bad % 1000000, (h.flags & kFlagNotSpd) ? "; rows also met non-positive pivots" : "");
     if (h.flags & kFlagNotSpd) return fail(c, ALX_ERR_NOT_SPD, "%llu rows met a non-positive pivot (first: row %lld); they were set to zero", h.not_spd, h.first_bad);
-    if (h.flags & kFlagTimeout) return fail(c, ALX_ERR_CUDA, "a bounded wait inside a kernel ran out (wait site %lld, block %lld)", h.first_bad / 1000000, h.first_bad % 1000000);
     return fail(c, ALX_ERR_CUDA, "device status flags 0x%x", h.flags);
 }
 
@@ -183,8 +215,9 @@ alx_status build_buckets(alx_ctx *c, int side, int64_t *scratch_a, int64_t *scra
     c->n_split_rows[side] = n_split;
     c->n_chunks[side] = 0;
     if (n_split > 0) {
+        Scratch tmp(c);
         int64_t *counts = nullptr;
-        ALX_ALLOC(c, counts, n_split);
+        ALX_TMP(c, tmp, counts, n_split);
         ALX_ALLOC(c, c->split_first[side], n_split + 1);
         const int32_t *split_rows = c->order[side] + offs[ALX_N_CLASSES - 1];
         ALX_CUDA(c, launch_chunk_counts(c->ptr[side], split_rows, n_split, c->split, counts, c->stream, &c->launches));
@@ -198,7 +231,6 @@ alx_status build_buckets(alx_ctx *c, int side, int64_t *scratch_a, int64_t *scra
         ALX_CUDA(c, launch_chunk_fill(c->ptr[side], split_rows, n_split, c->split, c->split_first[side],
                                       c->chunk_desc[side], c->stream, &c->launches));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
-        dev_free(c, counts);
     }
     for (int k = 0; k < ALX_N_CLASSES; ++k) c->stats.rows_in_class[side][k] = offs[k + 1] - offs[k];
     c->stats.n_chunks[side] = c->n_chunks[side];
@@ -272,6 +304,10 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
         c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;
+        c->dual_flag_latched = 0;
+        if (c->dual_candidates > 0)
+            ALX_CUDA(c, cudaMemcpyAsync(&c->dual_flag_latched, dual_flag_ptr(c->dual_ws), sizeof(int), cudaMemcpyDeviceToHost,
+                                        c->stream));
     } else {
         ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side],
                                        c->n_split_rows[side], c->table[fixed], c->bf16, c->opt.d, c->Bmat,
@@ -426,12 +462,14 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     const int64_t nmax = n_rows > n_cols ? n_rows : n_cols;
     const int64_t nb = bucket_blocks(nmax);
     const int64_t scan_elems = scan_scratch_elems(nb * kNClasses > nmax ? nb * kNClasses : nmax) + 16;
-    int64_t *scan_scratch = nullptr, *blk_counts = nullptr, *blk_offs = nullptr;
+    Scratch tmp(c);
+    int64_t *scan_scratch = nullptr, *blk_counts = nullptr, *blk_offs = nullptr, *class_entries = nullptr;
     int32_t *counts = nullptr;
-    ALX_ALLOC(c, scan_scratch, scan_elems);
-    ALX_ALLOC(c, blk_counts, nb * kNClasses);
-    ALX_ALLOC(c, blk_offs, nb * kNClasses + 1);
-    ALX_ALLOC(c, counts, n_cols);
+    ALX_TMP(c, tmp, scan_scratch, scan_elems);
+    ALX_TMP(c, tmp, blk_counts, nb * kNClasses);
+    ALX_TMP(c, tmp, blk_offs, nb * kNClasses + 1);
+    ALX_TMP(c, tmp, counts, n_cols);
+    ALX_TMP(c, tmp, class_entries, 2 * kNClasses);
 
     // transpose: count, prefix sum, degree classes of the columns, fill, sort each column, labels
     ALX_ALLOC(c, c->ptr[1], n_cols + 1);
@@ -453,18 +491,24 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     }
     st = build_buckets(c, ALX_ROWS, blk_counts, blk_offs, scan_scratch, scan_elems);
     if (st != ALX_OK) return st;
+    for (int s = 0; s < 2; ++s)
+        ALX_CUDA(c, launch_class_entries(c->ptr[s], c->order[s], c->class_offs_dev[s], c->n[s], class_entries + s * kNClasses,
+                                         c->stream, &c->launches));
+    ALX_CUDA(c, cudaMemcpyAsync(c->stats.entries_in_class, class_entries, 2 * kNClasses * sizeof(int64_t),
+                                cudaMemcpyDeviceToHost, c->stream));
     ALX_CUDA(c, cudaStreamSynchronize(c->stream));
-    dev_free(c, counts);
-    dev_free(c, blk_offs);
-    dev_free(c, blk_counts);
-    dev_free(c, scan_scratch);
+    tmp.release(counts);
+    tmp.release(blk_offs);
+    tmp.release(blk_counts);
+    tmp.release(scan_scratch);
+    tmp.release(class_entries);
 
     const int d = c->opt.d;
     int64_t sums[2] = {c->n_chunks[0], c->n_chunks[1]};
     for (int s = 0; s < 2; ++s) c->stats.long_rows[s] = c->stats.long_entries[s] = 0;
     if (tensor_path(c)) {    // one more sum per long whole row
         int64_t *total = nullptr;
-        ALX_ALLOC(c, total, 2);
+        ALX_TMP(c, tmp, total, 2);
         for (int s = 0; s < 2; ++s) {
             const int64_t first = c->class_offs[s][long_class_begin(c->class_offs[s])];
             const int64_t n_long = c->class_offs[s][kNClasses - 1] - first;
@@ -474,7 +518,7 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
         }
         ALX_CUDA(c, cudaMemcpyAsync(c->stats.long_entries, total, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
-        dev_free(c, total);
+        tmp.release(total);
     }
     const int64_t max_chunks = sums[0] > sums[1] ? sums[0] : sums[1];
     if (max_chunks > 0) ALX_ALLOC(c, c->split_partials, max_chunks * (int64_t)(d * d + d));
@@ -492,6 +536,7 @@ alx_status alx_set_embeddings(alx_ctx *c, alx_side side, const void *src, alx_dt
     const int64_t count = c->n[side] * c->opt.d;
     const size_t src_bytes = (size_t)count * (src_dtype == ALX_BF16 ? 2 : 4);
     const void *dev_src = src;
+    Scratch tmp(c);
     void *staging = nullptr;
     if (!on_device) {
         if ((src_dtype == ALX_BF16) == (c->bf16 != 0)) {
@@ -501,14 +546,13 @@ alx_status alx_set_embeddings(alx_ctx *c, alx_side side, const void *src, alx_dt
             c->have_gram[side] = false;
             return ALX_OK;
         }
-        staging = dev_alloc(c, src_bytes);
+        staging = tmp.keep(dev_alloc(c, src_bytes));
         if (!staging) return fail(c, ALX_ERR_OOM, "staging allocation failed");
         ALX_CUDA(c, cudaMemcpyAsync(staging, src, src_bytes, cudaMemcpyHostToDevice, c->stream));
         dev_src = staging;
     }
     ALX_CUDA(c, launch_convert(dev_src, src_dtype == ALX_BF16, c->table[side], c->bf16, count, c->stream, &c->launches));
     ALX_CUDA(c, cudaStreamSynchronize(c->stream));
-    if (staging) dev_free(c, staging);
     c->have_table[side] = true;
     c->have_gram[side] = false;
     return ALX_OK;
@@ -527,13 +571,14 @@ alx_status alx_set_embedding_rows(alx_ctx *c, alx_side side, int64_t row_begin, 
     const size_t src_bytes = (size_t)count * (src_dtype == ALX_BF16 ? 2 : 4);
     char *dst = static_cast<char *>(c->table[side]) + (size_t)row_begin * c->opt.d * c->elem;
     const void *dev_src = src;
+    Scratch tmp(c);
     void *staging = nullptr;
     const bool same = (src_dtype == ALX_BF16) == (c->bf16 != 0);
     if (same) {
         ALX_CUDA(c, cudaMemcpyAsync(dst, src, src_bytes, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
     } else {
         if (!on_device) {
-            staging = dev_alloc(c, src_bytes);
+            staging = tmp.keep(dev_alloc(c, src_bytes));
             if (!staging) return fail(c, ALX_ERR_OOM, "staging allocation failed");
             ALX_CUDA(c, cudaMemcpyAsync(staging, src, src_bytes, cudaMemcpyHostToDevice, c->stream));
             dev_src = staging;
@@ -541,7 +586,6 @@ alx_status alx_set_embedding_rows(alx_ctx *c, alx_side side, int64_t row_begin, 
         ALX_CUDA(c, launch_convert(dev_src, src_dtype == ALX_BF16, dst, c->bf16, count, c->stream, &c->launches));
     }
     ALX_CUDA(c, cudaStreamSynchronize(c->stream));
-    if (staging) dev_free(c, staging);
     c->have_table[side] = true;
     c->have_gram[side] = false;
     return ALX_OK;
@@ -566,12 +610,12 @@ alx_status alx_get_embeddings(alx_ctx *c, alx_side side, void *dst, alx_dtype ds
     } else if (same) {
         ALX_CUDA(c, cudaMemcpyAsync(dst, src, dst_bytes, cudaMemcpyDeviceToHost, c->stream));
     } else {
-        void *staging = dev_alloc(c, dst_bytes);
+        Scratch tmp(c);
+        void *staging = tmp.keep(dev_alloc(c, dst_bytes));
         if (!staging) return fail(c, ALX_ERR_OOM, "staging allocation failed");
         ALX_CUDA(c, launch_convert(src, c->bf16, staging, dst_dtype == ALX_BF16, count, c->stream, &c->launches));
         ALX_CUDA(c, cudaMemcpyAsync(dst, staging, dst_bytes, cudaMemcpyDeviceToHost, c->stream));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
-        dev_free(c, staging);
     }
     return check_device_status(c);
 }
@@ -656,10 +700,11 @@ alx_status alx_half_epoch_capture(alx_ctx *c, alx_side side, const int64_t *row_
     DeviceGuard guard(c->device);
     const int64_t n = c->n[side];
     const int d = c->opt.d;
+    Scratch tmp(c);
     int32_t *slot = nullptr;
     float *cap = nullptr;
-    ALX_ALLOC(c, slot, n);
-    ALX_ALLOC(c, cap, (k > 0 ? k : 1) * d);
+    ALX_TMP(c, tmp, slot, n);
+    ALX_TMP(c, tmp, cap, (k > 0 ? k : 1) * d);
     std::vector<int32_t> h(n, -1);
     for (int64_t j = 0; j < k; ++j) h[row_ids[j]] = (int32_t)j;   // a repeated id keeps its last slot
     ALX_CUDA(c, cudaMemcpyAsync(slot, h.data(), sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream));
@@ -674,8 +719,6 @@ alx_status alx_half_epoch_capture(alx_ctx *c, alx_side side, const int64_t *row_
     } else {
         cudaStreamSynchronize(c->stream);
     }
-    dev_free(c, slot);
-    dev_free(c, cap);
     return st;
 }
 
@@ -771,12 +814,7 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
     if (c->main_timed) {
         if (cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]) == cudaSuccess) c->stats.ms_main_kernel = ms; else cudaGetLastError();
     }
-    c->stats.dual_rows = 0;
-    if (c->dual_candidates > 0 && c->dual_ws) {
-        int flag = 0;
-        ALX_CUDA(c, cudaMemcpy(&flag, dual_flag_ptr(c->dual_ws), sizeof flag, cudaMemcpyDeviceToHost));
-        c->stats.dual_rows = flag ? c->dual_candidates : 0;
-    }
+    c->stats.dual_rows = c->dual_candidates > 0 && c->dual_flag_latched ? c->dual_candidates : 0;
     {
         unsigned long long h[3] = {0, 0, 0};
         ALX_CUDA(c, cudaMemcpy(h, c->cg_counters, sizeof h, cudaMemcpyDeviceToHost));

@@ -90,6 +90,9 @@ int64_t scan_scratch_elems(int64_t n);
 cudaError_t launch_validate(const int64_t *rowptr, const int32_t *colidx, int64_t n_rows, int64_t n_cols,
                             int64_t nnz, DevStatus *st, cudaStream_t s, int64_t *launches);
 cudaError_t launch_degrees(const int64_t *ptr, int64_t n, int32_t *deg, cudaStream_t s, int64_t *launches);
+// entries held by the rows of each degree class: out[kNClasses] (device), class_offs = the kNClasses + 1 offsets into order
+cudaError_t launch_class_entries(const int64_t *ptr, const int32_t *order, const int64_t *class_offs_dev, int64_t n,
+                                 int64_t *out, cudaStream_t s, int64_t *launches);
 cudaError_t launch_sum_row_lengths(const int64_t *ptr, const int32_t *rows, int64_t count, int64_t *out, cudaStream_t s,
                                    int64_t *launches);
 cudaError_t launch_count_cols(const int32_t *colidx, int64_t nnz, int32_t *counts, cudaStream_t s, int64_t *launches);

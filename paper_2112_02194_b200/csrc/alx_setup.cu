@@ -2,8 +2,8 @@
 // column), degree-class ordering of rows, chunk descriptors of long rows, prefix sums, and the
 // storage-type conversion used when tables are copied in or out.
 //
-// The paper gives S as per-row histories and asks for "a similar pass over the item side"
-// (Alg. 1 line 11), which needs the transpose; its dense batching (Sec. 4.3) tames the long tail
+// The paper gives S as per-row histories; the item-side pass of Alg. 1 line 11 reads the same entries column by
+// column, which needs the transpose; its dense batching (Sec. 4.3) tames the long tail
 // of row lengths, which here is the job of the degree classes and the chunk descriptors.
 #include "alx_common.cuh"
 
@@ -440,6 +440,39 @@ __global__ void k_sum_row_lengths(const int64_t *__restrict__ ptr, const int32_t
         __syncthreads();
     }
     if (threadIdx.x == 0) *out = part[0];
+}
+
+// entries per degree class: position k of `order` belongs to the class whose offset range holds k
+__global__ void __launch_bounds__(256) k_class_entries(const int64_t *__restrict__ ptr, const int32_t *__restrict__ order,
+                                                       const int64_t *__restrict__ class_offs, int64_t n,
+                                                       unsigned long long *__restrict__ out)
+{
+    __shared__ unsigned long long part[kNClasses];
+    __shared__ int64_t offs[kNClasses + 1];
+    if (threadIdx.x <= kNClasses) offs[threadIdx.x] = class_offs[threadIdx.x];
+    if (threadIdx.x < kNClasses) part[threadIdx.x] = 0;
+    __syncthreads();
+    for (int64_t k = (int64_t)blockIdx.x * 256 + threadIdx.x; k < n; k += (int64_t)gridDim.x * 256) {
+        int c = 0;
+        while (c + 1 < kNClasses && k >= offs[c + 1]) ++c;
+        const int32_t u = order[k];
+        const unsigned long long len = (unsigned long long)(ptr[u + 1] - ptr[u]);
+        if (len) atomicAdd(&part[c], len);
+    }
+    __syncthreads();
+    if (threadIdx.x < kNClasses && part[threadIdx.x]) atomicAdd(&out[threadIdx.x], part[threadIdx.x]);
+}
+
+cudaError_t launch_class_entries(const int64_t *ptr, const int32_t *order, const int64_t *class_offs_dev, int64_t n,
+                                 int64_t *out, cudaStream_t s, int64_t *launches)
+{
+    cudaError_t e = cudaMemsetAsync(out, 0, sizeof(int64_t) * kNClasses, s);
+    if (e != cudaSuccess) return e;
+    const int64_t blocks = (n + 255) / 256;
+    k_class_entries<<<(unsigned)(blocks < 1184 ? (blocks > 0 ? blocks : 1) : 1184), 256, 0, s>>>(
+        ptr, order, class_offs_dev, n, reinterpret_cast<unsigned long long *>(out));
+    ++*launches;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_sum_row_lengths(const int64_t *ptr, const int32_t *rows, int64_t count, int64_t *out, cudaStream_t s,

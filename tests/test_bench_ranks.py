@@ -42,3 +42,30 @@ def test_roofline_terms_match_the_stated_per_unit_costs():
     assert abs(b - 265.2e9) / 265.2e9 < 0.01          # bytes per half-epoch of the 10M x 10M workload
     assert abs(t - 3.31e13) / 3.31e13 < 0.01
     assert abs(a - 7.74e12) / 7.74e12 < 0.01
+
+
+def test_replica_command_is_one_process_per_gpu_on_this_node():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.replica_command(["--gpus", "4", "--steps", "2"], 4, 29555)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29555"
+    k = cmd.index(os.path.join(ROOT, "bench.py"))
+    assert cmd[k + 1:] == ["--gpus", "4", "--steps", "2"]
+
+
+def test_plain_launch_with_two_gpus_spawns_two_ranks_and_prints_one_line():
+    """`python bench.py --gpus 2` without a launcher's environment starts the ranks itself.  Run on the reference arm
+    (CPU only): rank 0 alone works and prints, the other rank exits 0, the launcher passes the exit code on."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--workload", "small", "--steps", "1", "--warmup", "0"], env=env, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0
