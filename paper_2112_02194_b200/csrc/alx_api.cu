@@ -20,24 +20,27 @@ struct alx_ctx {
     cudaStream_t stream = nullptr;
     int bf16 = 0;
     size_t elem = 4;
-    int64_t n[2] = {0, 0};   // n[ALX_ROWS] = n_rows, n[ALX_COLS] = n_cols
+    int64_t n[4] = {0, 0, 0, 0};   // n[ALX_ROWS] = n_rows, n[ALX_COLS] = n_cols (and again for the doubled lists, see below)
     int64_t nnz = -1;
     int64_t split = ALX_DEFAULT_SPLIT;
     bool has_values = false;
     bool have_table[2] = {false, false};
     bool have_gram[2] = {false, false};
 
-    // per orientation: [ALX_ROWS] = CSR (rows of the matrix), [ALX_COLS] = CSC
-    int64_t *ptr[2] = {nullptr, nullptr};
-    int32_t *idx[2] = {nullptr, nullptr};
-    float *val[2] = {nullptr, nullptr};
-    int32_t *order[2] = {nullptr, nullptr};
-    int64_t *class_offs_dev[2] = {nullptr, nullptr};
-    int64_t class_offs[2][ALX_N_CLASSES + 1] = {};
-    int64_t *chunk_desc[2] = {nullptr, nullptr};
-    int64_t *split_first[2] = {nullptr, nullptr};
-    int64_t n_chunks[2] = {0, 0};
-    int64_t n_split_rows[2] = {0, 0};
+    // per orientation: [ALX_ROWS] = CSR (rows of the matrix), [ALX_COLS] = CSC.  Slots 2 and 3 (fp32 tables of 64 features
+    // on the tensor cores only): the same two orientations with every row's entry list doubled over the table of
+    // bfloat16 parts, which is what that path's kernels walk; with degree classes and chunks of their own.
+    int64_t *ptr[4] = {nullptr, nullptr, nullptr, nullptr};
+    int32_t *idx[4] = {nullptr, nullptr, nullptr, nullptr};
+    float *val[4] = {nullptr, nullptr, nullptr, nullptr};
+    int32_t *order[4] = {nullptr, nullptr, nullptr, nullptr};
+    int64_t *class_offs_dev[4] = {nullptr, nullptr, nullptr, nullptr};
+    int64_t class_offs[4][ALX_N_CLASSES + 1] = {};
+    int64_t *chunk_desc[4] = {nullptr, nullptr, nullptr, nullptr};
+    int64_t *split_first[4] = {nullptr, nullptr, nullptr, nullptr};
+    int64_t n_chunks[4] = {0, 0, 0, 0};
+    int64_t n_split_rows[4] = {0, 0, 0, 0};
+    void *fold_table = nullptr;   // that path's fixed table: [2 N x 128] bfloat16 parts of the fp32 table, rebuilt every half-epoch
 
     void *table[2] = {nullptr, nullptr};
     double *G64[2] = {nullptr, nullptr};   // Gramian of table [side]
@@ -232,14 +235,16 @@ alx_status build_buckets(alx_ctx *c, int side, int64_t *scratch_a, int64_t *scra
                                       c->chunk_desc[side], c->stream, &c->launches));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
     }
-    for (int k = 0; k < ALX_N_CLASSES; ++k) c->stats.rows_in_class[side][k] = offs[k + 1] - offs[k];
-    c->stats.n_chunks[side] = c->n_chunks[side];
+    if (side < 2) {
+        for (int k = 0; k < ALX_N_CLASSES; ++k) c->stats.rows_in_class[side][k] = offs[k + 1] - offs[k];
+        c->stats.n_chunks[side] = c->n_chunks[side];
+    }
     return ALX_OK;
 }
 
 void release_matrix(alx_ctx *c)
 {
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < 4; ++s) {
         dev_free(c, c->ptr[s]); c->ptr[s] = nullptr;
         dev_free(c, c->idx[s]); c->idx[s] = nullptr;
         dev_free(c, c->val[s]); c->val[s] = nullptr;
@@ -253,6 +258,11 @@ void release_matrix(alx_ctx *c)
 }
 
 bool tensor_path(const alx_ctx *c) { return c->bf16 && c->opt.d == 128 && c->opt.kernels != 1; }
+// fp32 tables of 64 features: tensor cores through bfloat16 parts and doubled entry lists (ids up to 2 N must fit int32)
+bool fold_path(const alx_ctx *c)
+{
+    return !c->bf16 && c->opt.d == 64 && c->opt.kernels != 1 && c->n[0] < (1ll << 30) && c->n[1] < (1ll << 30);
+}
 bool dual_form(const alx_ctx *c) { return tensor_path(c) && c->opt.kernels == 0; }
 CgOptions cg_options(const alx_ctx *c, int solved_side)
 {
@@ -295,7 +305,17 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     if (st != ALX_OK) return st;
     ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
     RowOut out{c->table[side], cap_slot, cap_out};
-    if (tensor_path(c)) {
+    if (fold_path(c)) {
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
+        ALX_CUDA(c, launch_split_table(static_cast<const float *>(c->table[fixed]), c->n[fixed], c->fold_table, c->stream,
+                                       &c->launches));
+        ALX_CUDA(c, launch_rows_fold(side_view(c, 2 + side), c->class_offs[2 + side], c->n_chunks[2 + side],
+                                     c->n_split_rows[2 + side], c->fold_table, 2 * c->n[fixed], c->Bmat, c->split_partials,
+                                     out, c->status, c->stream, &c->launches, c->ev[3], c->ev[4], cg_options(c, side)));
+        c->stats.kernel_path[side] = 1;
+        c->main_timed = true;
+        c->dual_candidates = 0;
+    } else if (tensor_path(c)) {
         ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
@@ -365,8 +385,8 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
     c->stream = static_cast<cudaStream_t>(opt->stream);
     c->bf16 = opt->storage == ALX_BF16;
     c->elem = c->bf16 ? 2 : 4;
-    c->n[ALX_ROWS] = opt->n_rows;
-    c->n[ALX_COLS] = opt->n_cols;
+    c->n[ALX_ROWS] = c->n[2 + ALX_ROWS] = opt->n_rows;
+    c->n[ALX_COLS] = c->n[2 + ALX_COLS] = opt->n_cols;
     c->split = opt->split ? opt->split : ALX_DEFAULT_SPLIT;
     DeviceGuard guard(dev);
     auto body = [&]() -> alx_status {
@@ -377,6 +397,7 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
             c->table[s] = t;
             ALX_ALLOC(c, c->G64[s], d * d);
             ALX_ALLOC(c, c->class_offs_dev[s], ALX_N_CLASSES + 1);
+            if (fold_path(c)) ALX_ALLOC(c, c->class_offs_dev[2 + s], ALX_N_CLASSES + 1);
         }
         ALX_ALLOC(c, c->Bmat, d * d);
         if (dual_form(c)) {
@@ -384,6 +405,10 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
             if (!c->dual_ws) return fail(c, ALX_ERR_OOM, "device allocation of the dual-form workspace failed");
         }
         const int64_t nmax = c->n[0] > c->n[1] ? c->n[0] : c->n[1];
+        if (fold_path(c)) {
+            c->fold_table = dev_alloc(c, (size_t)2 * nmax * 128 * 2);
+            if (!c->fold_table) return fail(c, ALX_ERR_OOM, "device allocation of the table of bfloat16 parts failed");
+        }
         int64_t n_part = gramian_partials(nmax);
         if (gramian_umma_partials() > n_part) n_part = gramian_umma_partials();
         ALX_ALLOC(c, c->gram_partials, n_part * d * d);
@@ -491,6 +516,19 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     }
     st = build_buckets(c, ALX_ROWS, blk_counts, blk_offs, scan_scratch, scan_elems);
     if (st != ALX_OK) return st;
+    if (fold_path(c)) {
+        // the doubled entry lists of both orientations, with degree classes and chunks of their own
+        for (int s = 0; s < 2; ++s) {
+            ALX_ALLOC(c, c->ptr[2 + s], c->n[s] + 1);
+            ALX_ALLOC(c, c->idx[2 + s], 2 * nz);
+            if (values) ALX_ALLOC(c, c->val[2 + s], 2 * nz);
+            ALX_ALLOC(c, c->order[2 + s], c->n[s]);
+            ALX_CUDA(c, launch_double_entries(c->ptr[s], c->idx[s], c->val[s], c->n[s], c->n[1 - s], c->ptr[2 + s],
+                                              c->idx[2 + s], c->val[2 + s], c->stream, &c->launches));
+            st = build_buckets(c, 2 + s, blk_counts, blk_offs, scan_scratch, scan_elems);
+            if (st != ALX_OK) return st;
+        }
+    }
     for (int s = 0; s < 2; ++s)
         ALX_CUDA(c, launch_class_entries(c->ptr[s], c->order[s], c->class_offs_dev[s], c->n[s], class_entries + s * kNClasses,
                                          c->stream, &c->launches));
@@ -504,24 +542,28 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     tmp.release(class_entries);
 
     const int d = c->opt.d;
-    int64_t sums[2] = {c->n_chunks[0], c->n_chunks[1]};
+    const int kb = fold_path(c) ? 2 : 0;      // the lists the row kernels walk
+    const int dk = fold_path(c) ? 128 : d;    // the width of the sums they form
+    int64_t sums[2] = {c->n_chunks[kb], c->n_chunks[kb + 1]};
     for (int s = 0; s < 2; ++s) c->stats.long_rows[s] = c->stats.long_entries[s] = 0;
-    if (tensor_path(c)) {    // one more sum per long whole row
+    if (tensor_path(c) || fold_path(c)) {    // one more sum per long whole row
         int64_t *total = nullptr;
         ALX_TMP(c, tmp, total, 2);
         for (int s = 0; s < 2; ++s) {
-            const int64_t first = c->class_offs[s][long_class_begin(c->class_offs[s])];
-            const int64_t n_long = c->class_offs[s][kNClasses - 1] - first;
+            const int64_t *offs = c->class_offs[kb + s];
+            const int64_t first = offs[long_class_begin(offs)];
+            const int64_t n_long = offs[kNClasses - 1] - first;
             sums[s] += n_long;
             c->stats.long_rows[s] = n_long;
-            ALX_CUDA(c, launch_sum_row_lengths(c->ptr[s], c->order[s] + first, n_long, total + s, c->stream, &c->launches));
+            ALX_CUDA(c, launch_sum_row_lengths(c->ptr[kb + s], c->order[kb + s] + first, n_long, total + s, c->stream, &c->launches));
         }
         ALX_CUDA(c, cudaMemcpyAsync(c->stats.long_entries, total, 2 * sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+        if (fold_path(c)) for (int s = 0; s < 2; ++s) c->stats.long_entries[s] /= 2;      // (every entry is listed twice there)
         tmp.release(total);
     }
     const int64_t max_chunks = sums[0] > sums[1] ? sums[0] : sums[1];
-    if (max_chunks > 0) ALX_ALLOC(c, c->split_partials, max_chunks * (int64_t)(d * d + d));
+    if (max_chunks > 0) ALX_ALLOC(c, c->split_partials, max_chunks * (int64_t)(dk * dk + dk));
     ALX_ALLOC(c, c->loss_partials_buf, loss_partials(nnz));
     c->stats.nnz = nnz;
     return ALX_OK;

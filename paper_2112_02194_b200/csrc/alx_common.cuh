@@ -90,6 +90,10 @@ int64_t scan_scratch_elems(int64_t n);
 cudaError_t launch_validate(const int64_t *rowptr, const int32_t *colidx, int64_t n_rows, int64_t n_cols,
                             int64_t nnz, DevStatus *st, cudaStream_t s, int64_t *launches);
 cudaError_t launch_degrees(const int64_t *ptr, int64_t n, int32_t *deg, cudaStream_t s, int64_t *launches);
+// Entry lists over a table of 2N rows (the bfloat16 parts of an fp32 table, see launch_rows_fold): row u of length L
+// becomes a row of 2L entries, its L ids followed by the same ids + N (labels repeated); vptr = 2 ptr.
+cudaError_t launch_double_entries(const int64_t *ptr, const int32_t *idx, const float *val, int64_t n, int64_t n_fixed,
+                                  int64_t *vptr, int32_t *vidx, float *vval, cudaStream_t s, int64_t *launches);
 // entries held by the rows of each degree class: out[kNClasses] (device), class_offs = the kNClasses + 1 offsets into order
 cudaError_t launch_class_entries(const int64_t *ptr, const int32_t *order, const int64_t *class_offs_dev, int64_t n,
                                  int64_t *out, cudaStream_t s, int64_t *launches);
@@ -172,6 +176,12 @@ struct CgOptions {
 // alx_umma.cu: tensor-core path, d = 128 and bf16 tables only
 int64_t gramian_umma_partials();
 cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches);
+cudaError_t launch_rows_fold(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks, int64_t n_split_rows,
+                             const void *T, int64_t n_table, const float *Bmat, float *split_partials, RowOut out,
+                             DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
+                             const CgOptions &cg);
+// fp32 table [n x 64] -> bfloat16 parts [2n x 128]
+cudaError_t launch_split_table(const float *X, int64_t n, void *T, cudaStream_t s, int64_t *launches);
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                              int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
                              RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,

@@ -442,6 +442,41 @@ __global__ void k_sum_row_lengths(const int64_t *__restrict__ ptr, const int32_t
     if (threadIdx.x == 0) *out = part[0];
 }
 
+// doubled entry lists: one warp per row
+__global__ void __launch_bounds__(256) k_double_entries(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
+                                                        const float *__restrict__ val, int64_t n, int64_t n_fixed,
+                                                        int64_t *__restrict__ vptr, int32_t *__restrict__ vidx,
+                                                        float *__restrict__ vval)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * 8;
+    for (int64_t u = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); u <= n; u += warps) {
+        const int64_t beg = ptr[u];
+        if (lane == 0) vptr[u] = 2 * beg;
+        if (u == n) break;
+        const int64_t len = ptr[u + 1] - beg;
+        for (int64_t j = lane; j < len; j += 32) {
+            const int32_t c = idx[beg + j];
+            vidx[2 * beg + j] = c;
+            vidx[2 * beg + len + j] = (int32_t)(c + n_fixed);
+            if (val) {
+                const float y = val[beg + j];
+                vval[2 * beg + j] = y;
+                vval[2 * beg + len + j] = y;
+            }
+        }
+    }
+}
+
+cudaError_t launch_double_entries(const int64_t *ptr, const int32_t *idx, const float *val, int64_t n, int64_t n_fixed,
+                                  int64_t *vptr, int32_t *vidx, float *vval, cudaStream_t s, int64_t *launches)
+{
+    const int64_t blocks = (n + 1 + 7) / 8;
+    k_double_entries<<<(unsigned)(blocks < 148 * 16 ? blocks : 148 * 16), 256, 0, s>>>(ptr, idx, val, n, n_fixed, vptr, vidx, vval);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 // entries per degree class: position k of `order` belongs to the class whose offset range holds k
 __global__ void __launch_bounds__(256) k_class_entries(const int64_t *__restrict__ ptr, const int32_t *__restrict__ order,
                                                        const int64_t *__restrict__ class_offs, int64_t n,

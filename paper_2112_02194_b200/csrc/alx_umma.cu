@@ -47,7 +47,7 @@ constexpr int kStageRows = 32;
 template <int MODE> struct Ring {
     static constexpr int kRows = (MODE == 0) ? 32 : 64;   // gathered rows per stage
     // (the conjugate-gradient rows kernel needs no operand tiles for a factorisation: their space goes to its ring)
-    static constexpr int kNStage = (MODE == 0 || MODE == 3) ? 8 : 12;
+    static constexpr int kNStage = (MODE == 0 || MODE >= 3) ? 8 : 12;
     static constexpr int kHalfBytes = kRows * 128;        // one 64-feature half of a stage
     static constexpr int kStageHBytes = 2 * kHalfBytes;
     static constexpr int kStageYBytes = 2 * kRows * 16;   // label tile, two 8-column chunks
@@ -65,8 +65,13 @@ constexpr int kGramSubRows = 256;                     // rows per tensor-memory 
 constexpr int kGramBlocks = 148;                      // fixed, so that the order of sums depends on sizes only
 
 // kModeRowsCg: whole rows as kModeRows, solved by conjugate gradients instead of the in-place Cholesky
-enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2, kModeRowsCg = 3 };
-__host__ __device__ constexpr bool is_rows(int mode) { return mode == kModeRows || mode == kModeRowsCg; }
+// kModeRowsFold: the feed of kModeRowsCg for fp32 tables of 64 features.  The fixed table is given as 2N rows of 128
+//                bfloat16 values, [x1 | x2] and [x1 | x3] with x = x1 + x2 + x3 to 2^-24, and every row's entry list names
+//                both rows of each of its entries; the 128 x 128 sums S then hold the 64 x 64 sum of outer products as
+//                S11 / 2 + S12 + S21 + S22 (and the right-hand side as s1 / 2 + s2), which the solver folds and solves.
+enum Mode { kModeRows = 0, kModeChunks = 1, kModeGramian = 2, kModeRowsCg = 3, kModeRowsFold = 4 };
+__host__ __device__ constexpr bool is_cg(int mode) { return mode == kModeRowsCg || mode == kModeRowsFold; }
+__host__ __device__ constexpr bool is_rows(int mode) { return mode == kModeRows || is_cg(mode); }
 
 // thread layout per mode: solver groups (one accumulator each), then one MMA warp, then the producer warps
 template <int MODE> struct Cfg {
@@ -83,7 +88,7 @@ template <int MODE> struct Cfg {
     static constexpr int kFullArrivals = (MODE == kModeRows) ? kProducerWarps : 1;
     // a stage is free again when the tensor core has read it -- and, in the conjugate-gradient rows kernel, when the
     // producer warp that gathered it has summed y x over its rows
-    static constexpr int kEmptyArrivals = (MODE == kModeRowsCg) ? 2 : 1;
+    static constexpr int kEmptyArrivals = is_cg(MODE) ? 2 : 1;
     static constexpr int kBlockThreads = kSolverThreads + 32 + kProducers * 32;
 };
 
@@ -150,12 +155,12 @@ template <int MODE> struct __align__(1024) SmemT {
     unsigned char h[kNStage][Ring<MODE>::kStageHBytes];
     unsigned char y[is_rows(MODE) ? 1 : kNStage][Ring<MODE>::kStageYBytes];      // label tiles (chunks mode only)
     uint64_t full[kNStage], empty[kNStage], acc_full[kMaxGroups], acc_empty[kMaxGroups];
-    uint64_t rhs_done[MODE == kModeRowsCg ? Ring<MODE>::kBRing : 1];   // conjugate-gradient rows kernel: an item's right-hand side is written
+    uint64_t rhs_done[is_cg(MODE) ? Ring<MODE>::kBRing : 1];   // conjugate-gradient rows kernel: an item's right-hand side is written
     uint32_t tmem_base;
     int abort_flag;
     // rows modes: the producer warps also sum y x_i of the rows they staged.  kModeRows: the four warps share every stage
     // (four partial sums per item); kModeRowsCg: a warp gathers whole items (one sum per item)
-    static constexpr int kRhsParts = (MODE == kModeRowsCg) ? 1 : kProducerWarps;
+    static constexpr int kRhsParts = is_cg(MODE) ? 1 : kProducerWarps;
     float ylab[kNStage][Ring<MODE>::kRows];      // labels of the staged rows
     int stage_meta[kNStage];                     // K steps of the stage (1 or 2) | 4 if it ends its item; -1: no more work
     int rows_staged[kProducerWarps][kNStage];    // kModeRows, per producer warp: how many of its 8 rows of the stage are defined
@@ -1417,17 +1422,284 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
 
 
 
+// ---------------------------------------------------------------------------------------------------------
+// kModeRowsFold: the 64 x 64 system of an fp32 table of 64 features (Eq. 4), folded out of the 128 x 128 sums.
+// A solver group's 128 threads hold the folded matrix in registers: thread (i, h) = (tid & 63, tid >> 6) has columns
+// 32 h .. 32 h + 31 of row i.  Conjugate gradients (Sec. 4.5) run on it with the vector in shared memory (two named
+// barriers per step); a row that does not converge, and every row under the Cholesky option, is factored in shared
+// memory column by column.
+constexpr int kFoldD = 64;
+constexpr int kFoldLd = 65;                              // row stride of the matrix in shared memory (bank = row + column)
+struct __align__(128) FoldGroupSmem {
+    float M[kFoldD * 66];                                // the exchange buffers of the fold, then the matrix of the direct solve
+    alignas(16) float vec[kFoldD];                       // the vector of the next product
+    float ws[2][kFoldD];                                 // the two column halves' parts of a product
+    alignas(16) float red[4][4];                         // per-warp sums of a step
+    float dinv[kFoldD];
+    float zs[kFoldD];
+    int bad;
+    int stop;
+};
+static_assert(kMaxGroups * sizeof(FoldGroupSmem) <= sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem),
+              "the fold's scratch takes the place of the 128-feature solver's");
+
+// Conjugate gradients on the folded matrix: a[k] = A[i][32 h + k], b and x0 = this row's components.  Same recurrences,
+// start rule and stopping rule as cg_in_tmem.  Returns true with x_i when |r| <= tol |b|.
+__device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, const float (&a)[32], int bar_id, int tid,
+                                        float b, float x0, float &x_out, int &matvecs)
+{
+    const int lane = tid & 31, w = tid >> 5, i = tid & 63, h = tid >> 6;
+    // product with the vector in gs.vec: my half row's part, with this thread's share of r.w (v = the vector's own
+    // component); the parts and the warps' sums go through shared memory behind one barrier
+    auto product_and_sums = [&](float v, float bb_term, float &gsum, float &dl, float &bsum) {
+        float acc0 = 0.f, acc1 = 0.f;
+        const float4 *vp = reinterpret_cast<const float4 *>(gs.vec + 32 * h);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float4 q = vp[k];
+            acc0 = fmaf(a[4 * k], q.x, acc0);
+            acc1 = fmaf(a[4 * k + 1], q.y, acc1);
+            acc0 = fmaf(a[4 * k + 2], q.z, acc0);
+            acc1 = fmaf(a[4 * k + 3], q.w, acc1);
+        }
+        const float part = acc0 + acc1;
+        gs.ws[h][i] = part;
+        float s0 = h == 0 ? v * v : 0.f, s1 = v * part, s2 = h == 0 ? bb_term : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, o);
+            s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+            s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+        }
+        if (lane == 0) *reinterpret_cast<float4 *>(&gs.red[w][0]) = make_float4(s0, s1, s2, 0.f);
+        group128_sync(bar_id);
+        const float4 r0 = *reinterpret_cast<const float4 *>(&gs.red[0][0]), r1 = *reinterpret_cast<const float4 *>(&gs.red[1][0]),
+                     r2 = *reinterpret_cast<const float4 *>(&gs.red[2][0]), r3 = *reinterpret_cast<const float4 *>(&gs.red[3][0]);
+        gsum = r0.x + r1.x;
+        dl = ((r0.y + r1.y) + r2.y) + r3.y;
+        bsum = r0.z + r1.z;
+        return gs.ws[0][i] + gs.ws[1][i];
+    };
+    bool warm = p.cg_warm != 0;
+    float x = warm ? x0 : 0.f, r = b, pdir = 0.f, sdir = 0.f;
+    float rg_old = 0.f, inv_alpha_old = 0.f, bb = 0.f;
+    int products = 0;
+    if (h == 0) gs.vec[i] = warm ? x0 : b;
+    group128_sync(bar_id);
+    if (warm) {                 // r = b - A x0
+        float g0, d0, b0;
+        r = b - product_and_sums(x0, 0.f, g0, d0, b0);
+        ++products;
+        // (the vector was read before the barrier inside the product; the parts and sums are read before the next one)
+        if (h == 0) gs.vec[i] = r;
+        group128_sync(bar_id);
+    }
+    bool ok = false;
+    for (int it = 0;; ++it) {
+        float gsum, dl, bsum;
+        const float wv = product_and_sums(r, b * b, gsum, dl, bsum);
+        ++products;
+        if (it == 0) bb = bsum;
+        if (it == 0 && warm && !(gsum <= bb)) {
+            // the start vector is further from the solution than zero is: start again from zero
+            warm = false;
+            x = 0.f;
+            r = b;
+            if (h == 0) gs.vec[i] = r;
+            group128_sync(bar_id);
+            it = -1;
+            continue;
+        }
+        if (gsum <= p.cg_tol2 * bb) { ok = true; break; }        // (also b = 0: x = 0)
+        if (it >= p.cg_max_iter) break;
+        const float rg = __fdividef(1.f, gsum);
+        const float beta = gsum * rg_old;                        // 0 at the first step
+        const float inv_alpha = dl * rg - beta * inv_alpha_old;  // p.A p / |r|^2
+        if (!(inv_alpha > 0.f) || !(inv_alpha <= 3.0e38f)) break;
+        const float alpha = __fdividef(1.f, inv_alpha);
+        pdir = fmaf(beta, pdir, r);
+        sdir = fmaf(beta, sdir, wv);
+        x = fmaf(alpha, pdir, x);
+        r = fmaf(-alpha, sdir, r);
+        rg_old = rg;
+        inv_alpha_old = inv_alpha;
+        if (h == 0) gs.vec[i] = r;
+        group128_sync(bar_id);
+    }
+    group128_sync(bar_id);          // (the scratch is free for whatever follows)
+    matvecs = products;
+    x_out = x;
+    return ok;
+}
+
+// Direct solve of the folded system: the matrix goes to shared memory, Cholesky column by column, then the two
+// substitutions, one column per step.  Returns x_i; a non-positive pivot sets gs.bad.
+__device__ __forceinline__ float fold_cholesky(FoldGroupSmem &gs, const float (&a)[32], int bar_id, int tid, float b)
+{
+    const int i = tid & 63, h = tid >> 6;
+    float *M = gs.M;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) M[i * kFoldLd + 32 * h + k] = a[k];
+    group128_sync(bar_id);
+    for (int k = 0; k < kFoldD; ++k) {
+        const float piv = M[k * kFoldLd + k];
+        if (!(piv > 0.f)) {             // (every thread reads the same value)
+            if (tid == 0) gs.bad = 1;
+            return 0.f;
+        }
+        const float inv = rsqrtf(piv);
+        if (tid == 0) gs.dinv[k] = inv;
+        if (h == 0 && i > k) M[i * kFoldLd + k] *= inv;
+        group128_sync(bar_id);
+        // trailing update of the lower triangle: row i, columns k + 1 .. i, every second one per half
+        if (i > k) {
+            const float lik = M[i * kFoldLd + k];
+            for (int c = k + 1 + h; c <= i; c += 2) M[i * kFoldLd + c] = fmaf(-lik, M[c * kFoldLd + k], M[i * kFoldLd + c]);
+        }
+        group128_sync(bar_id);
+    }
+    // L z = b, then L^T x = z: the thread of row i carries its component; column k is final at step k
+    float v = b;
+    for (int k = 0; k < kFoldD; ++k) {
+        if (tid == k) gs.zs[k] = v * gs.dinv[k];
+        group128_sync(bar_id);
+        if (i > k) v = fmaf(-M[i * kFoldLd + k], gs.zs[k], v);
+    }
+    group128_sync(bar_id);
+    v = gs.zs[i];
+    group128_sync(bar_id);
+    for (int k = kFoldD - 1; k >= 0; --k) {
+        if (tid == k) gs.zs[k] = v * gs.dinv[k];
+        group128_sync(bar_id);
+        if (i < k) v = fmaf(-M[k * kFoldLd + i], gs.zs[k], v);
+    }
+    group128_sync(bar_id);
+    const float x = gs.zs[i];
+    group128_sync(bar_id);
+    return x;
+}
+
+// Adds alpha0 G + lambda I (64 x 64, from global memory: 16 KB that stay in L1) to the folded half row, solves, stores.
+__device__ __forceinline__ void fold_solve_store(const Params &p, FoldGroupSmem &gs, float (&a)[32], int bar_id, int tid,
+                                                 int64_t u, float b, float x0, bool use_cg, unsigned &cg_rows,
+                                                 unsigned &cg_matvecs, unsigned &cg_fallbacks)
+{
+    const int i = tid & 63, h = tid >> 6;
+    const float4 *Bp = reinterpret_cast<const float4 *>(p.Bmat + i * kFoldD + 32 * h);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const float4 q = __ldg(Bp + k);
+        a[4 * k] += q.x; a[4 * k + 1] += q.y; a[4 * k + 2] += q.z; a[4 * k + 3] += q.w;
+    }
+    float x = 0.f;
+    bool solved = false;
+    if (use_cg) {
+        int matvecs = 0;
+        solved = fold_cg(p, gs, a, bar_id, tid, b, x0, x, matvecs);
+        if (tid == 0) {
+            ++cg_rows;
+            cg_matvecs += matvecs;
+            if (!solved) ++cg_fallbacks;
+        }
+    }
+    if (!solved) x = fold_cholesky(gs, a, bar_id, tid, b);
+    group128_sync(bar_id);
+    const bool ok = gs.bad == 0;
+    const float xo = ok ? x : 0.f;
+    if (h == 0) {
+        reinterpret_cast<float *>(p.out.table)[u * kFoldD + i] = xo;
+        if (p.out.cap_slot) {
+            const int cs = p.out.cap_slot[u];
+            if (cs >= 0) p.out.cap_out[(int64_t)cs * kFoldD + i] = xo;
+        }
+    }
+    if (!ok && tid == 0) {
+        atomicAdd(&p.st->not_spd, 1ull);
+        raise_flag(p.st, kFlagNotSpd, u);
+    }
+    group128_sync(bar_id);
+    if (tid == 0) gs.bad = 0;
+}
+
+// solver group of the kModeRowsFold kernel
+template <class SmemRows>
+__device__ void solver_rows_fold(const Params &p, SmemRows &sm, FoldGroupSmem &gs, int gidx, int tid)
+{
+    constexpr int kGroups = Cfg<kModeRows>::kGroups, kAccStride = Cfg<kModeRows>::kAccStride;
+    constexpr int kBRing = Ring<kModeRowsFold>::kBRing;
+    const int w = tid >> 5;
+    const int i = tid & 63, h = tid >> 6;
+    const int bar_id = 1 + gidx;
+    const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;   // my lane (= row tid of the sums)
+    float *xbuf = gs.M + (1 - h) * (kFoldD * 33);      // where my half sends: [0] rows 0..63 -> the other half, [1] the reverse
+    const float *rbuf = gs.M + h * (kFoldD * 33);
+    const float scale = h == 0 ? 0.5f : 1.f;           // S11 / 2 + S12 in rows 0..63, S21 + S22 in rows 64..127
+    unsigned cg_rows = 0, cg_matvecs = 0, cg_fallbacks = 0;
+    if (tid == 0) gs.bad = 0;
+    for (int it = gidx;; it += kGroups) {
+        const int64_t t = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
+        if (t >= p.n_items) break;
+        int64_t u, beg, end, slot;
+        item_range<kModeRowsFold>(p, t, u, beg, end, slot);
+        const float x0 = p.cg_warm ? reinterpret_cast<const float *>(p.out.table)[u * kFoldD + i] : 0.f;
+        const uint32_t aph = (uint32_t)((it / kGroups) & 1);
+        if (tid == 0) {
+            bool ok = mbar_wait_parked(&sm.acc_full[gidx], aph, &sm.abort_flag, 62);
+            ok = ok && mbar_wait_parked(&sm.rhs_done[it % kBRing], (uint32_t)((it / kBRing) & 1), &sm.abort_flag, 63);
+            gs.stop = ok ? 0 : 1;
+        }
+        group128_sync(bar_id);
+        if (gs.stop) break;
+        tc_fence_after();
+        const float *bp = &sm.bpart[it % kBRing][0][0];
+        const float b = 0.5f * bp[i] + bp[kFoldD + i];
+        // fold: the half that goes to the other half's threads first (through shared memory), then the half I keep
+        float a[32];
+        {
+            const int send0 = 32 * (1 - h);            // first of the 32 folded columns I send
+            float lo[16], hi[16];
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                tmem_ld16(trow + send0 + 16 * part, lo);
+                tmem_ld16(trow + kFoldD + send0 + 16 * part, hi);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) xbuf[i * 33 + 16 * part + k] = fmaf(scale, lo[k], hi[k]);
+            }
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                tmem_ld16(trow + 32 * h + 16 * part, lo);
+                tmem_ld16(trow + kFoldD + 32 * h + 16 * part, hi);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) a[16 * part + k] = fmaf(scale, lo[k], hi[k]);
+            }
+        }
+        // the sums have been read: the accumulator is free for the MMA warp's next item
+        tc_fence_before();
+        group128_sync(bar_id);
+        if (tid == 0) mbar_arrive(&sm.acc_empty[gidx]);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) a[k] += rbuf[i * 33 + k];
+        group128_sync(bar_id);      // the exchange buffers are free (the direct solve reuses them)
+        fold_solve_store(p, gs, a, bar_id, tid, u, b, x0, p.solver != 0, cg_rows, cg_matvecs, cg_fallbacks);
+    }
+    if (tid == 0 && p.cg_counters) {
+        if (cg_rows) atomicAdd(&p.cg_counters[0], (unsigned long long)cg_rows);
+        if (cg_matvecs) atomicAdd(&p.cg_counters[1], (unsigned long long)cg_matvecs);
+        if (cg_fallbacks) atomicAdd(&p.cg_counters[2], (unsigned long long)cg_fallbacks);
+    }
+}
+
 // The conjugate-gradient variant runs 24 warps: the 21 of the roles and three idle ones that complete the last
 // warpgroup, so that registers can move between warpgroups (setmaxnreg): the four producer warps form one warpgroup
 // (64 registers per thread), the MMA warp and the idle warps the next (32), and the solver warps take 96 (their
 // matrix-vector product holds two loads of 16 matrix entries, 8 duplicated vector entries and four packed sums).
-template <int MODE> constexpr int block_threads() { return MODE == kModeRowsCg ? 768 : Cfg<MODE>::kBlockThreads; }
+template <int MODE> constexpr int block_threads() { return is_cg(MODE) ? 768 : Cfg<MODE>::kBlockThreads; }
 
 template <int MODE>
 __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, const __grid_constant__ CUtensorMap tmap)
 {
     using C = Cfg<MODE>;
-    constexpr bool CG = MODE == kModeRowsCg;
+    constexpr bool CG = is_cg(MODE), FOLD = MODE == kModeRowsFold;
     // which rows this launch takes (block-uniform decisions, before any barrier or allocation)
     if (MODE == kModeRowsCg && p.policy && p.policy->use_cholesky) return;      // the Cholesky launch takes them all
     if (MODE == kModeRows && p.item_count && !(p.policy && p.policy->use_cholesky)) {
@@ -1463,7 +1735,9 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
         st_shared_zero16(smem_u32(&sm.y[0][0]) + k * 16);
     for (int k = tid; k < (int)sizeof(sm.h) / 16; k += kThreads)
         st_shared_zero16(smem_u32(&sm.h[0][0]) + k * 16);
-    if constexpr (CG) {
+    if constexpr (FOLD) {
+        // (alpha0 G + lambda I is 64 x 64 here and read from global memory; the space holds the groups' scratch)
+    } else if constexpr (CG) {
         for (int e = tid; e < D * D; e += kThreads)
             Bs[(e >> 7) * kLdBq + (e & 3) * kQStride + ((e & (D - 1)) >> 2)] = p.Bmat[e];
     } else if constexpr (MODE == kModeRows) {
@@ -1495,7 +1769,8 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
     if (rw < C::kMmaWarp) {
         const int gidx = rw / (C::kGroupThreads / 32);
         if constexpr (CG) setmaxnreg_inc<96>();
-        if constexpr (is_rows(MODE)) solver_rows_tmem<false, CG>(p, sm, rgs[gidx], Bs, gidx, rtid - gidx * C::kGroupThreads);
+        if constexpr (FOLD) solver_rows_fold(p, sm, reinterpret_cast<FoldGroupSmem *>(Bs)[gidx], gidx, rtid - gidx * C::kGroupThreads);
+        else if constexpr (is_rows(MODE)) solver_rows_tmem<false, CG>(p, sm, rgs[gidx], Bs, gidx, rtid - gidx * C::kGroupThreads);
         else copyout_role<MODE>(p, sm, gidx, rtid - gidx * C::kGroupThreads);
     } else if (CG && rw > kMmaWarp) {
         setmaxnreg_dec<32>();       // idle warps of the last warpgroup
@@ -1586,18 +1861,110 @@ __global__ void __launch_bounds__(4 * 128, 1) k_solve_sums(Params p)
     if (tid == 0 && sm.abort_flag) raise_flag(p.st, kFlagTimeout, (long long)sm.abort_flag * 1000000 + blockIdx.x);
 }
 
+// kModeRowsFold: rows whose sums the chunks kernel formed (split rows: their chunks in ascending order; long whole rows:
+// one sum each), folded straight from the workspace.  Four groups of 128 threads per block, no tensor memory.
+__global__ void __launch_bounds__(4 * 128) k_solve_sums_fold(Params p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    FoldGroupSmem *groups = reinterpret_cast<FoldGroupSmem *>(smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u));
+    const int tid = threadIdx.x & 127, gidx = threadIdx.x >> 7;
+    FoldGroupSmem &gs = groups[gidx];
+    const int i = tid & 63, h = tid >> 6, bar_id = 1 + gidx;
+    if (tid == 0) { gs.bad = 0; gs.stop = 0; }
+    group128_sync(bar_id);
+    unsigned cg_rows = 0, cg_matvecs = 0, cg_fallbacks = 0;
+    constexpr int64_t kSum = (int64_t)D * D + D;
+    for (int64_t t = (int64_t)blockIdx.x * 4 + gidx; t < p.n_items; t += (int64_t)gridDim.x * 4) {
+        int64_t u, c0, c1;
+        if (t < p.n_split_rows) {
+            u = p.sv.order[p.split_begin + t];
+            c0 = p.sv.split_first[t];
+            c1 = p.sv.split_first[t + 1];
+        } else {
+            const int64_t j = t - p.n_split_rows;
+            u = p.sv.order[p.long_end - 1 - j];
+            c0 = p.n_chunks + j;
+            c1 = c0 + 1;
+        }
+        float a[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) a[k] = 0.f;
+        float b = 0.f;
+        for (int64_t c = c0; c < c1; ++c) {
+            const float *S = p.partials + c * kSum;
+            const float *r0 = S + (int64_t)i * D + 32 * h, *r1 = S + (int64_t)(kFoldD + i) * D + 32 * h;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float4 q11 = *reinterpret_cast<const float4 *>(r0 + 4 * k), q12 = *reinterpret_cast<const float4 *>(r0 + kFoldD + 4 * k);
+                const float4 q21 = *reinterpret_cast<const float4 *>(r1 + 4 * k), q22 = *reinterpret_cast<const float4 *>(r1 + kFoldD + 4 * k);
+                a[4 * k] += (fmaf(0.5f, q11.x, q12.x) + q21.x) + q22.x;
+                a[4 * k + 1] += (fmaf(0.5f, q11.y, q12.y) + q21.y) + q22.y;
+                a[4 * k + 2] += (fmaf(0.5f, q11.z, q12.z) + q21.z) + q22.z;
+                a[4 * k + 3] += (fmaf(0.5f, q11.w, q12.w) + q21.w) + q22.w;
+            }
+            b += fmaf(0.5f, S[D * D + i], S[D * D + kFoldD + i]);
+        }
+        const float x0 = p.cg_warm ? reinterpret_cast<const float *>(p.out.table)[u * kFoldD + i] : 0.f;
+        fold_solve_store(p, gs, a, bar_id, tid, u, b, x0, p.solver != 0, cg_rows, cg_matvecs, cg_fallbacks);
+    }
+    if (tid == 0 && p.cg_counters) {
+        if (cg_rows) atomicAdd(&p.cg_counters[0], (unsigned long long)cg_rows);
+        if (cg_matvecs) atomicAdd(&p.cg_counters[1], (unsigned long long)cg_matvecs);
+        if (cg_fallbacks) atomicAdd(&p.cg_counters[2], (unsigned long long)cg_fallbacks);
+    }
+}
+
+// fp32 table of 64 features -> 2N rows of 128 bfloat16: row i = [x1 | x2], row N + i = [x1 | x3], x = x1 + x2 + x3 with
+// every part the nearest bfloat16 of what the parts before it leave (the remainders are exact in fp32)
+__global__ void __launch_bounds__(256) k_split_table(const float *__restrict__ X, int64_t n, __nv_bfloat16 *__restrict__ T)
+{
+    const int64_t e = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;      // four features of one row
+    if (e >= n * kFoldD) return;
+    const int64_t row = e / kFoldD;
+    const int f = (int)(e % kFoldD);
+    const float4 x = *reinterpret_cast<const float4 *>(X + e);
+    const float xs[4] = {x.x, x.y, x.z, x.w};
+    __nv_bfloat16 p1[4], p2[4], p3[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        p1[k] = __float2bfloat16_rn(xs[k]);
+        const float r1 = xs[k] - __bfloat162float(p1[k]);
+        p2[k] = __float2bfloat16_rn(r1);
+        p3[k] = __float2bfloat16_rn(r1 - __bfloat162float(p2[k]));
+    }
+    __nv_bfloat16 *t1 = T + row * D + f, *t2 = T + (n + row) * D + f;
+    *reinterpret_cast<uint2 *>(t1) = *reinterpret_cast<const uint2 *>(p1);
+    *reinterpret_cast<uint2 *>(t1 + kFoldD) = *reinterpret_cast<const uint2 *>(p2);
+    *reinterpret_cast<uint2 *>(t2) = *reinterpret_cast<const uint2 *>(p1);
+    *reinterpret_cast<uint2 *>(t2 + kFoldD) = *reinterpret_cast<const uint2 *>(p3);
+}
+
+__global__ void k_zero_rows_f32x64(const int32_t *__restrict__ rows, int64_t count, RowOut out)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count * kFoldD) return;
+    const int64_t u = rows[e / kFoldD];
+    const int f = (int)(e % kFoldD);
+    reinterpret_cast<float *>(out.table)[u * kFoldD + f] = 0.f;
+    if (out.cap_slot) {
+        const int cs = out.cap_slot[u];
+        if (cs >= 0) out.cap_out[(int64_t)cs * kFoldD + f] = 0.f;
+    }
+}
+
 template <int MODE> size_t smem_bytes()
 {
     // a large request in every mode (more than half of what an SM offers): at most one block per SM, so two
     // blocks never compete for the SM's 512 tensor-memory columns
     size_t b = sizeof(SmemT<MODE>) + 1024;
     if (MODE == kModeRows) b += sizeof(float) * D * kLdBq + kMaxGroups * sizeof(RowGroupSmem);
-    if (MODE == kModeRowsCg) b += sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem);
+    if (is_cg(MODE)) b += sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem);
     return b;
 }
 static_assert(sizeof(SmemT<1>) + 1024 <= 232448 && sizeof(SmemT<1>) > 116224, "ring depth of the streaming modes");
 static_assert(sizeof(SmemT<0>) + 1024 + sizeof(float) * D * kLdBq + kMaxGroups * sizeof(RowGroupSmem) <= 232448, "rows mode");
 static_assert(sizeof(SmemT<3>) + 1024 + sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem) <= 232448, "rows mode, CG");
+static_assert(sizeof(SmemT<4>) == sizeof(SmemT<3>), "the fold kernel has the conjugate-gradient kernel's feed");
 
 // Tensor map of a bfloat16 table [n x 128] for row gathers: boxes of one row by 64 features (128 bytes), 128-byte swizzle.
 // (The encoder is a driver entry point, looked up through the runtime so that the library needs no driver at link time.)
@@ -1747,6 +2114,75 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         k_zero_rows_bf16<<<(unsigned)((n_zero * D + 255) / 256), 256, 0, s>>>(sv.order + offs[0], n_zero, out);
         ++*launches;
     }
+    return cudaGetLastError();
+}
+
+// Whole half-epoch of the rows of an fp32 table of 64 features on the tensor cores: sv is the doubled entry list over the
+// 2N-row bfloat16 table T (see kModeRowsFold), offs its degree classes.
+cudaError_t launch_rows_fold(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows, const void *T,
+                             int64_t n_table, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
+                             cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
+                             const CgOptions &cg)
+{
+    const int sms = sm_count();
+    Params p{};
+    p.sv = sv;
+    p.X = reinterpret_cast<const __nv_bfloat16 *>(T);
+    p.n_table = n_table;
+    p.Bmat = Bmat;
+    p.partials = split_partials;
+    p.out = out;
+    p.st = st;
+    p.solver = cg.enabled ? 1 : 0;
+    p.cg_max_iter = cg.max_iter;
+    p.cg_tol2 = cg.tol * cg.tol;
+    p.cg_warm = cg.warm_start ? 1 : 0;
+    p.cg_counters = cg.counters;
+    cudaError_t e;
+    const int c_long = long_class_begin(offs);
+    const int64_t n_long = offs[kNClasses - 1] - offs[c_long];
+    if (n_chunks + n_long > 0) {
+        p.n_chunks = n_chunks;
+        p.long_end = offs[kNClasses - 1];
+        p.n_items = n_chunks + n_long;
+        e = launch_mode<kModeChunks>(p, (int)(p.n_items < sms ? p.n_items : sms), s);
+        ++*launches;
+        if (e != cudaSuccess) return e;
+        p.split_begin = offs[kNClasses - 1];
+        p.n_split_rows = n_split_rows;
+        p.n_items = n_split_rows + n_long;
+        const size_t smem = 4 * sizeof(FoldGroupSmem) + 128;
+        e = cudaFuncSetAttribute(k_solve_sums_fold, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        const int64_t blocks = (p.n_items + 3) / 4;
+        k_solve_sums_fold<<<(int)(blocks < 2 * sms ? blocks : 2 * sms), 4 * 128, smem, s>>>(p);
+        ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    const int64_t n_whole = offs[c_long] - offs[1];
+    if (n_whole > 0) {
+        p.n_items = n_whole;
+        p.last_item = offs[c_long] - 1;
+        if (main_begin) cudaEventRecord(main_begin, s);
+        e = launch_mode<kModeRowsFold>(p, (int)(n_whole < sms ? n_whole : sms), s);
+        ++*launches;
+        if (e != cudaSuccess) return e;
+        if (main_end) cudaEventRecord(main_end, s);
+    }
+    const int64_t n_zero = offs[1] - offs[0];
+    if (n_zero > 0) {
+        k_zero_rows_f32x64<<<(unsigned)((n_zero * kFoldD + 255) / 256), 256, 0, s>>>(sv.order + offs[0], n_zero, out);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split_table(const float *X, int64_t n, void *T, cudaStream_t s, int64_t *launches)
+{
+    if (n <= 0) return cudaSuccess;
+    k_split_table<<<(unsigned)((n * kFoldD / 4 + 255) / 256), 256, 0, s>>>(X, n, reinterpret_cast<__nv_bfloat16 *>(T));
+    ++*launches;
     return cudaGetLastError();
 }
 

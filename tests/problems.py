@@ -97,4 +97,8 @@ def small_suite():
                          split=256, values=True, n_cols=2500, zero_labels=0.2),
         lambda: powerlaw("uniform_d32_bf16", 2000, 50000, 1.1, 900, 32, 0.05, 0.002, "bf16", "uniform", 19, n_cols=1700,
                          empty_rows=2),
+        # fp32 tables of 64 features on the tensor cores (bfloat16 parts, doubled entry lists): labelled entries, rows
+        # split at 256 observations, whole rows of more than 512 (their sums come from the chunks kernel)
+        lambda: powerlaw("split_labels_d64_f32", 2000, 90000, 1.0, 2500, 64, 0.05, 0.002, "f32", "zipf", 21, split=512,
+                         values=True, n_cols=3000, zero_labels=0.1, empty_rows=2),
     ]

@@ -70,7 +70,7 @@ def _check_half_step(p, side, X_gpu, X_ref, X_raw, x32, deg, ptr, idx, vals64, X
 SUITE = problems.small_suite()
 IDS = ["tiny", "zipf_d64_f32", "local_d128_bf16", "split_d128_bf16", "split_d32_f32_labels", "alpha0_d16_bf16",
        "default_split_d64_bf16", "long_labels_d128_bf16", "split_labels_d128_bf16", "zero_labels_d128_f32",
-       "uniform_d32_bf16"]
+       "uniform_d32_bf16", "split_labels_d64_f32"]
 
 
 @pytest.fixture(scope="module", params=list(range(len(SUITE))), ids=IDS)
@@ -115,10 +115,10 @@ def test_epoch_embeddings_residual_and_loss(prob):
     _epoch_checks(prob)
 
 
-@pytest.mark.parametrize("name", ["local_d128_bf16", "split_d128_bf16"])
+@pytest.mark.parametrize("name", ["local_d128_bf16", "split_d128_bf16", "zipf_d64_f32", "split_labels_d64_f32"])
 def test_fp32_alu_kernels_on_the_tensor_path_problems(name):
-    """kernels = 1 forces the FP32-ALU kernels where the tensor-core kernels would run (d = 128, bfloat16 tables):
-    the same gates against the oracle."""
+    """kernels = 1 forces the FP32-ALU kernels where the tensor-core kernels would run (d = 128 with bfloat16 tables,
+    d = 64 with fp32 tables): the same gates against the oracle."""
     _epoch_checks(_problem(name), kernels=1)
 
 
@@ -445,6 +445,52 @@ def test_conjugate_gradient_solve_meets_the_gates_and_tracks_the_oracle(name):
     for n in range(0, ids.size, 3):
         A, b = ials.row_system(p.rowptr, p.colidx, vals64, H0, G, p.alpha, p.lam, int(ids[n]))
         for label in ("cg", "fallback"):
+            worst = max(worst, np.linalg.norm(A @ sols[label][n] - b) / np.linalg.norm(b))
+    assert worst <= 1e-4, worst
+
+
+@pytest.mark.parametrize("name", ["zipf_d64_f32", "split_labels_d64_f32"])
+def test_fp32_tables_of_64_features_on_the_tensor_cores(name):
+    """d = 64 with fp32 tables: the outer products run on the tensor cores over bfloat16 parts of the fixed table
+    (x = x1 + x2 + x3), the 64 x 64 system is folded out of the 128 x 128 sums and solved by conjugate gradients
+    (Sec. 4.5) or, on request or when they do not converge, by Cholesky.  Every non-empty row, all three routes and
+    the FP32-ALU kernels against the exact row update and the residual gate."""
+    p = _problem(name)
+    deg = np.diff(p.rowptr)
+    ids = np.nonzero(deg > 0)[0].astype(np.int64)
+    H0 = p.f64(p.H0)
+    G = ials.gramian(H0)
+    vals64 = None if p.values is None else p.values.astype(np.float64)
+    sols, stats = {}, {}
+    for label, kw in (("cg", dict(cg_start=1)), ("chol", dict(solver=1)), ("fallback", dict(cg_max_iter=2, cg_start=1)),
+                      ("alu", dict(kernels=1))):
+        a = make_ctx(p, **kw)
+        sols[label] = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+        stats[label] = a.get_stats()
+        assert stats[label].not_spd == 0
+        assert stats[label].kernel_path[0] == (0 if label == "alu" else 1)
+        a.destroy()
+    assert stats["cg"].cg_rows == ids.size and stats["cg"].cg_fallbacks == 0
+    assert stats["chol"].cg_rows == 0 and stats["alu"].cg_rows == 0
+    assert stats["fallback"].cg_rows == ids.size and stats["fallback"].cg_fallbacks > 0.5 * ids.size
+    if p.split == 0:
+        assert stats["cg"].long_rows[0] > 0      # whole rows of more than 512 observations took the chunks kernel
+    _, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G, return_raw=True)
+    _, _, o_iters = ials.half_step_cg(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G,
+                                     tol=1e-5, max_iter=48)
+    mean_products = stats["cg"].cg_products / stats["cg"].cg_rows
+    assert abs(mean_products - (o_iters.mean() + 1)) <= 1.0, (mean_products, o_iters.mean())
+    nz = np.linalg.norm(W_raw, axis=1) > 0      # (rows whose labels are all 0 have the solution 0)
+    for label in sols:
+        assert rel_fro(sols[label], W_raw) <= 1e-4, label
+        assert row_rel(sols[label][nz], W_raw[nz]).max() <= 1e-3, label
+        assert np.all(sols[label][~nz] == 0.0), label
+    worst = 0.0
+    for n in range(0, ids.size, 5):
+        if not nz[n]:
+            continue
+        A, b = ials.row_system(p.rowptr, p.colidx, vals64, H0, G, p.alpha, p.lam, int(ids[n]))
+        for label in ("cg", "chol", "fallback"):
             worst = max(worst, np.linalg.norm(A @ sols[label][n] - b) / np.linalg.norm(b))
     assert worst <= 1e-4, worst
 
