@@ -233,6 +233,48 @@ alx_status alx_get_buckets(alx_ctx *ctx, alx_side side, int32_t *order, int64_t 
 
 alx_status alx_get_stats(alx_ctx *ctx, alx_stats *out);
 
+/*
+ * Evaluation (Sec. 4.6; the protocol of Sec. 5; the metric of Table 2).  Not part of a training epoch.
+ *
+ * alx_fold_in: embeddings of rows that were not trained.  Sec. 5 obtains the embedding of a held-out source row from
+ * the part of its links that is kept, through Eq. 4 with the trained column table held fixed: one more rows half-step,
+ * on new rows.  rowptr[n_new + 1] / colidx[nnz] / values[nnz] (or NULL: y = 1) give the new rows as CSR over the
+ * context's columns, with the rules of alx_set_csr; x_out receives n_new x d floats, the solutions after the round
+ * to the storage type (the values a trained table would hold).  The arrays are host or device memory as on_device
+ * says, x_out included.  The context's own matrix and tables are not touched; the call allocates what the half-step
+ * needs for n_new rows, runs the same kernels as alx_half_epoch and synchronises.  A row with no entry gets 0.
+ * ALX_ERR_BAD_STATE before the column table holds anything, ALX_ERR_BAD_CSR as alx_set_csr.
+ */
+alx_status alx_fold_in(alx_ctx *ctx, const int64_t *rowptr, const int32_t *colidx, const float *values, int64_t n_new,
+                       int64_t nnz, int on_device, float *x_out);
+
+#define ALX_MAX_TOPK 256
+/*
+ * alx_topk: exact Top-K retrieval (Sec. 4.6: the best k items of a user by inner product; every item is scored, no
+ * approximate search).  queries: m x d floats; the items are the rows of table `items` (ALX_COLS for the protocol
+ * of Sec. 5) as stored.  For query q the ids of the k largest <q, h_i> go to ids_out[q * k ..], best first; equal
+ * scores are ordered by ascending id (the paper states no tie rule); scores_out (m x k, may be NULL) receives the
+ * scores.  exclude_ptr[m + 1] / exclude_idx (may both be NULL) list, per query and ascending, ids that must not be
+ * returned (the kept links of a fold-in row, for example; the paper does not say whether it leaves them out).  Where
+ * fewer than k items qualify the row is filled with id -1 and score -inf.  1 <= k <= ALX_MAX_TOPK.
+ * Scores are fp32: for d = 128 with bfloat16 tables products of bfloat16 parts summed in fp32 on the tensor cores
+ * (the query as three parts, so to fp32 accuracy); otherwise fp32 FMAs.  Two items whose exact scores differ by less
+ * than that rounding may come out in either order.  All arrays host or device as on_device says; synchronises.
+ */
+alx_status alx_topk(alx_ctx *ctx, alx_side items, const float *queries, int64_t m, int32_t k, const int64_t *exclude_ptr,
+                    const int32_t *exclude_idx, int on_device, int32_t *ids_out, float *scores_out);
+
+/*
+ * alx_recall_at_k: Recall@K as Table 2 reports it, read as: for every query with at least one ground-truth id, the
+ * number of ground-truth ids among its first k retrieved ids divided by the number of its ground-truth ids; the mean
+ * over those queries (the paper names the metric without a formula).  ids: m rows of k_stride retrieved ids (best
+ * first, -1 = none), of which the first k count; truth_ptr[m + 1] / truth_idx: ground truth per query, ascending.
+ * *recall receives the mean, *n_counted (may be NULL) the number of queries it is over.  Sums in a fixed order.
+ */
+alx_status alx_recall_at_k(alx_ctx *ctx, const int32_t *ids, int64_t m, int32_t k_stride, int32_t k,
+                           const int64_t *truth_ptr, const int32_t *truth_idx, int on_device, double *recall,
+                           int64_t *n_counted);
+
 /* Diagnostic for roofline reports: measured FP32 fused-multiply-add throughput of the device in
    TFLOP/s (a register-resident FMA loop on every SM, best of three).  No counterpart in the paper.
    Allocates and frees 256 bytes with cudaMalloc; synchronises. */

@@ -51,7 +51,7 @@ EXPORTS = ["alx_create", "alx_create_ex", "alx_destroy", "alx_set_csr", "alx_set
            "alx_epoch", "alx_half_epoch_capture", "alx_loss", "alx_get_embeddings", "alx_get_gramian",
            "alx_gramian", "alx_fp32_peak_tflops", "alx_get_transpose", "alx_get_buckets", "alx_get_stats", "alx_synchronize",
            "alx_last_error", "alx_version", "alx_gramian_noalloc", "alx_gramian_noalloc_max_rows",
-           "alx_noalloc_last_error"]
+           "alx_noalloc_last_error", "alx_fold_in", "alx_topk", "alx_recall_at_k"]
 
 _lib = None
 
@@ -85,6 +85,9 @@ def load_library() -> ctypes.CDLL:
     lib.alx_get_buckets.argtypes = [P, c_int, P, P, P, POINTER(c_int64)]
     lib.alx_get_stats.argtypes = [P, POINTER(alx_stats)]
     lib.alx_synchronize.argtypes = [P]
+    lib.alx_fold_in.argtypes = [P, P, P, P, c_int64, c_int64, c_int, P]
+    lib.alx_topk.argtypes = [P, c_int, P, c_int64, c_int32, P, P, c_int, P, P]
+    lib.alx_recall_at_k.argtypes = [P, P, c_int64, c_int32, c_int32, P, P, c_int, POINTER(c_double), POINTER(c_int64)]
     lib.alx_fp32_peak_tflops.argtypes = [P, POINTER(c_double)]
     lib.alx_last_error.argtypes = [P]
     lib.alx_last_error.restype = c_char_p
@@ -266,6 +269,46 @@ class Alx:
         out = np.empty((ids.size, self.d), dtype=np.float32)
         self._check(self.lib.alx_half_epoch_capture(self.ctx, side, _np_ptr(ids), int(ids.size), _np_ptr(out)))
         return out
+
+    # ---- evaluation (host arrays in, host arrays out)
+    def fold_in(self, rowptr, colidx, values=None):
+        """Embeddings (float32, after the round to the storage type) of new rows given as CSR over the columns."""
+        rp = np.ascontiguousarray(rowptr, dtype=np.int64)
+        ci = np.ascontiguousarray(colidx, dtype=np.int32)
+        va = None if values is None else np.ascontiguousarray(values, dtype=np.float32)
+        n_new = rp.size - 1
+        out = np.empty((n_new, self.d), dtype=np.float32)
+        self._check(self.lib.alx_fold_in(self.ctx, _np_ptr(rp), _np_ptr(ci), None if va is None else _np_ptr(va), n_new,
+                                         int(ci.size), 0, _np_ptr(out)))
+        return out
+
+    def topk(self, items_side, queries, k, exclude=None, scores=True):
+        """(ids [m, k] int32, scores [m, k] float32 or None); exclude = (ptr, idx) CSR of ids to leave out per query."""
+        q = np.ascontiguousarray(queries, dtype=np.float32)
+        m = q.shape[0]
+        ids = np.empty((m, k), dtype=np.int32)
+        sc = np.empty((m, k), dtype=np.float32) if scores else None
+        ep = ei = None
+        if exclude is not None:
+            ep = np.ascontiguousarray(exclude[0], dtype=np.int64)
+            ei = np.ascontiguousarray(exclude[1], dtype=np.int32)
+            if ei.size == 0:
+                ei = np.zeros(1, dtype=np.int32)
+        self._check(self.lib.alx_topk(self.ctx, items_side, _np_ptr(q), m, k, None if ep is None else _np_ptr(ep),
+                                      None if ei is None else _np_ptr(ei), 0, _np_ptr(ids), None if sc is None else _np_ptr(sc)))
+        return ids, sc
+
+    def recall_at_k(self, ids, k, truth_ptr, truth_idx):
+        """(mean recall over the queries with ground truth, how many those are)"""
+        a = np.ascontiguousarray(ids, dtype=np.int32)
+        tp = np.ascontiguousarray(truth_ptr, dtype=np.int64)
+        ti = np.ascontiguousarray(truth_idx, dtype=np.int32)
+        if ti.size == 0:
+            ti = np.zeros(1, dtype=np.int32)
+        r, n = c_double(), c_int64()
+        self._check(self.lib.alx_recall_at_k(self.ctx, _np_ptr(a), a.shape[0], a.shape[1], k, _np_ptr(tp), _np_ptr(ti), 0,
+                                             byref(r), byref(n)))
+        return r.value, n.value
 
     def loss(self):
         total = c_double()

@@ -358,7 +358,15 @@ alx_status alx_create(int64_t n_rows, int64_t n_cols, int32_t d, float lambda, f
     return alx_create_ex(&o, out);   /* solver, cg_max_iter, cg_tol = 0: the defaults */
 }
 
-alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
+namespace {
+alx_status create_impl(const alx_options *opt, const alx_ctx *parent, alx_ctx **out);
+}
+
+alx_status alx_create_ex(const alx_options *opt, alx_ctx **out) { return create_impl(opt, nullptr, out); }
+
+namespace {
+// parent: the new context borrows the parent's column table (alx_fold_in) instead of holding one of its own
+alx_status create_impl(const alx_options *opt, const alx_ctx *parent, alx_ctx **out)
 {
     if (!opt || !out) return ALX_ERR_INVALID_ARG;
     if (opt->n_rows < 1 || opt->n_cols < 1 || opt->n_rows >= (1ll << 31) || opt->n_cols >= (1ll << 31))
@@ -392,7 +400,7 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
     auto body = [&]() -> alx_status {
         const int d = opt->d;
         for (int s = 0; s < 2; ++s) {
-            void *t = dev_alloc(c, (size_t)c->n[s] * d * c->elem);
+            void *t = parent && s == ALX_COLS ? parent->table[s] : dev_alloc(c, (size_t)c->n[s] * d * c->elem);
             if (!t) return fail(c, ALX_ERR_OOM, "device allocation of a %lld x %d table failed", (long long)c->n[s], d);
             c->table[s] = t;
             ALX_ALLOC(c, c->G64[s], d * d);
@@ -434,6 +442,7 @@ alx_status alx_create_ex(const alx_options *opt, alx_ctx **out)
     *out = c;
     return ALX_OK;
 }
+}  // namespace
 
 alx_status alx_destroy(alx_ctx *c)
 {
@@ -840,6 +849,126 @@ alx_status alx_get_buckets(alx_ctx *c, alx_side side, int32_t *order, int64_t *c
     if (chunk_desc && c->n_chunks[side] > 0)
         ALX_CUDA(c, cudaMemcpyAsync(chunk_desc, c->chunk_desc[side], sizeof(int64_t) * 4 * c->n_chunks[side], cudaMemcpyDeviceToHost, c->stream));
     ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ALX_OK;
+}
+
+alx_status alx_fold_in(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx, const float *values, int64_t n_new,
+                       int64_t nnz, int on_device, float *x_out)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (n_new < 0 || nnz < 0 || n_new >= (1ll << 31) || (n_new > 0 && (!rowptr || !x_out)) || (nnz > 0 && !colidx))
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_fold_in");
+    if (!c->have_table[ALX_COLS]) return fail(c, ALX_ERR_BAD_STATE, "the column table has not been set or solved yet");
+    if (n_new == 0) return ALX_OK;
+    DeviceGuard guard(c->device);
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    // a context of its own for the new rows: same options, the column table borrowed, the rows half-step of Eq. 4
+    alx_options o = c->opt;
+    o.n_rows = n_new;
+    o.device = c->device;
+    alx_ctx *k = nullptr;
+    alx_status st = create_impl(&o, c, &k);
+    if (st != ALX_OK) return fail(c, st, "alx_fold_in: the context for the new rows could not be created");
+    k->have_table[ALX_COLS] = true;
+    st = alx_set_csr(k, rowptr, colidx, values, nnz, on_device);
+    if (st == ALX_OK) st = alx_half_epoch(k, ALX_ROWS);
+    if (st == ALX_OK) st = alx_get_embeddings(k, ALX_ROWS, x_out, ALX_F32, 0, n_new, on_device);
+    if (st == ALX_OK) st = alx_synchronize(k);
+    c->launches += k->launches;
+    if (st != ALX_OK) c->err = "alx_fold_in: " + k->err;
+    alx_destroy(k);
+    return st;
+}
+
+alx_status alx_topk(alx_ctx *c, alx_side items, const float *queries, int64_t m, int32_t k, const int64_t *exclude_ptr,
+                    const int32_t *exclude_idx, int on_device, int32_t *ids_out, float *scores_out)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if ((items != ALX_ROWS && items != ALX_COLS) || m < 0 || k < 1 || k > ALX_MAX_TOPK || (m > 0 && (!queries || !ids_out)) ||
+        (exclude_ptr && !exclude_idx && m > 0))
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_topk");
+    if (!c->have_table[items]) return fail(c, ALX_ERR_BAD_STATE, "the table has not been set or solved yet");
+    if (m == 0) return ALX_OK;
+    DeviceGuard guard(c->device);
+    const int d = c->opt.d;
+    const int64_t n_items = c->n[items];
+    Scratch tmp(c);
+    const float *Q = queries;
+    const int64_t *ex_ptr = exclude_ptr;
+    const int32_t *ex_idx = exclude_idx;
+    int32_t *ids_dev = ids_out;
+    float *scores_dev = scores_out;
+    int64_t n_ex = 0;
+    if (!on_device) {
+        float *q_dev = nullptr;
+        ALX_TMP(c, tmp, q_dev, m * d);
+        ALX_CUDA(c, cudaMemcpyAsync(q_dev, queries, sizeof(float) * m * d, cudaMemcpyHostToDevice, c->stream));
+        Q = q_dev;
+        if (exclude_ptr) {
+            n_ex = exclude_ptr[m];
+            if (n_ex < 0) return fail(c, ALX_ERR_INVALID_ARG, "alx_topk: negative length of the exclusion lists");
+            int64_t *p_dev = nullptr;
+            int32_t *i_dev = nullptr;
+            ALX_TMP(c, tmp, p_dev, m + 1);
+            ALX_TMP(c, tmp, i_dev, n_ex > 0 ? n_ex : 1);
+            ALX_CUDA(c, cudaMemcpyAsync(p_dev, exclude_ptr, sizeof(int64_t) * (m + 1), cudaMemcpyHostToDevice, c->stream));
+            if (n_ex > 0) ALX_CUDA(c, cudaMemcpyAsync(i_dev, exclude_idx, sizeof(int32_t) * n_ex, cudaMemcpyHostToDevice, c->stream));
+            ex_ptr = p_dev;
+            ex_idx = i_dev;
+        }
+        ALX_TMP(c, tmp, ids_dev, m * k);
+        if (scores_out) ALX_TMP(c, tmp, scores_dev, m * k);
+    }
+    const int slabs = topk_slabs(n_items, m);
+    float *ls = nullptr;
+    int32_t *li = nullptr, *lc = nullptr;
+    ALX_TMP(c, tmp, ls, (int64_t)slabs * m * k);
+    ALX_TMP(c, tmp, li, (int64_t)slabs * m * k);
+    ALX_TMP(c, tmp, lc, (int64_t)slabs * m);
+    ALX_CUDA(c, cudaMemsetAsync(lc, 0, sizeof(int32_t) * slabs * m, c->stream));
+    ALX_CUDA(c, launch_topk(c->table[items], c->bf16 != 0, n_items, d, Q, m, k, ex_ptr, ex_idx, slabs, ls, li, lc, ids_dev,
+                            scores_dev, c->opt.kernels != 1, c->stream, &c->launches));
+    if (!on_device) {
+        ALX_CUDA(c, cudaMemcpyAsync(ids_out, ids_dev, sizeof(int32_t) * m * k, cudaMemcpyDeviceToHost, c->stream));
+        if (scores_out) ALX_CUDA(c, cudaMemcpyAsync(scores_out, scores_dev, sizeof(float) * m * k, cudaMemcpyDeviceToHost, c->stream));
+    }
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    return check_device_status(c);
+}
+
+alx_status alx_recall_at_k(alx_ctx *c, const int32_t *ids, int64_t m, int32_t k_stride, int32_t k, const int64_t *truth_ptr,
+                           const int32_t *truth_idx, int on_device, double *recall, int64_t *n_counted)
+{
+    if (!c) return ALX_ERR_INVALID_ARG;
+    if (m < 0 || k < 1 || k > k_stride || !recall || (m > 0 && (!ids || !truth_ptr)))
+        return fail(c, ALX_ERR_INVALID_ARG, "bad argument to alx_recall_at_k");
+    DeviceGuard guard(c->device);
+    Scratch tmp(c);
+    const int32_t *ids_dev = ids;
+    const int64_t *tp = truth_ptr;
+    const int32_t *ti = truth_idx;
+    if (!on_device && m > 0) {
+        const int64_t nt = truth_ptr[m];
+        if (nt < 0 || (nt > 0 && !truth_idx)) return fail(c, ALX_ERR_INVALID_ARG, "alx_recall_at_k: bad ground-truth lists");
+        int32_t *a = nullptr, *t = nullptr;
+        int64_t *p = nullptr;
+        ALX_TMP(c, tmp, a, m * k_stride);
+        ALX_TMP(c, tmp, p, m + 1);
+        ALX_TMP(c, tmp, t, nt > 0 ? nt : 1);
+        ALX_CUDA(c, cudaMemcpyAsync(a, ids, sizeof(int32_t) * m * k_stride, cudaMemcpyHostToDevice, c->stream));
+        ALX_CUDA(c, cudaMemcpyAsync(p, truth_ptr, sizeof(int64_t) * (m + 1), cudaMemcpyHostToDevice, c->stream));
+        if (nt > 0) ALX_CUDA(c, cudaMemcpyAsync(t, truth_idx, sizeof(int32_t) * nt, cudaMemcpyHostToDevice, c->stream));
+        ids_dev = a; tp = p; ti = t;
+    }
+    double *per_query = nullptr, *out2 = nullptr;
+    ALX_TMP(c, tmp, per_query, m > 0 ? m : 1);
+    ALX_TMP(c, tmp, out2, 2);
+    ALX_CUDA(c, launch_recall(ids_dev, m, k_stride, k, tp, ti, per_query, out2, c->stream, &c->launches));
+    double h[2] = {0.0, 0.0};
+    ALX_CUDA(c, cudaMemcpyAsync(h, out2, sizeof h, cudaMemcpyDeviceToHost, c->stream));
+    ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+    *recall = h[1] > 0.0 ? h[0] / h[1] : 0.0;
+    if (n_counted) *n_counted = (int64_t)h[1];
     return ALX_OK;
 }
 

@@ -176,6 +176,20 @@ struct CgOptions {
 // alx_umma.cu: tensor-core path, d = 128 and bf16 tables only
 int64_t gramian_umma_partials();
 cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaStream_t s, int64_t *launches);
+// ---- evaluation (alx_eval.cu, alx_topk_umma.cu)
+// slabs of items per query tile (each slab's best k are listed separately and merged)
+int topk_slabs(int64_t n_items, int64_t m);
+// exact Top-K of <q, h_i>: H [n_items x d] (storage type), Q [m x d] fp32; lists: [slabs][m][k] scratch;
+// ids_out [m x k] (-1 where fewer than k items qualify), scores_out [m x k] or nullptr; ex_*: per-query ids to leave out
+cudaError_t launch_topk(const void *H, bool bf16, int64_t n_items, int d, const float *Q, int64_t m, int k,
+                        const int64_t *ex_ptr, const int32_t *ex_idx, int slabs, float *list_s, int32_t *list_id,
+                        int32_t *list_cnt, int32_t *ids_out, float *scores_out, bool tensor_cores, cudaStream_t s,
+                        int64_t *launches);
+cudaError_t launch_topk_umma(const void *H, int64_t n_items, const float *Q, int64_t m, int k, const int64_t *ex_ptr,
+                             const int32_t *ex_idx, int slabs, int64_t slab, float *list_s, int32_t *list_id,
+                             int32_t *list_cnt, cudaStream_t s, int64_t *launches);
+cudaError_t launch_recall(const int32_t *ids, int64_t m, int k_stride, int k, const int64_t *tptr, const int32_t *tidx,
+                          double *per_query, double *out2, cudaStream_t s, int64_t *launches);
 cudaError_t launch_rows_fold(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks, int64_t n_split_rows,
                              const void *T, int64_t n_table, const float *Bmat, float *split_partials, RowOut out,
                              DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
