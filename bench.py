@@ -314,6 +314,24 @@ def run_ours(args, w):
         half_ms["cg_fallbacks"].append(s2.cg_fallbacks)
     fp32_peak = a.fp32_peak_tflops()
     loss = a.loss()[0]
+    evaluation = None
+    if args.eval:
+        # exact Top-50 of 2048 queries (rows of W) over every row of H, device buffers, outside the timed region
+        mq, kq = 2048, 50
+        Wq = torch.empty((mq, d), dtype=torch.float32, device=dev)
+        a.get_embeddings(ALX_ROWS, row_begin=0, row_count=mq, out=Wq)
+        ids_t = torch.empty((mq, kq), dtype=torch.int32, device=dev)
+        sc_t = torch.empty((mq, kq), dtype=torch.float32, device=dev)
+        t_top = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            a.topk_device(ALX_COLS, Wq, kq, ids_t, sc_t)
+            torch.cuda.synchronize()
+            t_top.append(time.perf_counter() - t0)
+        evaluation = {"topk": {"queries": mq, "k": kq, "items": n, "seconds": min(t_top),
+                               "scores_per_s": mq * n / min(t_top), "tflops": 2.0 * mq * n * d / min(t_top) / 1e12,
+                               "note": "alx_topk on device buffers, best of 3 (includes its scratch allocation and the merge)"}}
     ms, units = aggregate_over_ranks(ms_local, float(nnz), world, dev)
     value = units / (ms * 1e-3)
 
@@ -442,7 +460,7 @@ def run_ours(args, w):
                           "paper_context": "about 20 min/epoch for 365M nodes / 29.9B edges on 256 TPU v3 cores"},
                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
                "cpu_baseline": cpu_baseline,
-               "extra": {"solver": {"option": args.solver, "cg_rows": half_ms["cg_rows"], "cg_products": half_ms["cg_products"],
+               "extra": {"evaluation": evaluation, "solver": {"option": args.solver, "cg_rows": half_ms["cg_rows"], "cg_products": half_ms["cg_products"],
                                     "cg_fallbacks": half_ms["cg_fallbacks"],
                                     "note": "[rows half-epoch, columns half-epoch] of the half-epoch pair after the timed region"},
                          "epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
@@ -469,6 +487,7 @@ def main():
     ap.add_argument("--cg-start", type=int, default=0, choices=[0, 1],
                     help="alx_options.cg_start: 0 = the stored embedding, 1 = zero")
     ap.add_argument("--cg-tol", type=float, default=0.0, help="alx_options.cg_tol (0 = the library's default)")
+    ap.add_argument("--eval", action="store_true", help="also time the exact Top-K retrieval on the trained tables (extra.evaluation)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")
     args = ap.parse_args()

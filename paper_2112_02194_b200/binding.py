@@ -298,6 +298,14 @@ class Alx:
                                       None if ei is None else _np_ptr(ei), 0, _np_ptr(ids), None if sc is None else _np_ptr(sc)))
         return ids, sc
 
+    def topk_device(self, items_side, queries, k, ids_out, scores_out=None):
+        """Top-K with torch CUDA tensors: queries [m, d] float32, ids_out [m, k] int32, scores_out [m, k] float32."""
+        assert queries.is_cuda and queries.is_contiguous() and queries.dtype == self.torch.float32
+        assert ids_out.is_cuda and ids_out.is_contiguous() and ids_out.dtype == self.torch.int32
+        m = queries.shape[0]
+        self._check(self.lib.alx_topk(self.ctx, items_side, queries.data_ptr(), m, k, None, None, 1, ids_out.data_ptr(),
+                                      None if scores_out is None else scores_out.data_ptr()))
+
     def recall_at_k(self, ids, k, truth_ptr, truth_idx):
         """(mean recall over the queries with ground truth, how many those are)"""
         a = np.ascontiguousarray(ids, dtype=np.int32)

@@ -926,8 +926,11 @@ alx_status alx_topk(alx_ctx *c, alx_side items, const float *queries, int64_t m,
     ALX_TMP(c, tmp, li, (int64_t)slabs * m * k);
     ALX_TMP(c, tmp, lc, (int64_t)slabs * m);
     ALX_CUDA(c, cudaMemsetAsync(lc, 0, sizeof(int32_t) * slabs * m, c->stream));
+    const bool tensor_cores = c->opt.kernels != 1 && c->bf16 && d == 128;
+    unsigned char *q_parts = nullptr;
+    if (tensor_cores) ALX_TMP(c, tmp, q_parts, topk_query_scratch_bytes(m));
     ALX_CUDA(c, launch_topk(c->table[items], c->bf16 != 0, n_items, d, Q, m, k, ex_ptr, ex_idx, slabs, ls, li, lc, ids_dev,
-                            scores_dev, c->opt.kernels != 1, c->stream, &c->launches));
+                            scores_dev, tensor_cores, q_parts, c->status, c->stream, &c->launches));
     if (!on_device) {
         ALX_CUDA(c, cudaMemcpyAsync(ids_out, ids_dev, sizeof(int32_t) * m * k, cudaMemcpyDeviceToHost, c->stream));
         if (scores_out) ALX_CUDA(c, cudaMemcpyAsync(scores_out, scores_dev, sizeof(float) * m * k, cudaMemcpyDeviceToHost, c->stream));

@@ -183,11 +183,14 @@ int topk_slabs(int64_t n_items, int64_t m);
 // ids_out [m x k] (-1 where fewer than k items qualify), scores_out [m x k] or nullptr; ex_*: per-query ids to leave out
 cudaError_t launch_topk(const void *H, bool bf16, int64_t n_items, int d, const float *Q, int64_t m, int k,
                         const int64_t *ex_ptr, const int32_t *ex_idx, int slabs, float *list_s, int32_t *list_id,
-                        int32_t *list_cnt, int32_t *ids_out, float *scores_out, bool tensor_cores, cudaStream_t s,
-                        int64_t *launches);
+                        int32_t *list_cnt, int32_t *ids_out, float *scores_out, bool tensor_cores, void *scratch_q,
+                        DevStatus *st, cudaStream_t s, int64_t *launches);
+// the tensor-core scoring kernel (d = 128, bfloat16 table); scratch_q: topk_query_scratch_bytes(m) bytes for the queries'
+// bfloat16 parts
+int64_t topk_query_scratch_bytes(int64_t m);
 cudaError_t launch_topk_umma(const void *H, int64_t n_items, const float *Q, int64_t m, int k, const int64_t *ex_ptr,
                              const int32_t *ex_idx, int slabs, int64_t slab, float *list_s, int32_t *list_id,
-                             int32_t *list_cnt, cudaStream_t s, int64_t *launches);
+                             int32_t *list_cnt, void *scratch_q, DevStatus *st, cudaStream_t s, int64_t *launches);
 cudaError_t launch_recall(const int32_t *ids, int64_t m, int k_stride, int k, const int64_t *tptr, const int32_t *tidx,
                           double *per_query, double *out2, cudaStream_t s, int64_t *launches);
 cudaError_t launch_rows_fold(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks, int64_t n_split_rows,

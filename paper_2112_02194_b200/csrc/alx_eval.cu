@@ -12,6 +12,7 @@
 //                   into three bfloat16 parts (products exact, sums in fp32)
 #include "alx_common.cuh"
 #include "alx_ptx.cuh"
+#include "alx_topk.cuh"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -19,44 +20,6 @@
 namespace alx {
 
 namespace {
-
-constexpr int kTopkQueries = 128;      // queries per block (= threads of the selection)
-
-__device__ __forceinline__ bool excluded(const int64_t *ex_ptr, const int32_t *ex_idx, int64_t q, int32_t id)
-{
-    if (!ex_ptr) return false;
-    int64_t lo = ex_ptr[q], hi = ex_ptr[q + 1];
-    while (lo < hi) {
-        const int64_t mid = (lo + hi) >> 1;
-        const int32_t v = ex_idx[mid];
-        if (v == id) return true;
-        if (v < id) lo = mid + 1; else hi = mid;
-    }
-    return false;
-}
-
-// One query's list of the best k so far, sorted by (score descending, id ascending).  Items arrive in ascending id, so a
-// newcomer goes behind every element of equal score.
-struct TopList {
-    float *s;
-    int32_t *id;
-    int k, cnt;
-    float tau;      // score of the k-th element once the list is full
-    __device__ __forceinline__ bool wants(float v) const { return cnt < k ? (v == v) : v > tau; }
-    __device__ __forceinline__ void insert(float v, int32_t item)
-    {
-        int pos = cnt < k ? cnt : k - 1;
-        while (pos > 0 && s[pos - 1] < v) {
-            s[pos] = s[pos - 1];
-            id[pos] = id[pos - 1];
-            --pos;
-        }
-        s[pos] = v;
-        id[pos] = item;
-        if (cnt < k) ++cnt;
-        if (cnt == k) tau = s[k - 1];
-    }
-};
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
@@ -213,14 +176,15 @@ int topk_slabs(int64_t n_items, int64_t m)
 
 cudaError_t launch_topk(const void *H, bool bf16, int64_t n_items, int d, const float *Q, int64_t m, int k,
                         const int64_t *ex_ptr, const int32_t *ex_idx, int slabs, float *list_s, int32_t *list_id,
-                        int32_t *list_cnt, int32_t *ids_out, float *scores_out, bool tensor_cores, cudaStream_t s,
-                        int64_t *launches)
+                        int32_t *list_cnt, int32_t *ids_out, float *scores_out, bool tensor_cores, void *scratch_q,
+                        DevStatus *st, cudaStream_t s, int64_t *launches)
 {
     if (m <= 0) return cudaSuccess;
     int64_t slab = (n_items + slabs - 1) / slabs;
     slab = (slab + 127) / 128 * 128;
-    if (false && tensor_cores && bf16 && d == 128) {
-        cudaError_t e = launch_topk_umma(H, n_items, Q, m, k, ex_ptr, ex_idx, slabs, slab, list_s, list_id, list_cnt, s, launches);
+    if (tensor_cores && bf16 && d == 128) {
+        cudaError_t e = launch_topk_umma(H, n_items, Q, m, k, ex_ptr, ex_idx, slabs, slab, list_s, list_id, list_cnt, scratch_q, st, s,
+                                         launches);
         if (e != cudaSuccess) return e;
     } else {
 #define ALX_TOPK_CASE(DD)                                                                                            \

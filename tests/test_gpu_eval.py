@@ -52,11 +52,20 @@ def test_topk_with_exact_scores_is_identical_to_the_full_sort(d, storage, n_item
     a = _ctx(50, n_items, d, storage, graphs.to_storage_bits(H, storage))
     ex = _exclusions(m, n_items, 7)
     for k, exclude in ((50, None), (20, ex), (1, None)):
+        before = a.get_stats().kernel_launches
         ids, sc = a.topk(COLS, Q, k, exclude=exclude)
+        # d = 128 with bfloat16 tables scores on the tensor cores: query split, scoring, merge; otherwise scoring, merge
+        assert a.get_stats().kernel_launches - before == (3 if (d, storage) == (128, "bf16") else 2)
         o_ids, o_sc = ev.topk(Q, H, k, exclude=exclude)
         np.testing.assert_array_equal(ids, o_ids)
         np.testing.assert_array_equal(sc.astype(np.float64), o_sc)
     a.destroy()
+    if (d, storage) == (128, "bf16"):       # the same table through the fp32 scoring kernel
+        b = _ctx(50, n_items, d, storage, graphs.to_storage_bits(H, storage), kernels=1)
+        ids, sc = b.topk(COLS, Q, 50)
+        o_ids, o_sc = ev.topk(Q, H, 50)
+        np.testing.assert_array_equal(ids, o_ids)
+        b.destroy()
 
 
 def test_topk_fills_short_rows_with_minus_one():
