@@ -260,7 +260,7 @@ def run_ours(args, w):
     t_gen = time.perf_counter() - t_gen
 
     a = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0), solver=args.solver,
-            cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol, cg_start=args.cg_start)
+            cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol, cg_start=args.cg_start, dual_cond_limit=args.dual_cond_limit)
     t_set = time.perf_counter()
     a.set_csr(rowptr, colidx)
     torch.cuda.synchronize()
@@ -288,9 +288,15 @@ def run_ours(args, w):
     half_ms = {"rows": [], "cols": [], "gramian": [], "row_kernels": [], "main_kernel": [], "dual_rows": [],
                "cg_rows": [], "cg_products": [], "cg_fallbacks": []}
     ev[0].record()
+    trace = []
     for k in range(args.steps):
-        a.half_epoch(ALX_ROWS)
-        a.half_epoch(ALX_COLS)
+        for side in (ALX_ROWS, ALX_COLS):
+            a.half_epoch(side)
+            if args.trace:      # (reading the statistics waits for the stream: the epoch times of a traced run are not bench values)
+                s1 = a.get_stats()
+                trace.append({"epoch": k, "side": side, "ms": s1.ms_half_epoch, "main_ms": s1.ms_main_kernel,
+                              "cg_rows": s1.cg_rows, "cg_products": s1.cg_products, "cg_fallbacks": s1.cg_fallbacks,
+                              "dual_rows": s1.dual_rows, "cholesky_by_policy": list(s1.cholesky_by_policy)})
         ev[k + 1].record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -421,7 +427,7 @@ def run_ours(args, w):
         o_W = torch.empty_like(h_W, pin_memory=True)
         o_H = torch.empty_like(h_H, pin_memory=True)
         b = Alx(n, n, d, w["lam"], w["alpha"], storage=storage, split=w.get("split", 0), solver=args.solver,
-                cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol, cg_start=args.cg_start)
+                cg_max_iter=args.cg_max_iter, cg_tol=args.cg_tol, cg_start=args.cg_start, dual_cond_limit=args.dual_cond_limit)
         reps = 2 if w["name"] != "small" else 3
         times = []
         for r in range(reps):
@@ -460,7 +466,7 @@ def run_ours(args, w):
                           "paper_context": "about 20 min/epoch for 365M nodes / 29.9B edges on 256 TPU v3 cores"},
                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
                "cpu_baseline": cpu_baseline,
-               "extra": {"evaluation": evaluation, "solver": {"option": args.solver, "cg_rows": half_ms["cg_rows"], "cg_products": half_ms["cg_products"],
+               "extra": {"evaluation": evaluation, "trace": trace or None, "solver": {"option": args.solver, "cg_rows": half_ms["cg_rows"], "cg_products": half_ms["cg_products"],
                                     "cg_fallbacks": half_ms["cg_fallbacks"],
                                     "note": "[rows half-epoch, columns half-epoch] of the half-epoch pair after the timed region"},
                          "epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
@@ -487,6 +493,8 @@ def main():
     ap.add_argument("--cg-start", type=int, default=0, choices=[0, 1],
                     help="alx_options.cg_start: 0 = the stored embedding, 1 = zero")
     ap.add_argument("--cg-tol", type=float, default=0.0, help="alx_options.cg_tol (0 = the library's default)")
+    ap.add_argument("--dual-cond-limit", type=float, default=0.0, help="alx_options.dual_cond_limit (0 = the library's default)")
+    ap.add_argument("--trace", action="store_true", help="per half-epoch statistics of the timed epochs in extra.trace (perturbs the timing)")
     ap.add_argument("--eval", action="store_true", help="also time the exact Top-K retrieval on the trained tables (extra.evaluation)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")

@@ -54,6 +54,7 @@ typedef enum { ALX_SOLVER_AUTO = 0, ALX_SOLVER_CHOLESKY = 1 } alx_solver;
 typedef enum { ALX_CG_START_STORED = 0, ALX_CG_START_ZERO = 1 } alx_cg_start;
 #define ALX_DEFAULT_CG_MAX_ITER 48
 #define ALX_DEFAULT_CG_TOL 1e-5f
+#define ALX_DEFAULT_DUAL_COND_LIMIT 8192.f
 #define ALX_DEFAULT_CG_SWITCH_PRODUCTS 28.f
 
 /* number of degree classes and the default split threshold, see alx_get_buckets */
@@ -100,6 +101,11 @@ typedef struct alx_options {
                                 row's embedding as stored in the table being solved (close to the solution once training
                                 is under way; costs one product for r = b - A x0, and falls back to zero when |r| > |b|);
                                 ALX_CG_START_ZERO (1): x = 0, so that a row's work does not depend on the table's history */
+    float dual_cond_limit;   /* 0 => ALX_DEFAULT_DUAL_COND_LIMIT.  Rows with at most 32 observations (d = 128, bfloat16 tables)
+                                or 16 (d = 64, fp32 tables) are solved in the dual form of Eq. 4 while
+                                ||B||_F ||B^-1||_F <= this limit, B = alpha0 G + lambda I (the form's rounding error grows
+                                with the condition of B; the product is d for a multiple of the identity and about
+                                sqrt(d) cond_2(B) when one direction dominates) */
 } alx_options;
 
 typedef struct alx_stats {
@@ -130,6 +136,8 @@ typedef struct alx_stats {
    (Problem statement, Sec. 3: S subset of U x I x R, W in R^{U x d}, H in R^{I x d}.) */
 alx_status alx_create(int64_t n_rows, int64_t n_cols, int32_t d, float lambda, float alpha0, alx_ctx **out);
 alx_status alx_create_ex(const alx_options *opt, alx_ctx **out);
+/* Free the context and every device buffer it owns (waits for its stream first).  NULL is accepted.
+   Plumbing of this boundary: no counterpart in the paper. */
 alx_status alx_destroy(alx_ctx *ctx);
 
 /*
@@ -144,7 +152,9 @@ alx_status alx_destroy(alx_ctx *ctx);
 alx_status alx_set_csr(alx_ctx *ctx, const int64_t *rowptr, const int32_t *colidx, const float *values,
                        int64_t nnz, int on_device);
 
-/* Overwrite one table from n x d row-major data of type src_dtype (converted with round-to-nearest-even). */
+/* Overwrite one table from n x d row-major data of type src_dtype (converted with round-to-nearest-even).
+   The paper's counterpart is the initialisation of W and H before the first epoch (Alg. 1 takes them as given; it
+   states no distribution); otherwise plumbing of this boundary.  Synchronises. */
 alx_status alx_set_embeddings(alx_ctx *ctx, alx_side side, const void *src, alx_dtype src_dtype, int on_device);
 
 /* The same for rows row_begin .. row_begin + row_count - 1 only (src holds row_count x d values).  For tables that
@@ -203,7 +213,8 @@ alx_status alx_half_epoch_capture(alx_ctx *ctx, alx_side solved_side, const int6
  */
 alx_status alx_loss(alx_ctx *ctx, double *total, double *components);
 
-/* Copy rows [row_begin, row_begin + row_count) of one table to dst (row_count x d, dst_dtype). Synchronises. */
+/* Copy rows [row_begin, row_begin + row_count) of one table to dst (row_count x d, dst_dtype). Synchronises.
+   The tables are the method's output (W, H of Sec. 3); the call itself is plumbing with no counterpart in the paper. */
 alx_status alx_get_embeddings(alx_ctx *ctx, alx_side side, void *dst, alx_dtype dst_dtype, int64_t row_begin,
                               int64_t row_count, int on_device);
 
@@ -231,6 +242,7 @@ alx_status alx_get_transpose(alx_ctx *ctx, int64_t *colptr, int32_t *rowidx, flo
 alx_status alx_get_buckets(alx_ctx *ctx, alx_side side, int32_t *order, int64_t *class_offsets,
                            int64_t *chunk_desc, int64_t *n_chunks);
 
+/* Counters and device times of the context (see alx_stats).  Diagnostics: no counterpart in the paper. */
 alx_status alx_get_stats(alx_ctx *ctx, alx_stats *out);
 
 /*

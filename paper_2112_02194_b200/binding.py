@@ -33,7 +33,7 @@ class alx_options(Structure):
                 ("alpha0", c_float), ("storage", c_int32), ("device", c_int32), ("stream", c_void_p),
                 ("alloc", ALLOC_FN), ("free", FREE_FN), ("alloc_user", c_void_p), ("split", c_int64),
                 ("kernels", c_int32), ("solver", c_int32), ("cg_max_iter", c_int32), ("cg_tol", c_float),
-                ("cg_switch_products", c_float), ("cg_start", c_int32)]
+                ("cg_switch_products", c_float), ("cg_start", c_int32), ("dual_cond_limit", c_float)]
 
 
 class alx_stats(Structure):
@@ -117,7 +117,8 @@ class Alx:
     """One context.  Methods carry the C names without the ``alx_`` prefix and only marshal arguments."""
 
     def __init__(self, n_rows, n_cols, d, lam, alpha0, storage="f32", split=0, kernels=0, device=None,
-                 use_torch_allocator=True, solver=0, cg_max_iter=0, cg_tol=0.0, cg_start=0, cg_switch_products=0.0):
+                 use_torch_allocator=True, solver=0, cg_max_iter=0, cg_tol=0.0, cg_start=0, cg_switch_products=0.0,
+                 dual_cond_limit=0.0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("alx needs a CUDA device (B200, sm_100a); there is no CPU path")
@@ -137,6 +138,7 @@ class Alx:
         opt.kernels = kernels
         opt.solver, opt.cg_max_iter, opt.cg_tol = int(solver), int(cg_max_iter), float(cg_tol)
         opt.cg_start = int(cg_start)
+        opt.dual_cond_limit = float(dual_cond_limit)
         opt.cg_switch_products = float(cg_switch_products)
         if use_torch_allocator:
             dev = torch.device("cuda", self.device)

@@ -264,6 +264,7 @@ bool fold_path(const alx_ctx *c)
     return !c->bf16 && c->opt.d == 64 && c->opt.kernels != 1 && c->n[0] < (1ll << 30) && c->n[1] < (1ll << 30);
 }
 bool dual_form(const alx_ctx *c) { return tensor_path(c) && c->opt.kernels == 0; }
+float dual_cond_limit(const alx_ctx *c) { return c->opt.dual_cond_limit > 0.f ? c->opt.dual_cond_limit : ALX_DEFAULT_DUAL_COND_LIMIT; }
 CgOptions cg_options(const alx_ctx *c, int solved_side)
 {
     CgOptions o;
@@ -285,12 +286,14 @@ alx_status gramian_of(alx_ctx *c, int table_side)
         ALX_CUDA(c, launch_gramian_umma(c->table[table_side], c->n[table_side], c->gram_partials, c->stream, &c->launches));
         ALX_CUDA(c, launch_gramian_reduce(c->gram_partials, gramian_umma_partials(), c->opt.d, c->G64[table_side], c->Bmat,
                                           c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
-        if (dual_form(c)) ALX_CUDA(c, launch_dual_prepare(c->Bmat, c->dual_ws, c->stream, &c->launches));
+        if (dual_form(c)) ALX_CUDA(c, launch_dual_prepare(c->Bmat, c->dual_ws, dual_cond_limit(c), c->stream, &c->launches));
         c->have_gram[table_side] = true;
         return ALX_OK;
     }
     ALX_CUDA(c, launch_gramian(c->table[table_side], c->bf16, c->n[table_side], c->opt.d, c->gram_partials,
                                c->G64[table_side], c->Bmat, c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
+    if (fold_path(c) && c->dual_ws)
+        ALX_CUDA(c, launch_dual64_prepare(c->Bmat, c->dual_ws, dual_cond_limit(c), c->stream, &c->launches));
     c->have_gram[table_side] = true;
     return ALX_OK;
 }
@@ -309,12 +312,22 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
         ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_split_table(static_cast<const float *>(c->table[fixed]), c->n[fixed], c->fold_table, c->stream,
                                        &c->launches));
+        // rows of 1 .. 16 observations (class 1 of the entry lists as given = classes 1 and 2 of the doubled ones): dual form
+        const int64_t n_dual = c->dual_ws ? c->class_offs[side][2] - c->class_offs[side][1] : 0;
+        if (n_dual > 0)
+            ALX_CUDA(c, launch_rows_dual64(side_view(c, side), c->class_offs[side][1], n_dual, c->table[fixed], c->dual_ws, out,
+                                           c->stream, &c->launches));
         ALX_CUDA(c, launch_rows_fold(side_view(c, 2 + side), c->class_offs[2 + side], c->n_chunks[2 + side],
                                      c->n_split_rows[2 + side], c->fold_table, 2 * c->n[fixed], c->Bmat, c->split_partials,
-                                     out, c->status, c->stream, &c->launches, c->ev[3], c->ev[4], cg_options(c, side)));
+                                     out, c->status, c->stream, &c->launches, c->ev[3], c->ev[4], cg_options(c, side),
+                                     n_dual > 0 ? dual64_flag_ptr(c->dual_ws) : nullptr));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
-        c->dual_candidates = 0;
+        c->dual_candidates = n_dual;
+        c->dual_flag_latched = 0;
+        if (n_dual > 0)
+            ALX_CUDA(c, cudaMemcpyAsync(&c->dual_flag_latched, dual64_flag_ptr(c->dual_ws), sizeof(int), cudaMemcpyDeviceToHost,
+                                        c->stream));
     } else if (tensor_path(c)) {
         ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
@@ -379,7 +392,7 @@ alx_status create_impl(const alx_options *opt, const alx_ctx *parent, alx_ctx **
     if (opt->split != 0 && opt->split < 16) return ALX_ERR_INVALID_ARG;
     if (opt->solver != ALX_SOLVER_AUTO && opt->solver != ALX_SOLVER_CHOLESKY) return ALX_ERR_INVALID_ARG;
     if (opt->cg_start != ALX_CG_START_STORED && opt->cg_start != ALX_CG_START_ZERO) return ALX_ERR_INVALID_ARG;
-    if (!(opt->cg_switch_products >= 0.f)) return ALX_ERR_INVALID_ARG;
+    if (!(opt->cg_switch_products >= 0.f) || !(opt->dual_cond_limit >= 0.f)) return ALX_ERR_INVALID_ARG;
     if (opt->cg_max_iter < 0 || opt->cg_max_iter > 1024 || !(opt->cg_tol >= 0.f) || opt->cg_tol > 1e-2f) return ALX_ERR_INVALID_ARG;
     int dev = opt->device;
     if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return ALX_ERR_CUDA;
@@ -408,8 +421,8 @@ alx_status create_impl(const alx_options *opt, const alx_ctx *parent, alx_ctx **
             if (fold_path(c)) ALX_ALLOC(c, c->class_offs_dev[2 + s], ALX_N_CLASSES + 1);
         }
         ALX_ALLOC(c, c->Bmat, d * d);
-        if (dual_form(c)) {
-            c->dual_ws = dev_alloc(c, dual_workspace_bytes());
+        if (dual_form(c) || (fold_path(c) && c->opt.kernels == 0)) {
+            c->dual_ws = dev_alloc(c, dual_form(c) ? dual_workspace_bytes() : dual64_workspace_bytes());
             if (!c->dual_ws) return fail(c, ALX_ERR_OOM, "device allocation of the dual-form workspace failed");
         }
         const int64_t nmax = c->n[0] > c->n[1] ? c->n[0] : c->n[1];

@@ -196,7 +196,7 @@ cudaError_t launch_recall(const int32_t *ids, int64_t m, int k_stride, int k, co
 cudaError_t launch_rows_fold(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks, int64_t n_split_rows,
                              const void *T, int64_t n_table, const float *Bmat, float *split_partials, RowOut out,
                              DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
-                             const CgOptions &cg);
+                             const CgOptions &cg, const int *dual_flag);
 // fp32 table [n x 64] -> bfloat16 parts [2n x 128]
 cudaError_t launch_split_table(const float *X, int64_t n, void *T, cudaStream_t s, int64_t *launches);
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
@@ -206,7 +206,13 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host,
 
 // alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();
-cudaError_t launch_dual_prepare(const float *Bmat, void *ws, cudaStream_t s, int64_t *launches);
+cudaError_t launch_dual_prepare(const float *Bmat, void *ws, float cond_limit, cudaStream_t s, int64_t *launches);
+// fp32 tables of 64 features (alx_dual64.cu): B^-1 (fp32) + flag; rows of 1 .. 16 observations in the dual form
+size_t dual64_workspace_bytes();
+int *dual64_flag_ptr(void *ws);
+cudaError_t launch_dual64_prepare(const float *Bmat, void *ws, float cond_limit, cudaStream_t s, int64_t *launches);
+cudaError_t launch_rows_dual64(const SideView &sv, int64_t first, int64_t count, const void *X, void *ws, RowOut out,
+                               cudaStream_t s, int64_t *launches);
 const int *dual_flag_ptr(const void *ws);
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
                              const void *ws, RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches);

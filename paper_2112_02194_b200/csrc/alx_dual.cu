@@ -37,7 +37,6 @@ constexpr int kGroupThreads = 128;
 constexpr int kSolverThreads = kSlots * kGroupThreads;
 constexpr int kMmaWarp = kSolverThreads / 32;
 constexpr int kBlockThreads = kSolverThreads + 32 + kProducerWarps * 32;
-constexpr double kCondLimit = 2048.0;         // on ||B||_F ||B^-1||_F (128 for a multiple of the identity)
 
 // byte offset of element (row, feature) inside a K-major tile with 128-byte swizzle: rows of 64 features
 // (128 bytes), groups of 8 rows (1024 bytes), the 16-byte chunk index XORed with the row's index in its group
@@ -55,9 +54,10 @@ __host__ __device__ constexpr uint32_t idesc_bf16_k_major(int M, int N)
 
 // ---------------------------------------------------------------------------------------------------------
 // B^-1 in fp64 by Cholesky (one block of 128 threads, thread i = row i), written as three bfloat16 parts in the
-// operand layout of the dual kernel; flag = 1 if B is positive definite and ||B||_F ||B^-1||_F <= kCondLimit.
+// operand layout of the dual kernel; flag = 1 if B is positive definite and ||B||_F ||B^-1||_F <= cond_limit
+// (the product is 128 for a multiple of the identity).
 __global__ void __launch_bounds__(128, 1) k_binv_prepare(const float *__restrict__ Bmat, unsigned char *__restrict__ tiles,
-                                                         int *__restrict__ flag)
+                                                         int *__restrict__ flag, double cond_limit)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *A = reinterpret_cast<double *>(smem_raw);          // [128][129]: lower = L, strict upper = (L^-1)^T
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(128, 1) k_binv_prepare(const float *__restrict
     if (i == 0) {
         double a = 0.0, b = 0.0;
         for (int k = 0; k < D; ++k) { a += red[k]; b += dinv[k]; }
-        *flag = (s_ok && sqrt(a) * sqrt(b) <= kCondLimit) ? 1 : 0;
+        *flag = (s_ok && sqrt(a) * sqrt(b) <= cond_limit) ? 1 : 0;
     }
 }
 
@@ -602,13 +602,13 @@ template <int KP> cudaError_t launch_dual_instance(DualParams p, int sms, cudaSt
 size_t dual_workspace_bytes() { return (size_t)kBinvBytes + 256; }
 
 // B^-1 (three operand tiles at `ws`) and the flag (at ws + kBinvBytes) for the dual kernel
-cudaError_t launch_dual_prepare(const float *Bmat, void *ws, cudaStream_t s, int64_t *launches)
+cudaError_t launch_dual_prepare(const float *Bmat, void *ws, float cond_limit, cudaStream_t s, int64_t *launches)
 {
     const size_t smem = sizeof(double) * (D * (D + 1) + 2 * D);
     cudaError_t e = cudaFuncSetAttribute(k_binv_prepare, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     unsigned char *w = static_cast<unsigned char *>(ws);
-    k_binv_prepare<<<1, 128, smem, s>>>(Bmat, w, reinterpret_cast<int *>(w + kBinvBytes));
+    k_binv_prepare<<<1, 128, smem, s>>>(Bmat, w, reinterpret_cast<int *>(w + kBinvBytes), (double)cond_limit);
     ++*launches;
     return cudaGetLastError();
 }

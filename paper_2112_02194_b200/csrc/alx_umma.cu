@@ -2122,7 +2122,7 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
 cudaError_t launch_rows_fold(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows, const void *T,
                              int64_t n_table, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
                              cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
-                             const CgOptions &cg)
+                             const CgOptions &cg, const int *dual_flag)
 {
     const int sms = sm_count();
     Params p{};
@@ -2161,6 +2161,11 @@ cudaError_t launch_rows_fold(const SideView &sv, const int64_t *offs, int64_t n_
         if (e != cudaSuccess) return e;
     }
     const int64_t n_whole = offs[c_long] - offs[1];
+    if (dual_flag && offs[3] > offs[1]) {
+        // rows of at most 32 doubled entries (16 observations) are solved in the dual form elsewhere while the flag is set
+        p.dual_flag = dual_flag;
+        p.n_items_primal = offs[c_long] - offs[3];
+    }
     if (n_whole > 0) {
         p.n_items = n_whole;
         p.last_item = offs[c_long] - 1;

@@ -106,6 +106,8 @@ def test_gramian_matches_oracle(prob):
         ref = ials.gramian(p.f64(tab))
         # 1e-6 for fp32 FMA sums; the tensor-core accumulator truncates (up to 2^-24 per 16-row step, always
         # towards zero, 16 steps per read-out), which adds a bias of up to ~1e-6 on the diagonal
+        print(f"{p.name} Gramian of side {side}: max |G - ref| / max |ref| = {np.abs(G - ref).max() / np.abs(ref).max():.2e}, "
+              f"diagonal bias {np.mean(np.diag(G - ref)) / np.mean(np.diag(ref)):+.2e}")
         assert np.abs(G - ref).max() <= 2e-6 * np.abs(ref).max()
         np.testing.assert_array_equal(G, G.T)
     a.destroy()
@@ -404,6 +406,37 @@ def test_dual_form_steps_aside_when_base_matrix_is_ill_conditioned():
     assert worst <= 1e-4, worst
 
 
+@pytest.mark.parametrize("name,offset,kmax", [("local_d128_bf16", 0.02, 32), ("zipf_d64_f32", 0.05, 16)])
+def test_dual_form_meets_the_residual_gate_close_to_its_condition_limit(name, offset, kmax):
+    """||B||_F ||B^-1||_F of about 7300 (d = 128) and 8100 (d = 64), just inside the default limit of 8192 (cond_2(B) about 860
+    and 1200): the short rows are solved in the dual form and every one of them meets the residual gate with room to
+    spare (the form's error grows with the condition of B, which is what the limit is for)."""
+    from synth import graphs
+    p = _problem(name)
+    rng = np.random.Generator(np.random.PCG64(77))
+    H0 = offset + 0.1 / np.sqrt(p.d) * rng.standard_normal((p.n_cols, p.d))
+    p.H0 = graphs.to_storage_bits(H0, p.storage)
+    p.alpha, p.lam = 0.5, 0.01
+    deg = np.diff(p.rowptr)
+    ids = np.nonzero((deg > 0) & (deg <= kmax))[0].astype(np.int64)
+    a = make_ctx(p)
+    x32 = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+    st = a.get_stats()
+    a.destroy()
+    assert st.dual_rows == ids.size and st.not_spd == 0
+    H0r = p.f64(p.H0)
+    G = ials.gramian(H0r)
+    B = p.alpha * G + p.lam * np.eye(p.d)
+    fro = np.linalg.norm(B) * np.linalg.norm(np.linalg.inv(B))
+    assert 6000 < fro < 8192, fro
+    worst = 0.0
+    for n in range(ids.size):
+        A, b = ials.row_system(p.rowptr, p.colidx, None, H0r, G, p.alpha, p.lam, int(ids[n]))
+        worst = max(worst, np.linalg.norm(A @ x32[n] - b) / np.linalg.norm(b))
+    print(f"{name}: ||B|| ||B^-1|| = {fro:.0f}, worst residual of {ids.size} dual-form rows {worst:.2e}")
+    assert worst <= 5e-5, worst
+
+
 def _whole_rows(p):
     """rows of 33 .. 1024 observations: the ones the whole-rows tensor-core kernel solves"""
     deg = np.diff(p.rowptr)
@@ -462,7 +495,9 @@ def test_fp32_tables_of_64_features_on_the_tensor_cores(name):
     G = ials.gramian(H0)
     vals64 = None if p.values is None else p.values.astype(np.float64)
     sols, stats = {}, {}
-    for label, kw in (("cg", dict(cg_start=1)), ("chol", dict(solver=1)), ("fallback", dict(cg_max_iter=2, cg_start=1)),
+    # kernels = 2: the 64 x 64 form for every row; kernels = 0 (default): rows of at most 16 observations in the dual form
+    for label, kw in (("cg", dict(cg_start=1, kernels=2)), ("chol", dict(solver=1, kernels=2)),
+                      ("fallback", dict(cg_max_iter=2, cg_start=1, kernels=2)), ("dual", dict(cg_start=1)),
                       ("alu", dict(kernels=1))):
         a = make_ctx(p, **kw)
         sols[label] = a.half_epoch_capture(ROWS, ids).astype(np.float64)
@@ -470,9 +505,11 @@ def test_fp32_tables_of_64_features_on_the_tensor_cores(name):
         assert stats[label].not_spd == 0
         assert stats[label].kernel_path[0] == (0 if label == "alu" else 1)
         a.destroy()
-    assert stats["cg"].cg_rows == ids.size and stats["cg"].cg_fallbacks == 0
+    assert stats["cg"].cg_rows == ids.size and stats["cg"].cg_fallbacks == 0 and stats["cg"].dual_rows == 0
     assert stats["chol"].cg_rows == 0 and stats["alu"].cg_rows == 0
     assert stats["fallback"].cg_rows == ids.size and stats["fallback"].cg_fallbacks > 0.5 * ids.size
+    n_short = int(((deg > 0) & (deg <= 16)).sum())
+    assert n_short > 500 and stats["dual"].dual_rows == n_short and stats["dual"].cg_rows == ids.size - n_short
     if p.split == 0:
         assert stats["cg"].long_rows[0] > 0      # whole rows of more than 512 observations took the chunks kernel
     _, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G, return_raw=True)
@@ -490,7 +527,7 @@ def test_fp32_tables_of_64_features_on_the_tensor_cores(name):
         if not nz[n]:
             continue
         A, b = ials.row_system(p.rowptr, p.colidx, vals64, H0, G, p.alpha, p.lam, int(ids[n]))
-        for label in ("cg", "chol", "fallback"):
+        for label in ("cg", "chol", "fallback", "dual"):
             worst = max(worst, np.linalg.norm(A @ sols[label][n] - b) / np.linalg.norm(b))
     assert worst <= 1e-4, worst
 
