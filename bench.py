@@ -481,13 +481,83 @@ def run_ours(args, w):
         torch.distributed.destroy_process_group()
 
 
+def run_cfg1(args):
+    """Configuration 1 (2000 x 1500, 40 000 uniform cells, d = 16, fp32 tables): 2.6 MB of data and 2e7 flop per epoch, bound
+    by launch latency.  Reported as time per epoch; no roofline is claimed for it."""
+    import torch
+    from paper_2112_02194_b200 import ALX_COLS, ALX_ROWS, Alx
+    torch.cuda.set_device(0)
+    rowptr, colidx = graphs.uniform_cells_csr(2000, 1500, 40000, 0xA1C50001)
+    W0 = graphs.init_embeddings(2000, 16, 0x1A150001, 2, "f32")
+    H0 = graphs.init_embeddings(1500, 16, 0x1A150001, 3, "f32")
+    a = Alx(2000, 1500, 16, 0.1, 0.01, storage="f32")
+    a.set_csr(rowptr, colidx, None)
+    a.set_embeddings(ALX_ROWS, W0)
+    a.set_embeddings(ALX_COLS, H0)
+    for _ in range(args.warmup):
+        a.epoch()
+    a.synchronize()
+    launches0 = a.get_stats().kernel_launches
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev[0].record()
+    for _ in range(args.steps):
+        a.epoch()
+    ev[1].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev[0].elapsed_time(ev[1]) / args.steps
+    launches = a.get_stats().kernel_launches - launches0
+    oW, oH = np.empty_like(W0), np.empty_like(H0)
+    t0 = time.perf_counter()
+    a.load_host(rowptr, colidx, None, W0, H0)
+    a.epoch_to_host(oW, oH)
+    t_e2e = time.perf_counter() - t0
+    a.destroy()
+    nnz = int(colidx.size)
+    print(json.dumps({"metric": METRIC, "value": nnz / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+                      "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                      "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "cfg1", "description": "2000 x 1500, 40 000 uniform cells, d=16, fp32 tables",
+                                 "nnz": nnz, "l2": "fits in L2: latency-bound case, reported as time only"},
+                      "clocks": clocks, "gpu_launches": int(launches), "roofline": None, "cpu_baseline": None,
+                      "e2e": {"value": nnz / t_e2e, "unit": UNIT, "ms_per_step": t_e2e * 1e3,
+                              "h2d_bytes_per_step": int(rowptr.nbytes + colidx.nbytes + W0.nbytes + H0.nbytes),
+                              "d2h_bytes_per_step": int(W0.nbytes + H0.nbytes)}}))
+
+
+def run_cfg1_reference(args):
+    """The oracle's whole epoch on configuration 1 (it is small enough to run in full)."""
+    if dist_env()[0] != 0:
+        return
+    from oracle import ials
+    ials.build()
+    rowptr, colidx = graphs.uniform_cells_csr(2000, 1500, 40000, 0xA1C50001)
+    W0 = graphs.init_embeddings(2000, 16, 0x1A150001, 2, "f32").astype(np.float64)
+    H0 = graphs.init_embeddings(1500, 16, 0x1A150001, 3, "f32").astype(np.float64)
+    for _ in range(args.warmup):
+        ials.epoch(rowptr, colidx, None, W0, H0, 0.01, 0.1, "f32")
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ials.epoch(rowptr, colidx, None, W0, H0, 0.01, 0.1, "f32")
+    ms = (time.perf_counter() - t0) * 1e3 / max(args.steps, 1)
+    value = colidx.size / (ms * 1e-3)
+    info = {"kind": "oracle", "cores": os.cpu_count() or 1, "unit": UNIT, "value": value,
+            "sample": "the whole epoch of configuration 1 (2000 x 1500, 40 000 entries), fp64, OpenMP over rows"}
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+                      "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                      "dtype": "f64", "data": "synthetic", "config": {"workload": "cfg1"}, "cpu_baseline": info,
+                      "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS) + ["cfg1"])
     ap.add_argument("--solver", type=int, default=0, choices=[0, 1],
                     help="alx_options.solver: 0 = conjugate gradients where available (Cholesky otherwise), 1 = Cholesky")
     ap.add_argument("--cg-max-iter", type=int, default=0, help="alx_options.cg_max_iter (0 = the library's default)")
@@ -500,6 +570,8 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the host-buffer leg")
     ap.add_argument("--skip-cpu", action="store_true", help="profiling runs: leave out the CPU oracle leg")
     args = ap.parse_args()
+    if args.workload == "cfg1":
+        return run_cfg1(args) if args.impl == "ours" else run_cfg1_reference(args)
     w = dict(WORKLOADS[args.workload], name=args.workload)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # started as a plain script: become the launcher of one replica process per GPU

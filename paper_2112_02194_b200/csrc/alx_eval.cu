@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kTopkQueries) k_topk_simple(const T *__restric
 #pragma unroll
     for (int f = 0; f < DD; ++f) qv[f] = live ? Q[q * DD + f] : 0.f;
     const int64_t lq = (int64_t)blockIdx.y * m + (live ? q : 0);
-    TopList top{list_s + lq * k, list_id + lq * k, k, 0, 0.f};
+    TopList top{list_s + lq * k, list_id + lq * k, k, 0, 0.f, 1};
     const int64_t i0 = (int64_t)blockIdx.y * slab;
     const int64_t i1 = i0 + slab < n_items ? i0 + slab : n_items;
     for (int64_t base = i0; base < i1; base += kTile) {

@@ -21,24 +21,27 @@ __device__ __forceinline__ bool excluded(const int64_t *ex_ptr, const int32_t *e
 
 // One query's list of the best k so far, sorted by (score descending, id ascending).  Items arrive in ascending id, so a
 // newcomer goes behind every element of equal score.
+// (stride: distance between consecutive elements of the list, 1 in global memory; in shared memory the lists of a
+// block's 128 queries are interleaved, element p of query t at p * 128 + t, so that no two threads share a bank)
 struct TopList {
     float *s;
     int32_t *id;
     int k, cnt;
     float tau;      // score of the k-th element once the list is full
+    int stride;
     __device__ __forceinline__ bool wants(float v) const { return cnt < k ? (v == v) : v > tau; }
     __device__ __forceinline__ void insert(float v, int32_t item)
     {
         int pos = cnt < k ? cnt : k - 1;
-        while (pos > 0 && s[pos - 1] < v) {
-            s[pos] = s[pos - 1];
-            id[pos] = id[pos - 1];
+        while (pos > 0 && s[(pos - 1) * stride] < v) {
+            s[pos * stride] = s[(pos - 1) * stride];
+            id[pos * stride] = id[(pos - 1) * stride];
             --pos;
         }
-        s[pos] = v;
-        id[pos] = item;
+        s[pos * stride] = v;
+        id[pos * stride] = item;
         if (cnt < k) ++cnt;
-        if (cnt == k) tau = s[k - 1];
+        if (cnt == k) tau = s[(k - 1) * stride];
     }
 };
 
