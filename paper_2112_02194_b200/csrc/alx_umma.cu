@@ -1,4 +1,5 @@
-// Tensor-core (tcgen05 / tensor memory) kernels for d = 128 with bfloat16 tables:
+// Tensor-core (tcgen05 / tensor memory) kernels for d = 128 with bfloat16 tables (and, through bfloat16 parts of the
+// table and doubled entry lists, for d = 64 with fp32 tables: kModeRowsFold below):
 //   - the Gramian X^T X of the fixed table                                   (Alg. 1 line 2)
 //   - per row: sum x_i (x) x_i and sum y x_i over the row's observations      (Alg. 1 lines 6-9),
 //     then the solve of Eq. 4 and the store                                   (Alg. 1 line 10)
@@ -20,8 +21,9 @@
 //                    converge is left to a second launch.  kModeRows: thread i owns row i, the group adds
 //                    alpha0 G + lambda I on first touch and factors in place with a blocked right-looking
 //                    Cholesky (tcgen05.ld / tcgen05.st of 16-column row segments, trailing updates on the
-//                    tensor core), solves and stores the row.  Gramian pieces and chunks: two groups of 256
-//                    threads copy the sums out.
+//                    tensor core), solves and stores the row.  kModeRowsFold: the group folds the 64 x 64 system out
+//                    of its accumulator into registers and solves it there (conjugate gradients, or Cholesky in
+//                    shared memory).  Gramian pieces and chunks: two groups of 256 threads copy the sums out.
 // Stage and accumulator hand-over is by mbarriers; every wait is bounded and a block that gives up
 // sets a status flag, releases its tensor memory and returns.
 #include "alx_chol.cuh"
