@@ -105,7 +105,10 @@ typedef struct alx_options {
                                 or 16 (d = 64, fp32 tables) are solved in the dual form of Eq. 4 while
                                 ||B||_F ||B^-1||_F <= this limit, B = alpha0 G + lambda I (the form's rounding error grows
                                 with the condition of B; the product is d for a multiple of the identity and about
-                                sqrt(d) cond_2(B) when one direction dominates) */
+                                sqrt(d) cond_2(B) when one direction dominates).  Beyond the limit, with solver =
+                                ALX_SOLVER_AUTO and d = 128: the dual-form solutions become the start vectors of a
+                                conjugate-gradient pass over those rows (alx_stats.dual_polished_rows); otherwise the
+                                rows take the d x d solve like every other row */
 } alx_options;
 
 typedef struct alx_stats {
@@ -128,6 +131,8 @@ typedef struct alx_stats {
     int64_t cg_fallbacks;                    /* and how many of those rows went on to the Cholesky solve (not converged) */
     int32_t cholesky_by_policy[2];           /* [side]: 1 if the side's LAST half-epoch took Cholesky for every row because
                                                 its conjugate-gradient run before that spent too many products per row */
+    int64_t dual_polished_rows;              /* LAST half-epoch: dual-form rows that went through a conjugate-gradient pass */
+    int64_t dual_polish_products;            /* because B was beyond the condition limit (see dual_cond_limit), and its products */
     int64_t entries_in_class[2][ALX_N_CLASSES]; /* [side][class]: the observed entries held by the rows of each degree class
                                                    (sums to nnz over the classes of a side) */
 } alx_stats;

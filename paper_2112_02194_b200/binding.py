@@ -43,6 +43,7 @@ class alx_stats(Structure):
                 ("kernel_path", c_int32 * 2), ("ms_main_kernel", c_double), ("dual_rows", c_int64),
                 ("long_rows", c_int64 * 2), ("long_entries", c_int64 * 2), ("cg_rows", c_int64),
                 ("cg_products", c_int64), ("cg_fallbacks", c_int64), ("cholesky_by_policy", c_int32 * 2),
+                ("dual_polished_rows", c_int64), ("dual_polish_products", c_int64),
                 ("entries_in_class", (c_int64 * ALX_N_CLASSES) * 2)]
 
 

@@ -53,7 +53,7 @@ struct alx_ctx {
     double *loss_partials_buf = nullptr;
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
-    unsigned long long *cg_counters = nullptr;   // tensor path: rows solved by conjugate gradients, products, fall-backs (last half-epoch)
+    unsigned long long *cg_counters = nullptr;   // tensor path, last half-epoch: rows solved by conjugate gradients, products, fall-backs; dual-form rows polished, their products
     int32_t *cg_fallback_list = nullptr;         // tensor path with conjugate gradients: the rows left to the Cholesky solve
     CgPolicy *cg_policy = nullptr;               // [2]: per side, what the solver choice of its next half-epoch rests on
 
@@ -286,7 +286,8 @@ alx_status gramian_of(alx_ctx *c, int table_side)
         ALX_CUDA(c, launch_gramian_umma(c->table[table_side], c->n[table_side], c->gram_partials, c->stream, &c->launches));
         ALX_CUDA(c, launch_gramian_reduce(c->gram_partials, gramian_umma_partials(), c->opt.d, c->G64[table_side], c->Bmat,
                                           c->opt.alpha0, c->opt.lambda, c->stream, &c->launches));
-        if (dual_form(c)) ALX_CUDA(c, launch_dual_prepare(c->Bmat, c->dual_ws, dual_cond_limit(c), c->stream, &c->launches));
+        if (dual_form(c)) ALX_CUDA(c, launch_dual_prepare(c->Bmat, c->dual_ws, dual_cond_limit(c), c->opt.solver == ALX_SOLVER_AUTO, c->stream,
+                                                         &c->launches));
         c->have_gram[table_side] = true;
         return ALX_OK;
     }
@@ -309,7 +310,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
     RowOut out{c->table[side], cap_slot, cap_out};
     if (fold_path(c)) {
-        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 5 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_split_table(static_cast<const float *>(c->table[fixed]), c->n[fixed], c->fold_table, c->stream,
                                        &c->launches));
         // rows of 1 .. 16 observations (class 1 of the entry lists as given = classes 1 and 2 of the doubled ones): dual form
@@ -329,7 +330,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
             ALX_CUDA(c, cudaMemcpyAsync(&c->dual_flag_latched, dual64_flag_ptr(c->dual_ws), sizeof(int), cudaMemcpyDeviceToHost,
                                         c->stream));
     } else if (tensor_path(c)) {
-        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 5 * sizeof(unsigned long long), c->stream));
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
                                      &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed],
@@ -436,13 +437,13 @@ alx_status create_impl(const alx_options *opt, const alx_ctx *parent, alx_ctx **
         ALX_ALLOC(c, c->loss_result, 4);
         ALX_ALLOC(c, c->status, 1);
         ALX_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(DevStatus), c->stream));
-        ALX_ALLOC(c, c->cg_counters, 3);
+        ALX_ALLOC(c, c->cg_counters, 5);
         if (tensor_path(c) && c->opt.solver == ALX_SOLVER_AUTO) {
             ALX_ALLOC(c, c->cg_fallback_list, nmax);
             ALX_ALLOC(c, c->cg_policy, 2);
             ALX_CUDA(c, cudaMemsetAsync(c->cg_policy, 0, 2 * sizeof(CgPolicy), c->stream));
         }
-        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 3 * sizeof(unsigned long long), c->stream));
+        ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 5 * sizeof(unsigned long long), c->stream));
         for (auto &e : c->ev) ALX_CUDA(c, cudaEventCreate(&e));
         ALX_CUDA(c, cudaStreamSynchronize(c->stream));
         return ALX_OK;
@@ -1003,11 +1004,13 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
     }
     c->stats.dual_rows = c->dual_candidates > 0 && c->dual_flag_latched ? c->dual_candidates : 0;
     {
-        unsigned long long h[3] = {0, 0, 0};
+        unsigned long long h[5] = {0, 0, 0, 0, 0};
         ALX_CUDA(c, cudaMemcpy(h, c->cg_counters, sizeof h, cudaMemcpyDeviceToHost));
         c->stats.cg_rows = (int64_t)h[0];
         c->stats.cg_products = (int64_t)h[1];
         c->stats.cg_fallbacks = (int64_t)h[2];
+        c->stats.dual_polished_rows = (int64_t)h[3];
+        c->stats.dual_polish_products = (int64_t)h[4];
         c->stats.cholesky_by_policy[0] = c->stats.cholesky_by_policy[1] = 0;
         if (c->cg_policy) {
             CgPolicy pol[2];

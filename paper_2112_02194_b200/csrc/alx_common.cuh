@@ -206,7 +206,8 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host,
 
 // alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();
-cudaError_t launch_dual_prepare(const float *Bmat, void *ws, float cond_limit, cudaStream_t s, int64_t *launches);
+cudaError_t launch_dual_prepare(const float *Bmat, void *ws, float cond_limit, bool allow_start, cudaStream_t s,
+                                int64_t *launches);
 // fp32 tables of 64 features (alx_dual64.cu): B^-1 (fp32) + flag; rows of 1 .. 16 observations in the dual form
 size_t dual64_workspace_bytes();
 int *dual64_flag_ptr(void *ws);

@@ -54,10 +54,11 @@ __host__ __device__ constexpr uint32_t idesc_bf16_k_major(int M, int N)
 
 // ---------------------------------------------------------------------------------------------------------
 // B^-1 in fp64 by Cholesky (one block of 128 threads, thread i = row i), written as three bfloat16 parts in the
-// operand layout of the dual kernel; flag = 1 if B is positive definite and ||B||_F ||B^-1||_F <= cond_limit
+// operand layout of the dual kernel; flag = 1 if B is positive definite and ||B||_F ||B^-1||_F <= cond_limit,
+// 2 if it is positive definite but beyond the limit and the caller can use the dual solutions as start vectors, else 0
 // (the product is 128 for a multiple of the identity).
 __global__ void __launch_bounds__(128, 1) k_binv_prepare(const float *__restrict__ Bmat, unsigned char *__restrict__ tiles,
-                                                         int *__restrict__ flag, double cond_limit)
+                                                         int *__restrict__ flag, double cond_limit, int allow_start)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     double *A = reinterpret_cast<double *>(smem_raw);          // [128][129]: lower = L, strict upper = (L^-1)^T
@@ -129,7 +130,7 @@ __global__ void __launch_bounds__(128, 1) k_binv_prepare(const float *__restrict
     if (i == 0) {
         double a = 0.0, b = 0.0;
         for (int k = 0; k < D; ++k) { a += red[k]; b += dinv[k]; }
-        *flag = (s_ok && sqrt(a) * sqrt(b) <= cond_limit) ? 1 : 0;
+        *flag = !s_ok ? 0 : (sqrt(a) * sqrt(b) <= cond_limit) ? 1 : (allow_start ? 2 : 0);
     }
 }
 
@@ -545,7 +546,7 @@ template <int KP> __global__ void __launch_bounds__(kBlockThreads, 1) k_dual(Dua
     unsigned char *aligned = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     DualSmem &sm = *reinterpret_cast<DualSmem *>(aligned);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (*p.flag == 0) return;       // B is not well conditioned: the primal kernel takes these rows (block-uniform)
+    if (*p.flag == 0) return;       // the primal kernel takes these rows (block-uniform)
 
     if (tid == 0) {
         for (int s = 0; s < kSlots; ++s) {
@@ -602,13 +603,14 @@ template <int KP> cudaError_t launch_dual_instance(DualParams p, int sms, cudaSt
 size_t dual_workspace_bytes() { return (size_t)kBinvBytes + 256; }
 
 // B^-1 (three operand tiles at `ws`) and the flag (at ws + kBinvBytes) for the dual kernel
-cudaError_t launch_dual_prepare(const float *Bmat, void *ws, float cond_limit, cudaStream_t s, int64_t *launches)
+cudaError_t launch_dual_prepare(const float *Bmat, void *ws, float cond_limit, bool allow_start, cudaStream_t s,
+                                int64_t *launches)
 {
     const size_t smem = sizeof(double) * (D * (D + 1) + 2 * D);
     cudaError_t e = cudaFuncSetAttribute(k_binv_prepare, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     unsigned char *w = static_cast<unsigned char *>(ws);
-    k_binv_prepare<<<1, 128, smem, s>>>(Bmat, w, reinterpret_cast<int *>(w + kBinvBytes), (double)cond_limit);
+    k_binv_prepare<<<1, 128, smem, s>>>(Bmat, w, reinterpret_cast<int *>(w + kBinvBytes), (double)cond_limit, allow_start ? 1 : 0);
     ++*launches;
     return cudaGetLastError();
 }

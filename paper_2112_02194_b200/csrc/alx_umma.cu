@@ -121,6 +121,7 @@ struct Params {
     float cg_tol2;               // conjugate gradients: stop at |r|^2 <= cg_tol2 |b|^2
     int cg_warm;                 // conjugate gradients: start from the row's stored embedding instead of zero
     unsigned long long *cg_counters;   // [3]: rows solved by conjugate gradients, their matrix-vector products, rows that fell back
+    const int *polish_flag;      // set: this launch only runs while the flag reads 2 (the dual-form rows need a polish, see launch_rows_umma)
 };
 
 constexpr int kLdB = D + 4;
@@ -1703,6 +1704,7 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
     using C = Cfg<MODE>;
     constexpr bool CG = is_cg(MODE), FOLD = MODE == kModeRowsFold;
     // which rows this launch takes (block-uniform decisions, before any barrier or allocation)
+    if (is_rows(MODE) && p.polish_flag && *p.polish_flag != 2) return;
     if (MODE == kModeRowsCg && p.policy && p.policy->use_cholesky) return;      // the Cholesky launch takes them all
     if (MODE == kModeRows && p.item_count && !(p.policy && p.policy->use_cholesky)) {
         p.n_items = (int64_t)*p.item_count;                 // the rows conjugate gradients left over
@@ -2091,6 +2093,27 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         p.fallback_count = cg.counters + 2;
         const int grid = (int)(n_whole < sms ? n_whole : sms);
         if (main_begin) cudaEventRecord(main_begin, s);
+        if (cg.enabled && p.dual_flag) {
+            // The dual form beyond its condition limit (flag 2): its solutions, already in the table, are the start
+            // vectors of a conjugate-gradient pass over the same rows, which works on the d x d system itself and stops
+            // at the same residual as every other row (a few products instead of a solve from scratch); rows that do
+            // not converge get the Cholesky solve.  With the flag at 1 (or 0) both launches return at once.
+            Params q = p;
+            q.n_items = offs[3] - offs[1];
+            q.last_item = offs[3] - 1;
+            q.dual_flag = nullptr;
+            q.polish_flag = p.dual_flag;
+            q.cg_warm = 1;
+            q.cg_counters = cg.counters + 3;
+            const int grid_q = (int)(q.n_items < sms ? q.n_items : sms);
+            e = launch_mode<kModeRowsCg>(q, grid_q, s);
+            if (e != cudaSuccess) return e;
+            q.item_list = cg.fallback_list;
+            q.item_count = cg.counters + 2;
+            e = launch_mode<kModeRows>(q, grid_q, s);
+            if (e != cudaSuccess) return e;
+            *launches += 2;
+        }
         if (cg.enabled) {
             // solver of this half-epoch: conjugate gradients unless the side's last run took too many products
             k_cg_policy<<<1, 32, 0, s>>>(cg.policy, cg.switch_products);

@@ -381,9 +381,11 @@ def test_dual_form_for_short_rows_matches_oracle_and_primal_form():
     assert worst <= 1e-4, worst
 
 
-def test_dual_form_steps_aside_when_base_matrix_is_ill_conditioned():
-    """alpha0 G + lambda I with a condition number of about 4e4: the dual form would lose four digits, so the
-    library must take the primal form for every row (and still meet the residual gate)."""
+def test_dual_form_beyond_its_condition_limit_is_polished_or_steps_aside():
+    """alpha0 G + lambda I with a condition number of about 4e4: the dual form alone would lose four digits.  With
+    conjugate gradients available its solutions are only the start vectors of a conjugate-gradient pass over the same
+    rows (which stops at the usual residual); with the Cholesky-only option the d x d solve takes every row.  Either
+    way every short row meets the residual gate."""
     from synth import graphs
     p = _problem("local_d128_bf16")
     rng = np.random.Generator(np.random.PCG64(77))
@@ -391,19 +393,27 @@ def test_dual_form_steps_aside_when_base_matrix_is_ill_conditioned():
     p.H0 = graphs.to_storage_bits(H0, p.storage)
     p.alpha, p.lam = 0.5, 0.01
     ids = _class1_rows(p)
-    a = make_ctx(p)
-    x32 = a.half_epoch_capture(ROWS, ids).astype(np.float64)
-    st = a.get_stats()
-    assert st.dual_rows == 0 and st.kernel_path[0] == 1 and st.not_spd == 0
-    a.destroy()
     H0r = p.f64(p.H0)
     G = ials.gramian(H0r)
     assert np.linalg.cond(p.alpha * G + p.lam * np.eye(p.d)) > 1e4
-    worst = 0.0
-    for n in range(0, ids.size, 7):
-        A, b = ials.row_system(p.rowptr, p.colidx, None, H0r, G, p.alpha, p.lam, int(ids[n]))
-        worst = max(worst, np.linalg.norm(A @ x32[n] - b) / np.linalg.norm(b))
-    assert worst <= 1e-4, worst
+    for kw in (dict(), dict(solver=1)):
+        a = make_ctx(p, **kw)
+        x32 = a.half_epoch_capture(ROWS, ids).astype(np.float64)
+        st = a.get_stats()
+        a.destroy()
+        assert st.kernel_path[0] == 1 and st.not_spd == 0
+        if kw:
+            assert st.dual_rows == 0 and st.dual_polished_rows == 0
+        else:
+            assert st.dual_rows == ids.size and st.dual_polished_rows == ids.size
+            # started from the dual solution (rounded to bfloat16), the pass needs a fraction of a solve from scratch
+            print(f"polish: {st.dual_polish_products / st.dual_polished_rows:.1f} products per row")
+            assert st.dual_polish_products <= 12 * st.dual_polished_rows
+        worst = 0.0
+        for n in range(0, ids.size, 7):
+            A, b = ials.row_system(p.rowptr, p.colidx, None, H0r, G, p.alpha, p.lam, int(ids[n]))
+            worst = max(worst, np.linalg.norm(A @ x32[n] - b) / np.linalg.norm(b))
+        assert worst <= 1e-4, worst
 
 
 @pytest.mark.parametrize("name,offset,kmax", [("local_d128_bf16", 0.02, 32), ("zipf_d64_f32", 0.05, 16)])
