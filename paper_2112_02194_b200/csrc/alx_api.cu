@@ -272,7 +272,7 @@ CgOptions cg_options(const alx_ctx *c, int solved_side)
     o.warm_start = c->opt.cg_start == ALX_CG_START_STORED && c->have_table[solved_side];
     o.enabled = c->opt.solver == ALX_SOLVER_AUTO;
     o.max_iter = c->opt.cg_max_iter > 0 ? c->opt.cg_max_iter : ALX_DEFAULT_CG_MAX_ITER;
-    o.tol = c->opt.cg_tol > 0.f ? c->opt.cg_tol : ALX_DEFAULT_CG_TOL;
+    o.tol = c->opt.cg_tol > 0.f ? c->opt.cg_tol : (c->bf16 ? ALX_DEFAULT_CG_TOL_BF16 : ALX_DEFAULT_CG_TOL);
     o.counters = c->cg_counters;
     o.fallback_list = c->cg_fallback_list;
     o.policy = c->cg_policy ? c->cg_policy + solved_side : nullptr;

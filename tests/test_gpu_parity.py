@@ -252,11 +252,12 @@ def test_overlapped_host_calls_match_the_separate_calls(which):
     np.testing.assert_array_equal(W_out, W_ref)
     np.testing.assert_array_equal(H_out, H_ref)
     # and once more on the same context (the second stream and its event are reused).  The context remembers what the
-    # conjugate gradients of each side cost last time and may pick Cholesky now: the same solution, not the same bits
+    # conjugate gradients of each side cost last time and may pick Cholesky now: the same solution to within what the
+    # solver's stopping rule allows (a tenth of the table tolerance), not the same bits
     b.load_host(p.rowptr, p.colidx, p.values, W0, H0)
     b.epoch_to_host(W_out, H_out)
     for got, ref in ((W_out, W_ref), (H_out, H_ref)):
-        assert rel_fro(p.f64(got), p.f64(ref)) <= 1e-2 * p.emb_tol
+        assert rel_fro(p.f64(got), p.f64(ref)) <= 0.1 * p.emb_tol
     b.destroy()
     # with one solver throughout, the second round gives the same bits too
     c = Alx(p.n_rows, p.n_cols, p.d, p.lam, p.alpha, storage=p.storage, split=p.split, solver=1)
@@ -456,7 +457,7 @@ def _whole_rows(p):
 @pytest.mark.parametrize("name", ["local_d128_bf16", "long_labels_d128_bf16"])
 def test_conjugate_gradient_solve_meets_the_gates_and_tracks_the_oracle(name):
     """Sec. 4.5: conjugate gradients (the default solve of the whole-rows tensor-core kernel), started at 0 and
-    stopped at |r| <= 1e-5 |b|.  Judged by the residual of the fp32 solution and its distance to the exact row update;
+    stopped at |r| <= 3e-5 |b| (the default for bfloat16 tables).  Judged by the residual of the fp32 solution and its distance to the exact row update;
     the number of products is compared with the oracle's textbook iteration (the iterates themselves are unpinned)."""
     p = _problem(name)
     ids = _whole_rows(p)
@@ -477,7 +478,7 @@ def test_conjugate_gradient_solve_meets_the_gates_and_tracks_the_oracle(name):
     assert stats["fallback"].cg_rows == ids.size and stats["fallback"].cg_fallbacks > 0.9 * ids.size
     _, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G, return_raw=True)
     _, _, o_iters = ials.half_step_cg(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G,
-                                     tol=1e-5, max_iter=48)
+                                     tol=3e-5, max_iter=48)
     # products = steps + 1 (the product of the step at which convergence is seen); fp32 may need a step more or less
     mean_products = stats["cg"].cg_products / stats["cg"].cg_rows
     assert abs(mean_products - (o_iters.mean() + 1)) <= 1.0, (mean_products, o_iters.mean())
@@ -489,6 +490,7 @@ def test_conjugate_gradient_solve_meets_the_gates_and_tracks_the_oracle(name):
         A, b = ials.row_system(p.rowptr, p.colidx, vals64, H0, G, p.alpha, p.lam, int(ids[n]))
         for label in ("cg", "fallback"):
             worst = max(worst, np.linalg.norm(A @ sols[label][n] - b) / np.linalg.norm(b))
+    print(f"{name}: worst residual of the conjugate-gradient rows {worst:.2e}, {mean_products:.1f} products per row")
     assert worst <= 1e-4, worst
 
 
