@@ -49,7 +49,9 @@ struct alx_ctx {
     float *split_partials = nullptr;
     void *dual_ws = nullptr;      // tensor path: B^-1 operand tiles and the flag of the dual form
     int64_t dual_candidates = 0;  // rows of classes 1 and 2 of the last half-epoch (solved in the dual form if the flag is set)
-    int dual_flag_latched = 0;    // that flag as the last half-epoch's kernels saw it (the loss and the Gramian calls rewrite it)
+    int dual_flag_latched = 0;
+    int64_t dual_candidates32 = 0; // of them, the rows of 17 .. 32 observations (which the whole-rows kernel may have taken instead)
+    CgPolicy policy_latched{};    // the side's policy record as the last half-epoch's kernels saw it    // that flag as the last half-epoch's kernels saw it (the loss and the Gramian calls rewrite it)
     double *loss_partials_buf = nullptr;
     double *loss_result = nullptr;
     DevStatus *status = nullptr;
@@ -338,10 +340,16 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
         c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;
+        c->dual_candidates32 = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][2] : 0;
         c->dual_flag_latched = 0;
-        if (c->dual_candidates > 0)
+        c->policy_latched = CgPolicy{};
+        if (c->dual_candidates > 0) {
             ALX_CUDA(c, cudaMemcpyAsync(&c->dual_flag_latched, dual_flag_ptr(c->dual_ws), sizeof(int), cudaMemcpyDeviceToHost,
                                         c->stream));
+            if (c->cg_policy && c->opt.solver == ALX_SOLVER_AUTO)
+                ALX_CUDA(c, cudaMemcpyAsync(&c->policy_latched, c->cg_policy + side, sizeof(CgPolicy), cudaMemcpyDeviceToHost,
+                                            c->stream));
+        }
     } else {
         ALX_CUDA(c, launch_rows_simple(side_view(c, side), c->class_offs[side], c->n_chunks[side],
                                        c->n_split_rows[side], c->table[fixed], c->bf16, c->opt.d, c->Bmat,
@@ -1002,7 +1010,8 @@ alx_status alx_get_stats(alx_ctx *c, alx_stats *out)
     if (c->main_timed) {
         if (cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]) == cudaSuccess) c->stats.ms_main_kernel = ms; else cudaGetLastError();
     }
-    c->stats.dual_rows = c->dual_candidates > 0 && c->dual_flag_latched ? c->dual_candidates : 0;
+    c->stats.dual_rows = c->dual_candidates > 0 && c->dual_flag_latched
+                             ? c->dual_candidates - (c->policy_latched.short_rows_by_cg ? c->dual_candidates32 : 0) : 0;
     {
         unsigned long long h[5] = {0, 0, 0, 0, 0};
         ALX_CUDA(c, cudaMemcpy(h, c->cg_counters, sizeof h, cudaMemcpyDeviceToHost));

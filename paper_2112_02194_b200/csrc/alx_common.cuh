@@ -154,7 +154,13 @@ struct CgPolicy {
     unsigned long long rows, products;
     int use_cholesky;     // this half-epoch: 1 = the in-place Cholesky takes every row of the whole-rows kernel
     int calls;
+    int short_rows_by_cg; // this half-epoch: 1 = rows of 17 .. 32 observations go to the whole-rows kernel, not the dual form
+    int pad_;
 };
+// The dual-form kernel for rows of 17 .. 32 observations costs about as much as ten products of the whole-rows kernel
+// (measured: 28 ns against 10 + 1.8 per product ns per row): where the side's last conjugate-gradient run stayed at or
+// below this many products per row, those rows go there
+constexpr float kShortRowsByCgProducts = 11.f;
 // Conjugate gradients pay while a row takes fewer than about 28 products on average (measured on B200: about 2900 + 300
 // per product cycles of an SM per row, against 12 600 for the in-place Cholesky; alx_options.cg_switch_products); beyond
 // that the side's next half-epochs go to Cholesky, with one conjugate-gradient half-epoch every kCgReprobe to see whether
@@ -215,8 +221,10 @@ cudaError_t launch_dual64_prepare(const float *Bmat, void *ws, float cond_limit,
 cudaError_t launch_rows_dual64(const SideView &sv, int64_t first, int64_t count, const void *X, void *ws, RowOut out,
                                cudaStream_t s, int64_t *launches);
 const int *dual_flag_ptr(const void *ws);
+// route: set where conjugate gradients run; the kernel of the rows of 17 .. 32 observations returns at once when it says so
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
-                             const void *ws, RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches);
+                             const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, cudaStream_t s,
+                             int64_t *launches);
 
 // alx_loss.cu
 int64_t loss_partials(int64_t nnz);

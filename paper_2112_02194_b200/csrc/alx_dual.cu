@@ -140,6 +140,7 @@ struct DualParams {
     const __nv_bfloat16 *X;        // fixed table [N x 128]
     const unsigned char *binv;     // three operand tiles of B^-1
     const int *flag;
+    const CgPolicy *route;         // rows of 17 .. 32 observations: nothing to do when the whole-rows kernel takes them
     int64_t first;                 // position in sv.order of the first row of the class
     int64_t count;                 // rows of the class
     int64_t n_tiles;
@@ -547,6 +548,7 @@ template <int KP> __global__ void __launch_bounds__(kBlockThreads, 1) k_dual(Dua
     DualSmem &sm = *reinterpret_cast<DualSmem *>(aligned);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (*p.flag == 0) return;       // the primal kernel takes these rows (block-uniform)
+    if (KP == 32 && p.route && p.route->short_rows_by_cg) return;
 
     if (tid == 0) {
         for (int s = 0; s < kSlots; ++s) {
@@ -620,9 +622,11 @@ const int *dual_flag_ptr(const void *ws) { return reinterpret_cast<const int *>(
 // rows order[first16 .. first16 + count16) of the solved side have 1 .. 16 observations each, the count32 rows after
 // them 17 .. 32
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
-                             const void *ws, RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches)
+                             const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, cudaStream_t s,
+                             int64_t *launches)
 {
     DualParams p{};
+    p.route = route;
     p.sv = sv;
     p.X = reinterpret_cast<const __nv_bfloat16 *>(X);
     p.binv = static_cast<const unsigned char *>(ws);

@@ -122,6 +122,8 @@ struct Params {
     int cg_warm;                 // conjugate gradients: start from the row's stored embedding instead of zero
     unsigned long long *cg_counters;   // [3]: rows solved by conjugate gradients, their matrix-vector products, rows that fell back
     const int *polish_flag;      // set: this launch only runs while the flag reads 2 (the dual-form rows need a polish, see launch_rows_umma)
+    const CgPolicy *route;       // set where conjugate gradients run: whether the rows of 17 .. 32 observations are this kernel's
+    int64_t n_class2;            // how many rows those are (they follow the longer rows in the walk)
 };
 
 constexpr int kLdB = D + 4;
@@ -1704,14 +1706,18 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
     using C = Cfg<MODE>;
     constexpr bool CG = is_cg(MODE), FOLD = MODE == kModeRowsFold;
     // which rows this launch takes (block-uniform decisions, before any barrier or allocation)
-    if (is_rows(MODE) && p.polish_flag && *p.polish_flag != 2) return;
+    const bool short_rows_here = is_rows(MODE) && p.route && p.route->short_rows_by_cg;
+    if (is_rows(MODE) && p.polish_flag) {
+        if (*p.polish_flag != 2) return;
+        if (short_rows_here) { p.n_items -= p.n_class2; p.last_item -= p.n_class2; }      // (those rows are not dual-form rows then)
+    }
     if (MODE == kModeRowsCg && p.policy && p.policy->use_cholesky) return;      // the Cholesky launch takes them all
     if (MODE == kModeRows && p.item_count && !(p.policy && p.policy->use_cholesky)) {
         p.n_items = (int64_t)*p.item_count;                 // the rows conjugate gradients left over
         if ((int64_t)blockIdx.x >= p.n_items) return;
     } else {
         if (MODE == kModeRows) p.item_list = nullptr;       // (every row: the walk through the degree classes)
-        if (is_rows(MODE) && p.dual_flag && *p.dual_flag) p.n_items = p.n_items_primal;
+        if (is_rows(MODE) && p.dual_flag && *p.dual_flag) p.n_items = p.n_items_primal + (short_rows_here ? p.n_class2 : 0);
         if (is_rows(MODE) && (int64_t)blockIdx.x >= p.n_items) return;
     }
     extern __shared__ unsigned char smem_raw[];
@@ -1806,6 +1812,7 @@ __global__ void k_cg_policy(CgPolicy *pol, float switch_products)
     if (pol->rows > 0 && (float)pol->products > switch_products * (float)pol->rows) use = 1;
     if (use && (calls % kCgReprobe) == kCgReprobe - 1) use = 0;
     pol->use_cholesky = use;
+    pol->short_rows_by_cg = (!use && pol->rows > 0 && (float)pol->products <= kShortRowsByCgProducts * (float)pol->rows) ? 1 : 0;
 }
 // After them: keep the run's counts (they are cleared at the start of every half-epoch).
 __global__ void k_cg_record(CgPolicy *pol, const unsigned long long *counters)
@@ -2074,9 +2081,17 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
         if (e != cudaSuccess) return e;
     }
     const int64_t n_whole = offs[c_long] - offs[1];
+    if (cg.enabled && n_whole > 0) {
+        // solver of this half-epoch: conjugate gradients unless the side's last run took too many products; and where the
+        // rows of 17 .. 32 observations go
+        k_cg_policy<<<1, 32, 0, s>>>(cg.policy, cg.switch_products);
+        ++*launches;
+        p.route = cg.policy;
+        p.n_class2 = offs[3] - offs[2];
+    }
     if (dual_ws && offs[3] > offs[1]) {
         // rows with 1 .. 32 observations (classes 1 and 2): dual form, if the flag (set on the device) allows it
-        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], offs[3] - offs[2], X, dual_ws, out, st, s, launches);
+        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], offs[3] - offs[2], X, dual_ws, out, st, p.route, s, launches);
         if (e != cudaSuccess) return e;
         p.dual_flag = dual_flag_ptr(dual_ws);
         p.n_items_primal = offs[c_long] - offs[3];
@@ -2115,8 +2130,6 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
             *launches += 2;
         }
         if (cg.enabled) {
-            // solver of this half-epoch: conjugate gradients unless the side's last run took too many products
-            k_cg_policy<<<1, 32, 0, s>>>(cg.policy, cg.switch_products);
             p.policy = cg.policy;
             e = launch_mode<kModeRowsCg>(p, grid, s);
             if (e != cudaSuccess) return e;
@@ -2126,7 +2139,7 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
             p.item_list = cg.fallback_list;
             p.item_count = cg.counters + 2;
             e = launch_mode<kModeRows>(p, grid, s);
-            *launches += 4;
+            *launches += 3;
         } else {
             e = launch_mode<kModeRows>(p, grid, s);
             ++*launches;
