@@ -11,6 +11,7 @@
 
 #include "../../include/alx.h"
 #include "alx_common.cuh"
+#include <nvtx3/nvToolsExt.h>      // header-only: ranges show up in a profiler's timeline, and cost nothing without one
 
 using namespace alx;
 
@@ -95,6 +96,14 @@ alx_status fail(alx_ctx *c, alx_status code, const char *fmt, ...)
             return fail((c), e_ == cudaErrorMemoryAllocation ? ALX_ERR_OOM : ALX_ERR_CUDA,         \
                         "%s failed: %s", #expr, cudaGetErrorString(e_));                           \
     } while (0)
+
+// a named range on the profiler's timeline for as long as the object lives
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
 
 struct DeviceGuard {
     int prev = -1;
@@ -306,10 +315,16 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
     if (c->nnz < 0) return fail(c, ALX_ERR_BAD_STATE, "alx_half_epoch before alx_set_csr");
     const int fixed = 1 - side;
     if (!c->have_table[fixed]) return fail(c, ALX_ERR_BAD_STATE, "the fixed table has not been set");
+    NvtxRange range(side == ALX_ROWS ? "alx half-epoch: rows" : "alx half-epoch: columns");
     ALX_CUDA(c, cudaEventRecord(c->ev[0], c->stream));
-    alx_status st = gramian_of(c, fixed);
+    alx_status st;
+    {
+        NvtxRange r("alx Gramian + base matrix");
+        st = gramian_of(c, fixed);
+    }
     if (st != ALX_OK) return st;
     ALX_CUDA(c, cudaEventRecord(c->ev[1], c->stream));
+    NvtxRange rows_range("alx rows: gather, sums, solve, store");
     RowOut out{c->table[side], cap_slot, cap_out};
     if (fold_path(c)) {
         ALX_CUDA(c, cudaMemsetAsync(c->cg_counters, 0, 5 * sizeof(unsigned long long), c->stream));
@@ -486,6 +501,7 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
     if (!c) return ALX_ERR_INVALID_ARG;
     if (!rowptr || nnz < 0 || (nnz > 0 && !colidx)) return fail(c, ALX_ERR_INVALID_ARG, "null array or negative nnz");
     DeviceGuard guard(c->device);
+    NvtxRange range("alx_set_csr: validate, transpose, degree classes");
     release_matrix(c);
     const int64_t n_rows = c->n[ALX_ROWS], n_cols = c->n[ALX_COLS];
     const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
@@ -912,6 +928,7 @@ alx_status alx_topk(alx_ctx *c, alx_side items, const float *queries, int64_t m,
     if (!c->have_table[items]) return fail(c, ALX_ERR_BAD_STATE, "the table has not been set or solved yet");
     if (m == 0) return ALX_OK;
     DeviceGuard guard(c->device);
+    NvtxRange range("alx_topk");
     const int d = c->opt.d;
     const int64_t n_items = c->n[items];
     Scratch tmp(c);
