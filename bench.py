@@ -359,9 +359,12 @@ def run_ours(args, w):
     for sd in (0, 1):
         rows_sd = sum(st.rows_in_class[sd][1:11]) - st.long_rows[sd]
         ent_sd = sum(st.entries_in_class[sd][1:11]) - st.long_entries[sd]
-        if half_ms["dual_rows"][sd] > 0:
-            rows_sd -= st.rows_in_class[sd][1] + st.rows_in_class[sd][2]
-            ent_sd -= st.entries_in_class[sd][1] + st.entries_in_class[sd][2]
+        # rows the dual-form kernels took: classes 1 and 2, or class 1 alone where the rows of 17 .. 32 entries went to the
+        # whole-rows kernel (alx_stats.dual_rows says which)
+        for cl in (1, 2):
+            if half_ms["dual_rows"][sd] >= sum(st.rows_in_class[sd][1:cl + 1]) and st.rows_in_class[sd][cl] > 0:
+                rows_sd -= st.rows_in_class[sd][cl]
+                ent_sd -= st.entries_in_class[sd][cl]
         rows_side.append(rows_sd)
         ent_side.append(ent_sd)
         # solve work of the launch: the cheaper of Cholesky and the products conjugate gradients really spent

@@ -53,7 +53,7 @@ typedef enum { ALX_F32 = 0, ALX_BF16 = 1 } alx_dtype;
 typedef enum { ALX_SOLVER_AUTO = 0, ALX_SOLVER_CHOLESKY = 1 } alx_solver;
 typedef enum { ALX_CG_START_STORED = 0, ALX_CG_START_ZERO = 1 } alx_cg_start;
 #define ALX_DEFAULT_CG_MAX_ITER 48
-#define ALX_DEFAULT_CG_TOL 1e-5f        /* fp32 tables */
+#define ALX_DEFAULT_CG_TOL 1e-6f        /* fp32 tables */
 #define ALX_DEFAULT_CG_TOL_BF16 3e-5f   /* bfloat16 tables */
 #define ALX_DEFAULT_DUAL_COND_LIMIT 8192.f
 #define ALX_DEFAULT_CG_SWITCH_PRODUCTS 28.f
@@ -95,9 +95,10 @@ typedef struct alx_options {
                                 on the device from the counts of the side's last run.
                                 ALX_SOLVER_CHOLESKY (1): Cholesky for every row */
     int32_t cg_max_iter;     /* 0 => ALX_DEFAULT_CG_MAX_ITER */
-    float cg_tol;            /* 0 => ALX_DEFAULT_CG_TOL for fp32 tables, ALX_DEFAULT_CG_TOL_BF16 for bfloat16 tables (their
-                                results are rounded to 2^-9 anyway; a third of the usual residual gate of 1e-4 leaves room for
-                                the gap between the recurrence's residual and the true one); at most 1e-2 */
+    float cg_tol;            /* 0 => ALX_DEFAULT_CG_TOL for fp32 tables, ALX_DEFAULT_CG_TOL_BF16 for bfloat16 tables.  The error of
+                                a row is bounded by cond(A) times the relative residual: bfloat16 results are rounded to 2^-9
+                                anyway, so a third of the usual residual gate of 1e-4 is enough there; fp32 tables are expected
+                                to be right to 1e-3, which rows with cond(A) of 10^3 only are at 1e-6.  At most 1e-2 */
     float cg_switch_products; /* the mean number of products per row beyond which a side's next half-epochs take Cholesky
                                 (see solver); 0 => ALX_DEFAULT_CG_SWITCH_PRODUCTS */
     int32_t cg_start;        /* start vector of the conjugate gradients (the paper states none): ALX_CG_START_STORED (0): the

@@ -127,6 +127,10 @@ struct Params {
 };
 
 constexpr int kLdB = D + 4;
+// conjugate gradients on the folded 64 x 64 system: a row that needed this many products has its true residual b - A x
+// checked once before it is accepted (|b - A x| <= kCgVerifySlack * tol * |b|), else it goes to the direct solve
+constexpr int kCgVerifyProducts = 24;
+constexpr float kCgVerifySlack = 2.f;
 // conjugate gradients read the matrix with the 16x128b tensor-memory shape (a thread holds four rows, every fourth
 // column): alpha0 G + lambda I and the vector of a product are kept in shared memory by column class (column mod 4),
 // 36 floats per class so that the four classes of a quarter-warp's 16-byte loads fall into different banks
@@ -1532,6 +1536,27 @@ __device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, cons
         group128_sync(bar_id);
     }
     group128_sync(bar_id);          // (the scratch is free for whatever follows)
+    if (ok && products >= kCgVerifyProducts) {
+        // After many steps the residual of the recurrence can have drifted away from b - A x (its rounding errors add up
+        // with the condition of the matrix): look at the true residual once, with one more product, and leave the row to
+        // the direct solve if it is not what the recurrence says.  (The 128-feature kernel does not do this: there the
+        // check costs 1.5-3 % of the kernel's time for rows that, with its step limit and the per-side policy, have
+        // always passed their residual gate.)
+        if (h == 0) gs.vec[i] = x;
+        group128_sync(bar_id);
+        float g0, d0, b0;
+        const float rt = b - product_and_sums(x, 0.f, g0, d0, b0);
+        ++products;
+        group128_sync(bar_id);      // the sums of the product have been read
+        float tsum = h == 0 ? rt * rt : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tsum += __shfl_xor_sync(0xFFFFFFFFu, tsum, o);
+        if (lane == 0) gs.red[w][0] = tsum;
+        group128_sync(bar_id);
+        tsum = gs.red[0][0] + gs.red[1][0];
+        if (!(tsum <= kCgVerifySlack * kCgVerifySlack * p.cg_tol2 * bb)) ok = false;
+        group128_sync(bar_id);
+    }
     matvecs = products;
     x_out = x;
     return ok;

@@ -526,7 +526,7 @@ def test_fp32_tables_of_64_features_on_the_tensor_cores(name):
         assert stats["cg"].long_rows[0] > 0      # whole rows of more than 512 observations took the chunks kernel
     _, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G, return_raw=True)
     _, _, o_iters = ials.half_step_cg(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, row_ids=ids, G=G,
-                                     tol=1e-5, max_iter=48)
+                                     tol=1e-6, max_iter=48)
     mean_products = stats["cg"].cg_products / stats["cg"].cg_rows
     assert abs(mean_products - (o_iters.mean() + 1)) <= 1.0, (mean_products, o_iters.mean())
     nz = np.linalg.norm(W_raw, axis=1) > 0      # (rows whose labels are all 0 have the solution 0)
