@@ -202,3 +202,55 @@ def test_protocol_on_a_planted_graph_recall_at_20_and_50(d, storage):
     # Recall@K is about K / 79 at best)
     assert rec[50][0] >= 0.4 and rec[20][0] >= 0.15
     assert (ids == o_ids).mean() > 0.9
+
+
+@pytest.mark.parametrize("d,storage", [(128, "bf16"), (32, "f32")])
+def test_topk_extremes_of_k_m_and_table_size(d, storage):
+    """k = 1 and k = 256 (the most the call takes), a single query, a table shorter than one tile and shorter than k, the
+    rows table as the items, and every item excluded for one query."""
+    from paper_2112_02194_b200 import Alx
+    n_rows, n_cols = 77, 200
+    H, Q = _integer_tables(n_cols, 5, d, 9)
+    W, _ = _integer_tables(n_rows, 1, d, 10)
+    a = Alx(n_rows, n_cols, d, 0.05, 0.01, storage=storage)
+    a.set_embeddings(ROWS, graphs.to_storage_bits(W, storage))
+    a.set_embeddings(COLS, graphs.to_storage_bits(H, storage))
+    for k in (1, 256):
+        ids, sc = a.topk(COLS, Q, k)
+        o_ids, o_sc = ev.topk(Q, H, k)
+        np.testing.assert_array_equal(ids, o_ids)
+        np.testing.assert_array_equal(sc.astype(np.float64), o_sc)
+    assert np.all(ids[:, 200:] == -1)
+    ids, _ = a.topk(COLS, Q[:1], 7)                       # one query
+    np.testing.assert_array_equal(ids, ev.topk(Q[:1], H, 7)[0])
+    ids, _ = a.topk(ROWS, Q, 100)                         # the rows table as the items: 77 of them
+    np.testing.assert_array_equal(ids, ev.topk(Q, W, 100)[0])
+    ptr = np.array([0, 200, 200, 200, 200, 200], dtype=np.int64)      # query 0: everything excluded
+    idx = np.arange(200, dtype=np.int32)
+    ids, sc = a.topk(COLS, Q, 10, exclude=(ptr, idx))
+    assert np.all(ids[0] == -1) and np.all(np.isneginf(sc[0]))
+    np.testing.assert_array_equal(ids[1:], ev.topk(Q[1:], H, 10)[0])
+    a.destroy()
+
+
+def test_evaluation_calls_refuse_bad_arguments_with_status_codes():
+    from paper_2112_02194_b200 import Alx, AlxError
+    a = Alx(10, 20, 16, 0.05, 0.01, storage="f32")
+    q = np.zeros((2, 16), dtype=np.float32)
+    with pytest.raises(AlxError) as e:                     # nothing in the table yet
+        a.topk(COLS, q, 3)
+    assert e.value.status == 2                             # ALX_ERR_BAD_STATE
+    with pytest.raises(AlxError) as e:
+        a.fold_in(np.array([0, 1], dtype=np.int64), np.array([3], dtype=np.int32))
+    assert e.value.status == 2
+    a.set_embeddings(COLS, np.zeros((20, 16), dtype=np.float32))
+    for k in (0, 257):
+        with pytest.raises(AlxError) as e:
+            a.topk(COLS, q, k)
+        assert e.value.status == 1                         # ALX_ERR_INVALID_ARG
+    with pytest.raises(AlxError) as e:                     # a link to a column that does not exist
+        a.fold_in(np.array([0, 1], dtype=np.int64), np.array([20], dtype=np.int32))
+    assert e.value.status == 5                             # ALX_ERR_BAD_CSR
+    x = a.fold_in(np.array([0, 0], dtype=np.int64), np.zeros(0, dtype=np.int32))      # a new row without links
+    assert x.shape == (1, 16) and np.all(x == 0.0)
+    a.destroy()
