@@ -87,3 +87,42 @@ def test_single_row_and_single_column_matrices(d, storage):
     # (an fp32 solve is backward stable: its error is bounded by cond(A) d 2^-23, and this matrix -- 180 copies of one outer
     # product on top of lambda I -- has a condition of 10^4 .. 10^5: the residual above is the gate that means something)
     assert np.linalg.norm(x32[0] - exact) <= max(p.emb_tol, d * 1.2e-7 * np.linalg.cond(A)) * np.linalg.norm(exact)
+
+
+@pytest.mark.parametrize("case", [0, 3], ids=["edges_d128_bf16", "edges_d64_f32_labels_split"])
+def test_six_epochs_on_the_boundary_problems_each_match_the_oracle_epoch(case):
+    """Several epochs in a row: the solver choice per side, the routing of the rows of 17..32 entries and the start vectors
+    all depend on the context's history.  Every epoch is compared with the oracle's epoch from the SAME start tables (the
+    GPU's own, read back before the epoch): tables within the tolerance, loss to 1e-4, and the loss must not rise.  (Two
+    free-running trajectories drift apart by the storage rounding of every epoch, which says nothing about an epoch.)"""
+    from oracle import ials
+    from tests.test_gpu_parity import make_ctx, rel_fro
+    name, d, storage, n_cols, split, values = CASES[case]
+    p = boundary_problem(name, d, storage, n_cols, split, values, seed=7 + 11 * case)
+    a = make_ctx(p)
+    dt = "bf16" if storage == "bf16" else "f32"
+    colptr, rowidx, vt = ials.transpose(p.n_rows, p.n_cols, p.rowptr, p.colidx, p.values)
+    v64 = None if p.values is None else p.values.astype(np.float64)
+    vt64 = None if vt is None else vt.astype(np.float64)
+    prev = a.loss()[0]
+    H = p.f64(p.H0)
+    for ep in range(6):
+        a.half_epoch(0)
+        dual_rows = a.get_stats().dual_rows
+        a.half_epoch(1)
+        W_ref = ials.half_step(p.rowptr, p.colidx, v64, H, p.alpha, p.lam, p.storage)
+        H_ref = ials.half_step(colptr, rowidx, vt64, W_ref, p.alpha, p.lam, p.storage)
+        W_gpu = p.f64(a.get_embeddings(0, dtype=dt))
+        H_gpu = p.f64(a.get_embeddings(1, dtype=dt))
+        tot = a.loss()[0]
+        ref = ials.loss(p.rowptr, p.colidx, v64, W_ref, H_ref, p.alpha, p.lam)[0]
+        st = a.get_stats()
+        print(f"{name} epoch {ep + 1}: W {rel_fro(W_gpu, W_ref):.2e} H {rel_fro(H_gpu, H_ref):.2e} loss {abs(tot - ref) / ref:.2e}, "
+              f"dual-form rows {dual_rows}, products per row {st.cg_products / max(st.cg_rows, 1):.1f}, Cholesky by policy "
+              f"{list(st.cholesky_by_policy)}")
+        assert rel_fro(W_gpu, W_ref) <= p.emb_tol and rel_fro(H_gpu, H_ref) <= p.emb_tol
+        assert abs(tot - ref) <= 1e-4 * ref
+        assert tot <= prev * (1 + 1e-6) and st.not_spd == 0
+        prev = tot
+        H = H_gpu
+    a.destroy()
