@@ -65,3 +65,41 @@ def test_embeddings_normal_and_block_consistent():
     b = graphs.init_embeddings(3000, 16, 7, 2, "bf16")
     back = graphs.storage_to_f64(b, "bf16")
     assert np.abs(back - full).max() <= np.abs(full).max() * 2.0 ** -8
+
+
+def test_planted_links_and_the_evaluation_split():
+    """The planted block matrix and the split of the evaluation protocol: seeded (same call, same arrays), rows ascending and
+    distinct, most of a row's links inside its group's pool, 10 % test rows taken out of the training matrix, a quarter of
+    every test row's links (at least one) held out and the rest kept, nothing lost or invented."""
+    from synth import planted
+    n, n_cols = 600, 480
+    rowptr, colidx = planted.planted_links(n, n_cols, n_groups=12, pool=40, deg_lo=8, deg_hi=20, p_in=0.85, seed=3)
+    rowptr2, colidx2 = planted.planted_links(n, n_cols, n_groups=12, pool=40, deg_lo=8, deg_hi=20, p_in=0.85, seed=3)
+    np.testing.assert_array_equal(rowptr, rowptr2)
+    np.testing.assert_array_equal(colidx, colidx2)
+    deg = np.diff(rowptr)
+    assert deg.min() >= 7 and deg.max() <= 20 and colidx.min() >= 0 and colidx.max() < n_cols
+    for u in range(n):
+        c = colidx[rowptr[u]:rowptr[u + 1]]
+        assert np.all(np.diff(c) > 0)
+    # rows of one group share a pool: two rows of the same group overlap far more than rows of different groups
+    sets = [set(colidx[rowptr[u]:rowptr[u + 1]].tolist()) for u in range(48)]
+    same = np.mean([len(sets[u] & sets[u + 12]) for u in range(24)])
+    other = np.mean([len(sets[u] & sets[u + 1]) for u in range(24)])
+    assert same > 3 * max(other, 0.1)
+    sp = planted.split_rows(rowptr, colidx, 0.10, 0.25, seed=4)
+    test_rows = sp["test_rows"]
+    assert test_rows.size == 60
+    tr_ptr, tr_idx = sp["train"]
+    assert np.all(np.diff(tr_ptr)[test_rows] == 0)
+    kept_ptr, kept_idx = sp["kept"]
+    truth_ptr, truth_idx = sp["truth"]
+    for j, u in enumerate(test_rows):
+        kept = kept_idx[kept_ptr[j]:kept_ptr[j + 1]]
+        truth = truth_idx[truth_ptr[j]:truth_ptr[j + 1]]
+        full = colidx[rowptr[u]:rowptr[u + 1]]
+        assert truth.size == max(1, int(round(0.25 * full.size)))
+        np.testing.assert_array_equal(np.sort(np.concatenate([kept, truth])), full)
+        assert np.all(np.diff(kept) > 0) and np.all(np.diff(truth) > 0)
+    train_rows = np.setdiff1d(np.arange(n), test_rows)
+    assert int(np.diff(tr_ptr)[train_rows].sum()) == int(deg[train_rows].sum()) == tr_idx.size
