@@ -126,3 +126,23 @@ def test_six_epochs_on_the_boundary_problems_each_match_the_oracle_epoch(case):
         prev = tot
         H = H_gpu
     a.destroy()
+
+
+OPTION_SETS = [
+    dict(solver=1), dict(kernels=1), dict(kernels=2), dict(cg_start=1), dict(cg_max_iter=3), dict(cg_max_iter=200),
+    dict(cg_tol=1e-7), dict(dual_cond_limit=1.0), dict(dual_cond_limit=1e9), dict(cg_switch_products=1.0),
+    dict(solver=1, kernels=2), dict(cg_start=1, dual_cond_limit=1.0, cg_max_iter=5), dict(kernels=2, cg_tol=3e-6, cg_start=1),
+]
+
+
+@pytest.mark.parametrize("case", [1, 3, 6], ids=["edges_d128_bf16_labels_split", "edges_d64_f32_labels_split", "edges_d32_f32"])
+@pytest.mark.parametrize("opt", range(len(OPTION_SETS)), ids=[",".join(f"{k}={v}" for k, v in o.items()) for o in OPTION_SETS])
+def test_every_option_gives_the_same_epoch(case, opt):
+    """The options choose HOW a row is solved (kernel family, solver, start vector, step limit, limits), never WHAT: one
+    epoch of a boundary problem under each setting, held to the gates of the storage type and of the residual.  These
+    problems have rows with cond(A) of a few thousand, where conjugate gradients stopped at a relative residual leave
+    an error of cond(A) times that: the solver's fp32 solution is therefore held to the storage type's tolerance here,
+    not to the 1e-3 that the direct solves and the better conditioned suites reach."""
+    name, d, storage, n_cols, split, values = CASES[case]
+    p = boundary_problem(name, d, storage, n_cols, split, values, seed=7 + 11 * case)
+    _epoch_checks(p, raw_gate=(p.emb_tol, 10 * p.emb_tol), **OPTION_SETS[opt])

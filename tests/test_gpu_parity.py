@@ -35,7 +35,7 @@ def row_rel(x, ref):
 ROW_MAX_FACTOR = 10.0
 
 
-def _check_half_step(p, side, X_gpu, X_ref, X_raw, x32, deg, ptr, idx, vals64, X_fixed, G):
+def _check_half_step(p, side, X_gpu, X_ref, X_raw, x32, deg, ptr, idx, vals64, X_fixed, G, raw_gate=(1e-3, 1e-2)):
     """The gates of one half-step: the table (Frobenius), every row (99.9th percentile and maximum of the per-row relative
     error), exact zeros for rows without observations, the residual of the solver's own fp32 solutions."""
     rr = row_rel(X_gpu, X_ref)
@@ -63,8 +63,9 @@ def _check_half_step(p, side, X_gpu, X_ref, X_raw, x32, deg, ptr, idx, vals64, X
         worst = max(worst, np.linalg.norm(A @ x32[u].astype(np.float64) - b) / nb)
     print(f"{p.name} {side}: worst residual of {check.size} rows {worst:.2e}")
     assert worst <= 1e-4, worst
+    # the solver's own fp32 solution against the exact one (before the storage cast): table and worst row
     xr = row_rel(x32.astype(np.float64), X_raw)
-    assert rel_fro(x32.astype(np.float64), X_raw) <= 1e-3 and xr.max() <= 1e-2, (rel_fro(x32.astype(np.float64), X_raw), xr.max())
+    assert rel_fro(x32.astype(np.float64), X_raw) <= raw_gate[0] and xr.max() <= raw_gate[1], (rel_fro(x32.astype(np.float64), X_raw), xr.max())
 
 
 SUITE = problems.small_suite()
@@ -124,7 +125,7 @@ def test_fp32_alu_kernels_on_the_tensor_path_problems(name):
     _epoch_checks(_problem(name), kernels=1)
 
 
-def _epoch_checks(p, **ctx_kw):
+def _epoch_checks(p, raw_gate=(1e-3, 1e-2), **ctx_kw):
     a = make_ctx(p, **ctx_kw)
     W0, H0 = p.f64(p.W0), p.f64(p.H0)
     colptr, rowidx, vt = ials.transpose(p.n_rows, p.n_cols, p.rowptr, p.colidx, p.values)
@@ -143,7 +144,7 @@ def _epoch_checks(p, **ctx_kw):
     G = ials.gramian(H0)
     W_ref, W_raw = ials.half_step(p.rowptr, p.colidx, vals64, H0, p.alpha, p.lam, p.storage, G=G, return_raw=True)
     deg = np.diff(p.rowptr)
-    _check_half_step(p, "rows", W_gpu, W_ref, W_raw, x32, deg, p.rowptr, p.colidx, vals64, H0, G)
+    _check_half_step(p, "rows", W_gpu, W_ref, W_raw, x32, deg, p.rowptr, p.colidx, vals64, H0, G, raw_gate)
 
     # --- columns half-step on the GPU's own new W (trajectories may differ by storage rounding): the same gates
     cids = np.arange(p.n_cols, dtype=np.int64)
@@ -152,7 +153,7 @@ def _epoch_checks(p, **ctx_kw):
     G_W = ials.gramian(W_gpu)
     H_ref_same, H_raw_same = ials.half_step(colptr, rowidx, vt64, W_gpu, p.alpha, p.lam, p.storage, G=G_W, return_raw=True)
     cdeg = np.diff(colptr)
-    _check_half_step(p, "columns", H_gpu, H_ref_same, H_raw_same, h32, cdeg, colptr, rowidx, vt64, W_gpu, G_W)
+    _check_half_step(p, "columns", H_gpu, H_ref_same, H_raw_same, h32, cdeg, colptr, rowidx, vt64, W_gpu, G_W, raw_gate)
     # and end to end against the oracle's own trajectory
     H_ref = ials.half_step(colptr, rowidx, vt64, W_ref, p.alpha, p.lam, p.storage)
     assert rel_fro(H_gpu, H_ref) <= p.emb_tol
