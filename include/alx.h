@@ -82,9 +82,13 @@ typedef struct alx_options {
                                 different thread blocks accumulate; 0 => ALX_DEFAULT_SPLIT; >= 16 */
     int32_t kernels;         /* 0 = best available for (d, storage): for d = 128 with bf16 tables the tensor-core
                                 kernels, rows with at most 32 observations solved in the dual (push-through) form
-                                of Eq. 4 while alpha0 G + lambda I is well conditioned; 1 = force the plain FP32-ALU
-                                kernels (reference path inside the library; every d, every storage); 2 = as 0 but
-                                every row in the primal form */
+                                of Eq. 4 while alpha0 G + lambda I is well conditioned (see dual_cond_limit; the rows of
+                                17 .. 32 observations go to the conjugate-gradient kernel instead where that is the cheaper
+                                solve); for d = 64 with fp32 tables the same tensor-core kernels over bfloat16 parts of
+                                the fixed table (x = x1 + x2 + x3, so to fp32 accuracy), rows with at most 16
+                                observations in the dual form; every other (d, storage) the FP32-ALU kernels.
+                                1 = force the plain FP32-ALU kernels (reference path inside the library; every d, every
+                                storage); 2 = as 0 but every row in the primal form */
     int32_t solver;          /* how the d x d system of Eq. 4 is solved (Sec. 4.5 compares the choices):
                                 ALX_SOLVER_AUTO (0): conjugate gradients where the library has them (the whole-rows
                                 tensor-core kernel), started as cg_start says and stopped at |r| <= cg_tol |b|; a row that has not
