@@ -94,6 +94,10 @@ cudaError_t launch_degrees(const int64_t *ptr, int64_t n, int32_t *deg, cudaStre
 // becomes a row of 2L entries, its L ids followed by the same ids + N (labels repeated); vptr = 2 ptr.
 cudaError_t launch_double_entries(const int64_t *ptr, const int32_t *idx, const float *val, int64_t n, int64_t n_fixed,
                                   int64_t *vptr, int32_t *vidx, float *vval, cudaStream_t s, int64_t *launches);
+// stable partition of a list of rows by length (see alx_setup.cu)
+cudaError_t launch_partition_by_length(const int64_t *ptr, const int32_t *rows, int64_t count, int limit, int32_t *out,
+                                       int64_t *block_counts, int64_t *block_offsets, int64_t *n_short_dev,
+                                       int64_t *scan_scratch, int64_t scan_elems, cudaStream_t s, int64_t *launches);
 // entries held by the rows of each degree class: out[kNClasses] (device), class_offs = the kNClasses + 1 offsets into order
 cudaError_t launch_class_entries(const int64_t *ptr, const int32_t *order, const int64_t *class_offs_dev, int64_t n,
                                  int64_t *out, cudaStream_t s, int64_t *launches);
@@ -208,7 +212,7 @@ cudaError_t launch_split_table(const float *X, int64_t n, void *T, cudaStream_t 
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                              int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
                              RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,
-                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table, const CgOptions &cg);
+                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table, const CgOptions &cg, const int32_t *order16 = nullptr, int64_t n8 = 0);
 
 // alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();
@@ -221,10 +225,12 @@ cudaError_t launch_dual64_prepare(const float *Bmat, void *ws, float cond_limit,
 cudaError_t launch_rows_dual64(const SideView &sv, int64_t first, int64_t count, const void *X, void *ws, RowOut out,
                                cudaStream_t s, int64_t *launches);
 const int *dual_flag_ptr(const void *ws);
-// route: set where conjugate gradients run; the kernel of the rows of 17 .. 32 observations returns at once when it says so
+// route: set where conjugate gradients run; the kernel of the rows of 17 .. 32 observations returns at once when it says so.
+// order16 (may be null): the count16 rows of 1 .. 16 observations again, those with at most 8 first (n8 of them): they
+// then go to a kernel instance with eight observations per row, which does twice the rows per tile
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
-                             const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, cudaStream_t s,
-                             int64_t *launches);
+                             const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, const int32_t *order16,
+                             int64_t n8, cudaStream_t s, int64_t *launches);
 
 // alx_loss.cu
 int64_t loss_partials(int64_t nnz);

@@ -8,7 +8,7 @@
 // 128 x 128 x 128 tensor-core product (rows padded to 16 (or 32) observations with zero embeddings, B^-1 split
 // into three bfloat16 parts), and per row: S_u = I + Z_u H_u^T (FP32 FMAs), S_u t = y_u by the in-warp Cholesky
 // the primal kernel uses for its diagonal blocks (padding rows are rows of the identity), w_u = Z_u^T t.
-// Two instances: rows of 1 .. 16 observations (two rows per warp) and rows of 17 .. 32 (one row per warp).
+// Three instances: rows of 1 .. 8 observations (four rows per warp), 9 .. 16 (two rows per warp) and 17 .. 32 (one row per warp).
 // The form is used only while B is well conditioned (its error grows with cond(B), which the primal form
 // avoids): k_binv_prepare sets a flag from ||B||_F ||B^-1||_F, the dual kernel does nothing when it is clear,
 // and the primal kernel then takes these rows as well.
@@ -27,7 +27,7 @@ namespace {
 using namespace ptx;
 
 constexpr int D = 128;
-constexpr int kMaxTileRows = 8;               // matrix rows per tile: 128 / (observations per row after padding)
+constexpr int kMaxTileRows = 16;              // matrix rows per tile at most: 128 / (observations per row after padding)
 constexpr int kSlots = 3;                     // tiles in flight
 constexpr int kTileBytes = 128 * D * 2;       // 128 padded observations x 128 features, bf16: two 64-feature panels
 constexpr int kPanelBytes = kTileBytes / 2;
@@ -177,7 +177,7 @@ __device__ __forceinline__ float rsqrt_fast(float x)
 // On return lane l holds row l of L in d[0 .. l], its component of L^-1 b in b and 1 / L[l][l] in my_inv.
 template <int KP> __device__ __forceinline__ bool factor_rows(float (&d)[KP], float &b, float &my_inv, int lane, float *xch)
 {
-    const int hb = (KP == 16) ? (lane & 16) : 0, l = lane & (KP - 1);
+    const int hb = lane & (32 - KP), l = lane & (KP - 1);      // first lane of my matrix, my row of it
     bool all_ok = true;
 #pragma unroll
     for (int j = 0; j < KP; j += 2) {
@@ -256,6 +256,37 @@ __device__ __forceinline__ float halfwarp_reduce16(float (&v)[16], int lane)
     const float send = up ? t2[0] : t2[1];
     const float keep = up ? t2[1] : t2[0];
     return keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+}
+
+// sum over the 8 lanes of a quarter-warp of v[c], for 16 values at once: lane l (of its eight) returns columns 2 l, 2 l + 1
+__device__ __forceinline__ void quarterwarp_reduce16(float (&v)[16], int lane, float &r0, float &r1)
+{
+    float t8[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const bool up = (lane & 4) != 0;
+        const float send = up ? v[c] : v[c + 8];
+        const float keep = up ? v[c + 8] : v[c];
+        t8[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 4);
+    }
+    float t4[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const bool up = (lane & 2) != 0;
+        const float send = up ? t8[c] : t8[c + 4];
+        const float keep = up ? t8[c + 4] : t8[c];
+        t4[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 2);
+    }
+    float t2[2];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        const bool up = (lane & 1) != 0;
+        const float send = up ? t4[c] : t4[c + 2];
+        const float keep = up ? t4[c + 2] : t4[c];
+        t2[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+    }
+    r0 = t2[0];
+    r1 = t2[1];
 }
 
 // Producer warp pw fills padded observations 32 pw .. 32 pw + 31 of every tile.  The index loads of a tile form a
@@ -403,8 +434,12 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         tc_fence_after();
         const int u = sm.row_u[g][mr];
         const int k_u = sm.row_k[g][mr];
-        const int k_other = __shfl_xor_sync(0xFFFFFFFFu, k_u, 16);
-        const int kmax = k_u > k_other ? k_u : k_other;       // warp-uniform: the row(s) of this warp
+        int kmax = k_u;                                       // warp-uniform: the longest of this warp's rows
+#pragma unroll
+        for (int o = KP; o < 32; o <<= 1) {
+            const int k_other = __shfl_xor_sync(0xFFFFFFFFu, kmax, o);
+            kmax = kmax > k_other ? kmax : k_other;
+        }
         // S row: s[j'] = sum_f Z[me][f] H[row mr, observation j'][f]
         float s[KP];
 #pragma unroll
@@ -418,7 +453,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
 #pragma unroll 1
         for (int cf = 0; cf < D / 16; ++cf) {
             if (cf + 1 < D / 16) tmem_ld16_nowait(trow + 16 * (cf + 1), zn);      // lands while this chunk is used
-            if constexpr (KP == 16) {
+            if constexpr (KP <= 16) {
 #pragma unroll
                 for (int jj = 0; jj < KP; jj += 2) {
                     // two observations per trip and two partial sums each: four independent chains of packed FMAs (one
@@ -481,8 +516,8 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         float my_inv = 0.f;
         // every thread of the group is past its reads of the tile: its memory now serves as scratch
         asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-        if (KP == 16 && tid == 0) mbar_arrive(&sm.empty[g]);    // the tile, its labels and row ids are not read again
-        float *scratch = (KP == 16) ? &sm.scratch16[g][0] : reinterpret_cast<float *>(&sm.h[g][0]);
+        if (KP <= 16 && tid == 0) mbar_arrive(&sm.empty[g]);    // the tile, its labels and row ids are not read again
+        float *scratch = (KP <= 16) ? &sm.scratch16[g][0] : reinterpret_cast<float *>(&sm.h[g][0]);
         float *xch = scratch + mr * (4 * KP);                   // per matrix row
         float *Lrow = scratch + (128 / KP) * (4 * KP) + mr * (KP * KP);       // per matrix row: L, row-major
         const bool ok = factor_rows<KP>(d, b, my_inv, lane, xch);
@@ -492,7 +527,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
             *reinterpret_cast<float4 *>(&Lrow[j * KP + 4 * q4]) = make_float4(d[4 * q4], d[4 * q4 + 1], d[4 * q4 + 2], d[4 * q4 + 3]);
         __syncwarp();
         float tj = 0.f;
-        const int hb = (KP == 16) ? (lane & 16) : 0;
+        const int hb = lane & (32 - KP);
 #pragma unroll
         for (int c = KP - 1; c >= 0; --c) {
             const float tc = __shfl_sync(0xFFFFFFFFu, b * my_inv, hb + c);
@@ -516,6 +551,24 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
                     z[c] = (lane & 16) ? other + z[c] : z[c] + other;
                 }
             }
+            if constexpr (KP == 8) {
+                // eight observations per row: the row's eight lanes end with two features each
+                float w0, w1;
+                quarterwarp_reduce16(z, lane, w0, w1);         // features 16 cf + 2 (lane & 7) and the next of row u
+                if (store) {
+                    const int f = 16 * cf + 2 * (lane & 7);
+                    const float v0 = row_ok ? w0 : 0.f, v1 = row_ok ? w1 : 0.f;
+                    *reinterpret_cast<__nv_bfloat162 *>(reinterpret_cast<__nv_bfloat16 *>(p.out.table) + (int64_t)u * D + f) =
+                        __floats2bfloat162_rn(v0, v1);
+                    if (p.out.cap_slot) {
+                        const int cs = p.out.cap_slot[u];
+                        if (cs >= 0) {
+                            p.out.cap_out[(int64_t)cs * D + f] = v0;
+                            p.out.cap_out[(int64_t)cs * D + f + 1] = v1;
+                        }
+                    }
+                }
+            } else {
             const float wr = halfwarp_reduce16(z, lane);       // feature 16 cf + (lane & 15) of row u
             const float wv = row_ok ? wr : 0.f;
             if (store && (KP == 16 || lane < 16)) {
@@ -525,6 +578,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
                     const int cs = p.out.cap_slot[u];
                     if (cs >= 0) p.out.cap_out[(int64_t)cs * D + f] = wv;
                 }
+            }
             }
         }
         if (!row_ok && u >= 0 && j == 0) {
@@ -536,7 +590,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
         if (tid == 0) {
             mbar_arrive(&sm.acc_empty[g]);
-            if (KP != 16) mbar_arrive(&sm.empty[g]);
+            if (KP > 16) mbar_arrive(&sm.empty[g]);
         }
     }
 }
@@ -622,8 +676,8 @@ const int *dual_flag_ptr(const void *ws) { return reinterpret_cast<const int *>(
 // rows order[first16 .. first16 + count16) of the solved side have 1 .. 16 observations each, the count32 rows after
 // them 17 .. 32
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
-                             const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, cudaStream_t s,
-                             int64_t *launches)
+                             const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, const int32_t *order16,
+                             int64_t n8, cudaStream_t s, int64_t *launches)
 {
     DualParams p{};
     p.route = route;
@@ -636,10 +690,25 @@ cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count1
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    p.first = first16;
-    p.count = count16;
-    cudaError_t e = launch_dual_instance<16>(p, sms, s, launches);
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
+    if (order16) {
+        // the rows of at most 8 observations, eight padded observations each (sixteen rows per tile), then the rest of the class
+        p.sv.order = order16;
+        p.first = 0;
+        p.count = n8;
+        e = launch_dual_instance<8>(p, sms, s, launches);
+        if (e != cudaSuccess) return e;
+        p.first = n8;
+        p.count = count16 - n8;
+        e = launch_dual_instance<16>(p, sms, s, launches);
+        if (e != cudaSuccess) return e;
+        p.sv.order = sv.order;
+    } else {
+        p.first = first16;
+        p.count = count16;
+        e = launch_dual_instance<16>(p, sms, s, launches);
+        if (e != cudaSuccess) return e;
+    }
     p.first = first16 + count16;
     p.count = count32;
     return launch_dual_instance<32>(p, sms, s, launches);

@@ -442,6 +442,95 @@ __global__ void k_sum_row_lengths(const int64_t *__restrict__ ptr, const int32_t
     if (threadIdx.x == 0) *out = part[0];
 }
 
+// Stable two-way partition of a list of rows by length (at most `limit` entries first, the others after them, both in
+// their old order): per-block counts, a scan of the counts, then a block-wide scatter.  Blocks of 1024 positions.
+constexpr int kPartBlock = 1024;
+__global__ void __launch_bounds__(256) k_part_count(const int64_t *__restrict__ ptr, const int32_t *__restrict__ rows, int64_t count,
+                                                    int limit, int64_t *__restrict__ block_counts)
+{
+    __shared__ int warp_sums[8];
+    const int64_t base = (int64_t)blockIdx.x * kPartBlock;
+    int mine = 0;
+    for (int k = threadIdx.x; k < kPartBlock; k += 256) {
+        const int64_t i = base + k;
+        if (i < count) {
+            const int32_t u = rows[i];
+            mine += (ptr[u + 1] - ptr[u] <= limit) ? 1 : 0;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = mine;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int w = 0; w < 8; ++w) t += warp_sums[w];
+        block_counts[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(256) k_part_scatter(const int64_t *__restrict__ ptr, const int32_t *__restrict__ rows, int64_t count,
+                                                      int limit, const int64_t *__restrict__ block_offsets, int64_t n_blocks,
+                                                      int32_t *__restrict__ out)
+{
+    __shared__ int warp_short[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t base = (int64_t)blockIdx.x * kPartBlock;
+    const int64_t n_short_total = block_offsets[n_blocks];
+    int64_t short_at = block_offsets[blockIdx.x];              // next free place among the short rows
+    int64_t long_at = n_short_total + (base - short_at);       // ... and among the others (every earlier row is in one of the two)
+    for (int round = 0; round < kPartBlock / 256; ++round) {
+        const int64_t i = base + round * 256 + threadIdx.x;
+        const bool live = i < count;
+        int32_t u = 0;
+        bool is_short = false;
+        if (live) {
+            u = rows[i];
+            is_short = ptr[u + 1] - ptr[u] <= limit;
+        }
+        const unsigned m_short = __ballot_sync(0xFFFFFFFFu, live && is_short);
+        const unsigned m_live = __ballot_sync(0xFFFFFFFFu, live);
+        if (lane == 0) warp_short[warp] = __popc(m_short);
+        __syncthreads();
+        int short_before = 0, short_round = 0;
+        for (int w = 0; w < 8; ++w) {
+            if (w < warp) short_before += warp_short[w];
+            short_round += warp_short[w];
+        }
+        const int live_before = warp * 32;                      // (a round's live threads are a prefix of the block)
+        const unsigned below = (1u << lane) - 1u;
+        if (live) {
+            if (is_short) out[short_at + short_before + __popc(m_short & below)] = u;
+            else out[long_at + (live_before - short_before) + __popc(m_live & ~m_short & below)] = u;
+        }
+        int live_round = 0;
+        {
+            const int64_t left = count - (base + round * 256);
+            live_round = left >= 256 ? 256 : (left > 0 ? (int)left : 0);
+        }
+        short_at += short_round;
+        long_at += live_round - short_round;
+        __syncthreads();
+    }
+}
+
+// out[0 .. count): the rows of `rows` with at most `limit` entries, then the others; *n_short_dev receives the number of the
+// former (device; block_counts and block_offsets: count / 1024 + 2 int64 each)
+cudaError_t launch_partition_by_length(const int64_t *ptr, const int32_t *rows, int64_t count, int limit, int32_t *out,
+                                       int64_t *block_counts, int64_t *block_offsets, int64_t *n_short_dev,
+                                       int64_t *scan_scratch, int64_t scan_elems, cudaStream_t s, int64_t *launches)
+{
+    if (count <= 0) return cudaMemsetAsync(n_short_dev, 0, sizeof(int64_t), s);
+    const int64_t nb = (count + kPartBlock - 1) / kPartBlock;
+    k_part_count<<<(unsigned)nb, 256, 0, s>>>(ptr, rows, count, limit, block_counts);
+    ++*launches;
+    cudaError_t e = scan_exclusive(block_counts, true, block_offsets, nb, scan_scratch, scan_elems, s, launches);
+    if (e != cudaSuccess) return e;
+    k_part_scatter<<<(unsigned)nb, 256, 0, s>>>(ptr, rows, count, limit, block_offsets, nb, out);
+    ++*launches;
+    e = cudaMemcpyAsync(n_short_dev, block_offsets + nb, sizeof(int64_t), cudaMemcpyDeviceToDevice, s);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 // doubled entry lists: one warp per row
 __global__ void __launch_bounds__(256) k_double_entries(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
                                                         const float *__restrict__ val, int64_t n, int64_t n_fixed,
