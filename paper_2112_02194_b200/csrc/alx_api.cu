@@ -43,7 +43,7 @@ struct alx_ctx {
     int64_t n_split_rows[4] = {0, 0, 0, 0};
     // tensor path with the dual form: the rows of 1 .. 16 entries once more per orientation, those with at most 8 entries first
     int32_t *order16[2] = {nullptr, nullptr};
-    int64_t n8[2] = {0, 0};
+    int64_t n4[2] = {0, 0}, n8[2] = {0, 0};      // ... and those with at most 4 before them
     void *fold_table = nullptr;   // that path's fixed table: [2 N x 128] bfloat16 parts of the fp32 table, rebuilt every half-epoch
 
     void *table[2] = {nullptr, nullptr};
@@ -266,7 +266,7 @@ void release_matrix(alx_ctx *c)
         dev_free(c, c->chunk_desc[s]); c->chunk_desc[s] = nullptr;
         dev_free(c, c->split_first[s]); c->split_first[s] = nullptr;
     }
-    for (int s = 0; s < 2; ++s) { dev_free(c, c->order16[s]); c->order16[s] = nullptr; c->n8[s] = 0; }
+    for (int s = 0; s < 2; ++s) { dev_free(c, c->order16[s]); c->order16[s] = nullptr; c->n4[s] = c->n8[s] = 0; }
     dev_free(c, c->split_partials); c->split_partials = nullptr;
     dev_free(c, c->loss_partials_buf); c->loss_partials_buf = nullptr;
     c->nnz = -1;
@@ -355,7 +355,7 @@ alx_status half_epoch_impl(alx_ctx *c, int side, const int32_t *cap_slot, float 
         ALX_CUDA(c, launch_rows_umma(side_view(c, side), c->class_offs[side], c->n_chunks[side], c->n_split_rows[side],
                                      c->table[fixed], c->Bmat, c->split_partials, out, c->status, c->stream,
                                      &c->launches, c->ev[3], c->ev[4], dual_form(c) ? c->dual_ws : nullptr, c->n[fixed],
-                                     cg_options(c, side), c->order16[side], c->n8[side]));
+                                     cg_options(c, side), c->order16[side], c->n4[side], c->n8[side]));
         c->stats.kernel_path[side] = 1;
         c->main_timed = true;
         c->dual_candidates = dual_form(c) ? c->class_offs[side][3] - c->class_offs[side][1] : 0;
@@ -581,8 +581,8 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
         }
     }
     if (dual_form(c)) {
-        // the rows of 1 .. 16 entries, split at 8 entries (a kernel instance with eight observations per row takes the
-        // first part at half the cost per row)
+        // the rows of 1 .. 16 entries, ordered by length class (at most 4, 5 .. 8, 9 .. 16): kernel instances with four and
+        // eight observations per row take the first two parts at a quarter and half of the cost per row
         for (int s = 0; s < 2; ++s) {
             const int64_t n16 = c->class_offs[s][2] - c->class_offs[s][1];
             if (n16 <= 0) continue;
@@ -591,10 +591,24 @@ alx_status alx_set_csr(alx_ctx *c, const int64_t *rowptr, const int32_t *colidx,
             ALX_TMP(c, tmp, pc, nb + 2);
             ALX_TMP(c, tmp, po, nb + 2);
             ALX_ALLOC(c, c->order16[s], n16);
-            ALX_CUDA(c, launch_partition_by_length(c->ptr[s], c->order[s] + c->class_offs[s][1], n16, 8, c->order16[s], pc, po,
+            ALX_CUDA(c, launch_partition_by_length(c->ptr[s], c->order[s] + c->class_offs[s][1], n16, 4, c->order16[s], pc, po,
                                                    class_entries + s, scan_scratch, scan_elems, c->stream, &c->launches));
-            ALX_CUDA(c, cudaMemcpyAsync(&c->n8[s], class_entries + s, sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
+            ALX_CUDA(c, cudaMemcpyAsync(&c->n4[s], class_entries + s, sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
             ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+            const int64_t rest = n16 - c->n4[s];
+            c->n8[s] = c->n4[s];
+            if (rest > 0) {
+                int32_t *part = nullptr;
+                ALX_TMP(c, tmp, part, rest);
+                ALX_CUDA(c, launch_partition_by_length(c->ptr[s], c->order16[s] + c->n4[s], rest, 8, part, pc, po, class_entries + s,
+                                                       scan_scratch, scan_elems, c->stream, &c->launches));
+                int64_t n58 = 0;
+                ALX_CUDA(c, cudaMemcpyAsync(&n58, class_entries + s, sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
+                ALX_CUDA(c, cudaMemcpyAsync(c->order16[s] + c->n4[s], part, sizeof(int32_t) * rest, cudaMemcpyDeviceToDevice, c->stream));
+                ALX_CUDA(c, cudaStreamSynchronize(c->stream));
+                c->n8[s] += n58;
+                tmp.release(part);
+            }
             tmp.release(pc);
             tmp.release(po);
         }

@@ -212,7 +212,7 @@ cudaError_t launch_split_table(const float *X, int64_t n, void *T, cudaStream_t 
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *class_offs_host, int64_t n_chunks,
                              int64_t n_split_rows, const void *X, const float *Bmat, float *split_partials,
                              RowOut out, DevStatus *st, cudaStream_t s, int64_t *launches, cudaEvent_t main_begin,
-                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table, const CgOptions &cg, const int32_t *order16 = nullptr, int64_t n8 = 0);
+                             cudaEvent_t main_end, const void *dual_ws, int64_t n_table, const CgOptions &cg, const int32_t *order16 = nullptr, int64_t n4 = 0, int64_t n8 = 0);
 
 // alx_dual.cu: rows with at most 32 observations in the dual form (d = 128, bf16 tables)
 size_t dual_workspace_bytes();
@@ -226,11 +226,12 @@ cudaError_t launch_rows_dual64(const SideView &sv, int64_t first, int64_t count,
                                cudaStream_t s, int64_t *launches);
 const int *dual_flag_ptr(const void *ws);
 // route: set where conjugate gradients run; the kernel of the rows of 17 .. 32 observations returns at once when it says so.
-// order16 (may be null): the count16 rows of 1 .. 16 observations again, those with at most 8 first (n8 of them): they
-// then go to a kernel instance with eight observations per row, which does twice the rows per tile
+// order16 (may be null): the count16 rows of 1 .. 16 observations again, ordered by length class: the n4 rows of at most 4
+// first, then those of 5 .. 8 (up to position n8), then the rest; the first two parts go to kernel instances with four and
+// eight observations per row, which do four times and twice the rows per tile
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
                              const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, const int32_t *order16,
-                             int64_t n8, cudaStream_t s, int64_t *launches);
+                             int64_t n4, int64_t n8, cudaStream_t s, int64_t *launches);
 
 // alx_loss.cu
 int64_t loss_partials(int64_t nnz);

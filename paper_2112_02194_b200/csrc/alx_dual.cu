@@ -8,7 +8,7 @@
 // 128 x 128 x 128 tensor-core product (rows padded to 16 (or 32) observations with zero embeddings, B^-1 split
 // into three bfloat16 parts), and per row: S_u = I + Z_u H_u^T (FP32 FMAs), S_u t = y_u by the in-warp Cholesky
 // the primal kernel uses for its diagonal blocks (padding rows are rows of the identity), w_u = Z_u^T t.
-// Three instances: rows of 1 .. 8 observations (four rows per warp), 9 .. 16 (two rows per warp) and 17 .. 32 (one row per warp).
+// Four instances: rows of 1 .. 4 observations (eight rows per warp), 5 .. 8 (four), 9 .. 16 (two) and 17 .. 32 (one row per warp).
 // The form is used only while B is well conditioned (its error grows with cond(B), which the primal form
 // avoids): k_binv_prepare sets a flag from ||B||_F ||B^-1||_F, the dual kernel does nothing when it is clear,
 // and the primal kernel then takes these rows as well.
@@ -27,7 +27,7 @@ namespace {
 using namespace ptx;
 
 constexpr int D = 128;
-constexpr int kMaxTileRows = 16;              // matrix rows per tile at most: 128 / (observations per row after padding)
+constexpr int kMaxTileRows = 32;              // matrix rows per tile at most: 128 / (observations per row after padding)
 constexpr int kSlots = 3;                     // tiles in flight
 constexpr int kTileBytes = 128 * D * 2;       // 128 padded observations x 128 features, bf16: two 64-feature panels
 constexpr int kPanelBytes = kTileBytes / 2;
@@ -258,6 +258,26 @@ __device__ __forceinline__ float halfwarp_reduce16(float (&v)[16], int lane)
     return keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
 }
 
+// sum over 4 lanes of v[c], for 16 values at once: lane l (of its four) returns columns 4 l .. 4 l + 3
+__device__ __forceinline__ void eighthwarp_reduce16(float (&v)[16], int lane, float (&r)[4])
+{
+    float t8[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const bool up = (lane & 2) != 0;
+        const float send = up ? v[c] : v[c + 8];
+        const float keep = up ? v[c + 8] : v[c];
+        t8[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 2);
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const bool up = (lane & 1) != 0;
+        const float send = up ? t8[c] : t8[c + 4];
+        const float keep = up ? t8[c + 4] : t8[c];
+        r[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+    }
+}
+
 // sum over the 8 lanes of a quarter-warp of v[c], for 16 values at once: lane l (of its eight) returns columns 2 l, 2 l + 1
 __device__ __forceinline__ void quarterwarp_reduce16(float (&v)[16], int lane, float &r0, float &r1)
 {
@@ -447,6 +467,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
         // rows of my matrix row start at a multiple of 8 rows: the swizzle term of row KP mr + jj is jj & 7, known
         // at compile time, and the row's offset is one runtime base plus constants
         const unsigned char *tile = &sm.h[g][0] + (KP * mr / 8) * 1024;
+        const int rsub = (KP < 8) ? (KP * mr) & 7 : 0;      // four observations per row: two rows share a group of 8 tile rows
         float z[16], zn[16];
         tmem_ld16(trow, z);
         // not unrolled: the body is KP dot products of 16 terms; eight copies of it would not fit the instruction cache
@@ -464,10 +485,11 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
 #pragma unroll
                         for (int t = 0; t < 2; ++t) {
                             const int jt = jj + t;
-                            const int base = (cf >> 2) * kPanelBytes + (jt >> 3) * 1024 + (jt & 7) * 128;
+                            const int jr = jt + rsub;      // (row of the observation inside its group of 8 tile rows, for KP < 8)
+                            const int base = (cf >> 2) * kPanelBytes + (jr >> 3) * 1024 + (jr & 7) * 128;
                             const int c0 = (cf & 3) * 2;
-                            const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + base + ((c0 ^ (jt & 7)) << 4));
-                            const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + base + (((c0 + 1) ^ (jt & 7)) << 4));
+                            const uint4 h0 = *reinterpret_cast<const uint4 *>(tile + base + ((c0 ^ (jr & 7)) << 4));
+                            const uint4 h1 = *reinterpret_cast<const uint4 *>(tile + base + (((c0 + 1) ^ (jr & 7)) << 4));
                             const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
                             // packed FP32 FMAs: even features in .x, odd features in .y (a bfloat16 pair unpacks to exactly that)
                             acc[t][0] = make_float2(s[jt], 0.f);
@@ -551,7 +573,26 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
                     z[c] = (lane & 16) ? other + z[c] : z[c] + other;
                 }
             }
-            if constexpr (KP == 8) {
+            if constexpr (KP == 4) {
+                // four observations per row: the row's four lanes end with four features each
+                float w4[4];
+                eighthwarp_reduce16(z, lane, w4);              // features 16 cf + 4 (lane & 3) .. + 3 of row u
+                if (store) {
+                    const int f = 16 * cf + 4 * (lane & 3);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) w4[e] = row_ok ? w4[e] : 0.f;
+                    __nv_bfloat162 *dst = reinterpret_cast<__nv_bfloat162 *>(reinterpret_cast<__nv_bfloat16 *>(p.out.table) + (int64_t)u * D + f);
+                    dst[0] = __floats2bfloat162_rn(w4[0], w4[1]);
+                    dst[1] = __floats2bfloat162_rn(w4[2], w4[3]);
+                    if (p.out.cap_slot) {
+                        const int cs = p.out.cap_slot[u];
+                        if (cs >= 0) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) p.out.cap_out[(int64_t)cs * D + f + e] = w4[e];
+                        }
+                    }
+                }
+            } else if constexpr (KP == 8) {
                 // eight observations per row: the row's eight lanes end with two features each
                 float w0, w1;
                 quarterwarp_reduce16(z, lane, w0, w1);         // features 16 cf + 2 (lane & 7) and the next of row u
@@ -677,7 +718,7 @@ const int *dual_flag_ptr(const void *ws) { return reinterpret_cast<const int *>(
 // them 17 .. 32
 cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count16, int64_t count32, const void *X,
                              const void *ws, RowOut out, DevStatus *st, const CgPolicy *route, const int32_t *order16,
-                             int64_t n8, cudaStream_t s, int64_t *launches)
+                             int64_t n4, int64_t n8, cudaStream_t s, int64_t *launches)
 {
     DualParams p{};
     p.route = route;
@@ -692,10 +733,14 @@ cudaError_t launch_rows_dual(const SideView &sv, int64_t first16, int64_t count1
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaError_t e;
     if (order16) {
-        // the rows of at most 8 observations, eight padded observations each (sixteen rows per tile), then the rest of the class
+        // the rows of at most 4 and of 5 .. 8 observations (32 and 16 rows per tile), then the rest of the class
         p.sv.order = order16;
         p.first = 0;
-        p.count = n8;
+        p.count = n4;
+        e = launch_dual_instance<4>(p, sms, s, launches);
+        if (e != cudaSuccess) return e;
+        p.first = n4;
+        p.count = n8 - n4;
         e = launch_dual_instance<8>(p, sms, s, launches);
         if (e != cudaSuccess) return e;
         p.first = n8;

@@ -2070,7 +2070,7 @@ cudaError_t launch_gramian_umma(const void *X, int64_t n, float *partials, cudaS
 cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_chunks, int64_t n_split_rows,
                              const void *X, const float *Bmat, float *split_partials, RowOut out, DevStatus *st,
                              cudaStream_t s, int64_t *launches, cudaEvent_t main_begin, cudaEvent_t main_end,
-                             const void *dual_ws, int64_t n_table, const CgOptions &cg, const int32_t *order16, int64_t n8)
+                             const void *dual_ws, int64_t n_table, const CgOptions &cg, const int32_t *order16, int64_t n4, int64_t n8)
 {
     const int sms = sm_count();
     Params p{};
@@ -2116,7 +2116,7 @@ cudaError_t launch_rows_umma(const SideView &sv, const int64_t *offs, int64_t n_
     }
     if (dual_ws && offs[3] > offs[1]) {
         // rows with 1 .. 32 observations (classes 1 and 2): dual form, if the flag (set on the device) allows it
-        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], offs[3] - offs[2], X, dual_ws, out, st, p.route, order16, n8, s, launches);
+        e = launch_rows_dual(sv, offs[1], offs[2] - offs[1], offs[3] - offs[2], X, dual_ws, out, st, p.route, order16, n4, n8, s, launches);
         if (e != cudaSuccess) return e;
         p.dual_flag = dual_flag_ptr(dual_ws);
         p.n_items_primal = offs[c_long] - offs[3];
