@@ -474,7 +474,7 @@ template <int KP> __device__ void dual_solver(const DualParams &p, DualSmem &sm,
 #pragma unroll 1
         for (int cf = 0; cf < D / 16; ++cf) {
             if (cf + 1 < D / 16) tmem_ld16_nowait(trow + 16 * (cf + 1), zn);      // lands while this chunk is used
-            if constexpr (KP <= 16) {
+            if constexpr (KP <= 32) {      // (every instance; the one-observation-per-trip form below is kept for reference)
 #pragma unroll
                 for (int jj = 0; jj < KP; jj += 2) {
                     // two observations per trip and two partial sums each: four independent chains of packed FMAs (one
