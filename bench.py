@@ -387,18 +387,30 @@ def run_ours(args, w):
     alu_cg_half = statistics.mean([alu_half - rows_side[sd] * chol_row - 2.0 * ent_side[sd] * d + alu_side[sd] for sd in (0, 1)])
     t_alu_cg = alu_cg_half / (fp32_peak * 1e12)
     t_roof_cg = max(t_bytes, t_tensor + t_alu_cg)
-    kernel_txt = ("k_umma<3> + k_umma<0>: whole rows (item gather by TMA, tcgen05 outer products into tensor memory, "
-                  "conjugate gradients on the matrix in tensor memory, Cholesky in tensor memory for rows that do not "
-                  "converge or sides the policy moved, store)" if st.kernel_path[0] == 1 else
-                  "k_rows_simple: whole rows on the FP32 ALUs (gather, outer products, Cholesky in shared memory, store)")
+    fold = st.kernel_path[0] == 1 and e == 4       # fp32 tables with d = 64 on the tensor cores: split operands
+    if st.kernel_path[0] != 1:
+        kernel_txt = "k_rows_simple: whole rows on the FP32 ALUs (gather, outer products, Cholesky in shared memory, store)"
+    elif fold:
+        kernel_txt = ("k_umma<4>: whole rows of 17..512 entries (item gather by TMA from the bfloat16 parts of the fp32 "
+                      "table, tcgen05 outer products into tensor memory, fold to the 64 x 64 matrix, conjugate gradients "
+                      "on the matrix in registers, Cholesky in shared memory for rows that do not converge, store)")
+    else:
+        kernel_txt = ("k_umma<3> + k_umma<0>: whole rows (item gather by TMA, tcgen05 outer products into tensor memory, "
+                      "conjugate gradients on the matrix in tensor memory, Cholesky in tensor memory for rows that do not "
+                      "converge or sides the policy moved, store)")
+    short_txt = ("rows with at most 16 entries, solved by k_dual64 outside the dominant kernel" if fold else
+                 "rows with at most 32 entries, solved by k_dual outside the dominant kernel")
+    long_txt = ("whole rows of more than 512 entries: sums by the chunks kernel, solve by k_solve_sums_fold, outside the "
+                "dominant kernel" if fold else
+                "whole rows of more than 1024 entries: sums by the chunks kernel, solve by k_solve_sums, outside the "
+                "dominant kernel")
     roof.update({"kernel": kernel_txt,
                  "main_kernel_ms": main_ms, "rows_per_launch": rows_whole, "entries_per_launch": ent_whole,
                  "per_side": {"rows": rows_side, "entries": ent_side, "alu_flop": alu_side},
                  "rows_in_dual_form": {"rows": half_ms["dual_rows"][0], "cols": half_ms["dual_rows"][1],
-                                       "note": "rows with at most 32 entries, solved by k_dual outside the dominant kernel"},
+                                       "note": short_txt},
                  "long_rows": {"rows": list(st.long_rows), "entries": list(st.long_entries),
-                               "note": "whole rows of more than 1024 entries: sums by the chunks kernel, solve by "
-                                       "k_solve_sums, outside the dominant kernel"},
+                               "note": long_txt},
                  "peak_source": f"HBM and bf16 {peaks['source']} (sustained bf16); FP32 FMA measured in this run",
                  "half_epoch_ms": {"rows": half_ms["rows"][0], "cols": half_ms["cols"][0],
                                    "gramian": statistics.mean(half_ms["gramian"]), "row_kernels": rows_ms},
