@@ -125,6 +125,16 @@ __device__ __forceinline__ void tma_gather4(uint32_t dst_smem, const void *tenso
         : "memory");
 }
 
+// ---- TMA tile load: one box of a 2-D tensor (x = first element, y = first row), swizzled as the tensor map says;
+// rows past the tensor's extent arrive as zeros and count toward the bytes like the others.
+__device__ __forceinline__ void tma_tile_2d(uint32_t dst_smem, const void *tensor_map, int x, int y, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst_smem), "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
 __device__ __forceinline__ void st_shared_zero16(uint32_t dst_smem)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst_smem), "r"(0u) : "memory");

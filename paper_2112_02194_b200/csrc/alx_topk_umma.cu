@@ -50,14 +50,6 @@ template <bool SMEM_LISTS> struct __align__(1024) TopkSmem {
 
 static_assert(sizeof(TopkSmem<true>) + 1024 <= 232448 && sizeof(TopkSmem<false>) + 1024 <= 232448, "shared memory of the Top-K kernel");
 
-__device__ __forceinline__ void tma_tile_2d(uint32_t dst_smem, const void *tensor_map, int x, int y, uint64_t *bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst_smem), "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar))
-        : "memory");
-}
-
 // bf16 operands, fp32 accumulator, both operands K-major: D (+)= A * B^T
 __host__ __device__ constexpr uint32_t idesc_bf16_k_major(int M, int N)
 {

@@ -565,7 +565,8 @@ __device__ void producer_role_items(const Params &p, const CUtensorMap *tmap, Sm
 // number of producer warps, whole stages of 64 rows each.  The rows come by TMA row gathers (four rows of one
 // 64-feature half per instruction, written with the 128-byte swizzle the tensor core reads), issued by lanes 0 .. 15 for
 // the 16 groups of four rows; the stage's mbarrier counts the bytes.  Rows past the end of the item take a row
-// coordinate past the end of the table, which the copy fills with zeros.
+// coordinate past the end of the table, which the copy fills with zeros.  The Gramian's rows are consecutive: there a
+// stage is two tile loads of 64 rows, issued by one lane.
 template <int MODE>
 __device__ void stream_producer_role(const Params &p, const CUtensorMap *tmap, SmemT<MODE> &sm, int pw, int lane)
 {
@@ -584,6 +585,19 @@ __device__ void stream_producer_role(const Params &p, const CUtensorMap *tmap, S
             const uint32_t ph = ring_ph;
             if (++ring_slot == kNStage) { ring_slot = 0; ring_ph ^= 1u; }
             if ((int)(g % P) != pw) continue;
+            if constexpr (MODE == kModeGramian) {
+                // consecutive rows of the table: one tile load per 64-feature half (the same lines and swizzle as the
+                // row gathers leave; the tensor map of this launch has boxes of 64 rows)
+                if (!mbar_wait_warp(&sm.empty[slot], ph ^ 1u, &sm.abort_flag, 10 + MODE)) { alive = false; break; }
+                if (lane == 0) {
+                    const uint32_t dst = smem_u32(&sm.h[slot][0]);
+                    mbar_arrive_expect_tx(&sm.full[slot], 2u * (uint32_t)Ring<MODE>::kHalfBytes);
+                    tma_tile_2d(dst, tmap, 0, (int)e0, &sm.full[slot]);
+                    tma_tile_2d(dst + Ring<MODE>::kHalfBytes, tmap, 64, (int)e0, &sm.full[slot]);
+                }
+                __syncwarp();
+                continue;
+            }
             // this lane's two rows of the stage (lane and 32 + lane)
             int32_t my_idx[2] = {past_end, past_end};
             float my_y[2] = {0.f, 0.f};
@@ -2002,9 +2016,10 @@ static_assert(sizeof(SmemT<0>) + 1024 + sizeof(float) * D * kLdBq + kMaxGroups *
 static_assert(sizeof(SmemT<3>) + 1024 + sizeof(float) * D * kLdBq + kMaxGroups * sizeof(CgGroupSmem) <= 232448, "rows mode, CG");
 static_assert(sizeof(SmemT<4>) == sizeof(SmemT<3>), "the fold kernel has the conjugate-gradient kernel's feed");
 
-// Tensor map of a bfloat16 table [n x 128] for row gathers: boxes of one row by 64 features (128 bytes), 128-byte swizzle.
+// Tensor map of a bfloat16 table [n x 128]: boxes of 64 features (128 bytes) by one row for the row gathers, by a stage's
+// 64 rows for the tile loads of the Gramian; 128-byte swizzle.
 // (The encoder is a driver entry point, looked up through the runtime so that the library needs no driver at link time.)
-cudaError_t table_tensor_map(const void *X, int64_t n, CUtensorMap *tm)
+cudaError_t table_tensor_map(const void *X, int64_t n, CUtensorMap *tm, int box_rows = 1)
 {
     typedef CUresult (*Encode)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -2020,7 +2035,7 @@ cudaError_t table_tensor_map(const void *X, int64_t n, CUtensorMap *tm)
     }
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)n};
     const cuuint64_t strides[1] = {(cuuint64_t)D * sizeof(__nv_bfloat16)};
-    const cuuint32_t box[2] = {64, 1};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(X), dims, strides, box, estr,
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -2034,7 +2049,7 @@ template <int MODE> cudaError_t launch_mode(const Params &p, int grid, cudaStrea
     cudaError_t e = cudaFuncSetAttribute(k_umma<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     CUtensorMap tm;
-    e = table_tensor_map(p.X, p.n_table, &tm);
+    e = table_tensor_map(p.X, p.n_table, &tm, MODE == kModeGramian ? Ring<MODE>::kRows : 1);
     if (e != cudaSuccess) return e;
     k_umma<MODE><<<grid, block_threads<MODE>(), smem, s>>>(p, tm);
     return cudaGetLastError();
