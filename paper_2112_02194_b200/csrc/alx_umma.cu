@@ -1154,6 +1154,18 @@ __device__ __forceinline__ float chol_in_tmem(SmemRows &sm, RowGroupSmem &gs, co
     return x;
 }
 
+// Sums of two values over the warp with five shuffles instead of ten: the first exchange leaves the pair sum of `a` in
+// the even lanes and of `b` in the odd lanes, four more rounds complete them.  Returns the total of `a` in even lanes,
+// of `b` in odd lanes (a fixed order of additions).
+__device__ __forceinline__ float warp_sum_pair(float a, float b, int lane)
+{
+    const bool odd = (lane & 1) != 0;
+    float m = (odd ? b : a) + __shfl_xor_sync(0xFFFFFFFFu, odd ? a : b, 1);
+#pragma unroll
+    for (int o = 2; o < 32; o <<= 1) m += __shfl_xor_sync(0xFFFFFFFFu, m, o);
+    return m;
+}
+
 // The 16x128b tensor-memory shape as the conjugate-gradient solve uses it: thread (g, q) = (lane / 4, lane % 4) of warp w
 // sees rows 32w + g + 8k (k = 0 .. 3) of the matrix at the columns of its class, q + 4j.  One load brings 32 columns by
 // 16 lanes: cur[2j] = (row k = 2h, column 32cb + q + 4j), cur[2j + 1] = (row k = 2h + 1, same column), j = 0 .. 7.
@@ -1231,7 +1243,7 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
     const int lane = tid & 31, w = tid >> 5, g = lane >> 2, q = lane & 3;
     const int own = 32 * w + g + 8 * q;                          // the row this thread owns
     float *vq = reinterpret_cast<float *>(&gs.pop[0][0]);       // the vector of the next product
-    float *red = vq + 4 * kQStride;                              // [4 warps][4]
+    float *red = vq + 4 * kQStride;                              // [3 sums][4 warps]
     float *vslot = vq + (own & 3) * kQStride + (own >> 2);
     // product with the vector in shared memory; this thread's component of the result
     auto product = [&]() {
@@ -1265,21 +1277,28 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
     for (int it = 0;; ++it) {
         const float wv = product();
         ++products;
-        float gsum = r * r, dl = r * wv, bsum = b * b;
+        // |r|^2 and r.w of the warp with one butterfly: after the first exchange the even lanes carry |r|^2, the odd
+        // lanes r.w (red: [4 warps] of |r|^2, then of r.w, then of |b|^2)
+        float gsum, dl;
+        {
+            const float mine = warp_sum_pair(r * r, r * wv, lane);
+            if (lane < 2) red[4 * lane + w] = mine;
+            if (it == 0) {
+                float bsum = b * b;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, o);
-            dl += __shfl_xor_sync(0xFFFFFFFFu, dl, o);
-            if (it == 0) bsum += __shfl_xor_sync(0xFFFFFFFFu, bsum, o);
+                for (int o = 16; o > 0; o >>= 1) bsum += __shfl_xor_sync(0xFFFFFFFFu, bsum, o);
+                if (lane == 0) red[8 + w] = bsum;
+            }
         }
-        if (lane == 0) *reinterpret_cast<float4 *>(red + 4 * w) = make_float4(gsum, dl, bsum, 0.f);
         group128_sync(bar_id);
         {
-            const float4 r0 = *reinterpret_cast<const float4 *>(red), r1 = *reinterpret_cast<const float4 *>(red + 4),
-                         r2 = *reinterpret_cast<const float4 *>(red + 8), r3 = *reinterpret_cast<const float4 *>(red + 12);
-            gsum = ((r0.x + r1.x) + r2.x) + r3.x;
-            dl = ((r0.y + r1.y) + r2.y) + r3.y;
-            if (it == 0) bb = ((r0.z + r1.z) + r2.z) + r3.z;
+            const float4 g4 = *reinterpret_cast<const float4 *>(red), d4 = *reinterpret_cast<const float4 *>(red + 4);
+            gsum = ((g4.x + g4.y) + g4.z) + g4.w;
+            dl = ((d4.x + d4.y) + d4.z) + d4.w;
+            if (it == 0) {
+                const float4 b4 = *reinterpret_cast<const float4 *>(red + 8);
+                bb = ((b4.x + b4.y) + b4.z) + b4.w;
+            }
         }
         if (it == 0 && warm && !(gsum <= bb)) {
             // the start vector is further from the solution than zero is (tables not trained yet): start again from zero
@@ -1474,7 +1493,7 @@ __device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, cons
     const int lane = tid & 31, w = tid >> 5, i = tid & 63, h = tid >> 6;
     // product with the vector in gs.vec: my half row's part, with this thread's share of r.w (v = the vector's own
     // component); the parts and the warps' sums go through shared memory behind one barrier
-    auto product_and_sums = [&](float v, float bb_term, float &gsum, float &dl, float &bsum) {
+    auto product_and_sums = [&](float v, float bb_term, bool want_b, float &gsum, float &dl, float &bsum) {
         float acc0 = 0.f, acc1 = 0.f;
         const float4 *vp = reinterpret_cast<const float4 *>(gs.vec + 32 * h);
 #pragma unroll
@@ -1487,20 +1506,20 @@ __device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, cons
         }
         const float part = acc0 + acc1;
         gs.ws[h][i] = part;
-        float s0 = h == 0 ? v * v : 0.f, s1 = v * part, s2 = h == 0 ? bb_term : 0.f;
+        // (red: [3 sums][4 warps]; |v|^2 and |b|^2 come from the warps of the first column half alone)
+        const float m = warp_sum_pair(h == 0 ? v * v : 0.f, v * part, lane);
+        if (lane < 2) gs.red[lane][w] = m;
+        if (want_b) {
+            float s2 = h == 0 ? bb_term : 0.f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, o);
-            s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
-            s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+            for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+            if (lane == 0) gs.red[2][w] = s2;
         }
-        if (lane == 0) *reinterpret_cast<float4 *>(&gs.red[w][0]) = make_float4(s0, s1, s2, 0.f);
         group128_sync(bar_id);
-        const float4 r0 = *reinterpret_cast<const float4 *>(&gs.red[0][0]), r1 = *reinterpret_cast<const float4 *>(&gs.red[1][0]),
-                     r2 = *reinterpret_cast<const float4 *>(&gs.red[2][0]), r3 = *reinterpret_cast<const float4 *>(&gs.red[3][0]);
-        gsum = r0.x + r1.x;
-        dl = ((r0.y + r1.y) + r2.y) + r3.y;
-        bsum = r0.z + r1.z;
+        const float4 g4 = *reinterpret_cast<const float4 *>(&gs.red[0][0]), d4 = *reinterpret_cast<const float4 *>(&gs.red[1][0]);
+        gsum = g4.x + g4.y;
+        dl = ((d4.x + d4.y) + d4.z) + d4.w;
+        bsum = want_b ? gs.red[2][0] + gs.red[2][1] : 0.f;
         return gs.ws[0][i] + gs.ws[1][i];
     };
     bool warm = p.cg_warm != 0;
@@ -1511,7 +1530,7 @@ __device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, cons
     group128_sync(bar_id);
     if (warm) {                 // r = b - A x0
         float g0, d0, b0;
-        r = b - product_and_sums(x0, 0.f, g0, d0, b0);
+        r = b - product_and_sums(x0, 0.f, false, g0, d0, b0);
         ++products;
         // (the vector was read before the barrier inside the product; the parts and sums are read before the next one)
         if (h == 0) gs.vec[i] = r;
@@ -1520,7 +1539,7 @@ __device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, cons
     bool ok = false;
     for (int it = 0;; ++it) {
         float gsum, dl, bsum;
-        const float wv = product_and_sums(r, b * b, gsum, dl, bsum);
+        const float wv = product_and_sums(r, b * b, it == 0, gsum, dl, bsum);
         ++products;
         if (it == 0) bb = bsum;
         if (it == 0 && warm && !(gsum <= bb)) {
@@ -1559,7 +1578,7 @@ __device__ __forceinline__ bool fold_cg(const Params &p, FoldGroupSmem &gs, cons
         if (h == 0) gs.vec[i] = x;
         group128_sync(bar_id);
         float g0, d0, b0;
-        const float rt = b - product_and_sums(x, 0.f, g0, d0, b0);
+        const float rt = b - product_and_sums(x, 0.f, false, g0, d0, b0);
         ++products;
         group128_sync(bar_id);      // the sums of the product have been read
         float tsum = h == 0 ? rt * rt : 0.f;
