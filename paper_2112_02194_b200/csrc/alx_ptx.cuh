@@ -173,6 +173,15 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Copy of 128 rows x 32 bytes from shared memory to the 128 lanes x 8 columns of tensor memory at taddr, issued by ONE
+// thread; it runs in the tensor pipe, in order with the tcgen05.mma that this thread issues after it.  The source is
+// read through a descriptor without swizzle: 32-bit element (row r, column c < 8) at
+// (r / 8) * stride offset + (c / 4) * leading offset + (r % 8) * 16 + (c % 4) * 4 bytes (confirmed with a pattern).
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t src_desc)
+{
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(src_desc) : "memory");
+}
+
 // D[tmem] (+)= A[smem desc] * B[smem desc], issued by ONE thread
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate)
 {

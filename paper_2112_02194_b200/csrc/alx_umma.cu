@@ -132,10 +132,10 @@ constexpr int kLdB = D + 4;
 constexpr int kCgVerifyProducts = 24;
 constexpr float kCgVerifySlack = 2.f;
 // conjugate gradients read the matrix with the 16x128b tensor-memory shape (a thread holds four rows, every fourth
-// column): alpha0 G + lambda I and the vector of a product are kept in shared memory by column class (column mod 4),
-// 36 floats per class so that the four classes of a quarter-warp's 16-byte loads fall into different banks
+// column): the vector of a product is kept in shared memory by column class (column mod 4), 36 floats per class so
+// that the four classes of a quarter-warp's 16-byte loads fall into different banks
 constexpr int kQStride = 36;
-constexpr int kLdBq = 4 * kQStride;      // floats per row of alpha0 G + lambda I in that layout
+constexpr int kLdBq = 4 * kQStride;      // floats reserved per row of alpha0 G + lambda I in the rows kernels' shared memory
 struct __align__(128) RowGroupSmem {   // scratch of one tensor-memory solver group
     // Panel of the current block step as tensor-core operands: row i = what thread i computed, split into
     // three bfloat16 parts (p = p1 + p2 + p3 to 2^-24), each part a K-major 128 x 16 tile without swizzle:
@@ -645,7 +645,7 @@ __device__ void stream_producer_role(const Params &p, const CUtensorMap *tmap, S
     }
 }
 
-template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, int lane)
+template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, int lane, uint32_t base_smem = 0)
 {
     constexpr int kNStage = Ring<MODE>::kNStage, kRows = Ring<MODE>::kRows;
     constexpr uint32_t kIdescMain = idesc_bf16_mn_major(128, 128);
@@ -698,6 +698,16 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
             tc_fence_after();
             const uint32_t d_main = tmem + a * Cfg<MODE>::kAccStride;
             bool first = true;
+            if constexpr (MODE == kModeRowsCg) {
+                // the accumulator starts as alpha0 G + lambda I (copied from shared memory by the tensor pipe, in
+                // order with the products that follow): the solver finds the complete matrix of Eq. 4
+                if (lane == 0) {
+#pragma unroll 1
+                    for (int c8 = 0; c8 < D / 8; ++c8)
+                        tmem_cp_128x256b(d_main + 8 * c8, smem_desc(base_smem + c8 * 4096, 128, 256, 0));
+                }
+                first = false;
+            }
             for (int s = 0; s < nst; ++s)
                 if (!stage(d_main, s + 1 < nst ? kRows / 16 : nk_last, first)) { alive = false; break; }
             if (alive && lane == 0) umma_commit(&sm.acc_full[a]);
@@ -1170,28 +1180,6 @@ __device__ __forceinline__ float warp_sum_pair(float a, float b, int lane)
 // sees rows 32w + g + 8k (k = 0 .. 3) of the matrix at the columns of its class, q + 4j.  One load brings 32 columns by
 // 16 lanes: cur[2j] = (row k = 2h, column 32cb + q + 4j), cur[2j + 1] = (row k = 2h + 1, same column), j = 0 .. 7.
 //
-// Adds alpha0 G + lambda I to the matrix in tensor memory (every column: the products read both triangles).
-// Bq[row * kLdBq + q * kQStride + j] = B[row][q + 4j].
-__device__ __forceinline__ void cg_add_base(uint32_t twarp, const float *Bq, int row0, int q)
-{
-#pragma unroll 2
-    for (int step = 0; step < 8; ++step) {
-        const int h = step & 1, cb = step >> 1;
-        const uint32_t taddr = twarp + ((uint32_t)(h * 16) << 16) + 32 * cb;
-        float cur[16];
-        tmem_ld_16x128b_x8(taddr, cur);
-        const float *b0 = Bq + (row0 + 16 * h) * kLdBq + q * kQStride + 8 * cb, *b1 = b0 + 8 * kLdBq;
-#pragma unroll
-        for (int j4 = 0; j4 < 2; ++j4) {
-            const float4 u = *reinterpret_cast<const float4 *>(b0 + 4 * j4), v = *reinterpret_cast<const float4 *>(b1 + 4 * j4);
-            cur[8 * j4 + 0] += u.x; cur[8 * j4 + 1] += v.x; cur[8 * j4 + 2] += u.y; cur[8 * j4 + 3] += v.y;
-            cur[8 * j4 + 4] += u.z; cur[8 * j4 + 5] += v.z; cur[8 * j4 + 6] += u.w; cur[8 * j4 + 7] += v.w;
-        }
-        tmem_st_16x128b_x8(taddr, cur);
-    }
-    tmem_st_wait();
-}
-
 // Partial sums of the product A v for this thread's four rows over its column class: acc01 = rows k = 0, 1; acc23 =
 // rows k = 2, 3.  The next load is in flight while the current one is multiplied.  vq: the vector by column class,
 // vq[q * kQStride + j] = v[q + 4j].
@@ -1233,11 +1221,12 @@ __device__ __forceinline__ void cg_matvec(uint32_t twarp, const float *vq, int q
 // row it owns (component of x, r, p and A p).  The vector of the next product goes through shared memory, stored by
 // column class.  One fused reduction per step: the recurrences are arranged so that the product is taken with the
 // residual (w = A r; p and s = A p follow by recurrence), and |r|^2 and r.w are reduced together (warp butterfly, then
-// the four warps in order: a fixed order).  alpha0 G + lambda I is added to the matrix in tensor memory first.
+// the four warps in order: a fixed order).  The accumulator started as alpha0 G + lambda I (the MMA warp copies it in
+// before the item's outer products), so the matrix in tensor memory is complete.
 // Returns true with the owned component of x when
 // |r| <= tol |b|; false when the step limit is reached or a step length is not positive (the matrix is left complete
 // in tensor memory, and the caller solves it directly).
-__device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, const float *Bq, uint32_t twarp, int bar_id,
+__device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, uint32_t twarp, int bar_id,
                                            int tid, float b, float x0, float &x_out, int &matvecs)
 {
     const int lane = tid & 31, w = tid >> 5, g = lane >> 2, q = lane & 3;
@@ -1264,7 +1253,6 @@ __device__ __forceinline__ bool cg_in_tmem(const Params &p, CgGroupSmem &gs, con
     float rg_old = 0.f, inv_alpha_old = 0.f, bb = 0.f;
     int products = 0;
     *vslot = warm ? x0 : b;
-    cg_add_base(twarp, Bq, 32 * w + g, q);
     group128_sync(bar_id);
     if (warm) {                 // r = b - A x0
         r = b - product();
@@ -1348,7 +1336,7 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
     const int bar_id = 1 + gidx;
     const uint32_t trow = sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride;
     const float *Brow = Bs + i * kLdB;
-    // (CG: Bs holds alpha0 G + lambda I by column class, see kLdBq)
+    // (CG: Bs holds alpha0 G + lambda I as the MMA warp's copy source; the solver does not read it)
     const int own_cg = 32 * w + (lane >> 2) + 8 * (lane & 3);
     uint32_t trail_parity = 0;
     unsigned cg_rows = 0, cg_matvecs = 0;      // thread 0 of the group counts (per block: far below 2^32)
@@ -1425,7 +1413,7 @@ __device__ void solver_rows_tmem(const Params &p, SmemRows &sm, GroupSmem &gs, c
         bool solved = true;
         if constexpr (CG) {
             int matvecs = 0;
-            solved = cg_in_tmem(p, gs, Bs, sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride, bar_id, tid, b, x0,
+            solved = cg_in_tmem(p, gs, sm.tmem_base + ((uint32_t)(w * 32) << 16) + gidx * kAccStride, bar_id, tid, b, x0,
                                 x, matvecs);
             own = own_cg;
             if (tid == 0) {
@@ -1806,8 +1794,12 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
     if constexpr (FOLD) {
         // (alpha0 G + lambda I is 64 x 64 here and read from global memory; the space holds the groups' scratch)
     } else if constexpr (CG) {
-        for (int e = tid; e < D * D; e += kThreads)
-            Bs[(e >> 7) * kLdBq + (e & 3) * kQStride + ((e & (D - 1)) >> 2)] = p.Bmat[e];
+        // alpha0 G + lambda I as the source of the tensor-memory copies that start every accumulator: sixteen blocks
+        // of 8 columns, each 128 rows x 32 bytes in the layout tmem_cp_128x256b reads (offsets 128 and 256 bytes)
+        for (int e = tid; e < D * D; e += kThreads) {
+            const int r = e >> 7, c = e & (D - 1);
+            Bs[(c >> 3) * 1024 + (r >> 3) * 64 + ((c & 7) >> 2) * 32 + (r & 7) * 4 + (c & 3)] = p.Bmat[e];
+        }
     } else if constexpr (MODE == kModeRows) {
         for (int e = tid; e < D * D; e += kThreads) Bs[(e >> 7) * kLdB + (e & (D - 1))] = p.Bmat[e];
         for (int g = 0; g < C::kGroups; ++g) {
@@ -1844,7 +1836,7 @@ __global__ void __launch_bounds__(block_threads<MODE>(), 1) k_umma(Params p, con
         setmaxnreg_dec<32>();       // idle warps of the last warpgroup
     } else if (rw == kMmaWarp) {
         if constexpr (CG) setmaxnreg_dec<32>();
-        mma_role<MODE>(p, sm, lane);
+        mma_role<MODE>(p, sm, lane, smem_u32(Bs));
     } else {
         if constexpr (CG) setmaxnreg_dec<64>();
         if constexpr (CG) producer_role_items<MODE>(p, &tmap, sm, rw - kFirstProducerWarp, lane);
