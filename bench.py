@@ -291,13 +291,28 @@ def run_ours(args, w):
     ev[0].record()
     trace = []
     for k in range(args.steps):
-        for side in (ALX_ROWS, ALX_COLS):
+        for side, key in ((ALX_ROWS, "rows"), (ALX_COLS, "cols")):
             a.half_epoch(side)
-            if args.trace:      # (reading the statistics waits for the stream: the epoch times of a traced run are not bench values)
+            last = k == args.steps - 1
+            if args.trace or last:
+                # Reading the statistics waits for the stream.  The last timed epoch is read (two waits of a few tens
+                # of microseconds between half-epochs of milliseconds): its per-phase CUDA-event times and solver
+                # counts are the ones the roofline record uses, taken inside the timed region.  A traced run reads
+                # every half-epoch: its epoch times are not bench values.
                 s1 = a.get_stats()
-                trace.append({"epoch": k, "side": side, "ms": s1.ms_half_epoch, "main_ms": s1.ms_main_kernel,
-                              "cg_rows": s1.cg_rows, "cg_products": s1.cg_products, "cg_fallbacks": s1.cg_fallbacks,
-                              "dual_rows": s1.dual_rows, "cholesky_by_policy": list(s1.cholesky_by_policy)})
+                if args.trace:
+                    trace.append({"epoch": k, "side": side, "ms": s1.ms_half_epoch, "main_ms": s1.ms_main_kernel,
+                                  "cg_rows": s1.cg_rows, "cg_products": s1.cg_products, "cg_fallbacks": s1.cg_fallbacks,
+                                  "dual_rows": s1.dual_rows, "cholesky_by_policy": list(s1.cholesky_by_policy)})
+                if last:
+                    half_ms[key].append(s1.ms_half_epoch)
+                    half_ms["gramian"].append(s1.ms_gramian)
+                    half_ms["row_kernels"].append(s1.ms_rows)
+                    half_ms["main_kernel"].append(s1.ms_main_kernel)
+                    half_ms["dual_rows"].append(s1.dual_rows)
+                    half_ms["cg_rows"].append(s1.cg_rows)
+                    half_ms["cg_products"].append(s1.cg_products)
+                    half_ms["cg_fallbacks"].append(s1.cg_fallbacks)
         ev[k + 1].record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -307,18 +322,6 @@ def run_ours(args, w):
     launches = st.kernel_launches - launches0
     step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
     ms_local = sum(step_ms) / args.steps
-    # per-phase times of one more half-epoch pair (outside the timed region)
-    for side, key in ((ALX_ROWS, "rows"), (ALX_COLS, "cols")):
-        a.half_epoch(side)
-        s2 = a.get_stats()
-        half_ms[key].append(s2.ms_half_epoch)
-        half_ms["gramian"].append(s2.ms_gramian)
-        half_ms["row_kernels"].append(s2.ms_rows)
-        half_ms["main_kernel"].append(s2.ms_main_kernel)
-        half_ms["dual_rows"].append(s2.dual_rows)
-        half_ms["cg_rows"].append(s2.cg_rows)
-        half_ms["cg_products"].append(s2.cg_products)
-        half_ms["cg_fallbacks"].append(s2.cg_fallbacks)
     fp32_peak = a.fp32_peak_tflops()
     loss = a.loss()[0]
     evaluation = None
@@ -417,7 +420,7 @@ def run_ours(args, w):
                                    "gramian": statistics.mean(half_ms["gramian"]), "row_kernels": rows_ms},
                  "roofline_half_epoch_ms": {"bytes": t_bytes * 1e3, "tensor": t_tensor * 1e3, "alu": t_alu * 1e3,
                                             "max(bytes, tensor+alu)": t_roof * 1e3},
-                 # mean half-epoch of the TIMED epochs (the pair above is one more epoch, run for the per-phase figures)
+                 # mean half-epoch of the timed epochs (the per-phase figures above are the last timed epoch's)
                  "frac_of_roofline_time": t_roof * 1e3 / (0.5 * ms_local),
                  "roofline_half_epoch_ms_solve_as_spent": {"alu": t_alu_cg * 1e3, "max(bytes, tensor+alu)": t_roof_cg * 1e3,
                                                            "frac": t_roof_cg * 1e3 / (0.5 * ms_local),
@@ -500,7 +503,7 @@ def run_ours(args, w):
                "cpu_baseline": cpu_baseline,
                "extra": {"evaluation": evaluation, "trace": trace or None, "solver": {"option": args.solver, "cg_rows": half_ms["cg_rows"], "cg_products": half_ms["cg_products"],
                                     "cg_fallbacks": half_ms["cg_fallbacks"],
-                                    "note": "[rows half-epoch, columns half-epoch] of the half-epoch pair after the timed region"},
+                                    "note": "[rows half-epoch, columns half-epoch] of the last timed epoch"},
                          "epoch_ms_each": step_ms, "loss_after": loss, "fp32_peak_tflops_measured": fp32_peak,
                          "setup_s": {"generate": t_gen, "alx_set_csr_device": t_set},
                          "rows_in_class": [list(st.rows_in_class[0]), list(st.rows_in_class[1])],
