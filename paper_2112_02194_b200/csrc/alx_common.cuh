@@ -161,10 +161,12 @@ struct CgPolicy {
     int short_rows_by_cg; // this half-epoch: 1 = rows of 17 .. 32 observations go to the whole-rows kernel, not the dual form
     int pad_;
 };
-// The dual-form kernel for rows of 17 .. 32 observations costs about as much as ten products of the whole-rows kernel
-// (measured: 28 ns against 10 + 1.8 per product ns per row): where the side's last conjugate-gradient run stayed at or
-// below this many products per row, those rows go there
-constexpr float kShortRowsByCgProducts = 11.f;
+// Rows of 17 .. 32 observations: dual form, or the whole-rows kernel's conjugate gradients where those are cheap.
+// Measured on the rows side of the 10M x 10M workload (1.32M such rows): with them in the whole-rows kernel the
+// half-epoch takes 152.3 ms against 161.1 ms at 10.9 products per row (6.7 ns per row saved); a product costs about
+// 1.8 ns per row, so the two meet near 14.5 products.  Where the side's last conjugate-gradient run stayed at or below
+// this many products per row, those rows go there
+constexpr float kShortRowsByCgProducts = 13.f;
 // Conjugate gradients pay while a row takes fewer than about 28 products on average (measured on B200: about 2900 + 300
 // per product cycles of an SM per row, against 12 600 for the in-place Cholesky; alx_options.cg_switch_products); beyond
 // that the side's next half-epochs go to Cholesky, with one conjugate-gradient half-epoch every kCgReprobe to see whether
