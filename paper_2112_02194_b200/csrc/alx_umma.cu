@@ -651,6 +651,7 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
     constexpr uint32_t kIdescMain = idesc_bf16_mn_major(128, 128);
     constexpr uint32_t kIdescY = idesc_bf16_mn_major(128, 16);
     const uint32_t tmem = sm.tmem_base;
+    const uint64_t base_desc = smem_desc(base_smem, 128, 256, 0);      // (conjugate-gradient rows kernel: alpha0 G + lambda I)
     int slot = 0;             // ring position and phase of the next stage
     uint32_t ph = 0;
     bool alive = true;
@@ -702,9 +703,9 @@ template <int MODE> __device__ void mma_role(const Params &p, SmemT<MODE> &sm, i
                 // the accumulator starts as alpha0 G + lambda I (copied from shared memory by the tensor pipe, in
                 // order with the products that follow): the solver finds the complete matrix of Eq. 4
                 if (lane == 0) {
+                    // (the address field of the descriptor counts 16-byte units: 4096 bytes per block of 8 columns)
 #pragma unroll 1
-                    for (int c8 = 0; c8 < D / 8; ++c8)
-                        tmem_cp_128x256b(d_main + 8 * c8, smem_desc(base_smem + c8 * 4096, 128, 256, 0));
+                    for (int c8 = 0; c8 < D / 8; ++c8) tmem_cp_128x256b(d_main + 8 * c8, base_desc + (uint64_t)(c8 * 256));
                 }
                 first = false;
             }
